@@ -1,0 +1,24 @@
+"""CPU oracle for the SJA round -- TEST INFRASTRUCTURE ONLY.
+
+Only ``tests/``, ``__graft_entry__.smoke()`` and the CPU-baseline legs of ``bench.py``
+may import this package.  It shares nothing with the CUDA path and does not import it.
+
+Contents
+--------
+``sja_oracle.c``   the naive step-by-step walk (R1-R6 in its header), built with gcc
+``brute.py``       exhaustive prefix enumeration in pure Python, for tiny inputs
+``scan.py``        the per-job prefix quantities written out with numpy
+``api.py``         ctypes wrapper around the compiled walk
+"""
+from .api import (  # noqa: F401
+    AWARD_DTYPE,
+    GAP_DTYPE,
+    NO_JOB,
+    build,
+    commit,
+    num_threads,
+    pair,
+    select,
+)
+from .brute import brute_pair, brute_select  # noqa: F401
+from .scan import boundary_table, dense_prefix  # noqa: F401

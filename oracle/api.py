@@ -1,0 +1,131 @@
+"""ctypes wrapper around ``sja_oracle.c`` (the naive walk).  Test infrastructure only."""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sja_oracle.c")
+_LIB = os.path.join(_HERE, "libsja_oracle.so")
+
+NO_JOB = 0xFFFFFFFF
+
+GAP_DTYPE = np.dtype(
+    [("slice", "<u4"), ("start_ms", "<u4"), ("T_ms", "<u4"), ("C_MiB", "<u4")]
+)
+AWARD_DTYPE = np.dtype(
+    [("job", "<u4"), ("end_step", "<u4"), ("dur_ms", "<u4"), ("granted", "<u4"),
+     ("score", "<u8")]
+)
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (-O2 -fopenmp) next to its source."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    tmp = _LIB + f".tmp{os.getpid()}"
+    cmd = ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-Wall", "-Wextra",
+           "-o", tmp, _SRC]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    build()
+    lib = ctypes.CDLL(_LIB)
+    u32p = ctypes.POINTER(ctypes.c_uint32)
+    u64p = ctypes.POINTER(ctypes.c_uint64)
+    u8p = ctypes.POINTER(ctypes.c_uint8)
+    vp = ctypes.c_void_p
+    lib.orc_pair.restype = ctypes.c_int
+    lib.orc_pair.argtypes = [vp, vp, vp, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint32,
+                             ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
+                             u32p, u32p, u64p]
+    lib.orc_select.restype = ctypes.c_int
+    lib.orc_select.argtypes = [ctypes.c_uint32, vp, vp, vp, vp, vp, vp, vp, vp,
+                               ctypes.c_uint32, vp, ctypes.c_uint32, vp]
+    lib.orc_commit.restype = ctypes.c_int64
+    lib.orc_commit.argtypes = [ctypes.c_uint32, vp, vp, ctypes.c_uint32, vp, vp]
+    lib.orc_num_threads.restype = ctypes.c_int
+    lib.orc_num_threads.argtypes = []
+    del u8p
+    _lib = lib
+    return lib
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data
+
+
+def _as(a, dtype):
+    if a is None:
+        return None
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def num_threads() -> int:
+    return int(_load().orc_num_threads())
+
+
+def pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: int):
+    """R1-R3 for one (gap, job) pair: ``None`` for decline, else ``(k, dur, work)``."""
+    lib = _load()
+    k = ctypes.c_uint32()
+    dur = ctypes.c_uint32()
+    work = ctypes.c_uint64()
+    ok = lib.orc_pair(prof.dur_ms.ctypes.data, prof.mem_MiB.ctypes.data,
+                      prof.safe_bits.ctypes.data, int(prof.off[j]), int(prof.off[j + 1]),
+                      int(p), int(ready_ms), int(start_ms), int(T_ms), int(C_MiB),
+                      ctypes.byref(k), ctypes.byref(dur), ctypes.byref(work))
+    if not ok:
+        return None
+    return int(k.value), int(dur.value), int(work.value)
+
+
+def select(prof, progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray,
+           policy: int) -> np.ndarray:
+    """R1-R5 for a batch of gaps; returns ``AWARD_DTYPE[G]`` (``granted`` all zero)."""
+    lib = _load()
+    off = _as(prof.off, np.uint64)
+    d = _as(prof.dur_ms, np.uint32)
+    m = _as(prof.mem_MiB, np.uint32)
+    s = _as(prof.safe_bits, np.uint32)
+    progress = _as(progress, np.uint32)
+    ready_ms = _as(ready_ms, np.uint32)
+    wait = _as(prof.wait_ms, np.uint32)
+    prio = _as(prof.prio, np.uint8)
+    gaps = np.ascontiguousarray(gaps, dtype=GAP_DTYPE)
+    awards = np.zeros(gaps.shape[0], dtype=AWARD_DTYPE)
+    rc = lib.orc_select(off.shape[0] - 1, _ptr(off), _ptr(d), _ptr(m), _ptr(s),
+                        _ptr(progress), _ptr(ready_ms), _ptr(wait), _ptr(prio),
+                        gaps.shape[0], _ptr(gaps), int(policy), _ptr(awards))
+    if rc != 0:
+        raise ValueError("oracle select: unknown policy or missing attribute array")
+    return awards
+
+
+def commit(progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray,
+           awards: np.ndarray) -> int:
+    """R6, in place on ``progress``, ``ready_ms`` and ``awards['granted']``."""
+    lib = _load()
+    assert progress.dtype == np.uint32 and progress.flags.c_contiguous
+    assert ready_ms.dtype == np.uint32 and ready_ms.flags.c_contiguous
+    assert awards.dtype == AWARD_DTYPE and awards.flags.c_contiguous
+    gaps = np.ascontiguousarray(gaps, dtype=GAP_DTYPE)
+    n = lib.orc_commit(progress.shape[0], _ptr(progress), _ptr(ready_ms),
+                       gaps.shape[0], _ptr(gaps), _ptr(awards))
+    if n < 0:
+        raise OverflowError("oracle commit: start + dur does not fit in 32 bits")
+    return int(n)

@@ -1,0 +1,71 @@
+"""Exhaustive prefix enumeration for tiny inputs -- TEST INFRASTRUCTURE ONLY.
+
+For one (gap, job) pair every end index k in (p, len] is tried; the window sum and the
+window maximum are recomputed from scratch for each k (no running state), the candidate
+set of Sections 3.1 / 3.8 / 3.9 is filtered literally, and the longest candidate is kept.
+This is O(len^2) per pair and is only meant to check the step-by-step walk.
+"""
+from __future__ import annotations
+
+NO_JOB = 0xFFFFFFFF
+_MASK64 = (1 << 64) - 1
+
+
+def _safe(bits, i: int) -> bool:
+    return bool((int(bits[i >> 5]) >> (i & 31)) & 1)
+
+
+def brute_pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: int):
+    """``None`` (decline) or ``(k, dur, work)`` of the longest feasible subjob."""
+    s, e = int(prof.off[j]), int(prof.off[j + 1])
+    length = e - s
+    if p >= length:
+        return None
+    if start_ms < ready_ms:
+        return None
+    d = [int(x) for x in prof.dur_ms[s:e]]
+    m = [int(x) for x in prof.mem_MiB[s:e]]
+    candidates = []
+    for k in range(p + 1, length + 1):
+        ends_safe = _safe(prof.safe_bits, s + k - 1) or k == length
+        if not ends_safe:
+            continue
+        if sum(d[p:k]) > T_ms:
+            continue
+        if max(m[p:k]) > C_MiB:
+            continue
+        candidates.append(k)
+    if not candidates:
+        return None
+    k = max(candidates)
+    dur = sum(d[p:k])
+    work = sum(d[i] * m[i] for i in range(p, k))
+    return k, dur, work
+
+
+def brute_select(prof, progress, ready_ms, gaps, policy: int):
+    """Per-gap winner by sorting all interested jobs; returns a list of dicts."""
+    out = []
+    n_jobs = len(prof.off) - 1
+    for g in range(len(gaps)):
+        start, T, C = int(gaps["start_ms"][g]), int(gaps["T_ms"][g]), int(gaps["C_MiB"][g])
+        entries = []
+        for j in range(n_jobs):
+            r = brute_pair(prof, j, int(progress[j]), int(ready_ms[j]), start, T, C)
+            if r is None:
+                continue
+            k, dur, work = r
+            cls = 0
+            score = work
+            if policy == 1:
+                score = (work * (1 + int(prof.wait_ms[j]) // 1000)) & _MASK64
+            elif policy == 2:
+                cls = int(prof.prio[j])
+            # larger class, then larger score, then smaller job id
+            entries.append((-cls, -score, j, k, dur, score))
+        if not entries:
+            out.append(dict(job=NO_JOB, end_step=0, dur_ms=0, score=0))
+        else:
+            _, _, j, k, dur, score = min(entries)
+            out.append(dict(job=j, end_step=k, dur_ms=dur, score=score))
+    return out

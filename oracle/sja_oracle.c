@@ -1,0 +1,220 @@
+/*
+ * CPU oracle for the SJA advertise / signal / select / commit round.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition the CUDA
+ * library is checked against.  It shares no code, header, table or helper with the
+ * CUDA path and must never be linked into, or called from, the product path.
+ *
+ * What it computes, and where the paper defines it:
+ *   - A subjob is a self-contained fragment of a job that fits the offered window
+ *     in time and stays below the slice capacity for its whole lifetime (Section 3.1).
+ *   - A job is admissible in a window of length T on a slice of capacity C when the
+ *     maximum of its (risk-adjusted) memory envelope U over the window is <= C
+ *     (Section 3.8, and the window-max test of Section 3.9).  The per-step mem_MiB
+ *     array is U sampled per step; memory is constant within a step.
+ *   - A subjob ends at a safe boundary, the natural cut point where a job can be
+ *     paused with a checkpoint (Section 3.7).
+ *   - Three-phase protocol: the scheduler advertises gaps, each job signals interest
+ *     or declines, the scheduler applies its policy and grants the slot; nothing is
+ *     materialised before the grant (Section 3.5).  Greedy slot filling without
+ *     lookahead is the intended design (Section 4.2).
+ *   - The granted job resumes later from the end of its last completed fragment
+ *     (Sections 3.1, 3.5).
+ *
+ * Integer formalisation used here (the paper is prose; every choice is a stated reading):
+ *   R1 eligibility : p_j < len_j and start_g >= ready_j.
+ *   R2 candidates  : k in (p_j, len_j] with step k-1 safe (the last step of a job always
+ *                    counts as safe), sum d[p_j..k) <= T_g, max m[p_j..k) <= C_g (inclusive).
+ *   R3 signal      : interest iff eligible and a candidate exists; the subjob is the
+ *                    longest one, k* = max candidates; dur = sum d, work = sum d*m (u64).
+ *   R4 score       : efficiency  work;
+ *                    fairness    work * (1 + wait_j/1000), truncating division, u64;
+ *                    SLA         lexicographic (prio_j, work), larger prio = more urgent.
+ *   R5 select      : per gap, the interested job with the largest key; ties go to the
+ *                    lowest job id; no interested job -> SJA_NO_JOB and zeros.
+ *   R6 commit      : a job that won several gaps accepts the one with the largest k*,
+ *                    ties to the lowest gap id; that gap is granted, the others are not;
+ *                    then p_j = k*, ready_j = start_g + dur.
+ *
+ * The walk below visits one step at a time, exactly in that order: no prefix arrays,
+ * no search, no blocking.  OpenMP only spreads independent gaps over host threads.
+ *
+ * Pins (tests/test_oracle_pins.py): exhaustive prefix enumeration on tiny inputs,
+ * closed forms, reductions to numpy cumsum / searchsorted, monotonicity and symmetry
+ * properties, the rigid-job special case, hand-computed policy examples, and the paper's
+ * illustrative scenario.  The paper prints no numeric award values, so beyond those pins
+ * the award values are "parity unpinned".
+ */
+#include <stddef.h>
+#include <stdint.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORC_NO_JOB 0xFFFFFFFFu
+
+typedef struct {
+    uint32_t slice, start_ms, T_ms, C_MiB;
+} orc_gap;
+
+typedef struct {
+    uint32_t job, end_step, dur_ms, granted;
+    uint64_t score;
+} orc_award;
+
+enum { ORC_EFFICIENCY = 0, ORC_FAIRNESS = 1, ORC_SLA = 2 };
+
+static int step_is_safe(const uint32_t *safe_bits, uint64_t i)
+{
+    return (int)((safe_bits[i >> 5] >> (i & 31u)) & 1u);
+}
+
+/*
+ * R1-R3 for one (gap, job) pair.  Returns 1 for interest (and fills k, dur, work),
+ * 0 for decline.  [s, e) is the job's range of global step indices, p its progress.
+ */
+int orc_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *safe_bits,
+             uint64_t s, uint64_t e, uint32_t p, uint32_t ready_ms,
+             uint32_t start_ms, uint32_t T_ms, uint32_t C_MiB,
+             uint32_t *k_out, uint32_t *dur_out, uint64_t *work_out)
+{
+    uint64_t len = e - s;
+    if ((uint64_t)p >= len) return 0;            /* R1: finished job */
+    if (start_ms < ready_ms) return 0;           /* R1: gap opens before the job is ready */
+
+    uint64_t acc = 0, work = 0;
+    uint32_t peak = 0;
+    int found = 0;
+    uint32_t best_k = 0, best_dur = 0;
+    uint64_t best_work = 0;
+    for (uint64_t i = s + p; i < e; ++i) {
+        acc += dur_ms[i];
+        if (mem_MiB[i] > peak) peak = mem_MiB[i];
+        work += (uint64_t)dur_ms[i] * (uint64_t)mem_MiB[i];
+        if (acc > (uint64_t)T_ms || peak > C_MiB) break;   /* R2: window or capacity broken */
+        if (step_is_safe(safe_bits, i) || i + 1 == e) {    /* R2: safe boundary after step i */
+            found = 1;
+            best_k = (uint32_t)(i + 1 - s);
+            best_dur = (uint32_t)acc;
+            best_work = work;
+        }
+    }
+    if (!found) return 0;
+    *k_out = best_k;
+    *dur_out = best_dur;
+    *work_out = best_work;
+    return 1;
+}
+
+/* R4: the policy key of an interested job, as (class, score). */
+static void policy_key(uint32_t policy, uint64_t work, uint32_t j,
+                       const uint32_t *wait_ms, const uint8_t *prio,
+                       uint32_t *cls_out, uint64_t *score_out)
+{
+    *cls_out = 0;
+    *score_out = work;
+    if (policy == ORC_FAIRNESS) {
+        *score_out = work * (uint64_t)(1u + wait_ms[j] / 1000u);
+    } else if (policy == ORC_SLA) {
+        *cls_out = prio[j];
+    }
+}
+
+/*
+ * R1-R5 for a batch of gaps.  progress / ready_ms are read, never written
+ * (no subjob state exists before a grant, Section 3.5).
+ * Returns 0, or -1 for an unknown policy / missing attribute array.
+ */
+int orc_select(uint32_t n_jobs, const uint64_t *off,
+               const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *safe_bits,
+               const uint32_t *progress, const uint32_t *ready_ms,
+               const uint32_t *wait_ms, const uint8_t *prio,
+               uint32_t n_gaps, const orc_gap *gaps, uint32_t policy,
+               orc_award *awards)
+{
+    if (policy > ORC_SLA) return -1;
+    if (policy == ORC_FAIRNESS && !wait_ms) return -1;
+    if (policy == ORC_SLA && !prio) return -1;
+
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t g = 0; g < (int64_t)n_gaps; ++g) {
+        orc_gap gap = gaps[g];
+        int have = 0;
+        uint32_t best_cls = 0, best_job = ORC_NO_JOB, best_k = 0, best_dur = 0;
+        uint64_t best_score = 0;
+        for (uint32_t j = 0; j < n_jobs; ++j) {
+            uint32_t k, dur;
+            uint64_t work;
+            if (!orc_pair(dur_ms, mem_MiB, safe_bits, off[j], off[j + 1], progress[j],
+                          ready_ms[j], gap.start_ms, gap.T_ms, gap.C_MiB, &k, &dur, &work))
+                continue;                                      /* decline */
+            uint32_t cls;
+            uint64_t score;
+            policy_key(policy, work, j, wait_ms, prio, &cls, &score);
+            /* jobs are visited in ascending id, so a strict ">" keeps the lowest id on ties */
+            if (!have || cls > best_cls || (cls == best_cls && score > best_score)) {
+                have = 1;
+                best_cls = cls;
+                best_score = score;
+                best_job = j;
+                best_k = k;
+                best_dur = dur;
+            }
+        }
+        orc_award a;
+        a.job = have ? best_job : ORC_NO_JOB;
+        a.end_step = have ? best_k : 0;
+        a.dur_ms = have ? best_dur : 0;
+        a.granted = 0;
+        a.score = have ? best_score : 0;
+        awards[g] = a;
+    }
+    return 0;
+}
+
+/*
+ * R6.  Marks granted gaps in awards[], advances progress / ready_ms of the granted
+ * jobs, returns the number of grants (or -1 if start + dur does not fit in 32 bits).
+ */
+int64_t orc_commit(uint32_t n_jobs, uint32_t *progress, uint32_t *ready_ms,
+                   uint32_t n_gaps, const orc_gap *gaps, orc_award *awards)
+{
+    int64_t granted = 0;
+    for (uint32_t g = 0; g < n_gaps; ++g) awards[g].granted = 0;
+    for (uint32_t g = 0; g < n_gaps; ++g) {
+        uint32_t j = awards[g].job;
+        if (j == ORC_NO_JOB || j >= n_jobs) continue;
+        /* is g the gap this job accepts?  largest k*, then lowest gap id */
+        int accept = 1;
+        for (uint32_t h = 0; h < n_gaps; ++h) {
+            if (h == g || awards[h].job != j) continue;
+            if (awards[h].end_step > awards[g].end_step ||
+                (awards[h].end_step == awards[g].end_step && h < g)) {
+                accept = 0;
+                break;
+            }
+        }
+        if (accept) awards[g].granted = 1;
+    }
+    for (uint32_t g = 0; g < n_gaps; ++g) {
+        if (!awards[g].granted) continue;
+        uint32_t j = awards[g].job;
+        uint64_t new_ready = (uint64_t)gaps[g].start_ms + (uint64_t)awards[g].dur_ms;
+        if (new_ready > 0xFFFFFFFFull) return -1;
+        progress[j] = awards[g].end_step;
+        ready_ms[j] = (uint32_t)new_ready;
+        ++granted;
+    }
+    return granted;
+}
+
+int orc_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
