@@ -1,0 +1,343 @@
+#!/usr/bin/env python
+"""Benchmark of the SJA advertise / signal / select / commit round.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 0..4] [--impl ours|reference]
+
+One "step" is one pass of the whole round over one synthetic workload: the segmented scan
+of all job profiles (sja_load_profiles), sja_advertise, sja_select and sja_commit.
+Metric: job-gap pairs evaluated per second (G*J pairs per step; every pair counts, however
+early it is declined).  Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2509_19086_b200 import workloads as wl  # noqa: E402
+
+METRIC = "job-gap pairs evaluated/s"
+UNIT = "pairs/s"
+POLICY_NAMES = {0: "efficiency", 1: "fairness", 2: "sla"}
+# kernels launched per step: count_boundaries, row_offsets, scan_profiles | select_search,
+# finalize_awards | commit_vote, commit_apply, commit_refresh
+KERNELS_PER_STEP = 8
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(smax)) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _pinned(a: np.ndarray):
+    """A pinned torch tensor holding a's bytes and a numpy view of it."""
+    import torch
+    t = torch.empty(a.nbytes, dtype=torch.uint8).pin_memory()
+    v = t.numpy().view(a.dtype).reshape(a.shape)
+    v[...] = a
+    return t, v
+
+
+def _to_device(a: np.ndarray, device):
+    """Copy a numpy array to the device as a typed torch tensor (u64 -> int64, u32 -> int32 views)."""
+    import torch
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.uint64:
+        t = torch.from_numpy(a.view(np.int64))
+    elif a.dtype == np.uint8:
+        t = torch.from_numpy(a)
+    else:
+        t = torch.from_numpy(a.view(np.uint8).reshape(-1).view(np.int32))
+    return t.to(device, non_blocking=False)
+
+
+def oracle_rate(prof, gaps, policy, target_s=12.0):
+    """Time the CPU oracle (as it stands) on a bounded sample of the workload's gaps."""
+    import oracle
+    J = prof.n_jobs
+    progress = np.zeros(J, np.uint32)
+    threads = oracle.num_threads()
+    probe = min(gaps.shape[0], max(threads, 8))
+    t0 = time.perf_counter()
+    oracle.select(prof, progress, prof.ready_ms, gaps[:probe], policy)
+    dt = time.perf_counter() - t0
+    n = int(min(gaps.shape[0], max(probe, probe * target_s / max(dt, 1e-6))))
+    n = max(threads, (n // threads) * threads) if n >= threads else n
+    n = min(n, gaps.shape[0])
+    t0 = time.perf_counter()
+    oracle.select(prof, progress, prof.ready_ms, gaps[:n], policy)
+    dt = time.perf_counter() - t0
+    return {"value": n * J / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"first {n} of {gaps.shape[0]} gaps x all {J} jobs, naive walk (gcc -O2 -fopenmp), {dt:.2f} s"}
+
+
+def run_reference(args, spec):
+    """The reference arm: the CPU oracle on the host cores, same workload / metric / unit."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    prof = wl.make_profiles(spec, threads=os.cpu_count() or 8)
+    gaps = wl.make_gaps(spec)
+    import oracle
+    J, G = prof.n_jobs, gaps.shape[0]
+    progress = np.zeros(J, np.uint32)
+    threads = oracle.num_threads()
+    # size one step's sample so that warmup + steps stay within a few minutes
+    t0 = time.perf_counter()
+    probe = min(G, max(threads, 8))
+    oracle.select(prof, progress, prof.ready_ms, gaps[:probe], spec.policy)
+    per_gap = (time.perf_counter() - t0) / probe
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    n = int(max(1, min(G, budget / max(per_gap, 1e-9))))
+    for _ in range(args.warmup):
+        oracle.select(prof, progress, prof.ready_ms, gaps[:n], spec.policy)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        aw = oracle.select(prof, progress, prof.ready_ms, gaps[:n], spec.policy)
+        p2, r2 = progress.copy(), prof.ready_ms.copy()
+        oracle.commit(p2, r2, gaps[:n], aw)
+    dt = time.perf_counter() - t0
+    value = args.steps * n * J / dt
+    sample = f"per step: first {n} of {G} gaps x all {J} jobs (select + commit), naive walk"
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32/u64",
+        "data": "synthetic", "config": {"workload": spec.name, "jobs": J, "gaps": G, "steps_total": prof.n_steps,
+                                        "policy": POLICY_NAMES[spec.policy]},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", type=int, default=2, help="index into the published configuration list")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--flags", type=int, default=0, help="sja_policy.flags (1 = per-pair search kernel)")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    spec = wl.SPECS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, spec)
+        return
+
+    import torch
+    from paper_2509_19086_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=device)
+
+    # replicas: every rank runs an independent scheduler instance on its own seeded workload
+    my_spec = wl.scaled(spec, index=spec.index + 1000 * rank) if rank else spec
+    prof = wl.make_profiles(my_spec, threads=max(1, (os.cpu_count() or 8) // max(1, world)))
+    gaps = wl.make_gaps(my_spec)
+    J, G, N = prof.n_jobs, int(gaps.shape[0]), prof.n_steps
+    pairs = J * G
+
+    stream = torch.cuda.Stream(device=device)
+    ctx = binding.Sja(device=local_rank, stream=stream.cuda_stream)
+
+    host_arrays = dict(off=prof.off, d=prof.dur_ms, m=prof.mem_MiB, s=prof.safe_bits, ready=prof.ready_ms)
+    if prof.wait_ms is not None:
+        host_arrays["wait"] = prof.wait_ms
+    if prof.prio is not None:
+        host_arrays["prio"] = prof.prio
+    pinned_keep, pinned = {}, {}
+    for k, a in host_arrays.items():
+        pinned_keep[k], pinned[k] = _pinned(a)
+    pinned_keep["gaps"], gaps_pinned = _pinned(gaps.view(np.uint8))
+    gaps_pinned = gaps_pinned.view(wl.GAP_DTYPE)
+    dev = {k: _to_device(a, device) for k, a in host_arrays.items()}
+    dev_gaps = _to_device(gaps, device)
+    torch.cuda.synchronize()
+
+    def step_device():
+        ctx.load_profiles(dev["off"], dev["d"], dev["m"], dev["s"], dev["ready"],
+                          wait_ms=dev.get("wait"), prio=dev.get("prio"))
+        ctx.advertise(dev_gaps)
+        ctx.select(my_spec.policy, flags=args.flags)
+        ctx.commit(want_count=False)
+
+    def step_e2e():
+        ctx.load_profiles(pinned["off"], pinned["d"], pinned["m"], pinned["s"], pinned["ready"],
+                          wait_ms=pinned.get("wait"), prio=pinned.get("prio"))
+        ctx.advertise(gaps_pinned)
+        aw = ctx.select(my_spec.policy, flags=args.flags, out="host")
+        n = ctx.commit(want_count=True)
+        return aw, n
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            step_device()
+        n_rows = ctx.scan_size()
+        ctx.profile_enable(True)
+        sampler = ClockSampler(local_rank)
+        barrier()
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            step_device()
+        e1.record(stream)
+        barrier()
+        ms_total = e0.elapsed_time(e1)
+        clocks = sampler.stop()
+        timing = ctx.profile_read()
+        ctx.profile_enable(False)
+
+        # end to end: pinned host inputs in, awards + grant count out, every step
+        step_e2e()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            aw, n_granted = step_e2e()
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+
+    t_ms = torch.tensor([ms_total, 1e3 * e2e_s], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = float(t_ms[0]), float(t_ms[1])
+    ms_per_step = ms_total / args.steps
+    value = world * pairs * args.steps / (ms_total * 1e-3)
+    e2e_value = world * pairs * args.e2e_steps / (e2e_ms * 1e-3)
+    h2d = sum(int(a.nbytes) for a in host_arrays.values()) + int(gaps.nbytes)
+    d2h = 24 * G + 4
+
+    peak, peak_kind = measured_peak()
+    scan_ms = timing["scan_ms"] / max(1, timing["scan_launches"])
+    scan_bytes = prof.raw_bytes() + 24 * n_rows
+    achieved = scan_bytes / (scan_ms * 1e-3) / 1e9 if scan_ms > 0 else 0.0
+    roofline = {
+        "kernel": "scan_profiles_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+        "bytes_per_launch": scan_bytes, "ms_per_launch": scan_ms,
+    }
+    breakdown = {k: timing[k] / args.steps for k in ("scan_ms", "prep_ms", "advertise_ms", "select_ms", "commit_ms")}
+    select_ms = breakdown["select_ms"]
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u32/u64", "data": "synthetic",
+        "config": {"workload": my_spec.name if rank == 0 else spec.name, "jobs": J, "gaps": G, "steps_total": N,
+                   "boundary_rows": n_rows, "policy": POLICY_NAMES[spec.policy], "parallelism": f"replicas x{world}",
+                   "l2": "inputs larger than L2 (profile arrays re-read from HBM every step)"
+                   if prof.raw_bytes() > 200e6 else "inputs smaller than L2",
+                   "flags": args.flags},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": e2e_ms / args.e2e_steps, "steps": args.e2e_steps},
+        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "roofline": roofline,
+        "kernel_ms_per_step": breakdown,
+        "select_pairs_per_s": pairs / (select_ms * 1e-3) if select_ms > 0 else None,
+        "profile_gb_per_s": prof.raw_bytes() / (scan_ms * 1e-3) / 1e9 if scan_ms > 0 else None,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = oracle_rate(prof, gaps, my_spec.policy)
+    ctx.close()
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

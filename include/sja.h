@@ -1,0 +1,199 @@
+/*
+ * libsja -- the advertise / signal / select / commit round of Scheduler-Driven Job
+ * Atomization (SJA) on one NVIDIA B200 (sm_100a).
+ *
+ * The paper defines the round in prose: the scheduler advertises execution gaps (a time
+ * window on a MIG slice of some capacity), every waiting job answers "interest" if it
+ * could safely generate a subjob for that time/capacity pair, the scheduler picks one
+ * interested job per gap by its policy, and only the granted job materialises the subjob
+ * (Section 3.5; admissibility test in Sections 3.8 and 3.9; greedy slot filling in
+ * Section 4.2).  This library fixes that prose as integer arithmetic:
+ *
+ *   job j        steps i = 0..len_j-1 with duration d[i] (ms), memory envelope m[i] (MiB,
+ *                the risk-adjusted envelope U of Section 3.9 sampled per step) and a
+ *                safe-boundary bit s[i] (a checkpoint cut after step i, Section 3.7); the
+ *                end of a job always counts as a boundary.  State: progress p_j (steps
+ *                already granted) and ready_j (ms).
+ *   gap g        (slice, start, T, C).
+ *   signal       j is interested in g iff p_j < len_j, start_g >= ready_j and some
+ *                k in (p_j, len_j] ends on a boundary with sum d[p_j..k) <= T_g and
+ *                max m[p_j..k) <= C_g (all bounds inclusive).  Its subjob is the longest
+ *                such k; dur = sum d, work = sum d*m over [p_j, k).
+ *   score        EFFICIENCY work; FAIRNESS work * (1 + wait_j/1000) (truncating division);
+ *                SLA (prio_j, work) compared lexicographically, larger prio more urgent.
+ *   select       per gap the interested job with the largest score, ties to the lowest job id.
+ *   commit       a job that won several gaps accepts the one with the largest k, ties to
+ *                the lowest gap id; p_j = k, ready_j = start_g + dur.
+ *
+ * All pointers are plain C pointers.  Every array argument is either a HOST pointer or a
+ * DEVICE pointer on the context's device, as said by the `where` argument of the call.
+ * The caller owns every buffer it passes; the library copies what it needs before the
+ * call's work completes on the context's stream and never keeps a caller pointer.
+ * Device-memspace calls are ordered on the context's stream and return without waiting;
+ * host-memspace outputs are complete when the call returns.  Device input arrays dur_ms,
+ * mem_MiB and safe_bits must be 16-byte aligned.
+ *
+ * No call aborts the process or traps the device.  Every call returns an sja_status;
+ * sja_last_error() gives a text for the most recent failure on that context.
+ * SJA_ERR_INVALID_ARG, SJA_ERR_BAD_PROFILE and SJA_ERR_STATE leave the context as it was.
+ * After SJA_ERR_CUDA the context is unusable except for sja_destroy().
+ * A context is not thread-safe; use one per host thread or lock around it.
+ */
+#ifndef SJA_H
+#define SJA_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sja_ctx sja_ctx; /* opaque; owns all device memory it allocates */
+
+typedef enum {
+    SJA_OK = 0,
+    SJA_ERR_INVALID_ARG = 1, /* NULL pointer, zero count, unknown policy, misaligned device array */
+    SJA_ERR_BAD_PROFILE = 2, /* off[0] != 0, off not monotone, a job longer than 2^32-1 steps, progress > len */
+    SJA_ERR_OVERFLOW = 3,    /* a job's total duration >= 2^32 ms, total work or a score too large, start + dur >= 2^32 */
+    SJA_ERR_STATE = 4,       /* call order: select before advertise/load, commit before select or twice */
+    SJA_ERR_OOM = 5,         /* device or host allocation failed */
+    SJA_ERR_CUDA = 6,        /* a CUDA call failed; context poisoned */
+    SJA_ERR_TIMEOUT = 7      /* reserved: no kernel of this library waits on another */
+} sja_status;
+
+typedef enum { SJA_MEM_HOST = 0, SJA_MEM_DEVICE = 1 } sja_memspace;
+
+/* One advertised execution gap: "time interval and slice capacity" (Section 3.5). 16 bytes. */
+typedef struct {
+    uint32_t slice;    /* MIG slice label, carried through, not used in scoring */
+    uint32_t start_ms; /* absolute start of the window */
+    uint32_t T_ms;     /* window length */
+    uint32_t C_MiB;    /* slice memory capacity */
+} sja_gap;
+
+typedef enum {
+    SJA_POLICY_EFFICIENCY = 0, /* score = work */
+    SJA_POLICY_FAIRNESS = 1,   /* score = work * (1 + wait_ms/1000); needs wait_ms at load */
+    SJA_POLICY_SLA = 2         /* key = (prio, work); needs prio at load; reported score = work */
+} sja_policy_kind;
+
+/* Bit 0 of sja_policy.flags: evaluate every pair with the per-pair binary search over the
+ * boundary table instead of the windowed merge kernel (same results; for testing). */
+#define SJA_FLAG_FORCE_SEARCH 1u
+
+typedef struct {
+    uint32_t kind;  /* sja_policy_kind */
+    uint32_t flags; /* SJA_FLAG_* */
+} sja_policy;
+
+#define SJA_NO_JOB 0xFFFFFFFFu
+
+/* The scheduler's decision for one gap (third protocol phase, Section 3.5). 24 bytes. */
+typedef struct {
+    uint32_t job;      /* winner, or SJA_NO_JOB (then end_step = dur_ms = score = 0) */
+    uint32_t end_step; /* k: the subjob is steps [p_job, k) of the winner */
+    uint32_t dur_ms;   /* its cumulative duration, <= T_ms */
+    uint32_t granted;  /* 0 until sja_commit; then 1 iff the winner accepted this gap */
+    uint64_t score;    /* policy score of the winner (work for SLA) */
+} sja_award;
+
+/* Device times (CUDA events on the context's stream) accumulated while profiling is on. */
+typedef struct {
+    float scan_ms;      /* segmented prefix scan kernel (profile -> boundary table) */
+    float prep_ms;      /* validation, row counting, row offsets and state initialisation of a load */
+    float advertise_ms; /* gap upload and ordering */
+    float select_ms;    /* feasibility + score + per-gap argmax kernels of sja_select */
+    float commit_ms;    /* commit kernels */
+    uint32_t scan_launches, prep_launches, advertise_launches, select_launches, commit_launches;
+} sja_timing;
+
+/*
+ * Create a context on CUDA device `device`.  `cuda_stream` is a cudaStream_t (as void*)
+ * all work is ordered on; NULL means the legacy default stream.  The stream stays the
+ * caller's.  *out is set only on SJA_OK.
+ */
+sja_status sja_create(sja_ctx** out, int device, void* cuda_stream);
+
+/* Free the context and every device buffer it owns.  NULL is accepted. */
+sja_status sja_destroy(sja_ctx* ctx);
+
+/*
+ * Load J job profiles (ragged CSR) and run the segmented scan (the "on demand"
+ * segmentation of Section 3.9: the envelope may be refined, so the scan is re-runnable;
+ * a new load replaces the previous one and clears any advertised gaps).
+ *   off        u64[J+1], off[0] = 0, non-decreasing; job j owns steps [off[j], off[j+1]).
+ *   dur_ms     u32[N], N = off[J]         per-step duration
+ *   mem_MiB    u32[N]                     per-step memory envelope
+ *   safe_bits  u32[ceil(N/32)]            bit (i % 32) of word (i / 32), LSB first
+ *   ready_ms   u32[J]                     earliest start of each job
+ *   progress   u32[J] or NULL (= all 0)   steps already granted; must be <= len_j
+ *   wait_ms    u32[J] or NULL             needed for SJA_POLICY_FAIRNESS
+ *   prio       u8[J]  or NULL             needed for SJA_POLICY_SLA
+ * For each job the scan computes, at every safe end index k above its progress point, the
+ * cumulative duration, the running maximum of the memory envelope (the window-max test of
+ * Section 3.9), the maximum over the segment since the previous boundary, and the prefix
+ * work sum d*m.  Waits for completion (it returns validation results).
+ */
+sja_status sja_load_profiles(sja_ctx* ctx, uint32_t J, const uint64_t* off,
+                             const uint32_t* dur_ms, const uint32_t* mem_MiB,
+                             const uint32_t* safe_bits, const uint32_t* ready_ms,
+                             const uint32_t* progress, const uint32_t* wait_ms,
+                             const uint8_t* prio, sja_memspace where);
+
+/*
+ * First protocol phase (Section 3.5): make G gaps visible to all jobs.  Replaces the
+ * previous batch.  Gaps are taken as given (overlaps on a slice are not checked).
+ */
+sja_status sja_advertise(sja_ctx* ctx, uint32_t G, const sja_gap* gaps, sja_memspace where);
+
+/*
+ * Second and third phase (Section 3.5): every (gap, job) pair is tested for the longest
+ * feasible subjob, interested jobs are scored under `policy`, one winner per gap is
+ * chosen.  Does not change any job state (no subjob state exists before a grant).
+ * `out` (G awards, in the order the gaps were advertised) may be NULL; the awards are
+ * kept in the context either way.  May be called repeatedly.
+ */
+sja_status sja_select(sja_ctx* ctx, const sja_policy* policy, sja_award* out, sja_memspace where);
+
+/*
+ * Grant (Section 3.5: only the selected job materialises its subjob; Sections 3.1, 3.5:
+ * the parent job later resumes from the end of the fragment).  Resolves jobs that won
+ * several gaps, advances progress and ready time of the granted jobs, refreshes their
+ * running-maximum column.  `n_granted` is a HOST pointer or NULL; when given, the call
+ * waits for completion.  One commit per select.
+ */
+sja_status sja_commit(sja_ctx* ctx, uint32_t* n_granted);
+
+/* Copy the G awards of the last select (with `granted` set if it was committed). */
+sja_status sja_get_awards(sja_ctx* ctx, sja_award* out, sja_memspace where);
+
+/* Copy the per-job state: progress u32[J] and ready_ms u32[J] (either may be NULL). */
+sja_status sja_get_state(sja_ctx* ctx, uint32_t* progress, uint32_t* ready_ms, sja_memspace where);
+
+/* Number of rows of the boundary table built by the last load (sum over jobs). */
+sja_status sja_scan_size(sja_ctx* ctx, uint64_t* n_boundaries);
+
+/*
+ * Copy out the scan result (any pointer may be NULL).  Row r of job j is at
+ * boff[j] + r, r = 0 .. boff[j+1]-boff[j]-1, ascending in k:
+ *   boff u64[J+1]; k u32 safe end index; D u32 cumulative duration of [p, k);
+ *   M u32 max m[p_now..k) from the job's CURRENT progress point (rows below it are stale);
+ *   S u32 max m over the segment since the previous boundary; W u64 sum d*m over [p, k).
+ * D and W count from the progress point given at load.
+ */
+sja_status sja_get_scan(sja_ctx* ctx, uint64_t* boff, uint32_t* k, uint32_t* D, uint32_t* M,
+                        uint32_t* S, uint64_t* W, sja_memspace where);
+
+/* Switch per-kernel CUDA-event timing on (1) or off (0); resets the counters. */
+sja_status sja_profile_enable(sja_ctx* ctx, int on);
+
+/* Wait for the stream and read the accumulated kernel times. */
+sja_status sja_profile_read(sja_ctx* ctx, sja_timing* out);
+
+/* Text of the most recent error on this context ("" if none).  Owned by the context. */
+const char* sja_last_error(const sja_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SJA_H */

@@ -1,0 +1,239 @@
+"""ctypes binding of libsja.so.  Argument marshalling only: every step runs in the library.
+
+Arrays may be numpy arrays (host memory) or torch CUDA tensors (device memory); the
+memory space is inferred per call and all arrays of one call must agree.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+
+from .build import LIB_PATH
+
+SJA_OK = 0
+STATUS_NAMES = {
+    0: "SJA_OK", 1: "SJA_ERR_INVALID_ARG", 2: "SJA_ERR_BAD_PROFILE", 3: "SJA_ERR_OVERFLOW",
+    4: "SJA_ERR_STATE", 5: "SJA_ERR_OOM", 6: "SJA_ERR_CUDA", 7: "SJA_ERR_TIMEOUT",
+}
+MEM_HOST, MEM_DEVICE = 0, 1
+POLICY_EFFICIENCY, POLICY_FAIRNESS, POLICY_SLA = 0, 1, 2
+FLAG_FORCE_SEARCH = 1
+NO_JOB = 0xFFFFFFFF
+
+GAP_DTYPE = np.dtype([("slice", "<u4"), ("start_ms", "<u4"), ("T_ms", "<u4"), ("C_MiB", "<u4")])
+AWARD_DTYPE = np.dtype([("job", "<u4"), ("end_step", "<u4"), ("dur_ms", "<u4"), ("granted", "<u4"),
+                        ("score", "<u8")])
+
+EXPORTS = [
+    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_commit",
+    "sja_get_awards", "sja_get_state", "sja_scan_size", "sja_get_scan", "sja_profile_enable",
+    "sja_profile_read", "sja_last_error",
+]
+
+
+class SjaPolicy(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_uint32), ("flags", ctypes.c_uint32)]
+
+
+class SjaTiming(ctypes.Structure):
+    _fields_ = [("scan_ms", ctypes.c_float), ("prep_ms", ctypes.c_float),
+                ("advertise_ms", ctypes.c_float), ("select_ms", ctypes.c_float),
+                ("commit_ms", ctypes.c_float),
+                ("scan_launches", ctypes.c_uint32), ("prep_launches", ctypes.c_uint32),
+                ("advertise_launches", ctypes.c_uint32), ("select_launches", ctypes.c_uint32),
+                ("commit_launches", ctypes.c_uint32)]
+
+
+class SjaError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """dlopen libsja.so; raises if it has not been built (there is no fallback path)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2509_19086_b200.build` "
+            "(needs nvcc); this package has no CPU fallback")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, u32, i32 = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_int
+    lib.sja_create.argtypes = [ctypes.POINTER(vp), i32, vp]
+    lib.sja_destroy.argtypes = [vp]
+    lib.sja_load_profiles.argtypes = [vp, u32, vp, vp, vp, vp, vp, vp, vp, vp, i32]
+    lib.sja_advertise.argtypes = [vp, u32, vp, i32]
+    lib.sja_select.argtypes = [vp, ctypes.POINTER(SjaPolicy), vp, i32]
+    lib.sja_commit.argtypes = [vp, ctypes.POINTER(u32)]
+    lib.sja_get_awards.argtypes = [vp, vp, i32]
+    lib.sja_get_state.argtypes = [vp, vp, vp, i32]
+    lib.sja_scan_size.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
+    lib.sja_get_scan.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32]
+    lib.sja_profile_enable.argtypes = [vp, i32]
+    lib.sja_profile_read.argtypes = [vp, ctypes.POINTER(SjaTiming)]
+    lib.sja_last_error.argtypes = [vp]
+    lib.sja_last_error.restype = ctypes.c_char_p
+    for name in EXPORTS:
+        if name != "sja_last_error":
+            getattr(lib, name).restype = i32
+    _lib = lib
+    return lib
+
+
+def _is_torch(a) -> bool:
+    return type(a).__module__.startswith("torch")
+
+
+def _ptr_space(a, space: Optional[int], np_dtype=None):
+    """(pointer, memspace, keepalive) of a numpy array or torch tensor."""
+    if a is None:
+        return None, space, None
+    if _is_torch(a):
+        if not a.is_cuda:
+            raise TypeError("torch tensors passed to libsja must live on the CUDA device")
+        if not a.is_contiguous():
+            raise TypeError("tensor must be contiguous")
+        sp = MEM_DEVICE
+        ptr, keep = a.data_ptr(), a
+    else:
+        arr = np.ascontiguousarray(a) if np_dtype is None else np.ascontiguousarray(a, dtype=np_dtype)
+        sp = MEM_HOST
+        ptr, keep = arr.ctypes.data, arr
+    if space is not None and space != sp:
+        raise TypeError("all arrays of one call must be in the same memory space")
+    return ptr, sp, keep
+
+
+class Sja:
+    """One scheduler context on one CUDA device (wraps ``sja_ctx``)."""
+
+    def __init__(self, device: int = 0, stream: Optional[int] = None):
+        self._lib = load_library()
+        self._h = ctypes.c_void_p()
+        st = self._lib.sja_create(ctypes.byref(self._h), int(device), ctypes.c_void_p(stream or 0))
+        if st != SJA_OK:
+            self._h = ctypes.c_void_p()
+            raise SjaError(st, "sja_create failed (is a CUDA device present?)")
+        self.n_jobs = 0
+        self.n_gaps = 0
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h:
+            self._lib.sja_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def _check(self, st: int) -> None:
+        if st != SJA_OK:
+            msg = self._lib.sja_last_error(self._h)
+            raise SjaError(st, msg.decode() if msg else "")
+
+    # -- sja_load_profiles
+    def load_profiles(self, off, dur_ms, mem_MiB, safe_bits, ready_ms, progress=None, wait_ms=None,
+                      prio=None) -> None:
+        n_jobs = int(off.shape[0]) - 1
+        keep = []
+        space = None
+        ptrs = []
+        for a, dt in ((off, np.uint64), (dur_ms, np.uint32), (mem_MiB, np.uint32), (safe_bits, np.uint32),
+                      (ready_ms, np.uint32), (progress, np.uint32), (wait_ms, np.uint32), (prio, np.uint8)):
+            p, space, k = _ptr_space(a, space, dt)
+            ptrs.append(p)
+            keep.append(k)
+        self._check(self._lib.sja_load_profiles(self._h, n_jobs, *ptrs, space))
+        self.n_jobs = n_jobs
+
+    # -- sja_advertise
+    def advertise(self, gaps) -> None:
+        if _is_torch(gaps):
+            p, space, keep = _ptr_space(gaps, None)
+            n = gaps.numel() * gaps.element_size() // GAP_DTYPE.itemsize
+        else:
+            gaps = np.ascontiguousarray(gaps, dtype=GAP_DTYPE)
+            p, space, keep = _ptr_space(gaps, None)
+            n = gaps.shape[0]
+        self._check(self._lib.sja_advertise(self._h, int(n), p, space))
+        self.n_gaps = int(n)
+
+    # -- sja_select
+    def select(self, policy: int, flags: int = 0, out=None):
+        """Run signal + score + select.  ``out``: None (awards stay in the context), the string
+        "host" (returns a numpy AWARD_DTYPE array), or a CUDA uint8 tensor of 24*G bytes."""
+        pol = SjaPolicy(int(policy), int(flags))
+        if out is None:
+            self._check(self._lib.sja_select(self._h, ctypes.byref(pol), None, MEM_HOST))
+            return None
+        if isinstance(out, str):
+            arr = np.empty(self.n_gaps, dtype=AWARD_DTYPE)
+            self._check(self._lib.sja_select(self._h, ctypes.byref(pol), arr.ctypes.data, MEM_HOST))
+            return arr
+        p, space, _ = _ptr_space(out, None)
+        self._check(self._lib.sja_select(self._h, ctypes.byref(pol), p, space))
+        return out
+
+    # -- sja_commit
+    def commit(self, want_count: bool = True) -> Optional[int]:
+        if want_count:
+            n = ctypes.c_uint32()
+            self._check(self._lib.sja_commit(self._h, ctypes.byref(n)))
+            return int(n.value)
+        self._check(self._lib.sja_commit(self._h, None))
+        return None
+
+    # -- sja_get_awards / sja_get_state
+    def get_awards(self) -> np.ndarray:
+        arr = np.empty(self.n_gaps, dtype=AWARD_DTYPE)
+        self._check(self._lib.sja_get_awards(self._h, arr.ctypes.data, MEM_HOST))
+        return arr
+
+    def get_state(self):
+        p = np.empty(self.n_jobs, dtype=np.uint32)
+        r = np.empty(self.n_jobs, dtype=np.uint32)
+        self._check(self._lib.sja_get_state(self._h, p.ctypes.data, r.ctypes.data, MEM_HOST))
+        return p, r
+
+    # -- sja_scan_size / sja_get_scan
+    def scan_size(self) -> int:
+        n = ctypes.c_uint64()
+        self._check(self._lib.sja_scan_size(self._h, ctypes.byref(n)))
+        return int(n.value)
+
+    def get_scan(self):
+        n = self.scan_size()
+        boff = np.empty(self.n_jobs + 1, dtype=np.uint64)
+        k = np.empty(n, np.uint32)
+        D = np.empty(n, np.uint32)
+        M = np.empty(n, np.uint32)
+        S = np.empty(n, np.uint32)
+        W = np.empty(n, np.uint64)
+        self._check(self._lib.sja_get_scan(self._h, boff.ctypes.data, k.ctypes.data, D.ctypes.data,
+                                           M.ctypes.data, S.ctypes.data, W.ctypes.data, MEM_HOST))
+        return dict(boff=boff, k=k, D=D, M=M, S=S, W=W)
+
+    # -- profiling
+    def profile_enable(self, on: bool = True) -> None:
+        self._check(self._lib.sja_profile_enable(self._h, 1 if on else 0))
+
+    def profile_read(self) -> dict:
+        t = SjaTiming()
+        self._check(self._lib.sja_profile_read(self._h, ctypes.byref(t)))
+        return {name: getattr(t, name) for name, _ in SjaTiming._fields_}

@@ -1,0 +1,639 @@
+// libsja: C-ABI entry points and host-side orchestration (see include/sja.h).
+#include "../../include/sja.h"
+
+#include <cuda_runtime.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <utility>
+#include <vector>
+
+#include "sja_common.cuh"
+#include "sja_round.cuh"
+#include "sja_scan.cuh"
+
+using namespace sja;
+
+namespace {
+
+struct DevBuf {
+    void* p = nullptr;
+    size_t cap = 0;
+    template <class T> T* as() const { return static_cast<T*>(p); }
+};
+
+enum ProfCat { CAT_SCAN = 0, CAT_PREP, CAT_ADVERTISE, CAT_SELECT, CAT_COMMIT, CAT_COUNT };
+
+struct ProfSpan { cudaEvent_t a, b; int cat; };
+
+}  // namespace
+
+struct sja_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    char err[320] = {0};
+    bool poisoned = false;
+    int n_sm = 148;
+
+    // profiles / scan
+    bool loaded = false;
+    uint32_t J = 0;
+    uint64_t N = 0, n_rows = 0;
+    bool have_wait = false, have_prio = false;
+    uint32_t load_flags = 0;
+    DevBuf st_off, st_d, st_m, st_s, st_p;            // staging for host inputs / load-time progress
+    DevBuf p, ready, pb, Dp, Wp, wait, prio;          // per-job state and attributes
+    DevBuf nbj, boff, boff_next, A, B, jobwin;        // boundary table
+    DevBuf flags, counter, n_granted;                 // small device words
+    uint32_t* h_words = nullptr;                      // pinned host scratch (8 x u64)
+
+    // gaps / awards
+    bool advertised = false, selected = false, committed = false;
+    uint32_t G = 0, last_policy = 0;
+    DevBuf gaps, awards, widx, partial, winners;
+
+    // profiling
+    bool prof = false;
+    std::vector<ProfSpan> spans;
+    std::vector<cudaEvent_t> free_events;
+    float acc_ms[CAT_COUNT] = {0};
+    uint32_t acc_n[CAT_COUNT] = {0};
+};
+
+namespace {
+
+sja_status fail(sja_ctx* c, sja_status st, const char* fmt, ...) {
+    if (c) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(c->err, sizeof(c->err), fmt, ap);
+        va_end(ap);
+    }
+    return st;
+}
+
+sja_status cuda_fail(sja_ctx* c, cudaError_t e, const char* what) {
+    if (e == cudaErrorMemoryAllocation) {
+        cudaGetLastError();
+        return fail(c, SJA_ERR_OOM, "%s: out of memory", what);
+    }
+    if (c) c->poisoned = true;
+    return fail(c, SJA_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+#define CU(call)                                                        \
+    do {                                                                \
+        cudaError_t e__ = (call);                                       \
+        if (e__ != cudaSuccess) return cuda_fail(c, e__, #call);        \
+    } while (0)
+
+#define TRY(call)                                   \
+    do {                                            \
+        sja_status s__ = (call);                    \
+        if (s__ != SJA_OK) return s__;              \
+    } while (0)
+
+// Makes the context's device current for the duration of a call.
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { prev = -1; cudaGetLastError(); }
+        if (prev != dev) ok = (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() {
+        int cur = -1;
+        if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+    }
+};
+
+sja_status reserve(sja_ctx* c, DevBuf& b, size_t bytes) {
+    if (bytes <= b.cap) return SJA_OK;
+    if (b.p) {
+        CU(cudaStreamSynchronize(c->stream));   // a kernel in flight may still use the old buffer
+        CU(cudaFree(b.p));
+        b.p = nullptr;
+        b.cap = 0;
+    }
+    size_t want = (bytes + 255) & ~(size_t)255;
+    cudaError_t e = cudaMalloc(&b.p, want);
+    if (e != cudaSuccess) { b.p = nullptr; return cuda_fail(c, e, "cudaMalloc"); }
+    b.cap = want;
+    return SJA_OK;
+}
+
+void release(DevBuf& b) {
+    if (b.p) cudaFree(b.p);
+    b.p = nullptr;
+    b.cap = 0;
+}
+
+struct ProfScope {
+    sja_ctx* c;
+    ProfSpan sp;
+    bool on;
+    ProfScope(sja_ctx* ctx, int cat) : c(ctx), on(ctx->prof) {
+        if (!on) return;
+        sp.cat = cat;
+        sp.a = take();
+        sp.b = take();
+        if (!sp.a || !sp.b) { on = false; return; }
+        cudaEventRecord(sp.a, c->stream);
+    }
+    ~ProfScope() {
+        if (!on) return;
+        cudaEventRecord(sp.b, c->stream);
+        c->spans.push_back(sp);
+    }
+    cudaEvent_t take() {
+        if (!c->free_events.empty()) {
+            cudaEvent_t e = c->free_events.back();
+            c->free_events.pop_back();
+            return e;
+        }
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        return e;
+    }
+};
+
+sja_status collect_spans(sja_ctx* c) {
+    if (c->spans.empty()) return SJA_OK;
+    CU(cudaStreamSynchronize(c->stream));
+    for (ProfSpan& s : c->spans) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, s.a, s.b) == cudaSuccess) {
+            c->acc_ms[s.cat] += ms;
+            c->acc_n[s.cat] += 1;
+        } else {
+            cudaGetLastError();
+        }
+        c->free_events.push_back(s.a);
+        c->free_events.push_back(s.b);
+    }
+    c->spans.clear();
+    return SJA_OK;
+}
+
+sja_status check_ctx(sja_ctx* c) {
+    if (!c) return SJA_ERR_INVALID_ARG;
+    if (c->poisoned) return fail(c, SJA_ERR_CUDA, "context unusable after an earlier CUDA error");
+    return SJA_OK;
+}
+
+sja_status copy_in(sja_ctx* c, void* dst, const void* src, size_t bytes, sja_memspace where) {
+    if (bytes == 0) return SJA_OK;
+    CU(cudaMemcpyAsync(dst, src, bytes, where == SJA_MEM_HOST ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice,
+                       c->stream));
+    return SJA_OK;
+}
+
+sja_status copy_out(sja_ctx* c, void* dst, const void* src, size_t bytes, sja_memspace where) {
+    if (bytes == 0) return SJA_OK;
+    CU(cudaMemcpyAsync(dst, src, bytes, where == SJA_MEM_HOST ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice,
+                       c->stream));
+    return SJA_OK;
+}
+
+// Read the device flag word (waits for the stream).
+sja_status read_flags(sja_ctx* c, uint32_t* out) {
+    CU(cudaMemcpyAsync(c->h_words, c->flags.p, 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaStreamSynchronize(c->stream));
+    *out = c->h_words[0];
+    return SJA_OK;
+}
+
+JobView job_view(const sja_ctx* c) {
+    JobView v;
+    v.boff = c->boff.as<uint64_t>();
+    v.pb = c->pb.as<uint32_t>();
+    v.Dp = c->Dp.as<uint32_t>();
+    v.Wp = c->Wp.as<uint64_t>();
+    v.ready = c->ready.as<uint32_t>();
+    v.wait = c->have_wait ? c->wait.as<uint32_t>() : nullptr;
+    v.prio = c->have_prio ? c->prio.as<uint8_t>() : nullptr;
+    v.A = c->A.as<uint4>();
+    v.B = c->B.as<uint2>();
+    v.J = c->J;
+    return v;
+}
+
+// De-interleave the boundary table for sja_get_scan.
+__global__ void export_rows_kernel(const uint4* __restrict__ A, const uint2* __restrict__ B, uint64_t n,
+                                   uint32_t* k, uint32_t* D, uint32_t* M, uint32_t* S, uint64_t* W) {
+    const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const uint4 a = A[i];
+    const uint2 b = B[i];
+    if (k) k[i] = b.x;
+    if (D) D[i] = a.x;
+    if (M) M[i] = a.y;
+    if (S) S[i] = b.y;
+    if (W) W[i] = pack64(a.z, a.w);
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+// =======================================================================================
+extern "C" {
+
+sja_status sja_create(sja_ctx** out, int device, void* cuda_stream) {
+    if (!out) return SJA_ERR_INVALID_ARG;
+    *out = nullptr;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess) { cudaGetLastError(); return SJA_ERR_CUDA; }
+    if (device < 0 || device >= n_dev) return SJA_ERR_INVALID_ARG;
+    sja_ctx* c = new (std::nothrow) sja_ctx();
+    if (!c) return SJA_ERR_OOM;
+    c->device = device;
+    c->stream = static_cast<cudaStream_t>(cuda_stream);
+    DeviceGuard guard(device);
+    sja_status st = SJA_OK;
+    do {
+        if (!guard.ok) { st = SJA_ERR_CUDA; break; }
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
+        c->n_sm = prop.multiProcessorCount;
+        if (cudaMallocHost(reinterpret_cast<void**>(&c->h_words), 64) != cudaSuccess) { st = SJA_ERR_OOM; break; }
+        if ((st = reserve(c, c->flags, 4)) != SJA_OK) break;
+        if ((st = reserve(c, c->counter, 4)) != SJA_OK) break;
+        if ((st = reserve(c, c->n_granted, 4)) != SJA_OK) break;
+        if (cudaMemsetAsync(c->flags.p, 0, 4, c->stream) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
+        if (cudaFuncSetAttribute(scan_profiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 SCAN_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
+    } while (0);
+    if (st != SJA_OK) {
+        cudaGetLastError();
+        sja_destroy(c);
+        return st;
+    }
+    *out = c;
+    return SJA_OK;
+}
+
+sja_status sja_destroy(sja_ctx* c) {
+    if (!c) return SJA_OK;
+    DeviceGuard guard(c->device);
+    cudaStreamSynchronize(c->stream);
+    DevBuf* bufs[] = {&c->st_off, &c->st_d, &c->st_m, &c->st_s, &c->st_p, &c->p, &c->ready, &c->pb, &c->Dp,
+                      &c->Wp, &c->wait, &c->prio, &c->nbj, &c->boff, &c->boff_next, &c->A, &c->B, &c->jobwin,
+                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->awards, &c->widx, &c->partial,
+                      &c->winners};
+    for (DevBuf* b : bufs) release(*b);
+    for (ProfSpan& s : c->spans) { cudaEventDestroy(s.a); cudaEventDestroy(s.b); }
+    for (cudaEvent_t e : c->free_events) cudaEventDestroy(e);
+    if (c->h_words) cudaFreeHost(c->h_words);
+    cudaGetLastError();
+    delete c;
+    return SJA_OK;
+}
+
+const char* sja_last_error(const sja_ctx* c) { return c ? c->err : ""; }
+
+sja_status sja_profile_enable(sja_ctx* c, int on) {
+    TRY(check_ctx(c));
+    DeviceGuard guard(c->device);
+    TRY(collect_spans(c));
+    for (int i = 0; i < CAT_COUNT; ++i) { c->acc_ms[i] = 0.f; c->acc_n[i] = 0; }
+    c->prof = on != 0;
+    return SJA_OK;
+}
+
+sja_status sja_profile_read(sja_ctx* c, sja_timing* out) {
+    TRY(check_ctx(c));
+    if (!out) return fail(c, SJA_ERR_INVALID_ARG, "sja_profile_read: out is NULL");
+    DeviceGuard guard(c->device);
+    TRY(collect_spans(c));
+    out->scan_ms = c->acc_ms[CAT_SCAN];
+    out->prep_ms = c->acc_ms[CAT_PREP];
+    out->advertise_ms = c->acc_ms[CAT_ADVERTISE];
+    out->select_ms = c->acc_ms[CAT_SELECT];
+    out->commit_ms = c->acc_ms[CAT_COMMIT];
+    out->scan_launches = c->acc_n[CAT_SCAN];
+    out->prep_launches = c->acc_n[CAT_PREP];
+    out->advertise_launches = c->acc_n[CAT_ADVERTISE];
+    out->select_launches = c->acc_n[CAT_SELECT];
+    out->commit_launches = c->acc_n[CAT_COMMIT];
+    return SJA_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const uint32_t* dur_ms,
+                             const uint32_t* mem_MiB, const uint32_t* safe_bits, const uint32_t* ready_ms,
+                             const uint32_t* progress, const uint32_t* wait_ms, const uint8_t* prio,
+                             sja_memspace where) {
+    TRY(check_ctx(c));
+    if (J == 0 || J == 0xFFFFFFFFu) return fail(c, SJA_ERR_INVALID_ARG, "sja_load_profiles: J out of range");
+    if (!off || !ready_ms) return fail(c, SJA_ERR_INVALID_ARG, "sja_load_profiles: off / ready_ms is NULL");
+    if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_load_profiles: bad memspace");
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
+
+    // N = off[J]
+    uint64_t N = 0;
+    if (where == SJA_MEM_HOST) {
+        if (off[0] != 0) return fail(c, SJA_ERR_BAD_PROFILE, "off[0] != 0");
+        N = off[J];
+    } else {
+        CU(cudaMemcpyAsync(c->h_words, off + J, 8, cudaMemcpyDeviceToHost, c->stream));
+        CU(cudaStreamSynchronize(c->stream));
+        memcpy(&N, c->h_words, 8);
+    }
+    if (N >= (1ull << 40)) return fail(c, SJA_ERR_BAD_PROFILE, "off[J] = %llu is implausible", (unsigned long long)N);
+    if (N > 0 && (!dur_ms || !mem_MiB || !safe_bits))
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_load_profiles: profile array is NULL");
+    const uint64_t n_words = (N + 31) / 32;
+
+    const uint64_t* d_off = off;
+    const uint32_t *d_d = dur_ms, *d_m = mem_MiB, *d_s = safe_bits;
+    if (where == SJA_MEM_HOST) {
+        TRY(reserve(c, c->st_off, (size_t)(J + 1) * 8));
+        TRY(reserve(c, c->st_d, (size_t)N * 4 + 16));
+        TRY(reserve(c, c->st_m, (size_t)N * 4 + 16));
+        TRY(reserve(c, c->st_s, (size_t)n_words * 4 + 16));
+        TRY(copy_in(c, c->st_off.p, off, (size_t)(J + 1) * 8, where));
+        TRY(copy_in(c, c->st_d.p, dur_ms, (size_t)N * 4, where));
+        TRY(copy_in(c, c->st_m.p, mem_MiB, (size_t)N * 4, where));
+        TRY(copy_in(c, c->st_s.p, safe_bits, (size_t)n_words * 4, where));
+        d_off = c->st_off.as<uint64_t>();
+        d_d = c->st_d.as<uint32_t>();
+        d_m = c->st_m.as<uint32_t>();
+        d_s = c->st_s.as<uint32_t>();
+    } else if (N > 0 && (!aligned16(dur_ms) || !aligned16(mem_MiB) || !aligned16(safe_bits))) {
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_load_profiles: device profile arrays must be 16-byte aligned");
+    }
+    TRY(reserve(c, c->st_p, (size_t)J * 4));
+    TRY(reserve(c, c->nbj, (size_t)J * 4));
+    TRY(reserve(c, c->boff_next, (size_t)(J + 1) * 8));
+    if (progress) TRY(copy_in(c, c->st_p.p, progress, (size_t)J * 4, where));
+    else CU(cudaMemsetAsync(c->st_p.p, 0, (size_t)J * 4, c->stream));
+
+    // pass 0: validate + count rows, then row offsets; nothing of the loaded state is touched yet
+    CU(cudaMemsetAsync(c->flags.p, 0, 4, c->stream));
+    {
+        ProfScope ps(c, CAT_PREP);
+        const uint32_t blocks = (uint32_t)std::min<uint64_t>(((uint64_t)J * 32 + 255) / 256, (uint64_t)c->n_sm * 32);
+        count_boundaries_kernel<<<blocks, 256, 0, c->stream>>>(d_off, d_s, c->st_p.as<uint32_t>(), J, N,
+                                                               c->nbj.as<uint32_t>(), c->flags.as<uint32_t>());
+        row_offsets_kernel<<<1, 1024, 0, c->stream>>>(c->nbj.as<uint32_t>(), J, c->boff_next.as<uint64_t>());
+    }
+    CU(cudaGetLastError());
+    CU(cudaMemcpyAsync(c->h_words, c->flags.p, 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaMemcpyAsync(c->h_words + 2, c->boff_next.as<uint64_t>() + J, 8, cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaStreamSynchronize(c->stream));
+    if (c->h_words[0] & FLAG_BAD_PROFILE)
+        return fail(c, SJA_ERR_BAD_PROFILE, "profile CSR invalid (offsets not monotone, job too long, or progress > len)");
+    uint64_t n_rows = 0;
+    memcpy(&n_rows, c->h_words + 2, 8);
+
+    // from here on the previous load is replaced
+    c->loaded = false;
+    c->advertised = c->selected = c->committed = false;
+    TRY(reserve(c, c->A, (size_t)n_rows * 16 + 16));
+    TRY(reserve(c, c->B, (size_t)n_rows * 8 + 16));
+    TRY(reserve(c, c->p, (size_t)J * 4));
+    TRY(reserve(c, c->ready, (size_t)J * 4));
+    TRY(reserve(c, c->pb, (size_t)J * 4));
+    TRY(reserve(c, c->Dp, (size_t)J * 4));
+    TRY(reserve(c, c->Wp, (size_t)J * 8));
+    TRY(reserve(c, c->jobwin, (size_t)J * 8));
+    if (wait_ms) TRY(reserve(c, c->wait, (size_t)J * 4));
+    if (prio) TRY(reserve(c, c->prio, (size_t)J));
+    std::swap(c->boff, c->boff_next);
+    {
+        ProfScope ps(c, CAT_PREP);
+        CU(cudaMemcpyAsync(c->p.p, c->st_p.p, (size_t)J * 4, cudaMemcpyDeviceToDevice, c->stream));
+        TRY(copy_in(c, c->ready.p, ready_ms, (size_t)J * 4, where));
+        if (wait_ms) TRY(copy_in(c, c->wait.p, wait_ms, (size_t)J * 4, where));
+        if (prio) TRY(copy_in(c, c->prio.p, prio, (size_t)J, where));
+        CU(cudaMemsetAsync(c->pb.p, 0, (size_t)J * 4, c->stream));
+        CU(cudaMemsetAsync(c->Dp.p, 0, (size_t)J * 4, c->stream));
+        CU(cudaMemsetAsync(c->Wp.p, 0, (size_t)J * 8, c->stream));
+        CU(cudaMemsetAsync(c->jobwin.p, 0, (size_t)J * 8, c->stream));
+        CU(cudaMemsetAsync(c->counter.p, 0, 4, c->stream));
+    }
+    c->J = J;
+    c->N = N;
+    c->n_rows = n_rows;
+    c->have_wait = wait_ms != nullptr;
+    c->have_prio = prio != nullptr;
+
+    ScanArgs a;
+    a.off = d_off; a.d = d_d; a.m = d_m; a.sbits = d_s;
+    a.p0 = c->st_p.as<uint32_t>();
+    a.wait = c->have_wait ? c->wait.as<uint32_t>() : nullptr;
+    a.prio = c->have_prio ? c->prio.as<uint8_t>() : nullptr;
+    a.boff = c->boff.as<uint64_t>();
+    a.A = c->A.as<uint4>();
+    a.B = c->B.as<uint2>();
+    a.N = N; a.J = J;
+    a.counter = c->counter.as<uint32_t>();
+    a.flags = c->flags.as<uint32_t>();
+    if (N > 0) {
+        ProfScope ps(c, CAT_SCAN);
+        const uint32_t ctas_per_sm = 2;
+        const uint32_t want = (J + SCAN_WARPS - 1) / SCAN_WARPS;
+        const uint32_t grid = std::min<uint32_t>(want, (uint32_t)c->n_sm * ctas_per_sm);
+        scan_profiles_kernel<<<grid, SCAN_WARPS * 32, SCAN_SMEM_BYTES, c->stream>>>(a);
+    }
+    CU(cudaGetLastError());
+    uint32_t flags = 0;
+    TRY(read_flags(c, &flags));
+    if (flags & FLAG_INTERNAL) return fail(c, SJA_ERR_CUDA, "scan self-check failed (row count mismatch)");
+    if (flags & FLAG_OVF_DURATION) return fail(c, SJA_ERR_OVERFLOW, "a job's total duration does not fit in 32 bits");
+    if (flags & FLAG_OVF_WORK) return fail(c, SJA_ERR_OVERFLOW, "a job's total work is >= 2^63");
+    c->load_flags = flags;
+    c->loaded = true;
+    return SJA_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+sja_status sja_advertise(sja_ctx* c, uint32_t G, const sja_gap* gaps, sja_memspace where) {
+    TRY(check_ctx(c));
+    if (G == 0 || !gaps) return fail(c, SJA_ERR_INVALID_ARG, "sja_advertise: no gaps");
+    if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_advertise: bad memspace");
+    if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_advertise before sja_load_profiles");
+    DeviceGuard guard(c->device);
+    TRY(reserve(c, c->gaps, (size_t)G * sizeof(sja_gap)));
+    TRY(reserve(c, c->awards, (size_t)G * sizeof(sja_award)));
+    TRY(reserve(c, c->widx, (size_t)G * 4));
+    TRY(reserve(c, c->winners, (size_t)G * 4));
+    {
+        ProfScope ps(c, CAT_ADVERTISE);
+        TRY(copy_in(c, c->gaps.p, gaps, (size_t)G * sizeof(sja_gap), where));
+    }
+    if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));   // caller may reuse its buffer
+    c->G = G;
+    c->advertised = true;
+    c->selected = c->committed = false;
+    return SJA_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+sja_status sja_select(sja_ctx* c, const sja_policy* policy, sja_award* out, sja_memspace where) {
+    TRY(check_ctx(c));
+    if (!policy) return fail(c, SJA_ERR_INVALID_ARG, "sja_select: policy is NULL");
+    if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_select: bad memspace");
+    const uint32_t kind = policy->kind;
+    if (kind > SJA_POLICY_SLA) return fail(c, SJA_ERR_INVALID_ARG, "sja_select: unknown policy %u", kind);
+    if (!c->loaded || !c->advertised) return fail(c, SJA_ERR_STATE, "sja_select before load / advertise");
+    if (kind == SJA_POLICY_FAIRNESS && !c->have_wait)
+        return fail(c, SJA_ERR_INVALID_ARG, "fairness policy needs wait_ms at load");
+    if (kind == SJA_POLICY_SLA && !c->have_prio) return fail(c, SJA_ERR_INVALID_ARG, "SLA policy needs prio at load");
+    if (kind == SJA_POLICY_FAIRNESS && (c->load_flags & FLAG_OVF_FAIR))
+        return fail(c, SJA_ERR_OVERFLOW, "fairness score may reach 2^63 for some job");
+    if (kind == SJA_POLICY_SLA && (c->load_flags & FLAG_OVF_SLA))
+        return fail(c, SJA_ERR_OVERFLOW, "SLA key needs work < 2^55 for every job");
+    DeviceGuard guard(c->device);
+
+    const uint32_t G = c->G, J = c->J;
+    const uint32_t n_chunks = (J + SEARCH_THREADS - 1) / SEARCH_THREADS;
+    TRY(reserve(c, c->partial, (size_t)n_chunks * G * sizeof(Partial)));
+    // split the gaps so that the grid covers the SMs a few times over
+    uint32_t splits = (uint32_t)((4ull * c->n_sm + n_chunks - 1) / n_chunks);
+    const uint32_t max_splits = (G + SEARCH_GT - 1) / SEARCH_GT;
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    uint32_t per_split = (G + splits - 1) / splits;
+    per_split = ((per_split + SEARCH_GT - 1) / SEARCH_GT) * SEARCH_GT;
+    splits = (G + per_split - 1) / per_split;
+    {
+        ProfScope ps(c, CAT_SELECT);
+        const JobView jv = job_view(c);
+        select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, 0, c->stream>>>(
+            jv, c->gaps.as<Gap>(), G, per_split, kind, nullptr, 0, c->partial.as<Partial>());
+        finalize_awards_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(jv, c->partial.as<Partial>(), n_chunks, G,
+                                                                         kind, c->awards.as<Award>(),
+                                                                         c->widx.as<uint32_t>());
+    }
+    CU(cudaGetLastError());
+    c->selected = true;
+    c->committed = false;
+    c->last_policy = kind;
+    if (out) {
+        TRY(copy_out(c, out, c->awards.p, (size_t)G * sizeof(sja_award), where));
+        if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));
+    }
+    return SJA_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+sja_status sja_commit(sja_ctx* c, uint32_t* n_granted) {
+    TRY(check_ctx(c));
+    if (!c->selected) return fail(c, SJA_ERR_STATE, "sja_commit without a preceding sja_select");
+    if (c->committed) return fail(c, SJA_ERR_STATE, "sja_commit called twice for one select");
+    DeviceGuard guard(c->device);
+    const uint32_t G = c->G;
+    {
+        ProfScope ps(c, CAT_COMMIT);
+        const uint32_t gb = (G + 255) / 256;
+        commit_vote_kernel<<<gb, 256, 0, c->stream>>>(c->awards.as<Award>(), G,
+                                                      c->jobwin.as<unsigned long long>(),
+                                                      c->n_granted.as<uint32_t>());
+        commit_apply_kernel<<<gb, 256, 0, c->stream>>>(
+            c->awards.as<Award>(), c->gaps.as<Gap>(), c->widx.as<uint32_t>(), G,
+            c->jobwin.as<unsigned long long>(), c->boff.as<uint64_t>(), c->A.as<uint4>(), c->p.as<uint32_t>(),
+            c->ready.as<uint32_t>(), c->pb.as<uint32_t>(), c->Dp.as<uint32_t>(), c->Wp.as<uint64_t>(),
+            c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(), c->flags.as<uint32_t>());
+        commit_refresh_kernel<<<(G * 32 + 255) / 256, 256, 0, c->stream>>>(
+            c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(), G, c->boff.as<uint64_t>(),
+            c->pb.as<uint32_t>(), c->A.as<uint4>(), c->B.as<uint2>(), c->jobwin.as<unsigned long long>());
+    }
+    CU(cudaGetLastError());
+    c->committed = true;
+    c->selected = false;
+    c->advertised = false;   // the granted gaps are used up; advertise the next batch
+    if (n_granted) {
+        CU(cudaMemcpyAsync(c->h_words, c->n_granted.p, 4, cudaMemcpyDeviceToHost, c->stream));
+        CU(cudaMemcpyAsync(c->h_words + 1, c->flags.p, 4, cudaMemcpyDeviceToHost, c->stream));
+        CU(cudaStreamSynchronize(c->stream));
+        *n_granted = c->h_words[0];
+        if (c->h_words[1] & FLAG_OVF_READY) {
+            CU(cudaMemsetAsync(c->flags.p, 0, 4, c->stream));
+            return fail(c, SJA_ERR_OVERFLOW, "start + dur does not fit in 32 bits for a granted job (ready time saturated)");
+        }
+    }
+    return SJA_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+sja_status sja_get_awards(sja_ctx* c, sja_award* out, sja_memspace where) {
+    TRY(check_ctx(c));
+    if (!out) return fail(c, SJA_ERR_INVALID_ARG, "sja_get_awards: out is NULL");
+    if (!c->selected && !c->committed) return fail(c, SJA_ERR_STATE, "sja_get_awards before sja_select");
+    DeviceGuard guard(c->device);
+    TRY(copy_out(c, out, c->awards.p, (size_t)c->G * sizeof(sja_award), where));
+    if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));
+    return SJA_OK;
+}
+
+sja_status sja_get_state(sja_ctx* c, uint32_t* progress, uint32_t* ready_ms, sja_memspace where) {
+    TRY(check_ctx(c));
+    if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_get_state before sja_load_profiles");
+    DeviceGuard guard(c->device);
+    if (progress) TRY(copy_out(c, progress, c->p.p, (size_t)c->J * 4, where));
+    if (ready_ms) TRY(copy_out(c, ready_ms, c->ready.p, (size_t)c->J * 4, where));
+    if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));
+    return SJA_OK;
+}
+
+sja_status sja_scan_size(sja_ctx* c, uint64_t* n_boundaries) {
+    TRY(check_ctx(c));
+    if (!n_boundaries) return fail(c, SJA_ERR_INVALID_ARG, "sja_scan_size: out is NULL");
+    if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_scan_size before sja_load_profiles");
+    *n_boundaries = c->n_rows;
+    return SJA_OK;
+}
+
+sja_status sja_get_scan(sja_ctx* c, uint64_t* boff, uint32_t* k, uint32_t* D, uint32_t* M, uint32_t* S,
+                        uint64_t* W, sja_memspace where) {
+    TRY(check_ctx(c));
+    if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_get_scan before sja_load_profiles");
+    DeviceGuard guard(c->device);
+    const uint64_t n = c->n_rows;
+    if (boff) TRY(copy_out(c, boff, c->boff.p, (size_t)(c->J + 1) * 8, where));
+    if (n == 0) {
+        if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));
+        return SJA_OK;
+    }
+    uint32_t *dk = k, *dD = D, *dM = M, *dS = S;
+    uint64_t* dW = W;
+    DevBuf tmp[5];
+    sja_status st = SJA_OK;
+    if (where == SJA_MEM_HOST) {
+        void** outs[5] = {(void**)&dk, (void**)&dD, (void**)&dM, (void**)&dS, (void**)&dW};
+        const void* hosts[5] = {k, D, M, S, W};
+        const size_t esz[5] = {4, 4, 4, 4, 8};
+        for (int i = 0; i < 5 && st == SJA_OK; ++i) {
+            if (!hosts[i]) continue;
+            st = reserve(c, tmp[i], (size_t)n * esz[i]);
+            *outs[i] = tmp[i].p;
+        }
+    }
+    if (st == SJA_OK) {
+        const uint64_t blocks = (n + 255) / 256;
+        export_rows_kernel<<<(uint32_t)blocks, 256, 0, c->stream>>>(c->A.as<uint4>(), c->B.as<uint2>(), n, dk, dD,
+                                                                    dM, dS, dW);
+        if (cudaGetLastError() != cudaSuccess) st = fail(c, SJA_ERR_CUDA, "export_rows_kernel launch failed");
+    }
+    if (st == SJA_OK && where == SJA_MEM_HOST) {
+        void* hosts[5] = {k, D, M, S, W};
+        const size_t esz[5] = {4, 4, 4, 4, 8};
+        for (int i = 0; i < 5; ++i)
+            if (hosts[i]) cudaMemcpyAsync(hosts[i], tmp[i].p, (size_t)n * esz[i], cudaMemcpyDeviceToHost, c->stream);
+    }
+    cudaError_t e = cudaStreamSynchronize(c->stream);
+    for (DevBuf& b : tmp) release(b);
+    if (st == SJA_OK && e != cudaSuccess) return cuda_fail(c, e, "sja_get_scan");
+    return st;
+}
+
+}  // extern "C"

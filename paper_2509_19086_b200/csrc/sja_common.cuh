@@ -1,0 +1,55 @@
+// Shared device-side definitions of libsja (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sja {
+
+// Device error / status bits (one u32 word per context, set with atomicOr, read by the host).
+enum : uint32_t {
+    FLAG_BAD_PROFILE = 1u << 0,   // CSR offsets / progress invalid
+    FLAG_OVF_DURATION = 1u << 1,  // a job's total duration does not fit in 32 bits
+    FLAG_OVF_WORK = 1u << 2,      // a job's total work >= 2^63
+    FLAG_OVF_FAIR = 1u << 3,      // total work * (1 + wait/1000) >= 2^63 for some job
+    FLAG_OVF_SLA = 1u << 4,       // total work >= 2^55 for some job (SLA key packing)
+    FLAG_OVF_READY = 1u << 5,     // start + dur >= 2^32 at commit
+    FLAG_INTERNAL = 1u << 6,      // self-check failed (boundary count mismatch)
+};
+
+constexpr uint32_t SJA_NO_JOB_DEV = 0xFFFFFFFFu;
+
+// One row of the boundary table, "search" half: everything a feasibility probe reads.
+// D = cumulative duration of [p_load, k), M = max m over [p_now, k), W = sum d*m over [p_load, k).
+// Stored as uint4 {D, M, W_lo, W_hi}.
+// "Aux" half, uint2 {k, S}: k = safe end index (steps from the job's first step),
+// S = max m over the segment since the previous boundary.
+
+__device__ __forceinline__ uint64_t pack64(uint32_t lo, uint32_t hi) {
+    return (uint64_t)lo | ((uint64_t)hi << 32);
+}
+
+// Warp-wide maximum of a u64 (all lanes get the result).
+__device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {
+    uint32_t hi = (uint32_t)(v >> 32), lo = (uint32_t)v;
+    uint32_t mhi = __reduce_max_sync(0xFFFFFFFFu, hi);
+    uint32_t mlo = __reduce_max_sync(0xFFFFFFFFu, hi == mhi ? lo : 0u);
+    return pack64(mlo, mhi);
+}
+
+constexpr uint64_t KEY_SLA_SHIFT = 55;  // SLA key = 1 + (prio << 55) + work, work < 2^55
+
+// Policy key of an interested job: 0 is reserved for "no candidate".
+// kind 0 efficiency, 1 fairness (factor = 1 + wait/1000), 2 SLA (factor = prio).
+__device__ __forceinline__ uint64_t policy_key(uint32_t kind, uint64_t work, uint32_t factor) {
+    if (kind == 1) return work * (uint64_t)factor + 1ull;
+    if (kind == 2) return ((uint64_t)factor << KEY_SLA_SHIFT) + work + 1ull;
+    return work + 1ull;
+}
+
+__device__ __forceinline__ uint64_t key_to_score(uint32_t kind, uint64_t key) {
+    uint64_t v = key - 1ull;
+    if (kind == 2) v &= (1ull << KEY_SLA_SHIFT) - 1ull;
+    return v;
+}
+
+}  // namespace sja

@@ -1,0 +1,346 @@
+// Segmented prefix scan: raw per-step profiles -> per-job boundary table.
+//
+// The window-max admissibility test (Sections 3.8 / 3.9) and the window-length bound
+// (Section 3.1) only ever need to be evaluated at safe boundaries (Section 3.7), because a
+// subjob may end nowhere else.  The scan therefore streams every step once (8 B + 1 bit)
+// and writes one 24-byte row per safe boundary.
+//
+// Work split: one warp streams one job (jobs are handed out by an atomic counter, so no
+// warp ever waits on another).  A warp moves 512 steps per iteration: coalesced 16-byte
+// cp.async copies into a per-warp shared-memory ring (XOR-swizzled at 16-byte granularity),
+// then each lane reads its 16 CONSECUTIVE steps back with conflict-free 128-bit shared
+// loads, reduces them locally, the warp combines the 32 lane aggregates with shuffles, and
+// each lane re-walks its 16 steps to emit rows at its safe bits.
+#pragma once
+#include "sja_common.cuh"
+
+namespace sja {
+
+constexpr int SCAN_BLK = 512;     // steps per warp iteration (16 per lane)
+constexpr int SCAN_STAGES = 3;    // cp.async ring depth per warp
+constexpr int SCAN_WARPS = 8;     // warps per CTA
+constexpr int SCAN_STAGE_BYTES = 2048 + 2048 + 64;  // d, m, 16 safe words
+constexpr int SCAN_SMEM_BYTES = SCAN_WARPS * SCAN_STAGES * SCAN_STAGE_BYTES;
+
+struct ScanArgs {
+    const uint64_t* off;     // [J+1]
+    const uint32_t* d;       // [N]
+    const uint32_t* m;       // [N]
+    const uint32_t* sbits;   // [ceil(N/32)]
+    const uint32_t* p0;      // [J] progress at load
+    const uint32_t* wait;    // [J] or nullptr
+    const uint8_t* prio;     // [J] or nullptr
+    const uint64_t* boff;    // [J+1] row offsets
+    uint4* A;                // rows {D, M, W_lo, W_hi}
+    uint2* B;                // rows {k, S}
+    uint64_t N;
+    uint32_t J;
+    uint32_t* counter;       // job hand-out counter (zeroed before launch)
+    uint32_t* flags;
+};
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+
+// 16-byte chunk c of a 2 KB stage array lives at chunk slot swz(c): lane L reading chunks
+// 4L..4L+3 and lane L writing chunks 32r+L both hit 8 distinct bank groups per quarter-warp.
+__device__ __forceinline__ uint32_t swz(uint32_t c) { return c ^ ((c >> 3) & 3u); }
+
+// ---------------------------------------------------------------------------------------
+// Pass 0: validate the CSR and count the boundary rows of every job (popcount of its safe
+// bits above the progress point; the end of a job always counts).  One warp per job.
+__global__ void __launch_bounds__(256) count_boundaries_kernel(
+    const uint64_t* __restrict__ off, const uint32_t* __restrict__ sbits,
+    const uint32_t* __restrict__ p0, uint32_t J, uint64_t N, uint32_t* __restrict__ nbj,
+    uint32_t* __restrict__ flags) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t warps = (gridDim.x * blockDim.x) >> 5;
+    for (uint32_t j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; j < J; j += warps) {
+        const uint64_t js = off[j], je = off[j + 1];
+        const uint32_t p = p0[j];
+        bool bad = (je < js) || (je > N) || (je - js > 0xFFFFFFFFull) || ((uint64_t)p > je - js);
+        if (j == 0 && js != 0) bad = true;
+        if (bad) {
+            if (lane == 0) atomicOr(flags, FLAG_BAD_PROFILE);
+            if (lane == 0) nbj[j] = 0;
+            continue;
+        }
+        const uint64_t s = js + p, e = je;
+        uint32_t cnt = 0;
+        if (s < e) {
+            const uint64_t w0 = s >> 5, w1 = (e - 1) >> 5;
+            for (uint64_t w = w0 + lane; w <= w1; w += 32) {
+                uint32_t x = __ldg(sbits + w);
+                if (w == w0) x &= 0xFFFFFFFFu << (uint32_t)(s & 31);
+                if (w == w1) x &= 0xFFFFFFFFu >> (31u - (uint32_t)((e - 1) & 31));
+                cnt += __popc(x);
+            }
+            cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+            const uint32_t lastbit = (__ldg(sbits + w1) >> (uint32_t)((e - 1) & 31)) & 1u;
+            cnt += 1u - lastbit;
+        }
+        if (lane == 0) nbj[j] = cnt;
+    }
+}
+
+// Exclusive prefix sum of the per-job row counts -> boff[J+1] (u64).  One CTA of 1024
+// threads walks the array in tiles of 8192 with a running carry.
+__global__ void __launch_bounds__(1024) row_offsets_kernel(const uint32_t* __restrict__ nbj,
+                                                           uint32_t J,
+                                                           uint64_t* __restrict__ boff) {
+    __shared__ uint64_t warp_sums[32];
+    __shared__ uint64_t warp_excl[32];
+    __shared__ uint64_t tile_total;
+    const uint32_t t = threadIdx.x, lane = t & 31u, wid = t >> 5;
+    uint64_t carry = 0;  // same value in every thread
+    for (uint64_t base = 0; base < J; base += 8192) {
+        uint32_t v[8];
+        uint64_t local = 0;
+        const uint64_t i0 = base + (uint64_t)t * 8;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            v[i] = (i0 + i < J) ? nbj[i0 + i] : 0u;
+            local += v[i];
+        }
+        uint64_t inc = local;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint64_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= (uint32_t)o) inc += y;
+        }
+        if (lane == 31) warp_sums[wid] = inc;
+        __syncthreads();
+        if (wid == 0) {
+            const uint64_t ws = warp_sums[lane];
+            uint64_t wi = ws;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint64_t y = __shfl_up_sync(0xFFFFFFFFu, wi, o);
+                if (lane >= (uint32_t)o) wi += y;
+            }
+            warp_excl[lane] = wi - ws;
+            if (lane == 31) tile_total = wi;
+        }
+        __syncthreads();
+        uint64_t run = carry + warp_excl[wid] + (inc - local);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (i0 + i < J) boff[i0 + i] = run;
+            run += v[i];
+        }
+        carry += tile_total;
+        __syncthreads();  // warp_sums / tile_total are rewritten by the next tile
+    }
+    if (t == 0) boff[J] = carry;
+}
+
+// ---------------------------------------------------------------------------------------
+// The scan proper.
+__global__ void __launch_bounds__(SCAN_WARPS * 32) scan_profiles_kernel(ScanArgs a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t wid = threadIdx.x >> 5;
+    unsigned char* wbase = smem_raw + (size_t)wid * SCAN_STAGES * SCAN_STAGE_BYTES;
+    const uint32_t wbase_s = (uint32_t)__cvta_generic_to_shared(wbase);
+
+    for (;;) {
+        uint32_t j = 0;
+        if (lane == 0) j = atomicAdd(a.counter, 1u);
+        j = __shfl_sync(0xFFFFFFFFu, j, 0);
+        if (j >= a.J) break;
+
+        const uint64_t js = __ldg(a.off + j), je = __ldg(a.off + j + 1);
+        const uint32_t p = __ldg(a.p0 + j);
+        const uint64_t s = js + p, e = je;
+        if (s >= e) continue;
+        const uint64_t blk0 = s & ~31ull;
+        const uint64_t nblk = (e - blk0 + (SCAN_BLK - 1)) / SCAN_BLK;
+        const uint64_t out_base = __ldg(a.boff + j);
+        const uint64_t out_end = __ldg(a.boff + j + 1);   // rows are never written past this
+
+        // issue the async copies of block t into ring slot t % STAGES
+        auto issue = [&](uint64_t t) {
+            if (t < nblk) {
+                const uint64_t bs = blk0 + t * SCAN_BLK;
+                const uint32_t st = wbase_s + (uint32_t)(t % SCAN_STAGES) * SCAN_STAGE_BYTES;
+#pragma unroll
+                for (uint32_t r = 0; r < 4; ++r) {
+                    const uint32_t c = r * 32u + lane;
+                    const uint64_t step = bs + 4ull * c;
+                    uint32_t bytes = 0;
+                    if (step + 4 > s && step < e) {
+                        const uint64_t left = (a.N - step) * 4ull;
+                        bytes = left < 16 ? (uint32_t)left : 16u;
+                    }
+                    const uint64_t src = bytes ? step : 0ull;
+                    const uint32_t dst = st + swz(c) * 16u;
+                    cp_async16(dst, a.d + src, bytes);
+                    cp_async16(dst + 2048u, a.m + src, bytes);
+                }
+                if (lane < 16) {
+                    const uint64_t w = (bs >> 5) + lane;
+                    const bool ok = (w << 5) < e && ((w << 5) + 32) > s;
+                    cp_async4(st + 4096u + lane * 4u, a.sbits + (ok ? w : 0ull), ok ? 4u : 0u);
+                }
+            }
+            cp_async_commit();
+        };
+
+        uint32_t carryD = 0;     // cumulative duration mod 2^32
+        uint64_t tot64 = 0;      // exact cumulative duration (overflow check)
+        uint64_t carryW = 0;     // cumulative work
+        uint32_t carrySeg = 0;   // max m since the last boundary
+        uint32_t carryRun = 0;   // max m since the progress point
+        uint32_t outpos = 0;     // rows written so far
+
+#pragma unroll
+        for (int t = 0; t < SCAN_STAGES - 1; ++t) issue((uint64_t)t);
+
+        for (uint64_t t = 0; t < nblk; ++t) {
+            issue(t + SCAN_STAGES - 1);
+            cp_async_wait<SCAN_STAGES - 1>();
+            __syncwarp();
+
+            const unsigned char* st = wbase + (size_t)(t % SCAN_STAGES) * SCAN_STAGE_BYTES;
+            const uint4* sd = reinterpret_cast<const uint4*>(st);
+            const uint4* sm = reinterpret_cast<const uint4*>(st + 2048);
+            const uint32_t* ss = reinterpret_cast<const uint32_t*>(st + 4096);
+            uint32_t dv[16], mv[16];
+#pragma unroll
+            for (uint32_t r = 0; r < 4; ++r) {
+                const uint32_t ph = swz(4u * lane + r);
+                const uint4 qd = sd[ph];
+                const uint4 qm = sm[ph];
+                dv[4 * r + 0] = qd.x; dv[4 * r + 1] = qd.y; dv[4 * r + 2] = qd.z; dv[4 * r + 3] = qd.w;
+                mv[4 * r + 0] = qm.x; mv[4 * r + 1] = qm.y; mv[4 * r + 2] = qm.z; mv[4 * r + 3] = qm.w;
+            }
+            uint32_t bits = (ss[lane >> 1] >> ((lane & 1u) * 16u)) & 0xFFFFu;
+            __syncwarp();  // every lane has read the slot; a later issue may overwrite it
+
+            const uint64_t bs = blk0 + t * SCAN_BLK;
+            const uint64_t lane_base = bs + 16ull * lane;
+            // valid steps of this lane: [lo, hi) within its 16
+            uint32_t lo = 0, hi = 16;
+            if (s > lane_base) lo = (s - lane_base) >= 16 ? 16u : (uint32_t)(s - lane_base);
+            if (e < lane_base + 16) hi = (e <= lane_base) ? 0u : (uint32_t)(e - lane_base);
+            uint32_t vm = (hi > lo) ? (((1u << hi) - 1u) & ~((1u << lo) - 1u)) : 0u;
+            if (vm != 0xFFFFu) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    if (!((vm >> i) & 1u)) { dv[i] = 0; mv[i] = 0; }
+            }
+            bits &= vm;
+            if (e - 1 >= lane_base && e - 1 < lane_base + 16) bits |= 1u << (uint32_t)(e - 1 - lane_base);
+
+            // ---- lane-local aggregates
+            uint64_t td = 0, tw = 0;
+            uint32_t lmax = 0, tail = 0;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                td += dv[i];
+                tw += (uint64_t)dv[i] * (uint64_t)mv[i];
+                lmax = max(lmax, mv[i]);
+                tail = max(tail, mv[i]);
+                if ((bits >> i) & 1u) tail = 0;
+            }
+            const uint32_t cnt = __popc(bits);
+
+            // ---- warp combine
+            // exact block duration (lane sums < 2^36): two 32-bit reductions
+            const uint32_t sum_lo = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)(td & 0xFFFFu));
+            const uint32_t sum_hi = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)(td >> 16));
+            const uint64_t blockD = ((uint64_t)sum_hi << 16) + sum_lo;
+
+            uint32_t incD = (uint32_t)td;
+            uint64_t incW = tw;
+            uint32_t incC = cnt;
+            uint32_t incR = lmax;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t yd = __shfl_up_sync(0xFFFFFFFFu, incD, o);
+                const uint64_t yw = __shfl_up_sync(0xFFFFFFFFu, incW, o);
+                const uint32_t yc = __shfl_up_sync(0xFFFFFFFFu, incC, o);
+                const uint32_t yr = __shfl_up_sync(0xFFFFFFFFu, incR, o);
+                if (lane >= (uint32_t)o) {
+                    incD += yd;
+                    incW += yw;
+                    incC += yc;
+                    incR = max(incR, yr);
+                }
+            }
+            // segmented max of the lane tails: a lane with a safe bit starts a new segment
+            const uint32_t hm = __ballot_sync(0xFFFFFFFFu, bits != 0u);
+            const uint32_t below = hm & (0xFFFFFFFFu >> (31u - lane));   // lanes 0..lane
+            const int head = below ? (31 - __clz((int)below)) : -1;
+            uint32_t x = tail;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o);
+                if ((int)lane - o >= head && (int)lane >= o) x = max(x, y);
+            }
+            uint32_t seg_in = __shfl_up_sync(0xFFFFFFFFu, x, 1);
+            const bool none_before = (hm & ((1u << lane) - 1u)) == 0u;   // no boundary in lanes < lane
+            if (lane == 0) seg_in = carrySeg;
+            else if (none_before) seg_in = max(seg_in, carrySeg);
+            uint32_t run_in = __shfl_up_sync(0xFFFFFFFFu, incR, 1);
+            run_in = (lane == 0) ? carryRun : max(run_in, carryRun);
+
+            // ---- emit rows at this lane's safe bits
+            uint32_t D = carryD + (incD - (uint32_t)td);
+            uint64_t W = carryW + (incW - tw);
+            uint32_t seg = seg_in, run = run_in;
+            uint64_t pos = out_base + outpos + (incC - cnt);
+            const uint32_t k0 = (uint32_t)(lane_base - js);   // steps before this lane (may wrap if masked)
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                D += dv[i];
+                W += (uint64_t)dv[i] * (uint64_t)mv[i];
+                seg = max(seg, mv[i]);
+                run = max(run, mv[i]);
+                if ((bits >> i) & 1u) {
+                    if (pos < out_end) {
+                        a.A[pos] = make_uint4(D, run, (uint32_t)W, (uint32_t)(W >> 32));
+                        a.B[pos] = make_uint2(k0 + (uint32_t)i + 1u, seg);
+                    }
+                    ++pos;
+                    seg = 0;
+                }
+            }
+
+            // ---- carries for the next block
+            carryD += __shfl_sync(0xFFFFFFFFu, incD, 31);
+            carryW += __shfl_sync(0xFFFFFFFFu, incW, 31);
+            outpos += __shfl_sync(0xFFFFFFFFu, incC, 31);
+            carryRun = max(carryRun, __shfl_sync(0xFFFFFFFFu, incR, 31));
+            const uint32_t x31 = __shfl_sync(0xFFFFFFFFu, x, 31);
+            carrySeg = hm ? x31 : max(x31, carrySeg);
+            tot64 += blockD;
+        }
+
+        if (lane == 0) {
+            uint32_t f = 0;
+            if (tot64 > 0xFFFFFFFFull) f |= FLAG_OVF_DURATION;
+            if (carryW >= (1ull << 63)) f |= FLAG_OVF_WORK;
+            if (carryW >= (1ull << KEY_SLA_SHIFT)) f |= FLAG_OVF_SLA;
+            if (a.wait) {
+                const uint64_t fac = 1ull + (uint64_t)(__ldg(a.wait + j) / 1000u);
+                if (__umul64hi(carryW, fac) != 0ull || carryW * fac >= (1ull << 63)) f |= FLAG_OVF_FAIR;
+            }
+            if ((uint64_t)outpos != out_end - out_base) f |= FLAG_INTERNAL;
+            if (f) atomicOr(a.flags, f);
+        }
+    }
+}
+
+}  // namespace sja

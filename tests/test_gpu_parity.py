@@ -1,0 +1,310 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element.
+
+All quantities are integers, so the bar is bit-exact equality.
+"""
+import numpy as np
+import pytest
+
+from paper_2509_19086_b200 import workloads as wl
+from tests.helpers import gaps_from_lists, profiles_from_lists, random_small_profiles
+
+pytestmark = pytest.mark.gpu
+
+U32MAX = 0xFFFFFFFF
+
+
+@pytest.fixture(scope="module")
+def sja_mod():
+    from paper_2509_19086_b200 import binding
+    return binding
+
+
+def _load(ctx, prof, progress=None):
+    ctx.load_profiles(prof.off, prof.dur_ms, prof.mem_MiB, prof.safe_bits, prof.ready_ms,
+                      progress=progress, wait_ms=prof.wait_ms, prio=prof.prio)
+
+
+def _assert_awards_equal(got, want, fields=("job", "end_step", "dur_ms", "score")):
+    for f in fields:
+        bad = np.nonzero(got[f] != want[f])[0]
+        assert bad.size == 0, (f, bad[:5], got[bad[:5]], want[bad[:5]])
+
+
+def _check_scan(oracle, ctx, prof, progress):
+    sc = ctx.get_scan()
+    J = prof.n_jobs
+    for j in range(J):
+        rows = oracle.boundary_table(prof, j, int(progress[j]))
+        b0, b1 = int(sc["boff"][j]), int(sc["boff"][j + 1])
+        assert b1 - b0 == len(rows), (j, b1 - b0, len(rows))
+        if not rows:
+            continue
+        exp = np.array(rows, dtype=np.uint64)
+        assert np.array_equal(sc["k"][b0:b1], exp[:, 0]), j
+        assert np.array_equal(sc["D"][b0:b1], exp[:, 1]), j
+        assert np.array_equal(sc["M"][b0:b1], exp[:, 2]), j
+        assert np.array_equal(sc["S"][b0:b1], exp[:, 3]), j
+        assert np.array_equal(sc["W"][b0:b1], exp[:, 4]), j
+
+
+# ------------------------------------------------------------------ scan (a1)
+def test_scan_matches_oracle_ragged_lengths(sja_mod, oracle_mod):
+    """Job lengths around every tile edge of the scan (16-step lanes, 512-step warp blocks)."""
+    rng = np.random.default_rng(101)
+    lens = [1, 2, 15, 16, 17, 31, 32, 33, 100, 511, 512, 513, 1023, 1024, 1025, 1500, 2047, 4096, 5000, 3, 0, 7]
+    jobs = []
+    for n in lens:
+        d = rng.integers(0, 60, n).tolist()
+        m = rng.integers(0, 90000, n).tolist()
+        s = (rng.random(n) < 0.12).astype(int).tolist()
+        jobs.append((d, m, s))
+    prof = profiles_from_lists(jobs, ready=rng.integers(0, 100, len(jobs)))
+    progress = np.array([int(rng.integers(0, n + 1)) for n in lens], dtype=np.uint32)
+    progress[:6] = 0
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof, progress)
+        _check_scan(oracle_mod, ctx, prof, progress)
+        # device-resident inputs take the same path without the staging copy
+        import torch
+        dev = {k: torch.from_numpy(np.ascontiguousarray(v).view(np.int64 if v.dtype == np.uint64 else np.int32)).cuda()
+               for k, v in dict(off=prof.off, d=prof.dur_ms, m=prof.mem_MiB, s=prof.safe_bits,
+                                r=prof.ready_ms, p=progress).items()}
+        ctx.load_profiles(dev["off"], dev["d"], dev["m"], dev["s"], dev["r"], progress=dev["p"])
+        _check_scan(oracle_mod, ctx, prof, progress)
+
+
+def test_scan_matches_oracle_dense_boundaries_and_large_values(sja_mod, oracle_mod):
+    """Every step safe (512 rows per warp block) and 32-bit-wide values (64-bit work sums)."""
+    rng = np.random.default_rng(102)
+    jobs = []
+    for n in (700, 40, 1300):
+        jobs.append((rng.integers(0, 2**20, n).tolist(), rng.integers(0, 2**32 - 1, n).tolist(), [1] * n))
+    jobs.append(([5] * 600, [7] * 600, [0] * 600))          # no interior boundary at all
+    prof = profiles_from_lists(jobs)
+    progress = np.zeros(len(jobs), np.uint32)
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof, progress)
+        _check_scan(oracle_mod, ctx, prof, progress)
+
+
+def test_scan_cfg1_sampled_jobs(sja_mod, oracle_mod):
+    spec = wl.SPECS[1]
+    prof = wl.make_profiles(spec)
+    progress = np.zeros(prof.n_jobs, np.uint32)
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof, progress)
+        sc = ctx.get_scan()
+        safe = wl.unpack_safe_bits(prof.safe_bits, prof.n_steps)
+        assert ctx.scan_size() == int(safe.sum())
+        rng = np.random.default_rng(5)
+        for j in rng.choice(prof.n_jobs, 40, replace=False):
+            rows = np.array(oracle_mod.boundary_table(prof, int(j), 0), dtype=np.uint64)
+            b0, b1 = int(sc["boff"][j]), int(sc["boff"][j + 1])
+            assert b1 - b0 == rows.shape[0]
+            got = np.stack([sc["k"][b0:b1], sc["D"][b0:b1], sc["M"][b0:b1], sc["S"][b0:b1], sc["W"][b0:b1]], 1)
+            assert np.array_equal(got.astype(np.uint64), rows)
+
+
+# ------------------------------------------------------------------ select (a2-a5)
+@pytest.mark.parametrize("flags", [0, 1])
+@pytest.mark.parametrize("policy", [0, 1, 2])
+def test_select_tiny_random_vs_oracle(sja_mod, oracle_mod, policy, flags):
+    rng = np.random.default_rng(200 + policy)
+    with sja_mod.Sja() as ctx:
+        for trial in range(12):
+            jobs = random_small_profiles(rng, int(rng.integers(1, 70)), 40, p_safe=float(rng.uniform(0.05, 0.9)),
+                                         dmax=30, mmax=100, allow_zero=(trial % 4 == 0))
+            J = len(jobs)
+            prof = profiles_from_lists(jobs, ready=rng.integers(0, 20, J), wait=rng.integers(0, 9000, J),
+                                       prio=rng.integers(0, 3, J))
+            lens = np.diff(prof.off).astype(np.int64)
+            progress = np.array([rng.integers(0, n + 1) for n in lens], dtype=np.uint32)
+            G = int(rng.integers(1, 90))
+            gaps = gaps_from_lists([(int(rng.integers(0, 7)), int(rng.integers(0, 30)), int(rng.integers(0, 400)),
+                                     int(rng.integers(0, 110))) for _ in range(G)])
+            _load(ctx, prof, progress)
+            ctx.advertise(gaps)
+            got = ctx.select(policy, flags=flags, out="host")
+            want = oracle_mod.select(prof, progress, prof.ready_ms, gaps, policy)
+            _assert_awards_equal(got, want)
+            assert not got["granted"].any()
+
+
+@pytest.mark.parametrize("cfg", [0, 1])
+def test_select_published_small_configs(sja_mod, oracle_mod, cfg):
+    spec = wl.SPECS[cfg]
+    prof = wl.make_profiles(spec)
+    gaps = wl.make_gaps(spec)
+    progress = np.zeros(prof.n_jobs, np.uint32)
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof)
+        ctx.advertise(gaps)
+        want = oracle_mod.select(prof, progress, prof.ready_ms, gaps, spec.policy)
+        for flags in (0, 1):
+            got = ctx.select(spec.policy, flags=flags, out="host")
+            _assert_awards_equal(got, want)
+        assert (got["job"] != U32MAX).sum() > 0
+        # select is free of side effects and repeatable
+        p, r = ctx.get_state()
+        assert not p.any() and np.array_equal(r, prof.ready_ms)
+        again = ctx.select(spec.policy, out="host")
+        assert again.tobytes() == got.tobytes()
+
+
+def test_select_fairness_and_sla_scaled_configs(sja_mod, oracle_mod):
+    for base, changes in ((2, dict(n_jobs=3000, fixed_len=700, n_gaps=300)),
+                          (3, dict(n_jobs=4000, zipf_max=6000, n_gaps=256))):
+        spec = wl.scaled(wl.SPECS[base], **changes)
+        prof = wl.make_profiles(spec)
+        gaps = wl.make_gaps(spec)
+        progress = np.zeros(prof.n_jobs, np.uint32)
+        with sja_mod.Sja() as ctx:
+            _load(ctx, prof)
+            ctx.advertise(gaps)
+            want = oracle_mod.select(prof, progress, prof.ready_ms, gaps, spec.policy)
+            for flags in (0, 1):
+                got = ctx.select(spec.policy, flags=flags, out="host")
+                _assert_awards_equal(got, want)
+
+
+def test_select_long_windows_and_many_capacity_classes(sja_mod, oracle_mod):
+    """Windows far longer than any staged tile and hundreds of distinct capacities."""
+    rng = np.random.default_rng(77)
+    spec = wl.scaled(wl.SPECS[1], n_jobs=700, fixed_len=900, n_gaps=400)
+    prof = wl.make_profiles(spec)
+    gaps = wl.make_gaps(spec)
+    gaps["T_ms"] = rng.integers(0, 40000, gaps.shape[0])
+    gaps["T_ms"][:5] = U32MAX
+    gaps["C_MiB"] = rng.integers(1, 90000, gaps.shape[0])
+    gaps["C_MiB"][:3] = U32MAX
+    progress = rng.integers(0, 900, prof.n_jobs).astype(np.uint32)
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof, progress)
+        ctx.advertise(gaps)
+        want = oracle_mod.select(prof, progress, prof.ready_ms, gaps, 0)
+        for flags in (0, 1):
+            got = ctx.select(0, flags=flags, out="host")
+            _assert_awards_equal(got, want)
+
+
+# ------------------------------------------------------------------ commit (a6), multi-round
+@pytest.mark.parametrize("flags", [0, 1])
+def test_streaming_rounds_bit_exact(sja_mod, oracle_mod, flags):
+    """Scaled streaming workload: per-round awards (with grants) and final state match the oracle."""
+    spec = wl.scaled(wl.SPECS[4], n_jobs=1500, fixed_len=300, n_gaps=200, n_rounds=60)
+    prof = wl.make_profiles(spec)
+    progress = np.zeros(prof.n_jobs, np.uint32)
+    ready = prof.ready_ms.copy()
+    total = 0
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof)
+        for r in range(spec.n_rounds):
+            gaps = wl.make_gaps(spec, r)
+            ctx.advertise(gaps)
+            ctx.select(spec.policy, flags=flags)
+            n_gpu = ctx.commit()
+            got = ctx.get_awards()
+            want = oracle_mod.select(prof, progress, ready, gaps, spec.policy)
+            n_cpu = oracle_mod.commit(progress, ready, gaps, want)
+            _assert_awards_equal(got, want, fields=("job", "end_step", "dur_ms", "score", "granted"))
+            assert n_gpu == n_cpu
+            total += n_cpu
+        p, rdy = ctx.get_state()
+        assert np.array_equal(p, progress) and np.array_equal(rdy, ready)
+        assert total > spec.n_rounds          # the workload really grants subjobs
+        assert (p == 300).any()               # and some jobs finish and must decline afterwards
+
+
+def test_commit_resolves_multiple_wins(sja_mod, oracle_mod):
+    """One dominant job wins every gap; it accepts the largest k, then the lowest gap id."""
+    jobs = [([10] * 20, [100] * 20, [1] * 20), ([10] * 20, [1] * 20, [1] * 20)]
+    prof = profiles_from_lists(jobs)
+    gaps = gaps_from_lists([(0, 0, 50, 200), (1, 0, 120, 200), (2, 0, 120, 200), (3, 0, 30, 200)])
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof)
+        ctx.advertise(gaps)
+        ctx.select(0)
+        assert ctx.commit() == 1
+        aw = ctx.get_awards()
+        assert aw["job"].tolist() == [0, 0, 0, 0]
+        assert aw["granted"].tolist() == [0, 1, 0, 0]
+        p, r = ctx.get_state()
+        assert p.tolist() == [12, 0] and r.tolist() == [120, 0]
+        want = oracle_mod.select(prof, np.zeros(2, np.uint32), prof.ready_ms, gaps, 0)
+        pr, rd = np.zeros(2, np.uint32), prof.ready_ms.copy()
+        oracle_mod.commit(pr, rd, gaps, want)
+        _assert_awards_equal(aw, want, fields=("job", "end_step", "dur_ms", "score", "granted"))
+
+
+# ------------------------------------------------------------------ host logic / errors
+def test_error_paths(sja_mod):
+    b = sja_mod
+    prof = profiles_from_lists([([1, 2], [3, 4], [0, 1]), ([5], [6], [1])], wait=None, prio=None)
+    gaps = gaps_from_lists([(0, 0, 10, 10)])
+    with b.Sja() as ctx:
+        with pytest.raises(b.SjaError) as e:
+            ctx.advertise(gaps)
+        assert e.value.status == 4                      # STATE: advertise before load
+        with pytest.raises(b.SjaError) as e:
+            ctx.commit()
+        assert e.value.status == 4
+        _load(ctx, prof)
+        with pytest.raises(b.SjaError) as e:
+            ctx.select(0)
+        assert e.value.status == 4                      # select before advertise
+        ctx.advertise(gaps)
+        for policy, status in ((1, 1), (2, 1), (9, 1)):  # fairness w/o wait, SLA w/o prio, unknown
+            with pytest.raises(b.SjaError) as e:
+                ctx.select(policy)
+            assert e.value.status == status
+        got = ctx.select(0, out="host")
+        assert got["job"][0] == 1                       # job1: work 30 > job0: 1*3+2*4 = 11
+        assert ctx.commit() == 1
+        with pytest.raises(b.SjaError) as e:
+            ctx.commit()
+        assert e.value.status == 4                      # twice
+        # bad CSR leaves the loaded state untouched
+        bad_off = np.array([0, 5, 3], dtype=np.uint64)
+        with pytest.raises(b.SjaError) as e:
+            ctx.load_profiles(bad_off, prof.dur_ms, prof.mem_MiB, prof.safe_bits, prof.ready_ms)
+        assert e.value.status == 2
+        with pytest.raises(b.SjaError) as e:
+            ctx.load_profiles(prof.off, prof.dur_ms, prof.mem_MiB, prof.safe_bits, prof.ready_ms,
+                              progress=np.array([3, 0], np.uint32))
+        assert e.value.status == 2                      # progress > len
+        p, r = ctx.get_state()
+        assert p.tolist() == [0, 1]
+        # duration overflow is reported at load
+        big = profiles_from_lists([([2**31, 2**31], [1, 1], [1, 1])])
+        with pytest.raises(b.SjaError) as e:
+            _load(ctx, big)
+        assert e.value.status == 3
+        # fairness score overflow is reported at select
+        huge = profiles_from_lists([([2**31 - 1], [2**32 - 1], [1])], wait=[4_000_000_000])
+        _load(ctx, huge)
+        ctx.advertise(gaps)
+        ctx.select(0)
+        with pytest.raises(b.SjaError) as e:
+            ctx.select(1)
+        assert e.value.status == 3
+
+
+def test_empty_and_degenerate_inputs(sja_mod, oracle_mod):
+    # all jobs empty; a job that is already finished; gaps nobody fits
+    prof = profiles_from_lists([([], [], []), ([], [], [])])
+    gaps = gaps_from_lists([(0, 0, 100, 100), (1, 5, 0, 0)])
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof)
+        assert ctx.scan_size() == 0
+        ctx.advertise(gaps)
+        got = ctx.select(0, out="host")
+        assert (got["job"] == U32MAX).all() and not got["score"].any()
+        assert ctx.commit() == 0
+        prof2 = profiles_from_lists([([4, 4], [9, 9], [1, 1]), ([0, 0], [0, 7], [1, 1])])
+        progress = np.array([2, 0], np.uint32)
+        _load(ctx, prof2, progress)
+        ctx.advertise(gaps_from_lists([(0, 0, 0, 7), (0, 0, 0, 6)]))
+        got = ctx.select(0, out="host")
+        want = oracle_mod.select(prof2, progress, prof2.ready_ms, gaps_from_lists([(0, 0, 0, 7), (0, 0, 0, 6)]), 0)
+        _assert_awards_equal(got, want)
+        assert got["job"].tolist() == [1, 1] and got["end_step"].tolist() == [2, 1]   # zero-work interest
