@@ -29,9 +29,9 @@ from paper_2509_19086_b200 import workloads as wl  # noqa: E402
 METRIC = "job-gap pairs evaluated/s"
 UNIT = "pairs/s"
 POLICY_NAMES = {0: "efficiency", 1: "fairness", 2: "sla"}
-# kernels launched per step: count_boundaries, row_offsets, scan_profiles | select_search,
-# finalize_awards | commit_vote, commit_apply, commit_refresh
-KERNELS_PER_STEP = 8
+# kernels launched per step: count_boundaries, row_offsets, scan_profiles | sort_gaps |
+# select_merge (or select_search), finalize_awards | commit_vote, commit_apply, commit_refresh
+KERNELS_PER_STEP = 9
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -54,13 +54,14 @@ class ClockSampler:
     def __init__(self, index: int):
         self.index = index
         self.proc = None
-        self.lines = []
+        self.lines = []          # (arrival time, csv line)
+        self.t0 = self.t1 = None
 
     def start(self):
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -69,7 +70,18 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.perf_counter(), line.strip()))
+
+    def wait_first_sample(self, timeout=10.0):
+        t = time.perf_counter()
+        while self.proc is not None and not self.lines and time.perf_counter() - t < timeout:
+            time.sleep(0.02)
+
+    def mark_begin(self):
+        self.t0 = time.perf_counter()
+
+    def mark_end(self):
+        self.t1 = time.perf_counter()
 
     def stop(self) -> dict:
         if self.proc is None:
@@ -81,7 +93,9 @@ class ClockSampler:
             self.proc.kill()
         sm, smax, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        lines = [ln for (t, ln) in self.lines
+                 if self.t0 is None or self.t1 is None or (self.t0 <= t <= self.t1 + 0.15)]
+        for ln in lines:
             parts = [p.strip() for p in ln.split(",")]
             if len(parts) < 6:
                 continue
@@ -184,17 +198,23 @@ def run_reference(args, spec):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", type=int, default=2, help="index into the published configuration list")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--flags", type=int, default=0, help="sja_policy.flags (1 = per-pair search kernel)")
+    ap.add_argument("--jobs", type=int, default=0, help="override the job count (profiling captures)")
+    ap.add_argument("--gaps", type=int, default=0, help="override the gap count (profiling captures)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     spec = wl.SPECS[args.workload]
+    if args.jobs:
+        spec = wl.scaled(spec, n_jobs=args.jobs, name=spec.name + f"-jobs{args.jobs}")
+    if args.gaps:
+        spec = wl.scaled(spec, n_gaps=args.gaps, name=spec.name + f"-gaps{args.gaps}")
 
     if args.impl == "reference":
         run_reference(args, spec)
@@ -267,27 +287,32 @@ def main():
         n_rows = ctx.scan_size()
         ctx.profile_enable(True)
         sampler = ClockSampler(local_rank)
-        barrier()
         sampler.start()
+        sampler.wait_first_sample()
+        barrier()
+        sampler.mark_begin()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         for _ in range(args.steps):
             step_device()
         e1.record(stream)
         barrier()
+        sampler.mark_end()
         ms_total = e0.elapsed_time(e1)
         clocks = sampler.stop()
         timing = ctx.profile_read()
         ctx.profile_enable(False)
 
         # end to end: pinned host inputs in, awards + grant count out, every step
-        step_e2e()
-        barrier()
-        t0 = time.perf_counter()
-        for _ in range(args.e2e_steps):
-            aw, n_granted = step_e2e()
-        torch.cuda.synchronize()
-        e2e_s = time.perf_counter() - t0
+        e2e_s = 0.0
+        if args.e2e_steps > 0:
+            step_e2e()
+            barrier()
+            t0 = time.perf_counter()
+            for _ in range(args.e2e_steps):
+                aw, n_granted = step_e2e()
+            torch.cuda.synchronize()
+            e2e_s = time.perf_counter() - t0
 
     t_ms = torch.tensor([ms_total, 1e3 * e2e_s], dtype=torch.float64, device=device)
     if dist is not None:
@@ -295,7 +320,7 @@ def main():
     ms_total, e2e_ms = float(t_ms[0]), float(t_ms[1])
     ms_per_step = ms_total / args.steps
     value = world * pairs * args.steps / (ms_total * 1e-3)
-    e2e_value = world * pairs * args.e2e_steps / (e2e_ms * 1e-3)
+    e2e_value = world * pairs * args.e2e_steps / (e2e_ms * 1e-3) if e2e_ms > 0 else None
     h2d = sum(int(a.nbytes) for a in host_arrays.values()) + int(gaps.nbytes)
     d2h = 24 * G + 4
 
@@ -322,7 +347,7 @@ def main():
                    "flags": args.flags},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": e2e_ms / args.e2e_steps, "steps": args.e2e_steps},
+                "ms_per_step": e2e_ms / max(1, args.e2e_steps), "steps": args.e2e_steps},
         "gpu_launches": KERNELS_PER_STEP * args.steps,
         "roofline": roofline,
         "kernel_ms_per_step": breakdown,

@@ -53,7 +53,9 @@ struct sja_ctx {
     // gaps / awards
     bool advertised = false, selected = false, committed = false;
     uint32_t G = 0, last_policy = 0;
-    DevBuf gaps, awards, widx, partial, winners;
+    bool gaps_sorted = false;          // sgaps is ordered by (C, T); else it is the caller's order
+    uint32_t n_classes = 0;            // distinct capacities of the batch (valid when sorted)
+    DevBuf gaps, sgaps, gap_info, awards, widx, partial, winners;
 
     // profiling
     bool prof = false;
@@ -266,6 +268,11 @@ sja_status sja_create(sja_ctx** out, int device, void* cuda_stream) {
         if (cudaMemsetAsync(c->flags.p, 0, 4, c->stream) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         if (cudaFuncSetAttribute(scan_profiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  SCAN_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
+        if (cudaFuncSetAttribute(select_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 MERGE_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
+        if (cudaFuncSetAttribute(sort_gaps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(SORT_MAX_GAPS * 12)) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
+        if ((st = reserve(c, c->gap_info, sizeof(GapInfo))) != SJA_OK) break;
     } while (0);
     if (st != SJA_OK) {
         cudaGetLastError();
@@ -282,7 +289,7 @@ sja_status sja_destroy(sja_ctx* c) {
     cudaStreamSynchronize(c->stream);
     DevBuf* bufs[] = {&c->st_off, &c->st_d, &c->st_m, &c->st_s, &c->st_p, &c->p, &c->ready, &c->pb, &c->Dp,
                       &c->Wp, &c->wait, &c->prio, &c->nbj, &c->boff, &c->boff_next, &c->A, &c->B, &c->jobwin,
-                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->awards, &c->widx, &c->partial,
+                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->awards, &c->widx, &c->partial,
                       &c->winners};
     for (DevBuf* b : bufs) release(*b);
     for (ProfSpan& s : c->spans) { cudaEventDestroy(s.a); cudaEventDestroy(s.b); }
@@ -462,14 +469,30 @@ sja_status sja_advertise(sja_ctx* c, uint32_t G, const sja_gap* gaps, sja_memspa
     if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_advertise before sja_load_profiles");
     DeviceGuard guard(c->device);
     TRY(reserve(c, c->gaps, (size_t)G * sizeof(sja_gap)));
+    TRY(reserve(c, c->sgaps, (size_t)G * sizeof(sja_gap)));
     TRY(reserve(c, c->awards, (size_t)G * sizeof(sja_award)));
     TRY(reserve(c, c->widx, (size_t)G * 4));
     TRY(reserve(c, c->winners, (size_t)G * 4));
+    const bool sortable = G <= SORT_MAX_GAPS;
     {
         ProfScope ps(c, CAT_ADVERTISE);
         TRY(copy_in(c, c->gaps.p, gaps, (size_t)G * sizeof(sja_gap), where));
+        if (sortable) {
+            uint32_t n_pow2 = 1;
+            while (n_pow2 < G) n_pow2 <<= 1;
+            sort_gaps_kernel<<<1, 1024, (size_t)n_pow2 * 12, c->stream>>>(c->gaps.as<Gap>(), G, n_pow2,
+                                                                         c->sgaps.as<Gap>(),
+                                                                         c->gap_info.as<GapInfo>());
+            CU(cudaMemcpyAsync(c->h_words + 4, c->gap_info.p, sizeof(GapInfo), cudaMemcpyDeviceToHost, c->stream));
+        } else {
+            copy_gaps_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(c->gaps.as<Gap>(), G, c->sgaps.as<Gap>());
+        }
     }
-    if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));   // caller may reuse its buffer
+    CU(cudaGetLastError());
+    // the class count steers the kernel choice of sja_select, and a host buffer may be reused on return
+    CU(cudaStreamSynchronize(c->stream));
+    c->gaps_sorted = sortable;
+    c->n_classes = sortable ? c->h_words[4] : 0;
     c->G = G;
     c->advertised = true;
     c->selected = c->committed = false;
@@ -495,23 +518,35 @@ sja_status sja_select(sja_ctx* c, const sja_policy* policy, sja_award* out, sja_
     DeviceGuard guard(c->device);
 
     const uint32_t G = c->G, J = c->J;
-    const uint32_t n_chunks = (J + SEARCH_THREADS - 1) / SEARCH_THREADS;
+    // The merge kernel pays one restart per capacity class; with very many classes (or an
+    // unsorted batch) the per-pair search is the better tool.
+    const bool use_merge = !(policy->flags & SJA_FLAG_FORCE_SEARCH) && c->gaps_sorted &&
+                           c->n_classes <= std::max<uint32_t>(64u, G / 16u);
+    const uint32_t jobs_per_cta = use_merge ? (uint32_t)MERGE_JOBS : (uint32_t)SEARCH_THREADS;
+    const uint32_t tile = use_merge ? (uint32_t)MERGE_GT : (uint32_t)SEARCH_GT;
+    const uint32_t n_chunks = (J + jobs_per_cta - 1) / jobs_per_cta;
     TRY(reserve(c, c->partial, (size_t)n_chunks * G * sizeof(Partial)));
-    // split the gaps so that the grid covers the SMs a few times over
-    uint32_t splits = (uint32_t)((4ull * c->n_sm + n_chunks - 1) / n_chunks);
-    const uint32_t max_splits = (G + SEARCH_GT - 1) / SEARCH_GT;
+    // split the gaps so that the grid covers the SMs several times over
+    uint32_t splits = (uint32_t)((8ull * c->n_sm + n_chunks - 1) / n_chunks);
+    const uint32_t max_splits = (G + tile - 1) / tile;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
     uint32_t per_split = (G + splits - 1) / splits;
-    per_split = ((per_split + SEARCH_GT - 1) / SEARCH_GT) * SEARCH_GT;
+    per_split = ((per_split + tile - 1) / tile) * tile;
     splits = (G + per_split - 1) / per_split;
     {
         ProfScope ps(c, CAT_SELECT);
         const JobView jv = job_view(c);
-        select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, 0, c->stream>>>(
-            jv, c->gaps.as<Gap>(), G, per_split, kind, nullptr, 0, c->partial.as<Partial>());
-        finalize_awards_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(jv, c->partial.as<Partial>(), n_chunks, G,
-                                                                         kind, c->awards.as<Award>(),
+        if (use_merge) {
+            select_merge_kernel<<<dim3(n_chunks, splits), MERGE_WARPS * 32, MERGE_SMEM_BYTES, c->stream>>>(
+                jv, c->sgaps.as<Gap>(), G, per_split, kind, c->partial.as<Partial>());
+        } else {
+            select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, 0, c->stream>>>(
+                jv, c->sgaps.as<Gap>(), G, per_split, kind, nullptr, 0, c->partial.as<Partial>());
+        }
+        finalize_awards_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(jv, c->partial.as<Partial>(), n_chunks,
+                                                                         c->sgaps.as<Gap>(), G, kind,
+                                                                         c->awards.as<Award>(),
                                                                          c->widx.as<uint32_t>());
     }
     CU(cudaGetLastError());

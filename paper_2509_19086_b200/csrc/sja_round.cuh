@@ -115,9 +115,9 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
 // ---------------------------------------------------------------------------------------
 // Final reduction: one thread per gap folds the candidate rows of all CTAs into the award.
 __global__ void __launch_bounds__(256) finalize_awards_kernel(
-    JobView jv, const Partial* __restrict__ partial, uint32_t n_rows, uint32_t G, uint32_t kind,
-    Award* __restrict__ awards, uint32_t* __restrict__ widx) {
-    const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
+    JobView jv, const Partial* __restrict__ partial, uint32_t n_rows, const Gap* __restrict__ sgaps, uint32_t G,
+    uint32_t kind, Award* __restrict__ awards, uint32_t* __restrict__ widx) {
+    const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;   // position in the advertised (sorted) order
     if (g >= G) return;
     Partial best;
     best.key = 0; best.job = 0xFFFFFFFFu; best.cnt = 0;
@@ -125,10 +125,11 @@ __global__ void __launch_bounds__(256) finalize_awards_kernel(
         const Partial c = partial[(size_t)r * G + g];
         if (c.key > best.key || (c.key == best.key && c.job < best.job)) best = c;
     }
+    const uint32_t orig = sgaps[g].slice;   // caller's gap index
     Award a;
     if (best.key == 0) {
         a.job = 0xFFFFFFFFu; a.end_step = 0; a.dur = 0; a.granted = 0; a.score = 0;
-        widx[g] = 0;
+        widx[orig] = 0;
     } else {
         const uint32_t j = best.job;
         const uint64_t row = jv.boff[j] + jv.pb[j] + best.cnt - 1;
@@ -137,9 +138,9 @@ __global__ void __launch_bounds__(256) finalize_awards_kernel(
         a.dur = jv.A[row].x - jv.Dp[j];
         a.granted = 0;
         a.score = key_to_score(kind, best.key);
-        widx[g] = best.cnt;
+        widx[orig] = best.cnt;
     }
-    awards[g] = a;
+    awards[orig] = a;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -218,6 +219,223 @@ __global__ void __launch_bounds__(256) commit_refresh_kernel(
         if (v_last == old_last) break;
         carry = v_last;
     }
+}
+
+}  // namespace sja
+
+namespace sja {
+
+// ---------------------------------------------------------------------------------------
+// Advertise: order the gaps by (capacity, window length).  Gaps of one capacity form a
+// "class" (the finite capacity set of Section 3.9); inside a class T ascends, so every job's
+// answer moves monotonically along its boundary rows and the select kernel can merge
+// instead of search.  One CTA, bitonic sort in shared memory (G <= SORT_MAX_GAPS).
+constexpr uint32_t SORT_MAX_GAPS = 16384;
+
+struct GapInfo { uint32_t n_classes; uint32_t t_max; uint32_t c_max; uint32_t pad; };
+
+__global__ void __launch_bounds__(1024) sort_gaps_kernel(const Gap* __restrict__ gaps, uint32_t G, uint32_t n_pow2,
+                                                         Gap* __restrict__ sorted, GapInfo* __restrict__ info) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint64_t* key = reinterpret_cast<uint64_t*>(smem_raw);
+    uint32_t* idx = reinterpret_cast<uint32_t*>(smem_raw + (size_t)n_pow2 * 8);
+    __shared__ uint32_t s_classes, s_tmax, s_cmax;
+    const uint32_t t = threadIdx.x;
+    if (t == 0) { s_classes = 0; s_tmax = 0; s_cmax = 0; }
+    for (uint32_t i = t; i < n_pow2; i += blockDim.x) {
+        if (i < G) {
+            const Gap g = gaps[i];
+            key[i] = ((uint64_t)g.C << 32) | g.T;
+            idx[i] = i;
+        } else {
+            key[i] = 0xFFFFFFFFFFFFFFFFull;   // padding sorts last (after real gaps with the same key: larger idx)
+            idx[i] = 0xFFFFFFFFu;
+        }
+    }
+    __syncthreads();
+    for (uint32_t k = 2; k <= n_pow2; k <<= 1) {
+        for (uint32_t j = k >> 1; j > 0; j >>= 1) {
+            for (uint32_t i = t; i < n_pow2; i += blockDim.x) {
+                const uint32_t l = i ^ j;
+                if (l > i) {
+                    const uint64_t ki = key[i], kl = key[l];
+                    const uint32_t ii = idx[i], il = idx[l];
+                    const bool up = (i & k) == 0;
+                    const bool gt = ki > kl || (ki == kl && ii > il);
+                    if (gt == up) { key[i] = kl; key[l] = ki; idx[i] = il; idx[l] = ii; }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    uint32_t classes = 0, tmax = 0, cmax = 0;
+    for (uint32_t i = t; i < G; i += blockDim.x) {
+        const Gap g = gaps[idx[i]];
+        Gap o;
+        o.slice = idx[i];   // the original position travels in the slice field
+        o.start = g.start; o.T = g.T; o.C = g.C;
+        sorted[i] = o;
+        if (i == 0 || (uint32_t)(key[i - 1] >> 32) != g.C) ++classes;
+        tmax = max(tmax, g.T);
+        cmax = max(cmax, g.C);
+    }
+    atomicAdd(&s_classes, classes);
+    atomicMax(&s_tmax, tmax);
+    atomicMax(&s_cmax, cmax);
+    __syncthreads();
+    if (t == 0) { info->n_classes = s_classes; info->t_max = s_tmax; info->c_max = s_cmax; info->pad = 0; }
+}
+
+// Identity order (used when the batch is too large for the one-CTA sort).
+__global__ void __launch_bounds__(256) copy_gaps_kernel(const Gap* __restrict__ gaps, uint32_t G,
+                                                        Gap* __restrict__ sorted) {
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= G) return;
+    Gap g = gaps[i];
+    g.slice = i;
+    sorted[i] = g;
+}
+
+// ---------------------------------------------------------------------------------------
+// Merge kernel.  Each lane owns MERGE_R jobs and walks the gaps of its CTA's range in the
+// advertised order (capacity class, then T ascending).  Per job it keeps a cursor into the
+// job's boundary rows above the progress point: the number w of rows that satisfy both
+// bounds for the current gap.  Inside a class w only moves forward, so a pair costs a few
+// compares.  The next rows of every job wait in a per-lane shared-memory ring that is
+// refilled with 16-byte cp.async copies, so an advance never waits on global memory in the
+// steady state.  Per gap the warp reduces its 32 x MERGE_R keys to one candidate
+// (largest key, then lowest job id), the CTA folds its warps, and one candidate per
+// (CTA, gap) goes to global memory.
+constexpr int MERGE_WARPS = 8;
+constexpr int MERGE_R = 2;
+constexpr int MERGE_RING = 8;       // rows per lane-job ring
+constexpr int MERGE_GT = 64;        // gaps per staging tile
+constexpr int MERGE_JOBS = MERGE_WARPS * MERGE_R * 32;
+constexpr int MERGE_RING_BYTES = MERGE_WARPS * MERGE_R * MERGE_RING * 32 * 16;
+constexpr int MERGE_SMEM_BYTES = MERGE_RING_BYTES + MERGE_GT * MERGE_WARPS * 16 + MERGE_GT * 16;
+
+__device__ __forceinline__ void mg_cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void mg_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void mg_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+__global__ void __launch_bounds__(MERGE_WARPS * 32) select_merge_kernel(
+    JobView jv, const Gap* __restrict__ sgaps, uint32_t G, uint32_t gaps_per_split, uint32_t kind,
+    Partial* __restrict__ partial_out) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint4* ring_all = reinterpret_cast<uint4*>(smem_raw);
+    Partial* stage = reinterpret_cast<Partial*>(smem_raw + MERGE_RING_BYTES);            // [GT][WARPS]
+    uint4* sg = reinterpret_cast<uint4*>(smem_raw + MERGE_RING_BYTES + MERGE_GT * MERGE_WARPS * 16);
+    const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
+
+    uint64_t base[MERGE_R], Wp[MERGE_R], nextW[MERGE_R], curKey[MERGE_R];
+    uint32_t n[MERGE_R], Dp[MERGE_R], ready[MERGE_R], factor[MERGE_R], w[MERGE_R], nextD[MERGE_R], nextM[MERGE_R];
+    uint4* ring[MERGE_R];
+    uint32_t ring_s[MERGE_R];
+    const uint32_t job0 = blockIdx.x * MERGE_JOBS + wid * MERGE_R * 32;   // first job of this warp
+#pragma unroll
+    for (int r = 0; r < MERGE_R; ++r) {
+        const uint32_t j = job0 + r * 32 + lane;
+        ring[r] = ring_all + (size_t)(wid * MERGE_R + r) * MERGE_RING * 32 + lane;
+        ring_s[r] = (uint32_t)__cvta_generic_to_shared(ring[r]);
+        base[r] = 0; Wp[r] = 0; nextW[r] = 0; curKey[r] = 0;
+        n[r] = 0; Dp[r] = 0; ready[r] = 0; factor[r] = 0; w[r] = 0; nextD[r] = 0; nextM[r] = 0;
+        if (j < jv.J) {
+            const uint64_t b0 = jv.boff[j], b1 = jv.boff[j + 1];
+            const uint32_t pb = jv.pb[j];
+            base[r] = b0 + pb;
+            n[r] = (uint32_t)(b1 - b0) - pb;
+            Dp[r] = jv.Dp[j];
+            Wp[r] = jv.Wp[j];
+            ready[r] = jv.ready[j];
+            factor[r] = policy_factor(jv, kind, j);
+        }
+    }
+    const uint32_t g_begin = blockIdx.y * gaps_per_split;
+    const uint32_t g_end = min(G, g_begin + gaps_per_split);
+    bool first = true;
+    uint32_t curC = 0;
+
+    for (uint32_t g0 = g_begin; g0 < g_end; g0 += MERGE_GT) {
+        const uint32_t gt = min((uint32_t)MERGE_GT, g_end - g0);
+        if (threadIdx.x < gt) sg[threadIdx.x] = __ldg(reinterpret_cast<const uint4*>(sgaps) + g0 + threadIdx.x);
+        __syncthreads();
+        for (uint32_t gi = 0; gi < gt; ++gi) {
+            const uint4 gq = sg[gi];
+            const uint32_t start = gq.y, T = gq.z, C = gq.w;
+            if (first || C != curC) {
+                // new capacity class: T restarts from its smallest value, so do the cursors
+                first = false;
+                curC = C;
+                mg_wait<0>();
+#pragma unroll
+                for (int r = 0; r < MERGE_R; ++r) {
+                    w[r] = 0;
+                    curKey[r] = 0;
+#pragma unroll
+                    for (int i = 0; i < MERGE_RING; ++i) {
+                        if ((uint32_t)i < n[r]) mg_cp_async16(ring_s[r] + i * 32 * 16, jv.A + base[r] + i);
+                        mg_commit();
+                    }
+                }
+                mg_wait<0>();
+#pragma unroll
+                for (int r = 0; r < MERGE_R; ++r) {
+                    if (n[r]) {
+                        const uint4 row = ring[r][0];
+                        nextD[r] = row.x - Dp[r];
+                        nextM[r] = row.y;
+                        nextW[r] = pack64(row.z, row.w);
+                    }
+                }
+            }
+            uint64_t best = 0;
+            uint32_t best_slot = 0, best_cnt = 0;
+#pragma unroll
+            for (int r = 0; r < MERGE_R; ++r) {
+                while (w[r] < n[r] && nextD[r] <= T && nextM[r] <= C) {
+                    curKey[r] = policy_key(kind, nextW[r] - Wp[r], factor[r]);
+                    if (w[r] + MERGE_RING < n[r])
+                        mg_cp_async16(ring_s[r] + (w[r] % MERGE_RING) * 32 * 16, jv.A + base[r] + w[r] + MERGE_RING);
+                    mg_commit();
+                    ++w[r];
+                    if (w[r] < n[r]) {
+                        mg_wait<MERGE_RING - 1>();
+                        const uint4 row = ring[r][(w[r] % MERGE_RING) * 32];
+                        nextD[r] = row.x - Dp[r];
+                        nextM[r] = row.y;
+                        nextW[r] = pack64(row.z, row.w);
+                    }
+                }
+                const uint64_t k = (start >= ready[r]) ? curKey[r] : 0ull;
+                if (k > best) { best = k; best_slot = (uint32_t)r * 32u + lane; best_cnt = w[r]; }
+            }
+            const uint64_t mk = warp_max_u64(best);
+            const uint32_t smin = __reduce_min_sync(0xFFFFFFFFu, (best == mk && mk != 0ull) ? best_slot : 0xFFFFFFFFu);
+            const uint32_t wcnt = __shfl_sync(0xFFFFFFFFu, best_cnt, smin & 31u);
+            if (lane == 0) {
+                Partial pr;
+                pr.key = mk;
+                pr.job = mk ? job0 + smin : 0xFFFFFFFFu;
+                pr.cnt = mk ? wcnt : 0u;
+                stage[gi * MERGE_WARPS + wid] = pr;
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x < gt) {
+            Partial bestp = stage[threadIdx.x * MERGE_WARPS];
+#pragma unroll
+            for (int ww = 1; ww < MERGE_WARPS; ++ww) {
+                const Partial c = stage[threadIdx.x * MERGE_WARPS + ww];
+                if (c.key > bestp.key || (c.key == bestp.key && c.job < bestp.job)) bestp = c;
+            }
+            partial_out[(size_t)blockIdx.x * G + g0 + threadIdx.x] = bestp;
+        }
+        __syncthreads();
+    }
+    mg_wait<0>();
 }
 
 }  // namespace sja
