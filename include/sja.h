@@ -156,6 +156,35 @@ sja_status sja_advertise(sja_ctx* ctx, uint32_t G, const sja_gap* gaps, sja_mems
 sja_status sja_select(sja_ctx* ctx, const sja_policy* policy, sja_award* out, sja_memspace where);
 
 /*
+ * sja_select for callers that must not allocate.  (The paper has no counterpart: this is
+ * a deployment variant of the call above, with identical results.)
+ *
+ * Who needs it: a scheduler loop that runs where device allocation is off limits -- for
+ * instance a service that handed all device memory to its own pool at start-up, so a
+ * cudaMalloc from a library would fail or fragment it, or a latency-bound control loop that
+ * cannot afford the device-wide synchronisation an allocation or free implies.  sja_select
+ * grows a context buffer for its per-CTA candidate rows whenever a larger job or gap count
+ * comes along; this call instead keeps those rows in a fixed array of
+ * SJA_STATIC_SCRATCH_BYTES that is part of the library image.  It calls no cudaMalloc,
+ * cudaFree or other allocating routine and records no profiling events.
+ *
+ * Cost and limit: every GPU on which the library is used holds the array until the process
+ * exits.  The call needs ceil(J / 512) * G candidate slots of 16 bytes (ceil(J / 256) * G
+ * with SJA_FLAG_FORCE_SEARCH or an unsorted / many-capacity batch); if that exceeds the
+ * array it returns SJA_ERR_INVALID_ARG with the numbers in sja_last_error() and does nothing.
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
+ * the context's device current); make that first call before starting any stream capture.
+ * All contexts and all calls on one device share the one array.  It keeps whatever the last
+ * call left in it; this call overwrites every slot it later reads, so no clearing is needed,
+ * but two calls that overlap on the GPU (different streams or contexts on the same device)
+ * race on it: serialise them.  Arguments, outputs, state rules and errors are otherwise those
+ * of sja_select, and sja_commit / sja_get_awards follow it in the same way.
+ */
+#define SJA_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+sja_status sja_select_static(sja_ctx* ctx, const sja_policy* policy, sja_award* out, sja_memspace where);
+
+/*
  * Grant (Section 3.5: only the selected job materialises its subjob; Sections 3.1, 3.5:
  * the parent job later resumes from the end of the fragment).  Resolves jobs that won
  * several gaps, advances progress and ready time of the granted jobs, refreshes their

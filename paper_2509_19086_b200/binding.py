@@ -28,7 +28,7 @@ AWARD_DTYPE = np.dtype([("job", "<u4"), ("end_step", "<u4"), ("dur_ms", "<u4"), 
                         ("score", "<u8")])
 
 EXPORTS = [
-    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_commit",
+    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit",
     "sja_get_awards", "sja_get_state", "sja_scan_size", "sja_get_scan", "sja_profile_enable",
     "sja_profile_read", "sja_last_error",
 ]
@@ -72,6 +72,7 @@ def load_library() -> ctypes.CDLL:
     lib.sja_load_profiles.argtypes = [vp, u32, vp, vp, vp, vp, vp, vp, vp, vp, i32]
     lib.sja_advertise.argtypes = [vp, u32, vp, i32]
     lib.sja_select.argtypes = [vp, ctypes.POINTER(SjaPolicy), vp, i32]
+    lib.sja_select_static.argtypes = [vp, ctypes.POINTER(SjaPolicy), vp, i32]
     lib.sja_commit.argtypes = [vp, ctypes.POINTER(u32)]
     lib.sja_get_awards.argtypes = [vp, vp, i32]
     lib.sja_get_state.argtypes = [vp, vp, vp, i32]
@@ -188,6 +189,22 @@ class Sja:
             return arr
         p, space, _ = _ptr_space(out, None)
         self._check(self._lib.sja_select(self._h, ctypes.byref(pol), p, space))
+        return out
+
+    # -- sja_select_static
+    def select_static(self, policy: int, flags: int = 0, out=None):
+        """sja_select_static: same arguments and results as :meth:`select`, but the library
+        allocates nothing on this path (fixed scratch; sizes beyond it raise SjaError)."""
+        pol = SjaPolicy(int(policy), int(flags))
+        if out is None:
+            self._check(self._lib.sja_select_static(self._h, ctypes.byref(pol), None, MEM_HOST))
+            return None
+        if isinstance(out, str):
+            arr = np.empty(self.n_gaps, dtype=AWARD_DTYPE)
+            self._check(self._lib.sja_select_static(self._h, ctypes.byref(pol), arr.ctypes.data, MEM_HOST))
+            return arr
+        p, space, _ = _ptr_space(out, None)
+        self._check(self._lib.sja_select_static(self._h, ctypes.byref(pol), p, space))
         return out
 
     # -- sja_commit

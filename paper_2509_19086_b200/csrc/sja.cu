@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <new>
 #include <utility>
 #include <vector>
@@ -238,6 +239,39 @@ __global__ void export_rows_kernel(const uint4* __restrict__ A, const uint2* __r
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------
+// Fixed scratch for sja_select_static: the per-CTA candidate rows of one select call.
+// It is part of the loaded module, so every GPU that loads this library holds these bytes
+// until the process exits.  In host code the name below is only a handle for the runtime,
+// never a device address; the address is looked up once per device by static_scratch_for().
+static __device__ __align__(256) unsigned char g_select_scratch[SJA_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int STATIC_MAX_DEVICES = 64;
+void* g_scratch_addr[STATIC_MAX_DEVICES] = {nullptr};
+std::mutex g_scratch_mutex;   // contexts on different host threads may reach the set-up together
+
+// Device address of g_select_scratch on `device`, which must be the current device.
+// The first call per device asks the runtime (this loads the module on that device);
+// later calls return the cached pointer.
+sja_status static_scratch_for(sja_ctx* c, int device, Partial** out) {
+    if (device < 0 || device >= STATIC_MAX_DEVICES)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_select_static: device index %d not supported", device);
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_addr[device]) {
+        void* ptr = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&ptr, g_select_scratch);
+        if (e != cudaSuccess) return cuda_fail(c, e, "cudaGetSymbolAddress(g_select_scratch)");
+        if (!ptr) return fail(c, SJA_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
+        g_scratch_addr[device] = ptr;
+    }
+    *out = static_cast<Partial*>(g_scratch_addr[device]);
+    return SJA_OK;
+}
 
 }  // namespace
 
@@ -549,6 +583,76 @@ sja_status sja_select(sja_ctx* c, const sja_policy* policy, sja_award* out, sja_
                                                                          c->awards.as<Award>(),
                                                                          c->widx.as<uint32_t>());
     }
+    CU(cudaGetLastError());
+    c->selected = true;
+    c->committed = false;
+    c->last_policy = kind;
+    if (out) {
+        TRY(copy_out(c, out, c->awards.p, (size_t)G * sizeof(sja_award), where));
+        if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));
+    }
+    return SJA_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// Same work as sja_select, but the candidate rows go to the module's fixed scratch array
+// instead of a context buffer, so no allocation can happen on this path: no cudaMalloc,
+// no cudaFree, no event creation (kernel timing is therefore not recorded here).
+sja_status sja_select_static(sja_ctx* c, const sja_policy* policy, sja_award* out, sja_memspace where) {
+    TRY(check_ctx(c));
+    if (!policy) return fail(c, SJA_ERR_INVALID_ARG, "sja_select_static: policy is NULL");
+    if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_select_static: bad memspace");
+    const uint32_t kind = policy->kind;
+    if (kind > SJA_POLICY_SLA) return fail(c, SJA_ERR_INVALID_ARG, "sja_select_static: unknown policy %u", kind);
+    if (!c->loaded || !c->advertised) return fail(c, SJA_ERR_STATE, "sja_select_static before load / advertise");
+    if (kind == SJA_POLICY_FAIRNESS && !c->have_wait)
+        return fail(c, SJA_ERR_INVALID_ARG, "fairness policy needs wait_ms at load");
+    if (kind == SJA_POLICY_SLA && !c->have_prio) return fail(c, SJA_ERR_INVALID_ARG, "SLA policy needs prio at load");
+    if (kind == SJA_POLICY_FAIRNESS && (c->load_flags & FLAG_OVF_FAIR))
+        return fail(c, SJA_ERR_OVERFLOW, "fairness score may reach 2^63 for some job");
+    if (kind == SJA_POLICY_SLA && (c->load_flags & FLAG_OVF_SLA))
+        return fail(c, SJA_ERR_OVERFLOW, "SLA key needs work < 2^55 for every job");
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
+
+    const uint32_t G = c->G, J = c->J;
+    const bool use_merge = !(policy->flags & SJA_FLAG_FORCE_SEARCH) && c->gaps_sorted &&
+                           c->n_classes <= std::max<uint32_t>(64u, G / 16u);
+    const uint32_t jobs_per_cta = use_merge ? (uint32_t)MERGE_JOBS : (uint32_t)SEARCH_THREADS;
+    const uint32_t tile = use_merge ? (uint32_t)MERGE_GT : (uint32_t)SEARCH_GT;
+    const uint32_t n_chunks = (J + jobs_per_cta - 1) / jobs_per_cta;
+    const uint64_t need = (uint64_t)n_chunks * G;   // candidate slots: one per (CTA job chunk, gap)
+    const uint64_t have = (uint64_t)SJA_STATIC_SCRATCH_BYTES / sizeof(Partial);
+    if (need > have)
+        return fail(c, SJA_ERR_INVALID_ARG,
+                    "sja_select_static: %u jobs x %u gaps need %llu candidate slots (ceil(J/%u) x G), the fixed "
+                    "scratch holds %llu; use sja_select for this size",
+                    J, G, (unsigned long long)need, jobs_per_cta, (unsigned long long)have);
+    Partial* scratch = nullptr;
+    TRY(static_scratch_for(c, c->device, &scratch));
+
+    uint32_t splits = (uint32_t)((8ull * c->n_sm + n_chunks - 1) / n_chunks);
+    const uint32_t max_splits = (G + tile - 1) / tile;
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    uint32_t per_split = (G + splits - 1) / splits;
+    per_split = ((per_split + tile - 1) / tile) * tile;
+    splits = (G + per_split - 1) / per_split;
+    // Every slot that finalize_awards_kernel reads is written by the select kernel of this
+    // same call (all chunks x all gaps), so nothing left over from an earlier call is ever
+    // read and nothing has to be cleared first.
+    const JobView jv = job_view(c);
+    if (use_merge) {
+        select_merge_kernel<<<dim3(n_chunks, splits), MERGE_WARPS * 32, MERGE_SMEM_BYTES, c->stream>>>(
+            jv, c->sgaps.as<Gap>(), G, per_split, kind, scratch);
+    } else {
+        select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, 0, c->stream>>>(
+            jv, c->sgaps.as<Gap>(), G, per_split, kind, nullptr, 0, scratch);
+    }
+    finalize_awards_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(jv, scratch, n_chunks, c->sgaps.as<Gap>(), G,
+                                                                     kind, c->awards.as<Award>(),
+                                                                     c->widx.as<uint32_t>());
     CU(cudaGetLastError());
     c->selected = true;
     c->committed = false;
