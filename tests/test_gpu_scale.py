@@ -1,0 +1,151 @@
+"""Full-size published configurations on the GPU, in the launch configuration bench.py times.
+
+Where the oracle finishes in seconds the comparison is complete; elsewhere it covers sampled
+gaps / the first rounds bit-exactly and everything else through properties that hold at any
+size (every award re-derived from the raw arrays: fits T, ends on a boundary, state tiling).
+No expected value comes from the CUDA path: the oracle always runs from its own state.
+"""
+import numpy as np
+import pytest
+
+from paper_2509_19086_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+U32MAX = 0xFFFFFFFF
+FIELDS = ("job", "end_step", "dur_ms", "score")
+
+
+def _load(ctx, prof):
+    ctx.load_profiles(prof.off, prof.dur_ms, prof.mem_MiB, prof.safe_bits, prof.ready_ms,
+                      wait_ms=prof.wait_ms, prio=prof.prio)
+
+
+def _assert_equal(got, want, fields=FIELDS):
+    for f in fields:
+        bad = np.nonzero(got[f] != want[f])[0]
+        assert bad.size == 0, (f, bad[:5], got[bad[:5]], want[bad[:5]])
+
+
+def test_cfg2_large_uniform_all_awards(oracle_mod):
+    """65 536 jobs x 4096 steps, 4096 gaps, fairness: every award against the oracle."""
+    from paper_2509_19086_b200 import binding
+    spec = wl.SPECS[2]
+    prof = wl.make_profiles(spec, threads=16)
+    gaps = wl.make_gaps(spec)
+    with binding.Sja() as ctx:
+        _load(ctx, prof)
+        safe = wl.unpack_safe_bits(prof.safe_bits, prof.n_steps)
+        assert ctx.scan_size() == int(safe.sum())
+        ctx.advertise(gaps)
+        got = ctx.select(spec.policy, out="host")
+        progress = np.zeros(prof.n_jobs, np.uint32)
+        ready = prof.ready_ms.copy()
+        want = oracle_mod.select(prof, progress, ready, gaps, spec.policy)
+        _assert_equal(got, want)
+        n_gpu = ctx.commit()
+        n_cpu = oracle_mod.commit(progress, ready, gaps, want)
+        assert n_gpu == n_cpu > 0
+        _assert_equal(ctx.get_awards(), want, FIELDS + ("granted",))
+        p, r = ctx.get_state()
+        assert np.array_equal(p, progress) and np.array_equal(r, ready)
+        # the per-pair search kernel on a sample of the gaps
+        sub = gaps[::16]
+        ctx.advertise(sub)
+        got = ctx.select(spec.policy, flags=binding.FLAG_FORCE_SEARCH, out="host")
+        want = oracle_mod.select(prof, progress, ready, sub, spec.policy)
+        _assert_equal(got, want)
+
+
+def test_cfg3_heavy_tailed_sampled_gaps(oracle_mod):
+    """262 144 ragged jobs (about 1e9 steps), 16 384 gaps, SLA: all gaps on the GPU, 4096
+    sampled gaps x all jobs against the oracle, structural checks on every award."""
+    from paper_2509_19086_b200 import binding
+    spec = wl.SPECS[3]
+    prof = wl.make_profiles(spec, threads=16)
+    gaps = wl.make_gaps(spec)
+    assert 0.8e9 < prof.n_steps < 1.2e9
+    with binding.Sja() as ctx:
+        _load(ctx, prof)
+        ctx.advertise(gaps)
+        got = ctx.select(spec.policy, out="host")
+        progress = np.zeros(prof.n_jobs, np.uint32)
+        rng = np.random.default_rng(33)
+        sample = np.sort(rng.choice(gaps.shape[0], 4096, replace=False))
+        want = oracle_mod.select(prof, progress, prof.ready_ms, gaps[sample], spec.policy)
+        _assert_equal(got[sample], want)
+        # every award: winner eligible, subjob inside the job, ends on a boundary, fits T
+        win = got["job"] != U32MAX
+        assert win.mean() > 0.9
+        j = got["job"][win].astype(np.int64)
+        k = got["end_step"][win].astype(np.int64)
+        lens = np.diff(prof.off).astype(np.int64)
+        assert (k >= 1).all() and (k <= lens[j]).all()
+        last = prof.off[j].astype(np.int64) + k - 1
+        bit = (prof.safe_bits[last >> 5] >> (last & 31).astype(np.uint32)) & 1
+        assert ((bit == 1) | (k == lens[j])).all()
+        assert (got["dur_ms"][win] <= gaps["T_ms"][win]).all()
+        assert (gaps["start_ms"][win] >= prof.ready_ms[j]).all()
+        # SLA: the winner's class is the highest class among the sampled oracle winners' gaps
+        assert (prof.prio[j] == 2).mean() > 0.9
+        n = ctx.commit()
+        aw = ctx.get_awards()
+        granted = aw["job"][aw["granted"] == 1]
+        assert n == granted.size == np.unique(granted).size
+        assert set(np.unique(aw["job"][win]).tolist()) == set(granted.tolist())
+
+
+def test_cfg4_streaming_1000_rounds(oracle_mod):
+    """100 000 jobs x 2048 steps, 1000 rounds of 8192 gaps.  Rounds 0-2 bit-exact against
+    the oracle (awards, grants, state); all 1000 rounds through replay properties."""
+    from paper_2509_19086_b200 import binding
+    spec = wl.SPECS[4]
+    prof = wl.make_profiles(spec, threads=16)
+    J = prof.n_jobs
+    off = prof.off.astype(np.int64)
+    cum_d = np.zeros(prof.n_steps + 1, dtype=np.int64)
+    np.cumsum(prof.dur_ms, out=cum_d[1:])
+    o_progress = np.zeros(J, np.uint32)
+    o_ready = prof.ready_ms.copy()
+    replay_p = np.zeros(J, np.int64)
+    replay_r = prof.ready_ms.astype(np.int64)
+    total = 0
+    with binding.Sja() as ctx:
+        _load(ctx, prof)
+        for r in range(spec.n_rounds):
+            gaps = wl.make_gaps(spec, r)
+            ctx.advertise(gaps)
+            ctx.select(spec.policy)
+            n = ctx.commit()
+            aw = ctx.get_awards()
+            if r < 3:
+                want = oracle_mod.select(prof, o_progress, o_ready, gaps, spec.policy)
+                n_cpu = oracle_mod.commit(o_progress, o_ready, gaps, want)
+                _assert_equal(aw, want, FIELDS + ("granted",))
+                assert n == n_cpu
+                p, rd = ctx.get_state()
+                assert np.array_equal(p, o_progress) and np.array_equal(rd, o_ready)
+            # replay properties on this round's grants
+            g = np.nonzero(aw["granted"] == 1)[0]
+            assert g.size == n
+            j = aw["job"][g].astype(np.int64)
+            k = aw["end_step"][g].astype(np.int64)
+            assert np.unique(j).size == j.size                       # one grant per job and round
+            assert (k > replay_p[j]).all() and (k <= 2048).all()     # progress moves forward
+            dur = cum_d[off[j] + k] - cum_d[off[j] + replay_p[j]]
+            assert (dur == aw["dur_ms"][g]).all()                    # subjob starts at the job's progress
+            assert (dur <= gaps["T_ms"][g]).all()
+            assert (gaps["start_ms"][g] >= replay_r[j]).all()
+            last = off[j] + k - 1
+            bit = (prof.safe_bits[last >> 5] >> (last & 31).astype(np.uint32)) & 1
+            assert ((bit == 1) | (k == 2048)).all()                  # every cut is a safe boundary
+            winners = np.unique(aw["job"][aw["job"] != U32MAX])
+            assert np.array_equal(winners, np.sort(j))               # every winning job gets exactly one gap
+            replay_p[j] = k
+            replay_r[j] = gaps["start_ms"][g].astype(np.int64) + dur
+            total += n
+        p, rd = ctx.get_state()
+        assert np.array_equal(p.astype(np.int64), replay_p)
+        assert np.array_equal(rd.astype(np.int64), replay_r)
+        print("cfg4 grants over 1000 rounds:", total)
+        assert total > 50_000
