@@ -147,6 +147,18 @@ __global__ void __launch_bounds__(1024) row_offsets_kernel(const uint32_t* __res
 
 // ---------------------------------------------------------------------------------------
 // The scan proper.
+//
+// Per 512-step block a warp knows, after one popcount scan, how many rows the block emits.
+// Usual case (at most SCAN_STAGE_ROWS rows): each lane walks its 16 steps ONCE, keeping
+// lane-local sums, and drops a lane-relative row into shared memory at every safe bit (the
+// just-consumed input slot of the ring is reused as the row buffer).  The warp then scans the
+// 32 lane totals and a second, row-indexed phase (32 rows per iteration, i.e. about a tenth of
+// the steps) adds each row's lane offset, derives the running maximum as a prefix maximum over
+// the rows' segment maxima, and writes the finished rows with fully coalesced 512-byte and
+// 256-byte stores.  Blocks with more rows (boundaries denser than one in three steps) take
+// the two-pass route: lane totals first, then a second walk that stores rows directly.
+constexpr int SCAN_STAGE_ROWS = 168;   // 168 * 24 B = 4032 B <= the 4096 B of a consumed d+m slot
+
 __global__ void __launch_bounds__(SCAN_WARPS * 32) scan_profiles_kernel(ScanArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t lane = threadIdx.x & 31u;
@@ -201,7 +213,7 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32) scan_profiles_kernel(ScanArgs
         uint64_t tot64 = 0;      // exact cumulative duration (overflow check)
         uint64_t carryW = 0;     // cumulative work
         uint32_t carrySeg = 0;   // max m since the last boundary
-        uint32_t carryRun = 0;   // max m since the progress point
+        uint32_t carryRun = 0;   // max m over all finished segments since the progress point
         uint32_t outpos = 0;     // rows written so far
 
 #pragma unroll
@@ -212,7 +224,7 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32) scan_profiles_kernel(ScanArgs
             cp_async_wait<SCAN_STAGES - 1>();
             __syncwarp();
 
-            const unsigned char* st = wbase + (size_t)(t % SCAN_STAGES) * SCAN_STAGE_BYTES;
+            unsigned char* st = wbase + (size_t)(t % SCAN_STAGES) * SCAN_STAGE_BYTES;
             const uint4* sd = reinterpret_cast<const uint4*>(st);
             const uint4* sm = reinterpret_cast<const uint4*>(st + 2048);
             const uint32_t* ss = reinterpret_cast<const uint32_t*>(st + 4096);
@@ -226,7 +238,7 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32) scan_profiles_kernel(ScanArgs
                 mv[4 * r + 0] = qm.x; mv[4 * r + 1] = qm.y; mv[4 * r + 2] = qm.z; mv[4 * r + 3] = qm.w;
             }
             uint32_t bits = (ss[lane >> 1] >> ((lane & 1u) * 16u)) & 0xFFFFu;
-            __syncwarp();  // every lane has read the slot; a later issue may overwrite it
+            __syncwarp();  // every lane has read the slot: it may now be reused as the row buffer
 
             const uint64_t bs = blk0 + t * SCAN_BLK;
             const uint64_t lane_base = bs + 16ull * lane;
@@ -234,7 +246,7 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32) scan_profiles_kernel(ScanArgs
             uint32_t lo = 0, hi = 16;
             if (s > lane_base) lo = (s - lane_base) >= 16 ? 16u : (uint32_t)(s - lane_base);
             if (e < lane_base + 16) hi = (e <= lane_base) ? 0u : (uint32_t)(e - lane_base);
-            uint32_t vm = (hi > lo) ? (((1u << hi) - 1u) & ~((1u << lo) - 1u)) : 0u;
+            const uint32_t vm = (hi > lo) ? (((1u << hi) - 1u) & ~((1u << lo) - 1u)) : 0u;
             if (vm != 0xFFFFu) {
 #pragma unroll
                 for (int i = 0; i < 16; ++i)
@@ -242,42 +254,72 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32) scan_profiles_kernel(ScanArgs
             }
             bits &= vm;
             if (e - 1 >= lane_base && e - 1 < lane_base + 16) bits |= 1u << (uint32_t)(e - 1 - lane_base);
+            const uint32_t k0 = (uint32_t)(lane_base - js);   // steps of the job before this lane
 
-            // ---- lane-local aggregates
-            uint64_t td = 0, tw = 0;
-            uint32_t lmax = 0, tail = 0;
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                td += dv[i];
-                tw += (uint64_t)dv[i] * (uint64_t)mv[i];
-                lmax = max(lmax, mv[i]);
-                tail = max(tail, mv[i]);
-                if ((bits >> i) & 1u) tail = 0;
-            }
+            // rows of this block: exclusive count per lane, total
             const uint32_t cnt = __popc(bits);
-
-            // ---- warp combine
-            // exact block duration (lane sums < 2^36): two 32-bit reductions
-            const uint32_t sum_lo = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)(td & 0xFFFFu));
-            const uint32_t sum_hi = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)(td >> 16));
-            const uint64_t blockD = ((uint64_t)sum_hi << 16) + sum_lo;
-
-            uint32_t incD = (uint32_t)td;
-            uint64_t incW = tw;
             uint32_t incC = cnt;
-            uint32_t incR = lmax;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t yc = __shfl_up_sync(0xFFFFFFFFu, incC, o);
+                if (lane >= (uint32_t)o) incC += yc;
+            }
+            const uint32_t c_total = __shfl_sync(0xFFFFFFFFu, incC, 31);
+            const bool staged = c_total <= (uint32_t)SCAN_STAGE_ROWS;   // warp-uniform
+
+            uint4* rowA = reinterpret_cast<uint4*>(st);
+            uint2* rowB = reinterpret_cast<uint2*>(st + 16 * SCAN_STAGE_ROWS);
+
+            // ---- walk the 16 steps: lane totals, and (staged route) lane-relative rows
+            uint32_t td = 0, tail = 0, orv = 0;
+            uint64_t tw = 0;
+            if (staged) {
+                uint32_t lpos = incC - cnt;
+                uint32_t meta = lane | 256u;   // bit 8: first row of this lane (takes the carried-in segment)
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    td += dv[i];
+                    tw += (uint64_t)dv[i] * (uint64_t)mv[i];
+                    tail = max(tail, mv[i]);
+                    orv |= dv[i];
+                    if ((bits >> i) & 1u) {
+                        rowA[lpos] = make_uint4(td, meta, (uint32_t)tw, (uint32_t)(tw >> 32));
+                        rowB[lpos] = make_uint2(k0 + (uint32_t)i + 1u, tail);
+                        ++lpos;
+                        tail = 0;
+                        meta = lane;
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    td += dv[i];
+                    tw += (uint64_t)dv[i] * (uint64_t)mv[i];
+                    tail = max(tail, mv[i]);
+                    orv |= dv[i];
+                    if ((bits >> i) & 1u) tail = 0;
+                }
+            }
+
+            // ---- warp combine of the lane totals
+            uint32_t incD = td;
+            uint64_t incW = tw;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const uint32_t yd = __shfl_up_sync(0xFFFFFFFFu, incD, o);
                 const uint64_t yw = __shfl_up_sync(0xFFFFFFFFu, incW, o);
-                const uint32_t yc = __shfl_up_sync(0xFFFFFFFFu, incC, o);
-                const uint32_t yr = __shfl_up_sync(0xFFFFFFFFu, incR, o);
-                if (lane >= (uint32_t)o) {
-                    incD += yd;
-                    incW += yw;
-                    incC += yc;
-                    incR = max(incR, yr);
-                }
+                if (lane >= (uint32_t)o) { incD += yd; incW += yw; }
+            }
+            // exact block duration for the overflow check.  If every d < 2^22 the 32-bit block
+            // sum cannot wrap (512 * 2^22 = 2^31); otherwise sum the lanes exactly in 64 bits.
+            uint64_t blockD = __shfl_sync(0xFFFFFFFFu, incD, 31);
+            if (__reduce_or_sync(0xFFFFFFFFu, orv) >= (1u << 22)) {
+                uint64_t t64 = 0;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) t64 += dv[i];
+                const uint32_t sum_lo = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)(t64 & 0xFFFFu));
+                const uint32_t sum_hi = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)(t64 >> 16));
+                blockD = ((uint64_t)sum_hi << 16) + sum_lo;
             }
             // segmented max of the lane tails: a lane with a safe bit starts a new segment
             const uint32_t hm = __ballot_sync(0xFFFFFFFFu, bits != 0u);
@@ -293,39 +335,85 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32) scan_profiles_kernel(ScanArgs
             const bool none_before = (hm & ((1u << lane) - 1u)) == 0u;   // no boundary in lanes < lane
             if (lane == 0) seg_in = carrySeg;
             else if (none_before) seg_in = max(seg_in, carrySeg);
-            uint32_t run_in = __shfl_up_sync(0xFFFFFFFFu, incR, 1);
-            run_in = (lane == 0) ? carryRun : max(run_in, carryRun);
+            const uint32_t baseD = carryD + (incD - td);     // duration before this lane's first step
+            const uint64_t baseW = carryW + (incW - tw);
+            const uint64_t out0 = out_base + outpos;
 
-            // ---- emit rows at this lane's safe bits
-            uint32_t D = carryD + (incD - (uint32_t)td);
-            uint64_t W = carryW + (incW - tw);
-            uint32_t seg = seg_in, run = run_in;
-            uint64_t pos = out_base + outpos + (incC - cnt);
-            const uint32_t k0 = (uint32_t)(lane_base - js);   // steps before this lane (may wrap if masked)
+            if (staged) {
+                __syncwarp();   // all lanes' rows are in the buffer
+                uint32_t runc = carryRun;
+                for (uint32_t rb = 0; rb < c_total; rb += 32) {
+                    const uint32_t idx = rb + lane;
+                    const bool ok = idx < c_total;
+                    uint4 ra = make_uint4(0, 0, 0, 0);
+                    uint2 rbv = make_uint2(0, 0);
+                    if (ok) { ra = rowA[idx]; rbv = rowB[idx]; }
+                    const uint32_t src = ra.y & 31u;
+                    const uint32_t sD = __shfl_sync(0xFFFFFFFFu, baseD, src);
+                    const uint64_t sW = __shfl_sync(0xFFFFFFFFu, baseW, src);
+                    const uint32_t sS = __shfl_sync(0xFFFFFFFFu, seg_in, src);
+                    const uint32_t segr = (ra.y & 256u) ? max(rbv.y, sS) : rbv.y;
+                    uint32_t v = ok ? segr : 0u;      // running max = prefix max over the rows' segment maxima
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                D += dv[i];
-                W += (uint64_t)dv[i] * (uint64_t)mv[i];
-                seg = max(seg, mv[i]);
-                run = max(run, mv[i]);
-                if ((bits >> i) & 1u) {
-                    if (pos < out_end) {
-                        a.A[pos] = make_uint4(D, run, (uint32_t)W, (uint32_t)(W >> 32));
-                        a.B[pos] = make_uint2(k0 + (uint32_t)i + 1u, seg);
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, v, o);
+                        if (lane >= (uint32_t)o) v = max(v, y);
                     }
-                    ++pos;
-                    seg = 0;
+                    v = max(v, runc);
+                    const uint64_t W = pack64(ra.z, ra.w) + sW;
+                    const uint64_t pos = out0 + idx;
+                    if (ok && pos < out_end) {
+                        a.A[pos] = make_uint4(ra.x + sD, v, (uint32_t)W, (uint32_t)(W >> 32));
+                        a.B[pos] = make_uint2(rbv.x, segr);
+                    }
+                    runc = __shfl_sync(0xFFFFFFFFu, v, 31);
                 }
+                carryRun = runc;
+            } else {
+                // two-pass route: per-lane running maximum needs the exclusive prefix max of the
+                // lane maxima (everything before this lane counts, finished segment or not)
+                uint32_t lmax = 0;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) lmax = max(lmax, mv[i]);
+                uint32_t incR = lmax;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t yr = __shfl_up_sync(0xFFFFFFFFu, incR, o);
+                    if (lane >= (uint32_t)o) incR = max(incR, yr);
+                }
+                const uint32_t before = max(carryRun, carrySeg);
+                uint32_t run = __shfl_up_sync(0xFFFFFFFFu, incR, 1);
+                run = (lane == 0) ? before : max(run, before);
+                uint32_t D = baseD;
+                uint64_t W = baseW;
+                uint32_t seg = seg_in;
+                uint64_t pos = out0 + (incC - cnt);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    D += dv[i];
+                    W += (uint64_t)dv[i] * (uint64_t)mv[i];
+                    seg = max(seg, mv[i]);
+                    run = max(run, mv[i]);
+                    if ((bits >> i) & 1u) {
+                        if (pos < out_end) {
+                            a.A[pos] = make_uint4(D, run, (uint32_t)W, (uint32_t)(W >> 32));
+                            a.B[pos] = make_uint2(k0 + (uint32_t)i + 1u, seg);
+                        }
+                        ++pos;
+                        seg = 0;
+                    }
+                }
+                carryRun = max(before, __shfl_sync(0xFFFFFFFFu, incR, 31));
             }
 
             // ---- carries for the next block
             carryD += __shfl_sync(0xFFFFFFFFu, incD, 31);
             carryW += __shfl_sync(0xFFFFFFFFu, incW, 31);
-            outpos += __shfl_sync(0xFFFFFFFFu, incC, 31);
-            carryRun = max(carryRun, __shfl_sync(0xFFFFFFFFu, incR, 31));
+            outpos += c_total;
             const uint32_t x31 = __shfl_sync(0xFFFFFFFFu, x, 31);
             carrySeg = hm ? x31 : max(x31, carrySeg);
             tot64 += blockD;
+            __syncwarp();   // the row buffer is read out before the next copies land in this slot
         }
 
         if (lane == 0) {
