@@ -32,7 +32,8 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         return LIB_PATH
     nvcc = os.environ.get("NVCC", "nvcc")
     tmp = LIB_PATH + f".tmp{os.getpid()}"
-    cmd = [nvcc] + NVCC_FLAGS + ["-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
+    extra = os.environ.get("SJA_NVCC_EXTRA", "").split()     # e.g. -DSJA_SCAN_STAGES=2 for tuning sweeps
+    cmd = [nvcc] + NVCC_FLAGS + extra + ["-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)

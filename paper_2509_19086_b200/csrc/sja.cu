@@ -478,7 +478,7 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
     a.flags = c->flags.as<uint32_t>();
     if (N > 0) {
         ProfScope ps(c, CAT_SCAN);
-        const uint32_t ctas_per_sm = 2;
+        const uint32_t ctas_per_sm = SCAN_CTAS_PER_SM;
         const uint32_t want = (J + SCAN_WARPS - 1) / SCAN_WARPS;
         const uint32_t grid = std::min<uint32_t>(want, (uint32_t)c->n_sm * ctas_per_sm);
         scan_profiles_kernel<<<grid, SCAN_WARPS * 32, SCAN_SMEM_BYTES, c->stream>>>(a);

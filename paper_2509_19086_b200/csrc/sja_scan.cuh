@@ -16,9 +16,19 @@
 
 namespace sja {
 
-constexpr int SCAN_BLK = 512;     // steps per warp iteration (16 per lane)
-constexpr int SCAN_STAGES = 3;    // cp.async ring depth per warp
-constexpr int SCAN_WARPS = 8;     // warps per CTA
+#ifndef SJA_SCAN_STAGES
+#define SJA_SCAN_STAGES 2
+#endif
+#ifndef SJA_SCAN_WARPS
+#define SJA_SCAN_WARPS 10
+#endif
+#ifndef SJA_SCAN_CTAS_PER_SM
+#define SJA_SCAN_CTAS_PER_SM 2
+#endif
+constexpr int SCAN_BLK = 512;                       // steps per warp iteration (16 per lane)
+constexpr int SCAN_STAGES = SJA_SCAN_STAGES;        // cp.async ring depth per warp
+constexpr int SCAN_WARPS = SJA_SCAN_WARPS;          // warps per CTA
+constexpr int SCAN_CTAS_PER_SM = SJA_SCAN_CTAS_PER_SM;
 constexpr int SCAN_STAGE_BYTES = 2048 + 2048 + 64;  // d, m, 16 safe words
 constexpr int SCAN_SMEM_BYTES = SCAN_WARPS * SCAN_STAGES * SCAN_STAGE_BYTES;
 
@@ -159,12 +169,14 @@ __global__ void __launch_bounds__(1024) row_offsets_kernel(const uint32_t* __res
 // the two-pass route: lane totals first, then a second walk that stores rows directly.
 constexpr int SCAN_STAGE_ROWS = 168;   // 168 * 24 B = 4032 B <= the 4096 B of a consumed d+m slot
 
-__global__ void __launch_bounds__(SCAN_WARPS * 32) scan_profiles_kernel(ScanArgs a) {
+__global__ void __launch_bounds__(SCAN_WARPS * 32, SCAN_CTAS_PER_SM) scan_profiles_kernel(ScanArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t wid = threadIdx.x >> 5;
     unsigned char* wbase = smem_raw + (size_t)wid * SCAN_STAGES * SCAN_STAGE_BYTES;
     const uint32_t wbase_s = (uint32_t)__cvta_generic_to_shared(wbase);
+    const uint32_t lane_sw = (lane ^ ((lane >> 3) & 3u)) * 16u;   // swz(32 r + lane) * 16 - 512 r
+    const uint32_t rd_x = (lane >> 1) & 3u;                        // swz(4 lane + r) = 4 lane + (r ^ rd_x)
 
     for (;;) {
         uint32_t j = 0;
@@ -186,24 +198,37 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32) scan_profiles_kernel(ScanArgs
             if (t < nblk) {
                 const uint64_t bs = blk0 + t * SCAN_BLK;
                 const uint32_t st = wbase_s + (uint32_t)(t % SCAN_STAGES) * SCAN_STAGE_BYTES;
+                if (bs >= s && bs + SCAN_BLK <= e) {
+                    // block entirely inside the job: plain 16-byte copies, no clipping
+                    const uint32_t* dp = a.d + bs + 4u * lane;
+                    const uint32_t* mp = a.m + bs + 4u * lane;
+                    const uint32_t dst = st + lane_sw;
 #pragma unroll
-                for (uint32_t r = 0; r < 4; ++r) {
-                    const uint32_t c = r * 32u + lane;
-                    const uint64_t step = bs + 4ull * c;
-                    uint32_t bytes = 0;
-                    if (step + 4 > s && step < e) {
-                        const uint64_t left = (a.N - step) * 4ull;
-                        bytes = left < 16 ? (uint32_t)left : 16u;
+                    for (uint32_t r = 0; r < 4; ++r) {
+                        cp_async16(dst + r * 512u, dp + r * 128u, 16u);
+                        cp_async16(dst + r * 512u + 2048u, mp + r * 128u, 16u);
                     }
-                    const uint64_t src = bytes ? step : 0ull;
-                    const uint32_t dst = st + swz(c) * 16u;
-                    cp_async16(dst, a.d + src, bytes);
-                    cp_async16(dst + 2048u, a.m + src, bytes);
-                }
-                if (lane < 16) {
-                    const uint64_t w = (bs >> 5) + lane;
-                    const bool ok = (w << 5) < e && ((w << 5) + 32) > s;
-                    cp_async4(st + 4096u + lane * 4u, a.sbits + (ok ? w : 0ull), ok ? 4u : 0u);
+                    if (lane < 16) cp_async4(st + 4096u + lane * 4u, a.sbits + (bs >> 5) + lane, 4u);
+                } else {
+#pragma unroll
+                    for (uint32_t r = 0; r < 4; ++r) {
+                        const uint32_t c = r * 32u + lane;
+                        const uint64_t step = bs + 4ull * c;
+                        uint32_t bytes = 0;
+                        if (step + 4 > s && step < e) {
+                            const uint64_t left = (a.N - step) * 4ull;
+                            bytes = left < 16 ? (uint32_t)left : 16u;
+                        }
+                        const uint64_t src = bytes ? step : 0ull;
+                        const uint32_t dst = st + swz(c) * 16u;
+                        cp_async16(dst, a.d + src, bytes);
+                        cp_async16(dst + 2048u, a.m + src, bytes);
+                    }
+                    if (lane < 16) {
+                        const uint64_t w = (bs >> 5) + lane;
+                        const bool ok = (w << 5) < e && ((w << 5) + 32) > s;
+                        cp_async4(st + 4096u + lane * 4u, a.sbits + (ok ? w : 0ull), ok ? 4u : 0u);
+                    }
                 }
             }
             cp_async_commit();
@@ -231,7 +256,7 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32) scan_profiles_kernel(ScanArgs
             uint32_t dv[16], mv[16];
 #pragma unroll
             for (uint32_t r = 0; r < 4; ++r) {
-                const uint32_t ph = swz(4u * lane + r);
+                const uint32_t ph = 4u * lane + (r ^ rd_x);
                 const uint4 qd = sd[ph];
                 const uint4 qm = sm[ph];
                 dv[4 * r + 0] = qd.x; dv[4 * r + 1] = qd.y; dv[4 * r + 2] = qd.z; dv[4 * r + 3] = qd.w;
@@ -242,18 +267,20 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32) scan_profiles_kernel(ScanArgs
 
             const uint64_t bs = blk0 + t * SCAN_BLK;
             const uint64_t lane_base = bs + 16ull * lane;
-            // valid steps of this lane: [lo, hi) within its 16
-            uint32_t lo = 0, hi = 16;
-            if (s > lane_base) lo = (s - lane_base) >= 16 ? 16u : (uint32_t)(s - lane_base);
-            if (e < lane_base + 16) hi = (e <= lane_base) ? 0u : (uint32_t)(e - lane_base);
-            const uint32_t vm = (hi > lo) ? (((1u << hi) - 1u) & ~((1u << lo) - 1u)) : 0u;
-            if (vm != 0xFFFFu) {
+            if (!(bs >= s && bs + SCAN_BLK < e)) {
+                // first / last block of the job: clip to [s, e), force the end-of-job boundary
+                uint32_t lo = 0, hi = 16;
+                if (s > lane_base) lo = (s - lane_base) >= 16 ? 16u : (uint32_t)(s - lane_base);
+                if (e < lane_base + 16) hi = (e <= lane_base) ? 0u : (uint32_t)(e - lane_base);
+                const uint32_t vm = (hi > lo) ? (((1u << hi) - 1u) & ~((1u << lo) - 1u)) : 0u;
+                if (vm != 0xFFFFu) {
 #pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    if (!((vm >> i) & 1u)) { dv[i] = 0; mv[i] = 0; }
+                    for (int i = 0; i < 16; ++i)
+                        if (!((vm >> i) & 1u)) { dv[i] = 0; mv[i] = 0; }
+                }
+                bits &= vm;
+                if (e - 1 >= lane_base && e - 1 < lane_base + 16) bits |= 1u << (uint32_t)(e - 1 - lane_base);
             }
-            bits &= vm;
-            if (e - 1 >= lane_base && e - 1 < lane_base + 16) bits |= 1u << (uint32_t)(e - 1 - lane_base);
             const uint32_t k0 = (uint32_t)(lane_base - js);   // steps of the job before this lane
 
             // rows of this block: exclusive count per lane, total
