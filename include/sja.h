@@ -169,7 +169,7 @@ sja_status sja_select(sja_ctx* ctx, const sja_policy* policy, sja_award* out, sj
  * cudaFree or other allocating routine and records no profiling events.
  *
  * Cost and limit: every GPU on which the library is used holds the array until the process
- * exits.  The call needs ceil(J / 512) * G candidate slots of 16 bytes (ceil(J / 256) * G
+ * exits.  The call needs ceil(J / 1024) * G candidate slots of 16 bytes (ceil(J / 256) * G
  * with SJA_FLAG_FORCE_SEARCH or an unsorted / many-capacity batch); if that exceeds the
  * array it returns SJA_ERR_INVALID_ARG with the numbers in sja_last_error() and does nothing.
  *

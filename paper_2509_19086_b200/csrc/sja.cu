@@ -238,6 +238,17 @@ __global__ void export_rows_kernel(const uint4* __restrict__ A, const uint2* __r
     if (W) W[i] = pack64(a.z, a.w);
 }
 
+void launch_merge(uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& jv, const Gap* sgaps, uint32_t G,
+                  uint32_t per_split, Partial* partial) {
+    const int threads = MERGE_WARPS * 32;
+    if (kind == SJA_POLICY_FAIRNESS)
+        select_merge_kernel<1><<<grid, threads, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split, partial);
+    else if (kind == SJA_POLICY_SLA)
+        select_merge_kernel<2><<<grid, threads, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split, partial);
+    else
+        select_merge_kernel<0><<<grid, threads, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split, partial);
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
@@ -302,7 +313,11 @@ sja_status sja_create(sja_ctx** out, int device, void* cuda_stream) {
         if (cudaMemsetAsync(c->flags.p, 0, 4, c->stream) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         if (cudaFuncSetAttribute(scan_profiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  SCAN_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
-        if (cudaFuncSetAttribute(select_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(select_merge_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 MERGE_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
+        if (cudaFuncSetAttribute(select_merge_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 MERGE_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
+        if (cudaFuncSetAttribute(select_merge_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  MERGE_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         if (cudaFuncSetAttribute(sort_gaps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)(SORT_MAX_GAPS * 12)) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
@@ -572,8 +587,8 @@ sja_status sja_select(sja_ctx* c, const sja_policy* policy, sja_award* out, sja_
         ProfScope ps(c, CAT_SELECT);
         const JobView jv = job_view(c);
         if (use_merge) {
-            select_merge_kernel<<<dim3(n_chunks, splits), MERGE_WARPS * 32, MERGE_SMEM_BYTES, c->stream>>>(
-                jv, c->sgaps.as<Gap>(), G, per_split, kind, c->partial.as<Partial>());
+            launch_merge(kind, dim3(n_chunks, splits), c->stream, jv, c->sgaps.as<Gap>(), G, per_split,
+                         c->partial.as<Partial>());
         } else {
             select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, 0, c->stream>>>(
                 jv, c->sgaps.as<Gap>(), G, per_split, kind, nullptr, 0, c->partial.as<Partial>());
@@ -644,8 +659,7 @@ sja_status sja_select_static(sja_ctx* c, const sja_policy* policy, sja_award* ou
     // read and nothing has to be cleared first.
     const JobView jv = job_view(c);
     if (use_merge) {
-        select_merge_kernel<<<dim3(n_chunks, splits), MERGE_WARPS * 32, MERGE_SMEM_BYTES, c->stream>>>(
-            jv, c->sgaps.as<Gap>(), G, per_split, kind, scratch);
+        launch_merge(kind, dim3(n_chunks, splits), c->stream, jv, c->sgaps.as<Gap>(), G, per_split, scratch);
     } else {
         select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, 0, c->stream>>>(
             jv, c->sgaps.as<Gap>(), G, per_split, kind, nullptr, 0, scratch);

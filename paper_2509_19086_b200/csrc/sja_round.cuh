@@ -300,19 +300,36 @@ __global__ void __launch_bounds__(256) copy_gaps_kernel(const Gap* __restrict__ 
 // Merge kernel.  Each lane owns MERGE_R jobs and walks the gaps of its CTA's range in the
 // advertised order (capacity class, then T ascending).  Per job it keeps a cursor into the
 // job's boundary rows above the progress point: the number w of rows that satisfy both
-// bounds for the current gap.  Inside a class w only moves forward, so a pair costs a few
-// compares.  The next rows of every job wait in a per-lane shared-memory ring that is
-// refilled with 16-byte cp.async copies, so an advance never waits on global memory in the
-// steady state.  Per gap the warp reduces its 32 x MERGE_R keys to one candidate
-// (largest key, then lowest job id), the CTA folds its warps, and one candidate per
-// (CTA, gap) goes to global memory.
-constexpr int MERGE_WARPS = 8;
-constexpr int MERGE_R = 2;
-constexpr int MERGE_RING = 8;       // rows per lane-job ring
-constexpr int MERGE_GT = 64;        // gaps per staging tile
+// bounds for the current gap.  Inside a class w only moves forward, so a pair costs one
+// compare against the duration threshold of the next row ("thr", set to the largest u32
+// when the next row is out of reach for this class) plus the key comparison.  The next
+// rows of every job wait in a per-lane shared-memory ring that is refilled with 16-byte
+// cp.async copies, so an advance never waits on global memory in the steady state.  All
+// MERGE_R cursors of a lane advance inside ONE divergent region per gap.  Per gap the warp
+// reduces its 32 x MERGE_R keys to one candidate (largest key, then lowest job id), the CTA
+// folds its warps, and one candidate per (CTA, gap) goes to global memory.
+#ifndef SJA_MERGE_WARPS
+#define SJA_MERGE_WARPS 8
+#endif
+#ifndef SJA_MERGE_R
+#define SJA_MERGE_R 4
+#endif
+#ifndef SJA_MERGE_RING
+#define SJA_MERGE_RING 4
+#endif
+#ifndef SJA_MERGE_CTAS_PER_SM
+#define SJA_MERGE_CTAS_PER_SM 2
+#endif
+constexpr int MERGE_WARPS = SJA_MERGE_WARPS;
+constexpr int MERGE_R = SJA_MERGE_R;          // jobs per lane
+constexpr int MERGE_RING = SJA_MERGE_RING;    // rows per lane-job ring (power of two)
+constexpr int MERGE_CTAS_PER_SM = SJA_MERGE_CTAS_PER_SM;
+constexpr int MERGE_GT = 64;                  // gaps per staging tile
 constexpr int MERGE_JOBS = MERGE_WARPS * MERGE_R * 32;
 constexpr int MERGE_RING_BYTES = MERGE_WARPS * MERGE_R * MERGE_RING * 32 * 16;
 constexpr int MERGE_SMEM_BYTES = MERGE_RING_BYTES + MERGE_GT * MERGE_WARPS * 16 + MERGE_GT * 16;
+static_assert((MERGE_RING & (MERGE_RING - 1)) == 0, "ring size must be a power of two");
+static_assert(MERGE_GT <= MERGE_WARPS * 32, "one thread per gap of a tile");
 
 __device__ __forceinline__ void mg_cp_async16(uint32_t dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(src) : "memory");
@@ -320,37 +337,62 @@ __device__ __forceinline__ void mg_cp_async16(uint32_t dst, const void* src) {
 __device__ __forceinline__ void mg_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void mg_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+__device__ __forceinline__ uint4 mg_lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr)
+                 : "memory");
+    return v;
+}
 
-__global__ void __launch_bounds__(MERGE_WARPS * 32) select_merge_kernel(
-    JobView jv, const Gap* __restrict__ sgaps, uint32_t G, uint32_t gaps_per_split, uint32_t kind,
-    Partial* __restrict__ partial_out) {
+// The u64 warp maximum as two 32-bit hardware reductions (high word, then low word among the
+// lanes that hold the maximal high word).
+struct WarpBest { uint64_t key; uint32_t writer; bool hit; };
+
+__device__ __forceinline__ WarpBest warp_argmax_lowest_lane(uint64_t best, uint32_t lane) {
+    WarpBest o;
+    o.key = warp_max_u64(best);
+    o.hit = (best == o.key) && (o.key != 0ull);
+    const uint32_t ball = __ballot_sync(0xFFFFFFFFu, o.hit);
+    o.writer = ball ? (uint32_t)(__ffs((int)ball) - 1) : 0u;   // lowest lane = lowest job id (lane-major jobs)
+    o.hit = o.hit && (lane == o.writer);
+    return o;
+}
+
+template <uint32_t KIND>
+__global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_merge_kernel(
+    JobView jv, const Gap* __restrict__ sgaps, uint32_t G, uint32_t gaps_per_split, Partial* __restrict__ partial_out) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint4* ring_all = reinterpret_cast<uint4*>(smem_raw);
     Partial* stage = reinterpret_cast<Partial*>(smem_raw + MERGE_RING_BYTES);            // [GT][WARPS]
     uint4* sg = reinterpret_cast<uint4*>(smem_raw + MERGE_RING_BYTES + MERGE_GT * MERGE_WARPS * 16);
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
+    const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(smem_raw);
 
-    uint64_t base[MERGE_R], Wp[MERGE_R], nextW[MERGE_R], curKey[MERGE_R];
-    uint32_t n[MERGE_R], Dp[MERGE_R], ready[MERGE_R], factor[MERGE_R], w[MERGE_R], nextD[MERGE_R], nextM[MERGE_R];
-    uint4* ring[MERGE_R];
+    // per lane-job state; job of (lane, r) = first job of the warp + lane * MERGE_R + r
+    const uint4* next_row[MERGE_R];   // row w + MERGE_RING of the job: the next one to prefetch
+    const uint4* row0[MERGE_R];
+    uint64_t Wp[MERGE_R], nextW[MERGE_R], curKey[MERGE_R];
+    uint32_t n[MERGE_R], Dp[MERGE_R], ready[MERGE_R], factor[MERGE_R];
+    uint32_t w[MERGE_R];      // rows that satisfy both bounds for the current gap
+    uint32_t thr[MERGE_R];    // duration of row w relative to the progress point, or 0xFFFFFFFF when closed
     uint32_t ring_s[MERGE_R];
+    uint32_t open = 0;        // bit r: row w of job r exists and its running max fits the current class
     const uint32_t job0 = blockIdx.x * MERGE_JOBS + wid * MERGE_R * 32;   // first job of this warp
 #pragma unroll
     for (int r = 0; r < MERGE_R; ++r) {
-        const uint32_t j = job0 + r * 32 + lane;
-        ring[r] = ring_all + (size_t)(wid * MERGE_R + r) * MERGE_RING * 32 + lane;
-        ring_s[r] = (uint32_t)__cvta_generic_to_shared(ring[r]);
-        base[r] = 0; Wp[r] = 0; nextW[r] = 0; curKey[r] = 0;
-        n[r] = 0; Dp[r] = 0; ready[r] = 0; factor[r] = 0; w[r] = 0; nextD[r] = 0; nextM[r] = 0;
+        const uint32_t j = job0 + lane * MERGE_R + r;
+        ring_s[r] = smem_s + ((wid * MERGE_R + r) * MERGE_RING * 32 + lane) * 16;
+        row0[r] = jv.A; next_row[r] = jv.A;
+        Wp[r] = 0; nextW[r] = 0; curKey[r] = 0;
+        n[r] = 0; Dp[r] = 0; ready[r] = 0xFFFFFFFFu; factor[r] = 0; w[r] = 0; thr[r] = 0xFFFFFFFFu;
         if (j < jv.J) {
             const uint64_t b0 = jv.boff[j], b1 = jv.boff[j + 1];
             const uint32_t pb = jv.pb[j];
-            base[r] = b0 + pb;
+            row0[r] = jv.A + b0 + pb;
             n[r] = (uint32_t)(b1 - b0) - pb;
             Dp[r] = jv.Dp[j];
             Wp[r] = jv.Wp[j];
             ready[r] = jv.ready[j];
-            factor[r] = policy_factor(jv, kind, j);
+            factor[r] = policy_factor(jv, KIND, j);
         }
     }
     const uint32_t g_begin = blockIdx.y * gaps_per_split;
@@ -358,70 +400,94 @@ __global__ void __launch_bounds__(MERGE_WARPS * 32) select_merge_kernel(
     bool first = true;
     uint32_t curC = 0;
 
+    // Cursor update and lane-local best candidate for one gap.
+    auto eval_gap = [&](const uint4 gq, uint64_t& best, uint32_t& best_r, uint32_t& best_cnt) {
+        const uint32_t start = gq.y, T = gq.z, C = gq.w;
+        if (first || C != curC) {
+            // new capacity class: T restarts from its smallest value, so do the cursors
+            first = false;
+            curC = C;
+            mg_wait<0>();
+#pragma unroll
+            for (int r = 0; r < MERGE_R; ++r) {
+                w[r] = 0;
+                curKey[r] = 0;
+#pragma unroll
+                for (int i = 0; i < MERGE_RING; ++i) {
+                    if ((uint32_t)i < n[r]) mg_cp_async16(ring_s[r] + i * 32 * 16, row0[r] + i);
+                    mg_commit();
+                }
+                next_row[r] = row0[r] + MERGE_RING;
+            }
+            mg_wait<0>();
+            open = 0;
+#pragma unroll
+            for (int r = 0; r < MERGE_R; ++r) {
+                thr[r] = 0xFFFFFFFFu;
+                if (n[r]) {
+                    const uint4 row = mg_lds128(ring_s[r]);
+                    nextW[r] = pack64(row.z, row.w);
+                    if (row.y <= C) { open |= 1u << r; thr[r] = row.x - Dp[r]; }
+                }
+            }
+        }
+        // one cheap test per job; the rare advances of all jobs of the lane share one region
+        bool need = false;
+#pragma unroll
+        for (int r = 0; r < MERGE_R; ++r) need |= (T >= thr[r]);
+        if (need) {
+#pragma unroll
+            for (int r = 0; r < MERGE_R; ++r) {
+                while (((open >> r) & 1u) && T >= thr[r]) {
+                    // row w qualifies: it becomes the candidate; fetch row w + 1 from the ring
+                    curKey[r] = policy_key(KIND, nextW[r] - Wp[r], factor[r]);
+                    if (w[r] + MERGE_RING < n[r])
+                        mg_cp_async16(ring_s[r] + (w[r] & (MERGE_RING - 1)) * 32 * 16, next_row[r]);
+                    mg_commit();
+                    ++next_row[r];
+                    ++w[r];
+                    open &= ~(1u << r);
+                    thr[r] = 0xFFFFFFFFu;
+                    if (w[r] < n[r]) {
+                        mg_wait<MERGE_RING - 1>();
+                        const uint4 row = mg_lds128(ring_s[r] + (w[r] & (MERGE_RING - 1)) * 32 * 16);
+                        nextW[r] = pack64(row.z, row.w);
+                        if (row.y <= C) { open |= 1u << r; thr[r] = row.x - Dp[r]; }
+                    }
+                }
+            }
+        }
+        best = 0; best_r = 0; best_cnt = 0;
+#pragma unroll
+        for (int r = 0; r < MERGE_R; ++r) {
+            const uint64_t k = (start >= ready[r]) ? curKey[r] : 0ull;
+            if (k > best) { best = k; best_r = (uint32_t)r; best_cnt = w[r]; }   // strict: lower r wins ties
+        }
+    };
+    auto publish = [&](const WarpBest& wb, uint32_t gi, uint32_t br, uint32_t bc) {
+        if (wb.key == 0ull) {
+            if (lane == 0) { Partial pr; pr.key = 0; pr.job = 0xFFFFFFFFu; pr.cnt = 0; stage[gi * MERGE_WARPS + wid] = pr; }
+        } else if (wb.hit) {
+            Partial pr; pr.key = wb.key; pr.job = job0 + lane * MERGE_R + br; pr.cnt = bc;
+            stage[gi * MERGE_WARPS + wid] = pr;
+        }
+    };
+
     for (uint32_t g0 = g_begin; g0 < g_end; g0 += MERGE_GT) {
         const uint32_t gt = min((uint32_t)MERGE_GT, g_end - g0);
         if (threadIdx.x < gt) sg[threadIdx.x] = __ldg(reinterpret_cast<const uint4*>(sgaps) + g0 + threadIdx.x);
         __syncthreads();
-        for (uint32_t gi = 0; gi < gt; ++gi) {
-            const uint4 gq = sg[gi];
-            const uint32_t start = gq.y, T = gq.z, C = gq.w;
-            if (first || C != curC) {
-                // new capacity class: T restarts from its smallest value, so do the cursors
-                first = false;
-                curC = C;
-                mg_wait<0>();
-#pragma unroll
-                for (int r = 0; r < MERGE_R; ++r) {
-                    w[r] = 0;
-                    curKey[r] = 0;
-#pragma unroll
-                    for (int i = 0; i < MERGE_RING; ++i) {
-                        if ((uint32_t)i < n[r]) mg_cp_async16(ring_s[r] + i * 32 * 16, jv.A + base[r] + i);
-                        mg_commit();
-                    }
-                }
-                mg_wait<0>();
-#pragma unroll
-                for (int r = 0; r < MERGE_R; ++r) {
-                    if (n[r]) {
-                        const uint4 row = ring[r][0];
-                        nextD[r] = row.x - Dp[r];
-                        nextM[r] = row.y;
-                        nextW[r] = pack64(row.z, row.w);
-                    }
-                }
-            }
-            uint64_t best = 0;
-            uint32_t best_slot = 0, best_cnt = 0;
-#pragma unroll
-            for (int r = 0; r < MERGE_R; ++r) {
-                while (w[r] < n[r] && nextD[r] <= T && nextM[r] <= C) {
-                    curKey[r] = policy_key(kind, nextW[r] - Wp[r], factor[r]);
-                    if (w[r] + MERGE_RING < n[r])
-                        mg_cp_async16(ring_s[r] + (w[r] % MERGE_RING) * 32 * 16, jv.A + base[r] + w[r] + MERGE_RING);
-                    mg_commit();
-                    ++w[r];
-                    if (w[r] < n[r]) {
-                        mg_wait<MERGE_RING - 1>();
-                        const uint4 row = ring[r][(w[r] % MERGE_RING) * 32];
-                        nextD[r] = row.x - Dp[r];
-                        nextM[r] = row.y;
-                        nextW[r] = pack64(row.z, row.w);
-                    }
-                }
-                const uint64_t k = (start >= ready[r]) ? curKey[r] : 0ull;
-                if (k > best) { best = k; best_slot = (uint32_t)r * 32u + lane; best_cnt = w[r]; }
-            }
-            const uint64_t mk = warp_max_u64(best);
-            const uint32_t smin = __reduce_min_sync(0xFFFFFFFFu, (best == mk && mk != 0ull) ? best_slot : 0xFFFFFFFFu);
-            const uint32_t wcnt = __shfl_sync(0xFFFFFFFFu, best_cnt, smin & 31u);
-            if (lane == 0) {
-                Partial pr;
-                pr.key = mk;
-                pr.job = mk ? job0 + smin : 0xFFFFFFFFu;
-                pr.cnt = mk ? wcnt : 0u;
-                stage[gi * MERGE_WARPS + wid] = pr;
-            }
+        // two gaps per iteration: their warp reductions are independent and overlap
+        for (uint32_t gi = 0; gi < gt; gi += 2) {
+            uint64_t bestA, bestB = 0;
+            uint32_t rA, cA, rB = 0, cB = 0;
+            eval_gap(sg[gi], bestA, rA, cA);
+            const bool two = gi + 1 < gt;
+            if (two) eval_gap(sg[gi + 1], bestB, rB, cB);
+            const WarpBest wa = warp_argmax_lowest_lane(bestA, lane);
+            const WarpBest wb = warp_argmax_lowest_lane(bestB, lane);
+            publish(wa, gi, rA, cA);
+            if (two) publish(wb, gi + 1, rB, cB);
         }
         __syncthreads();
         if (threadIdx.x < gt) {
