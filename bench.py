@@ -29,9 +29,9 @@ from paper_2509_19086_b200 import workloads as wl  # noqa: E402
 METRIC = "job-gap pairs evaluated/s"
 UNIT = "pairs/s"
 POLICY_NAMES = {0: "efficiency", 1: "fairness", 2: "sla"}
-# kernels launched per step: count_boundaries, row_offsets, scan_profiles | sort_gaps |
-# select_merge (or select_search), finalize_awards | commit_vote, commit_apply, commit_refresh
-KERNELS_PER_STEP = 9
+# kernels launched per step: count_boundaries, cta_offsets, row_offsets, scan_profiles | rank_gaps,
+# place_gaps | select_merge (or select_search), finalize_awards | commit_vote, commit_apply, commit_refresh
+KERNELS_PER_STEP = 11
 FALLBACK_HBM_GBS = 6650.0
 
 

@@ -47,7 +47,7 @@ struct sja_ctx {
     uint32_t load_flags = 0;
     DevBuf st_off, st_d, st_m, st_s, st_p;            // staging for host inputs / load-time progress
     DevBuf p, ready, pb, Dp, Wp, wait, prio;          // per-job state and attributes
-    DevBuf nbj, boff, boff_next, A, B, jobwin;        // boundary table
+    DevBuf nbj, cta_tot, cta_base, boff, boff_next, A, B, jobwin;   // row counting scratch, boundary table
     DevBuf flags, counter, n_granted;                 // small device words
     uint32_t* h_words = nullptr;                      // pinned host scratch (8 x u64)
 
@@ -56,7 +56,7 @@ struct sja_ctx {
     uint32_t G = 0, last_policy = 0;
     bool gaps_sorted = false;          // sgaps is ordered by (C, T); else it is the caller's order
     uint32_t n_classes = 0;            // distinct capacities of the batch (valid when sorted)
-    DevBuf gaps, sgaps, gap_info, awards, widx, partial, winners;
+    DevBuf gaps, sgaps, gap_info, gap_rank, awards, widx, partial, winners;
 
     // profiling
     bool prof = false;
@@ -319,8 +319,6 @@ sja_status sja_create(sja_ctx** out, int device, void* cuda_stream) {
                                  MERGE_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         if (cudaFuncSetAttribute(select_merge_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  MERGE_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
-        if (cudaFuncSetAttribute(sort_gaps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(SORT_MAX_GAPS * 12)) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         if ((st = reserve(c, c->gap_info, sizeof(GapInfo))) != SJA_OK) break;
     } while (0);
     if (st != SJA_OK) {
@@ -337,8 +335,8 @@ sja_status sja_destroy(sja_ctx* c) {
     DeviceGuard guard(c->device);
     cudaStreamSynchronize(c->stream);
     DevBuf* bufs[] = {&c->st_off, &c->st_d, &c->st_m, &c->st_s, &c->st_p, &c->p, &c->ready, &c->pb, &c->Dp,
-                      &c->Wp, &c->wait, &c->prio, &c->nbj, &c->boff, &c->boff_next, &c->A, &c->B, &c->jobwin,
-                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->awards, &c->widx, &c->partial,
+                      &c->Wp, &c->wait, &c->prio, &c->nbj, &c->cta_tot, &c->cta_base, &c->boff, &c->boff_next, &c->A, &c->B, &c->jobwin,
+                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->awards, &c->widx, &c->partial,
                       &c->winners};
     for (DevBuf* b : bufs) release(*b);
     for (ProfSpan& s : c->spans) { cudaEventDestroy(s.a); cudaEventDestroy(s.b); }
@@ -425,7 +423,10 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
         return fail(c, SJA_ERR_INVALID_ARG, "sja_load_profiles: device profile arrays must be 16-byte aligned");
     }
     TRY(reserve(c, c->st_p, (size_t)J * 4));
-    TRY(reserve(c, c->nbj, (size_t)J * 4));
+    const uint32_t n_count_ctas = (J + COUNT_JOBS_PER_CTA - 1) / COUNT_JOBS_PER_CTA;
+    TRY(reserve(c, c->nbj, (size_t)J * 8));                       // per-job row offset inside its CTA
+    TRY(reserve(c, c->cta_tot, (size_t)n_count_ctas * 8));
+    TRY(reserve(c, c->cta_base, (size_t)(n_count_ctas + 1) * 8));
     TRY(reserve(c, c->boff_next, (size_t)(J + 1) * 8));
     if (progress) TRY(copy_in(c, c->st_p.p, progress, (size_t)J * 4, where));
     else CU(cudaMemsetAsync(c->st_p.p, 0, (size_t)J * 4, c->stream));
@@ -434,10 +435,13 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
     CU(cudaMemsetAsync(c->flags.p, 0, 4, c->stream));
     {
         ProfScope ps(c, CAT_PREP);
-        const uint32_t blocks = (uint32_t)std::min<uint64_t>(((uint64_t)J * 32 + 255) / 256, (uint64_t)c->n_sm * 32);
-        count_boundaries_kernel<<<blocks, 256, 0, c->stream>>>(d_off, d_s, c->st_p.as<uint32_t>(), J, N,
-                                                               c->nbj.as<uint32_t>(), c->flags.as<uint32_t>());
-        row_offsets_kernel<<<1, 1024, 0, c->stream>>>(c->nbj.as<uint32_t>(), J, c->boff_next.as<uint64_t>());
+        count_boundaries_kernel<<<n_count_ctas, 256, 0, c->stream>>>(
+            d_off, d_s, c->st_p.as<uint32_t>(), J, N, c->nbj.as<uint64_t>(), c->cta_tot.as<uint64_t>(),
+            c->flags.as<uint32_t>());
+        cta_offsets_kernel<<<1, 1024, 0, c->stream>>>(c->cta_tot.as<uint64_t>(), n_count_ctas,
+                                                      c->cta_base.as<uint64_t>());
+        row_offsets_kernel<<<(J + 255) / 256, 256, 0, c->stream>>>(c->nbj.as<uint64_t>(), c->cta_base.as<uint64_t>(),
+                                                                   J, n_count_ctas, c->boff_next.as<uint64_t>());
     }
     CU(cudaGetLastError());
     CU(cudaMemcpyAsync(c->h_words, c->flags.p, 4, cudaMemcpyDeviceToHost, c->stream));
@@ -519,6 +523,7 @@ sja_status sja_advertise(sja_ctx* c, uint32_t G, const sja_gap* gaps, sja_memspa
     DeviceGuard guard(c->device);
     TRY(reserve(c, c->gaps, (size_t)G * sizeof(sja_gap)));
     TRY(reserve(c, c->sgaps, (size_t)G * sizeof(sja_gap)));
+    TRY(reserve(c, c->gap_rank, (size_t)G * 8));
     TRY(reserve(c, c->awards, (size_t)G * sizeof(sja_award)));
     TRY(reserve(c, c->widx, (size_t)G * 4));
     TRY(reserve(c, c->winners, (size_t)G * 4));
@@ -527,11 +532,19 @@ sja_status sja_advertise(sja_ctx* c, uint32_t G, const sja_gap* gaps, sja_memspa
         ProfScope ps(c, CAT_ADVERTISE);
         TRY(copy_in(c, c->gaps.p, gaps, (size_t)G * sizeof(sja_gap), where));
         if (sortable) {
-            uint32_t n_pow2 = 1;
-            while (n_pow2 < G) n_pow2 <<= 1;
-            sort_gaps_kernel<<<1, 1024, (size_t)n_pow2 * 12, c->stream>>>(c->gaps.as<Gap>(), G, n_pow2,
-                                                                         c->sgaps.as<Gap>(),
-                                                                         c->gap_info.as<GapInfo>());
+            // rank[G] and not_leader[G] share one buffer; both and the class counter start at zero
+            uint32_t* rank = c->gap_rank.as<uint32_t>();
+            CU(cudaMemsetAsync(rank, 0, (size_t)G * 8, c->stream));
+            CU(cudaMemsetAsync(c->gap_info.p, 0, sizeof(GapInfo), c->stream));
+            const uint32_t i_blocks = (G + RANK_THREADS - 1) / RANK_THREADS;
+            uint32_t slices = (uint32_t)((16ull * c->n_sm + i_blocks - 1) / i_blocks);   // enough CTAs to fill the GPU
+            slices = std::max(1u, std::min(slices, (G + 63u) / 64u));
+            const uint32_t slice_len = (G + slices - 1) / slices;
+            slices = (G + slice_len - 1) / slice_len;
+            rank_gaps_kernel<<<dim3(i_blocks, slices), RANK_THREADS, 0, c->stream>>>(c->gaps.as<Gap>(), G, slice_len,
+                                                                                      rank, rank + G);
+            place_gaps_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(c->gaps.as<Gap>(), G, rank, rank + G,
+                                                                      c->sgaps.as<Gap>(), c->gap_info.as<GapInfo>());
             CU(cudaMemcpyAsync(c->h_words + 4, c->gap_info.p, sizeof(GapInfo), cudaMemcpyDeviceToHost, c->stream));
         } else {
             copy_gaps_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(c->gaps.as<Gap>(), G, c->sgaps.as<Gap>());
@@ -593,7 +606,7 @@ sja_status sja_select(sja_ctx* c, const sja_policy* policy, sja_award* out, sja_
             select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, 0, c->stream>>>(
                 jv, c->sgaps.as<Gap>(), G, per_split, kind, nullptr, 0, c->partial.as<Partial>());
         }
-        finalize_awards_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(jv, c->partial.as<Partial>(), n_chunks,
+        finalize_awards_kernel<<<(uint32_t)(((uint64_t)G * FINALIZE_LANES + 255) / 256), 256, 0, c->stream>>>(jv, c->partial.as<Partial>(), n_chunks,
                                                                          c->sgaps.as<Gap>(), G, kind,
                                                                          c->awards.as<Award>(),
                                                                          c->widx.as<uint32_t>());
@@ -664,7 +677,7 @@ sja_status sja_select_static(sja_ctx* c, const sja_policy* policy, sja_award* ou
         select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, 0, c->stream>>>(
             jv, c->sgaps.as<Gap>(), G, per_split, kind, nullptr, 0, scratch);
     }
-    finalize_awards_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(jv, scratch, n_chunks, c->sgaps.as<Gap>(), G,
+    finalize_awards_kernel<<<(uint32_t)(((uint64_t)G * FINALIZE_LANES + 255) / 256), 256, 0, c->stream>>>(jv, scratch, n_chunks, c->sgaps.as<Gap>(), G,
                                                                      kind, c->awards.as<Award>(),
                                                                      c->widx.as<uint32_t>());
     CU(cudaGetLastError());

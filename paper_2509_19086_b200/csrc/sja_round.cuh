@@ -114,17 +114,31 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
 
 // ---------------------------------------------------------------------------------------
 // Final reduction: one thread per gap folds the candidate rows of all CTAs into the award.
+constexpr int FINALIZE_LANES = 8;   // lanes that share the candidate rows of one gap
+
 __global__ void __launch_bounds__(256) finalize_awards_kernel(
     JobView jv, const Partial* __restrict__ partial, uint32_t n_rows, const Gap* __restrict__ sgaps, uint32_t G,
     uint32_t kind, Award* __restrict__ awards, uint32_t* __restrict__ widx) {
-    const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;   // position in the advertised (sorted) order
-    if (g >= G) return;
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t g = t / FINALIZE_LANES;     // position in the advertised (sorted) order
+    const uint32_t sub = t % FINALIZE_LANES;
     Partial best;
     best.key = 0; best.job = 0xFFFFFFFFu; best.cnt = 0;
-    for (uint32_t r = 0; r < n_rows; ++r) {
-        const Partial c = partial[(size_t)r * G + g];
+    if (g < G) {
+        for (uint32_t r = sub; r < n_rows; r += FINALIZE_LANES) {
+            const Partial c = partial[(size_t)r * G + g];
+            if (c.key > best.key || (c.key == best.key && c.job < best.job)) best = c;
+        }
+    }
+#pragma unroll
+    for (int o = FINALIZE_LANES / 2; o > 0; o >>= 1) {
+        Partial c;
+        c.key = __shfl_xor_sync(0xFFFFFFFFu, best.key, o);
+        c.job = __shfl_xor_sync(0xFFFFFFFFu, best.job, o);
+        c.cnt = __shfl_xor_sync(0xFFFFFFFFu, best.cnt, o);
         if (c.key > best.key || (c.key == best.key && c.job < best.job)) best = c;
     }
+    if (g >= G || sub != 0) return;
     const uint32_t orig = sgaps[g].slice;   // caller's gap index
     Award a;
     if (best.key == 0) {
@@ -229,61 +243,64 @@ namespace sja {
 // Advertise: order the gaps by (capacity, window length).  Gaps of one capacity form a
 // "class" (the finite capacity set of Section 3.9); inside a class T ascends, so every job's
 // answer moves monotonically along its boundary rows and the select kernel can merge
-// instead of search.  One CTA, bitonic sort in shared memory (G <= SORT_MAX_GAPS).
-constexpr uint32_t SORT_MAX_GAPS = 16384;
+// instead of search.  The order is found by ranking: gap i goes to position
+// #{j : (C_j, T_j, j) < (C_i, T_i, i)}.  That is G^2 comparisons, but they are independent
+// (no barriers, no passes): thread (i, slice) counts over one slice of j held in shared
+// memory and adds its partial rank with one atomic; for the batch sizes of a scheduling
+// round (thousands of gaps) this takes a few microseconds.  The same sweep marks every gap
+// that has a predecessor of equal capacity, so the unmarked ones count the classes.
+constexpr uint32_t SORT_MAX_GAPS = 65536;
+constexpr int RANK_THREADS = 128;
+constexpr int RANK_TILE = 1024;   // keys per shared-memory tile
 
-struct GapInfo { uint32_t n_classes; uint32_t t_max; uint32_t c_max; uint32_t pad; };
+struct GapInfo { uint32_t n_classes; uint32_t pad[3]; };
 
-__global__ void __launch_bounds__(1024) sort_gaps_kernel(const Gap* __restrict__ gaps, uint32_t G, uint32_t n_pow2,
+__global__ void __launch_bounds__(RANK_THREADS) rank_gaps_kernel(const Gap* __restrict__ gaps, uint32_t G,
+                                                                 uint32_t slice_len, uint32_t* __restrict__ rank,
+                                                                 uint32_t* __restrict__ not_leader) {
+    __shared__ uint64_t skey[RANK_TILE];
+    const uint32_t i = blockIdx.x * RANK_THREADS + threadIdx.x;
+    uint64_t ki = 0;
+    if (i < G) { const Gap g = gaps[i]; ki = ((uint64_t)g.C << 32) | g.T; }
+    const uint32_t j_begin = blockIdx.y * slice_len;
+    const uint32_t j_end = min(G, j_begin + slice_len);
+    uint32_t cnt = 0, same = 0;
+    for (uint32_t t0 = j_begin; t0 < j_end; t0 += RANK_TILE) {
+        const uint32_t tn = min((uint32_t)RANK_TILE, j_end - t0);
+        __syncthreads();
+        for (uint32_t q = threadIdx.x; q < tn; q += RANK_THREADS) {
+            const Gap g = gaps[t0 + q];
+            skey[q] = ((uint64_t)g.C << 32) | g.T;
+        }
+        __syncthreads();
+        for (uint32_t q = 0; q < tn; ++q) {
+            const uint64_t kj = skey[q];
+            const bool less = kj < ki || (kj == ki && t0 + q < i);
+            cnt += less ? 1u : 0u;
+            same |= (less && (uint32_t)(kj >> 32) == (uint32_t)(ki >> 32)) ? 1u : 0u;
+        }
+    }
+    if (i < G) {
+        if (cnt) atomicAdd(rank + i, cnt);
+        if (same) atomicOr(not_leader + i, 1u);
+    }
+}
+
+__global__ void __launch_bounds__(256) place_gaps_kernel(const Gap* __restrict__ gaps, uint32_t G,
+                                                         const uint32_t* __restrict__ rank,
+                                                         const uint32_t* __restrict__ not_leader,
                                                          Gap* __restrict__ sorted, GapInfo* __restrict__ info) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    uint64_t* key = reinterpret_cast<uint64_t*>(smem_raw);
-    uint32_t* idx = reinterpret_cast<uint32_t*>(smem_raw + (size_t)n_pow2 * 8);
-    __shared__ uint32_t s_classes, s_tmax, s_cmax;
-    const uint32_t t = threadIdx.x;
-    if (t == 0) { s_classes = 0; s_tmax = 0; s_cmax = 0; }
-    for (uint32_t i = t; i < n_pow2; i += blockDim.x) {
-        if (i < G) {
-            const Gap g = gaps[i];
-            key[i] = ((uint64_t)g.C << 32) | g.T;
-            idx[i] = i;
-        } else {
-            key[i] = 0xFFFFFFFFFFFFFFFFull;   // padding sorts last (after real gaps with the same key: larger idx)
-            idx[i] = 0xFFFFFFFFu;
-        }
-    }
-    __syncthreads();
-    for (uint32_t k = 2; k <= n_pow2; k <<= 1) {
-        for (uint32_t j = k >> 1; j > 0; j >>= 1) {
-            for (uint32_t i = t; i < n_pow2; i += blockDim.x) {
-                const uint32_t l = i ^ j;
-                if (l > i) {
-                    const uint64_t ki = key[i], kl = key[l];
-                    const uint32_t ii = idx[i], il = idx[l];
-                    const bool up = (i & k) == 0;
-                    const bool gt = ki > kl || (ki == kl && ii > il);
-                    if (gt == up) { key[i] = kl; key[l] = ki; idx[i] = il; idx[l] = ii; }
-                }
-            }
-            __syncthreads();
-        }
-    }
-    uint32_t classes = 0, tmax = 0, cmax = 0;
-    for (uint32_t i = t; i < G; i += blockDim.x) {
-        const Gap g = gaps[idx[i]];
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool leader = i < G && not_leader[i] == 0u;
+    if (i < G) {
+        const Gap g = gaps[i];
         Gap o;
-        o.slice = idx[i];   // the original position travels in the slice field
+        o.slice = i;   // the original position travels in the slice field
         o.start = g.start; o.T = g.T; o.C = g.C;
-        sorted[i] = o;
-        if (i == 0 || (uint32_t)(key[i - 1] >> 32) != g.C) ++classes;
-        tmax = max(tmax, g.T);
-        cmax = max(cmax, g.C);
+        sorted[rank[i]] = o;
     }
-    atomicAdd(&s_classes, classes);
-    atomicMax(&s_tmax, tmax);
-    atomicMax(&s_cmax, cmax);
-    __syncthreads();
-    if (t == 0) { info->n_classes = s_classes; info->t_max = s_tmax; info->c_max = s_cmax; info->pad = 0; }
+    const uint32_t n = __popc(__ballot_sync(0xFFFFFFFFu, leader));
+    if ((threadIdx.x & 31u) == 0 && n) atomicAdd(&info->n_classes, n);
 }
 
 // Identity order (used when the batch is too large for the one-CTA sort).
