@@ -24,6 +24,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+from paper_2509_19086_b200 import replicas  # noqa: E402
 from paper_2509_19086_b200 import workloads as wl  # noqa: E402
 
 METRIC = "job-gap pairs evaluated/s"
@@ -237,7 +238,7 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     # replicas: every rank runs an independent scheduler instance on its own seeded workload
-    my_spec = wl.scaled(spec, index=spec.index + 1000 * rank) if rank else spec
+    my_spec = replicas.replica_spec(spec, rank)
     prof = wl.make_profiles(my_spec, threads=max(1, (os.cpu_count() or 8) // max(1, world)))
     gaps = wl.make_gaps(my_spec)
     J, G, N = prof.n_jobs, int(gaps.shape[0]), prof.n_steps
@@ -314,13 +315,10 @@ def main():
             torch.cuda.synchronize()
             e2e_s = time.perf_counter() - t0
 
-    t_ms = torch.tensor([ms_total, 1e3 * e2e_s], dtype=torch.float64, device=device)
-    if dist is not None:
-        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = float(t_ms[0]), float(t_ms[1])
+    total_pairs, (ms_total, e2e_ms) = replicas.aggregate(pairs, [ms_total, 1e3 * e2e_s], dist, device)
     ms_per_step = ms_total / args.steps
-    value = world * pairs * args.steps / (ms_total * 1e-3)
-    e2e_value = world * pairs * args.e2e_steps / (e2e_ms * 1e-3) if e2e_ms > 0 else None
+    value = replicas.throughput(total_pairs, args.steps, ms_total)
+    e2e_value = replicas.throughput(total_pairs, args.e2e_steps, e2e_ms) if e2e_ms > 0 else None
     h2d = sum(int(a.nbytes) for a in host_arrays.values()) + int(gaps.nbytes)
     d2h = 24 * G + 4
 
