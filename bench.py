@@ -34,6 +34,22 @@ POLICY_NAMES = {0: "efficiency", 1: "fairness", 2: "sla"}
 # place_gaps | select_merge (or select_search), finalize_awards | commit_vote, commit_apply, commit_refresh
 KERNELS_PER_STEP = 11
 FALLBACK_HBM_GBS = 6650.0
+# DRAM traffic of the scan kernel from its ncu capture on the 8192-job case (profiles/
+# scan_profiles_kernel_cfg2-jobs8192.md): dram__bytes_read.sum + dram__bytes_write.sum over 33 554 432 steps.
+# Traffic grows in proportion to the step count, so a full launch is this figure times N.  It is only reported
+# while csrc/sja_scan.cuh is the file the counters were taken from (first 16 hex digits of its sha256).
+NCU_SCAN_TRAFFIC_BYTES_PER_STEP = (273.046784e6 + 59.959040e6) / 33554432
+NCU_SCAN_SOURCE_SHA = "ad34fcb17e56902c"
+
+
+def scan_traffic(n_steps: int):
+    import hashlib
+    path = os.path.join(ROOT, "paper_2509_19086_b200", "csrc", "sja_scan.cuh")
+    try:
+        sha = hashlib.sha256(open(path, "rb").read()).hexdigest()[:16]
+    except OSError:
+        return None
+    return NCU_SCAN_TRAFFIC_BYTES_PER_STEP * n_steps if sha == NCU_SCAN_SOURCE_SHA else None
 
 
 def measured_peak():
@@ -328,7 +344,7 @@ def main():
     achieved = scan_bytes / (scan_ms * 1e-3) / 1e9 if scan_ms > 0 else 0.0
     roofline = {
         "kernel": "scan_profiles_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-        "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+        "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": scan_traffic(N),
         "bytes_per_launch": scan_bytes, "ms_per_launch": scan_ms,
     }
     breakdown = {k: timing[k] / args.steps for k in ("scan_ms", "prep_ms", "advertise_ms", "select_ms", "commit_ms")}
