@@ -326,10 +326,10 @@ __global__ void __launch_bounds__(256) copy_gaps_kernel(const Gap* __restrict__ 
 // reduces its 32 x MERGE_R keys to one candidate (largest key, then lowest job id), the CTA
 // folds its warps, and one candidate per (CTA, gap) goes to global memory.
 #ifndef SJA_MERGE_WARPS
-#define SJA_MERGE_WARPS 8
+#define SJA_MERGE_WARPS 16
 #endif
 #ifndef SJA_MERGE_R
-#define SJA_MERGE_R 4
+#define SJA_MERGE_R 2
 #endif
 #ifndef SJA_MERGE_RING
 #define SJA_MERGE_RING 4
@@ -341,7 +341,10 @@ constexpr int MERGE_WARPS = SJA_MERGE_WARPS;
 constexpr int MERGE_R = SJA_MERGE_R;          // jobs per lane
 constexpr int MERGE_RING = SJA_MERGE_RING;    // rows per lane-job ring (power of two)
 constexpr int MERGE_CTAS_PER_SM = SJA_MERGE_CTAS_PER_SM;
-constexpr int MERGE_GT = 64;                  // gaps per staging tile
+#ifndef SJA_MERGE_GT
+#define SJA_MERGE_GT 128
+#endif
+constexpr int MERGE_GT = SJA_MERGE_GT;        // gaps per staging tile
 constexpr int MERGE_JOBS = MERGE_WARPS * MERGE_R * 32;
 constexpr int MERGE_RING_BYTES = MERGE_WARPS * MERGE_R * MERGE_RING * 32 * 16;
 constexpr int MERGE_SMEM_BYTES = MERGE_RING_BYTES + MERGE_GT * MERGE_WARPS * 16 + MERGE_GT * 16;
@@ -474,12 +477,24 @@ __global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_me
                 }
             }
         }
-        best = 0; best_r = 0; best_cnt = 0;
+        // lane-local best over the MERGE_R jobs as a tournament (independent compares first);
+        // on equal keys the lower r, i.e. the lower job id, stays
+        uint64_t kk[MERGE_R];
+        uint32_t rr[MERGE_R], cc[MERGE_R];
 #pragma unroll
         for (int r = 0; r < MERGE_R; ++r) {
-            const uint64_t k = (start >= ready[r]) ? curKey[r] : 0ull;
-            if (k > best) { best = k; best_r = (uint32_t)r; best_cnt = w[r]; }   // strict: lower r wins ties
+            kk[r] = (start >= ready[r]) ? curKey[r] : 0ull;
+            rr[r] = (uint32_t)r;
+            cc[r] = w[r];
         }
+#pragma unroll
+        for (int span = 1; span < MERGE_R; span <<= 1) {
+#pragma unroll
+            for (int r = 0; r + span < MERGE_R; r += 2 * span) {
+                if (kk[r + span] > kk[r]) { kk[r] = kk[r + span]; rr[r] = rr[r + span]; cc[r] = cc[r + span]; }
+            }
+        }
+        best = kk[0]; best_r = rr[0]; best_cnt = cc[0];
     };
     auto publish = [&](const WarpBest& wb, uint32_t gi, uint32_t br, uint32_t bc) {
         if (wb.key == 0ull) {

@@ -250,3 +250,28 @@ def checksum64(a: np.ndarray) -> int:
     with np.errstate(over="ignore"):
         mixed = (w ^ (idx * np.uint64(0x9E3779B97F4A7C15))) * np.uint64(0xBF58476D1CE4E5B9)
         return int(np.bitwise_xor.reduce(mixed) ^ np.add.reduce(mixed))
+
+
+def _main() -> None:
+    """Print the reproducibility table: per configuration the step count and array checksums."""
+    import argparse
+    import time
+
+    ap = argparse.ArgumentParser(description="checksums of the seeded synthetic workloads")
+    ap.add_argument("configs", nargs="*", type=int, default=[0, 1, 2, 3, 4])
+    ap.add_argument("--threads", type=int, default=8)
+    args = ap.parse_args()
+    print("| cfg | seed | jobs | N steps | checksum(dur) | checksum(mem) | checksum(safe) | checksum(ready) | checksum(gaps r0) |")
+    print("|---|---|---|---|---|---|---|---|---|")
+    for c in args.configs:
+        spec = SPECS[c]
+        t0 = time.time()
+        prof = make_profiles(spec, threads=args.threads)
+        gaps = make_gaps(spec)
+        cs = [checksum64(a) for a in (prof.dur_ms, prof.mem_MiB, prof.safe_bits, prof.ready_ms, gaps)]
+        print(f"| {c} | {spec.seed} | {prof.n_jobs} | {prof.n_steps} | " + " | ".join(f"{x:016x}" for x in cs)
+              + f" | <!-- {time.time() - t0:.1f} s -->")
+
+
+if __name__ == "__main__":
+    _main()
