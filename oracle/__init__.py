@@ -9,6 +9,7 @@ Contents
 ``brute.py``       exhaustive prefix enumeration in pure Python, for tiny inputs
 ``scan.py``        the per-job prefix quantities written out with numpy
 ``api.py``         ctypes wrapper around the compiled walk
+``reauction.py``   the round repeated for gaps orphaned by multi-winners (built from the walk)
 """
 from .api import (  # noqa: F401
     AWARD_DTYPE,
@@ -21,4 +22,5 @@ from .api import (  # noqa: F401
     select,
 )
 from .brute import brute_pair, brute_select  # noqa: F401
+from .reauction import round_with_reauction  # noqa: F401
 from .scan import boundary_table, dense_prefix  # noqa: F401
