@@ -222,6 +222,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--flags", type=int, default=0, help="sja_policy.flags (1 = per-pair search kernel)")
+    ap.add_argument("--reauction", action="store_true",
+                    help="time sja_round_reauction (select + commit repeated for orphaned gaps) instead of one select + commit")
     ap.add_argument("--jobs", type=int, default=0, help="override the job count (profiling captures)")
     ap.add_argument("--gaps", type=int, default=0, help="override the gap count (profiling captures)")
     args = ap.parse_args()
@@ -277,12 +279,19 @@ def main():
     dev_gaps = _to_device(gaps, device)
     torch.cuda.synchronize()
 
+    launches = [0]
+
     def step_device():
         ctx.load_profiles(dev["off"], dev["d"], dev["m"], dev["s"], dev["ready"],
                           wait_ms=dev.get("wait"), prio=dev.get("prio"))
         ctx.advertise(dev_gaps)
-        ctx.select(my_spec.policy, flags=args.flags)
-        ctx.commit(want_count=False)
+        if args.reauction:
+            _, passes = ctx.round_reauction(my_spec.policy, flags=args.flags)
+            launches[0] += 6 + 6 * passes      # per pass: select, finalize, 3 commit kernels, orphan compaction
+        else:
+            ctx.select(my_spec.policy, flags=args.flags)
+            ctx.commit(want_count=False)
+            launches[0] += KERNELS_PER_STEP
 
     def step_e2e():
         ctx.load_profiles(pinned["off"], pinned["d"], pinned["m"], pinned["s"], pinned["ready"],
@@ -310,9 +319,11 @@ def main():
         sampler.mark_begin()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
+        launches[0] = 0
         for _ in range(args.steps):
             step_device()
         e1.record(stream)
+        timed_launches = launches[0]
         barrier()
         sampler.mark_end()
         ms_total = e0.elapsed_time(e1)
@@ -358,11 +369,11 @@ def main():
                    "boundary_rows": n_rows, "policy": POLICY_NAMES[spec.policy], "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2 (profile arrays re-read from HBM every step)"
                    if prof.raw_bytes() > 200e6 else "inputs smaller than L2",
-                   "flags": args.flags},
+                   "flags": args.flags, "reauction": bool(args.reauction)},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / max(1, args.e2e_steps), "steps": args.e2e_steps},
-        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "gpu_launches": timed_launches,
         "roofline": roofline,
         "kernel_ms_per_step": breakdown,
         "select_pairs_per_s": pairs / (select_ms * 1e-3) if select_ms > 0 else None,

@@ -193,6 +193,22 @@ sja_status sja_select_static(sja_ctx* ctx, const sja_policy* policy, sja_award* 
  */
 sja_status sja_commit(sja_ctx* ctx, uint32_t* n_granted);
 
+/*
+ * One whole round with re-auction of orphaned gaps: sja_select + sja_commit, then again for
+ * the gaps that had a winner but were not granted because that winner accepted another
+ * gap, until no such gap is left, a pass grants nothing, or max_passes passes ran
+ * (0 = no limit).  Jobs granted in an earlier pass of the call decline in later passes: one
+ * subjob per job and round (one progress point per job, Sections 3.1 and 3.5).  Greedy slot
+ * filling without lookahead is the paper's design (Section 4.2); the re-auction only keeps
+ * it from wasting windows that further jobs had signalled interest in.
+ * A pass-0-only call (max_passes = 1) equals sja_select followed by sja_commit.
+ * The award of a gap (sja_get_awards) is the one of the last pass the gap took part in.
+ * n_granted / n_passes are HOST pointers or NULL.  Waits for completion after every pass.
+ * Uses up the advertised batch like sja_commit.
+ */
+sja_status sja_round_reauction(sja_ctx* ctx, const sja_policy* policy, uint32_t max_passes, uint32_t* n_granted,
+                               uint32_t* n_passes);
+
 /* Copy the G awards of the last select (with `granted` set if it was committed). */
 sja_status sja_get_awards(sja_ctx* ctx, sja_award* out, sja_memspace where);
 

@@ -28,7 +28,7 @@ AWARD_DTYPE = np.dtype([("job", "<u4"), ("end_step", "<u4"), ("dur_ms", "<u4"), 
                         ("score", "<u8")])
 
 EXPORTS = [
-    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit",
+    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit", "sja_round_reauction",
     "sja_get_awards", "sja_get_state", "sja_scan_size", "sja_get_scan", "sja_profile_enable",
     "sja_profile_read", "sja_last_error",
 ]
@@ -74,6 +74,7 @@ def load_library() -> ctypes.CDLL:
     lib.sja_select.argtypes = [vp, ctypes.POINTER(SjaPolicy), vp, i32]
     lib.sja_select_static.argtypes = [vp, ctypes.POINTER(SjaPolicy), vp, i32]
     lib.sja_commit.argtypes = [vp, ctypes.POINTER(u32)]
+    lib.sja_round_reauction.argtypes = [vp, ctypes.POINTER(SjaPolicy), u32, ctypes.POINTER(u32), ctypes.POINTER(u32)]
     lib.sja_get_awards.argtypes = [vp, vp, i32]
     lib.sja_get_state.argtypes = [vp, vp, vp, i32]
     lib.sja_scan_size.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
@@ -215,6 +216,15 @@ class Sja:
             return int(n.value)
         self._check(self._lib.sja_commit(self._h, None))
         return None
+
+    # -- sja_round_reauction
+    def round_reauction(self, policy: int, flags: int = 0, max_passes: int = 0):
+        """select + commit, repeated for gaps orphaned by multi-winners; returns (n_granted, n_passes)."""
+        pol = SjaPolicy(int(policy), int(flags))
+        n, k = ctypes.c_uint32(), ctypes.c_uint32()
+        self._check(self._lib.sja_round_reauction(self._h, ctypes.byref(pol), int(max_passes),
+                                                  ctypes.byref(n), ctypes.byref(k)))
+        return int(n.value), int(k.value)
 
     # -- sja_get_awards / sja_get_state
     def get_awards(self) -> np.ndarray:

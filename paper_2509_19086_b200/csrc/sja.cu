@@ -57,6 +57,7 @@ struct sja_ctx {
     bool gaps_sorted = false;          // sgaps is ordered by (C, T); else it is the caller's order
     uint32_t n_classes = 0;            // distinct capacities of the batch (valid when sorted)
     DevBuf gaps, sgaps, gap_info, gap_rank, awards, widx, partial, winners;
+    DevBuf sgaps_alt, blocked, n_active;   // re-auction: second ordered gap list, per-job block flags, gap counter
 
     // profiling
     bool prof = false;
@@ -220,6 +221,7 @@ JobView job_view(const sja_ctx* c) {
     v.prio = c->have_prio ? c->prio.as<uint8_t>() : nullptr;
     v.A = c->A.as<uint4>();
     v.B = c->B.as<uint2>();
+    v.blocked = nullptr;
     v.J = c->J;
     return v;
 }
@@ -252,6 +254,74 @@ void launch_merge(uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
+
+// Policy argument checks shared by the select entry points.
+sja_status check_policy(sja_ctx* c, const sja_policy* policy, const char* who) {
+    if (!policy) return fail(c, SJA_ERR_INVALID_ARG, "%s: policy is NULL", who);
+    const uint32_t kind = policy->kind;
+    if (kind > SJA_POLICY_SLA) return fail(c, SJA_ERR_INVALID_ARG, "%s: unknown policy %u", who, kind);
+    if (!c->loaded || !c->advertised) return fail(c, SJA_ERR_STATE, "%s before load / advertise", who);
+    if (kind == SJA_POLICY_FAIRNESS && !c->have_wait)
+        return fail(c, SJA_ERR_INVALID_ARG, "fairness policy needs wait_ms at load");
+    if (kind == SJA_POLICY_SLA && !c->have_prio) return fail(c, SJA_ERR_INVALID_ARG, "SLA policy needs prio at load");
+    if (kind == SJA_POLICY_FAIRNESS && (c->load_flags & FLAG_OVF_FAIR))
+        return fail(c, SJA_ERR_OVERFLOW, "fairness score may reach 2^63 for some job");
+    if (kind == SJA_POLICY_SLA && (c->load_flags & FLAG_OVF_SLA))
+        return fail(c, SJA_ERR_OVERFLOW, "SLA key needs work < 2^55 for every job");
+    return SJA_OK;
+}
+
+// Launch signal + score + select for the first G_act entries of `sgaps` (ordered or not);
+// awards and widx are written at the gaps' original indices.  `blocked` may be nullptr.
+sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sgaps, uint32_t G_act,
+                      const uint32_t* blocked) {
+    const uint32_t J = c->J;
+    // The merge kernel pays one restart per capacity class; with very many classes (or an
+    // unsorted batch) the per-pair search is the better tool.
+    const bool use_merge = !(pflags & SJA_FLAG_FORCE_SEARCH) && c->gaps_sorted &&
+                           c->n_classes <= std::max<uint32_t>(64u, c->G / 16u);
+    const uint32_t jobs_per_cta = use_merge ? (uint32_t)MERGE_JOBS : (uint32_t)SEARCH_THREADS;
+    const uint32_t tile = use_merge ? (uint32_t)MERGE_GT : (uint32_t)SEARCH_GT;
+    const uint32_t n_chunks = (J + jobs_per_cta - 1) / jobs_per_cta;
+    TRY(reserve(c, c->partial, (size_t)n_chunks * c->G * sizeof(Partial)));
+    // split the gaps so that the grid covers the SMs several times over
+    uint32_t splits = (uint32_t)((8ull * c->n_sm + n_chunks - 1) / n_chunks);
+    const uint32_t max_splits = (G_act + tile - 1) / tile;
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    uint32_t per_split = (G_act + splits - 1) / splits;
+    per_split = ((per_split + tile - 1) / tile) * tile;
+    splits = (G_act + per_split - 1) / per_split;
+    ProfScope ps(c, CAT_SELECT);
+    JobView jv = job_view(c);
+    jv.blocked = blocked;
+    if (use_merge) {
+        launch_merge(kind, dim3(n_chunks, splits), c->stream, jv, sgaps, G_act, per_split, c->partial.as<Partial>());
+    } else {
+        select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, 0, c->stream>>>(
+            jv, sgaps, G_act, per_split, kind, nullptr, 0, c->partial.as<Partial>());
+    }
+    finalize_awards_kernel<<<(uint32_t)(((uint64_t)G_act * FINALIZE_LANES + 255) / 256), 256, 0, c->stream>>>(
+        jv, c->partial.as<Partial>(), n_chunks, sgaps, G_act, kind, c->awards.as<Award>(), c->widx.as<uint32_t>());
+    return SJA_OK;
+}
+
+// Launch the three commit kernels over all G awards.  `blocked` may be nullptr.
+void run_commit(sja_ctx* c, uint32_t* blocked) {
+    const uint32_t G = c->G;
+    ProfScope ps(c, CAT_COMMIT);
+    const uint32_t gb = (G + 255) / 256;
+    commit_vote_kernel<<<gb, 256, 0, c->stream>>>(c->awards.as<Award>(), G, c->jobwin.as<unsigned long long>(),
+                                                  c->n_granted.as<uint32_t>());
+    commit_apply_kernel<<<gb, 256, 0, c->stream>>>(
+        c->awards.as<Award>(), c->gaps.as<Gap>(), c->widx.as<uint32_t>(), G, c->jobwin.as<unsigned long long>(),
+        c->boff.as<uint64_t>(), c->A.as<uint4>(), c->p.as<uint32_t>(), c->ready.as<uint32_t>(), c->pb.as<uint32_t>(),
+        c->Dp.as<uint32_t>(), c->Wp.as<uint64_t>(), c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(),
+        c->flags.as<uint32_t>(), blocked);
+    commit_refresh_kernel<<<(G * 32 + 255) / 256, 256, 0, c->stream>>>(
+        c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(), G, c->boff.as<uint64_t>(), c->pb.as<uint32_t>(),
+        c->A.as<uint4>(), c->B.as<uint2>(), c->jobwin.as<unsigned long long>());
+}
 
 // ---------------------------------------------------------------------------------------
 // Fixed scratch for sja_select_static: the per-CTA candidate rows of one select call.
@@ -336,7 +406,7 @@ sja_status sja_destroy(sja_ctx* c) {
     cudaStreamSynchronize(c->stream);
     DevBuf* bufs[] = {&c->st_off, &c->st_d, &c->st_m, &c->st_s, &c->st_p, &c->p, &c->ready, &c->pb, &c->Dp,
                       &c->Wp, &c->wait, &c->prio, &c->nbj, &c->cta_tot, &c->cta_base, &c->boff, &c->boff_next, &c->A, &c->B, &c->jobwin,
-                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->awards, &c->widx, &c->partial,
+                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->awards, &c->widx, &c->partial,
                       &c->winners};
     for (DevBuf* b : bufs) release(*b);
     for (ProfSpan& s : c->spans) { cudaEventDestroy(s.a); cudaEventDestroy(s.b); }
@@ -564,59 +634,18 @@ sja_status sja_advertise(sja_ctx* c, uint32_t G, const sja_gap* gaps, sja_memspa
 // ---------------------------------------------------------------------------------------
 sja_status sja_select(sja_ctx* c, const sja_policy* policy, sja_award* out, sja_memspace where) {
     TRY(check_ctx(c));
-    if (!policy) return fail(c, SJA_ERR_INVALID_ARG, "sja_select: policy is NULL");
     if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE)
         return fail(c, SJA_ERR_INVALID_ARG, "sja_select: bad memspace");
-    const uint32_t kind = policy->kind;
-    if (kind > SJA_POLICY_SLA) return fail(c, SJA_ERR_INVALID_ARG, "sja_select: unknown policy %u", kind);
-    if (!c->loaded || !c->advertised) return fail(c, SJA_ERR_STATE, "sja_select before load / advertise");
-    if (kind == SJA_POLICY_FAIRNESS && !c->have_wait)
-        return fail(c, SJA_ERR_INVALID_ARG, "fairness policy needs wait_ms at load");
-    if (kind == SJA_POLICY_SLA && !c->have_prio) return fail(c, SJA_ERR_INVALID_ARG, "SLA policy needs prio at load");
-    if (kind == SJA_POLICY_FAIRNESS && (c->load_flags & FLAG_OVF_FAIR))
-        return fail(c, SJA_ERR_OVERFLOW, "fairness score may reach 2^63 for some job");
-    if (kind == SJA_POLICY_SLA && (c->load_flags & FLAG_OVF_SLA))
-        return fail(c, SJA_ERR_OVERFLOW, "SLA key needs work < 2^55 for every job");
+    TRY(check_policy(c, policy, "sja_select"));
     DeviceGuard guard(c->device);
-
-    const uint32_t G = c->G, J = c->J;
-    // The merge kernel pays one restart per capacity class; with very many classes (or an
-    // unsorted batch) the per-pair search is the better tool.
-    const bool use_merge = !(policy->flags & SJA_FLAG_FORCE_SEARCH) && c->gaps_sorted &&
-                           c->n_classes <= std::max<uint32_t>(64u, G / 16u);
-    const uint32_t jobs_per_cta = use_merge ? (uint32_t)MERGE_JOBS : (uint32_t)SEARCH_THREADS;
-    const uint32_t tile = use_merge ? (uint32_t)MERGE_GT : (uint32_t)SEARCH_GT;
-    const uint32_t n_chunks = (J + jobs_per_cta - 1) / jobs_per_cta;
-    TRY(reserve(c, c->partial, (size_t)n_chunks * G * sizeof(Partial)));
-    // split the gaps so that the grid covers the SMs several times over
-    uint32_t splits = (uint32_t)((8ull * c->n_sm + n_chunks - 1) / n_chunks);
-    const uint32_t max_splits = (G + tile - 1) / tile;
-    if (splits > max_splits) splits = max_splits;
-    if (splits < 1) splits = 1;
-    uint32_t per_split = (G + splits - 1) / splits;
-    per_split = ((per_split + tile - 1) / tile) * tile;
-    splits = (G + per_split - 1) / per_split;
-    {
-        ProfScope ps(c, CAT_SELECT);
-        const JobView jv = job_view(c);
-        if (use_merge) {
-            launch_merge(kind, dim3(n_chunks, splits), c->stream, jv, c->sgaps.as<Gap>(), G, per_split,
-                         c->partial.as<Partial>());
-        } else {
-            select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, 0, c->stream>>>(
-                jv, c->sgaps.as<Gap>(), G, per_split, kind, nullptr, 0, c->partial.as<Partial>());
-        }
-        finalize_awards_kernel<<<(uint32_t)(((uint64_t)G * FINALIZE_LANES + 255) / 256), 256, 0, c->stream>>>(jv, c->partial.as<Partial>(), n_chunks,
-                                                                         c->sgaps.as<Gap>(), G, kind,
-                                                                         c->awards.as<Award>(),
-                                                                         c->widx.as<uint32_t>());
-    }
+    const uint32_t kind = policy->kind;
+    TRY(run_select(c, kind, policy->flags, c->sgaps.as<Gap>(), c->G, nullptr));
     CU(cudaGetLastError());
     c->selected = true;
     c->committed = false;
     c->last_policy = kind;
     if (out) {
-        TRY(copy_out(c, out, c->awards.p, (size_t)G * sizeof(sja_award), where));
+        TRY(copy_out(c, out, c->awards.p, (size_t)c->G * sizeof(sja_award), where));
         if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));
     }
     return SJA_OK;
@@ -697,22 +726,7 @@ sja_status sja_commit(sja_ctx* c, uint32_t* n_granted) {
     if (!c->selected) return fail(c, SJA_ERR_STATE, "sja_commit without a preceding sja_select");
     if (c->committed) return fail(c, SJA_ERR_STATE, "sja_commit called twice for one select");
     DeviceGuard guard(c->device);
-    const uint32_t G = c->G;
-    {
-        ProfScope ps(c, CAT_COMMIT);
-        const uint32_t gb = (G + 255) / 256;
-        commit_vote_kernel<<<gb, 256, 0, c->stream>>>(c->awards.as<Award>(), G,
-                                                      c->jobwin.as<unsigned long long>(),
-                                                      c->n_granted.as<uint32_t>());
-        commit_apply_kernel<<<gb, 256, 0, c->stream>>>(
-            c->awards.as<Award>(), c->gaps.as<Gap>(), c->widx.as<uint32_t>(), G,
-            c->jobwin.as<unsigned long long>(), c->boff.as<uint64_t>(), c->A.as<uint4>(), c->p.as<uint32_t>(),
-            c->ready.as<uint32_t>(), c->pb.as<uint32_t>(), c->Dp.as<uint32_t>(), c->Wp.as<uint64_t>(),
-            c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(), c->flags.as<uint32_t>());
-        commit_refresh_kernel<<<(G * 32 + 255) / 256, 256, 0, c->stream>>>(
-            c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(), G, c->boff.as<uint64_t>(),
-            c->pb.as<uint32_t>(), c->A.as<uint4>(), c->B.as<uint2>(), c->jobwin.as<unsigned long long>());
-    }
+    run_commit(c, nullptr);
     CU(cudaGetLastError());
     c->committed = true;
     c->selected = false;
@@ -726,6 +740,54 @@ sja_status sja_commit(sja_ctx* c, uint32_t* n_granted) {
             CU(cudaMemsetAsync(c->flags.p, 0, 4, c->stream));
             return fail(c, SJA_ERR_OVERFLOW, "start + dur does not fit in 32 bits for a granted job (ready time saturated)");
         }
+    }
+    return SJA_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+sja_status sja_round_reauction(sja_ctx* c, const sja_policy* policy, uint32_t max_passes, uint32_t* n_granted,
+                               uint32_t* n_passes) {
+    TRY(check_ctx(c));
+    TRY(check_policy(c, policy, "sja_round_reauction"));
+    DeviceGuard guard(c->device);
+    const uint32_t kind = policy->kind, G = c->G, J = c->J;
+    TRY(reserve(c, c->sgaps_alt, (size_t)G * sizeof(sja_gap)));
+    TRY(reserve(c, c->blocked, (size_t)J * 4));
+    TRY(reserve(c, c->n_active, 4));
+    CU(cudaMemsetAsync(c->blocked.p, 0, (size_t)J * 4, c->stream));
+
+    const Gap* cur = c->sgaps.as<Gap>();
+    Gap* spare = c->sgaps_alt.as<Gap>();
+    Gap* const own = c->sgaps.as<Gap>();   // only ever written as the spare of a later pass, after it was read
+    uint32_t g_act = G, total = 0, passes = 0;
+    bool overflow = false;
+    while (g_act > 0 && (max_passes == 0 || passes < max_passes)) {
+        TRY(run_select(c, kind, policy->flags, cur, g_act, c->blocked.as<uint32_t>()));
+        run_commit(c, c->blocked.as<uint32_t>());
+        collect_orphans_kernel<<<1, 1024, 0, c->stream>>>(cur, g_act, c->awards.as<Award>(), spare,
+                                                          c->n_active.as<uint32_t>());
+        CU(cudaGetLastError());
+        CU(cudaMemcpyAsync(c->h_words, c->n_granted.p, 4, cudaMemcpyDeviceToHost, c->stream));
+        CU(cudaMemcpyAsync(c->h_words + 1, c->n_active.p, 4, cudaMemcpyDeviceToHost, c->stream));
+        CU(cudaMemcpyAsync(c->h_words + 2, c->flags.p, 4, cudaMemcpyDeviceToHost, c->stream));
+        CU(cudaStreamSynchronize(c->stream));
+        ++passes;
+        total += c->h_words[0];
+        if (c->h_words[2] & FLAG_OVF_READY) overflow = true;
+        if (c->h_words[0] == 0) break;          // nothing granted: the remaining gaps cannot be filled
+        g_act = c->h_words[1];
+        cur = spare;
+        spare = (spare == c->sgaps_alt.as<Gap>()) ? own : c->sgaps_alt.as<Gap>();
+    }
+    c->selected = false;
+    c->committed = true;
+    c->advertised = false;   // sgaps may have been overwritten; advertise the next batch
+    c->last_policy = kind;
+    if (n_granted) *n_granted = total;
+    if (n_passes) *n_passes = passes;
+    if (overflow) {
+        CU(cudaMemsetAsync(c->flags.p, 0, 4, c->stream));
+        return fail(c, SJA_ERR_OVERFLOW, "start + dur does not fit in 32 bits for a granted job (ready time saturated)");
     }
     return SJA_OK;
 }

@@ -18,6 +18,7 @@ struct JobView {
     const uint8_t* prio;    // may be nullptr
     const uint4* A;
     const uint2* B;
+    const uint32_t* blocked;  // may be nullptr; jobs with a non-zero entry decline every gap
     uint32_t J;
 };
 
@@ -54,6 +55,7 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
         const uint32_t pb = jv.pb[j];
         base = b0 + pb;
         n = (uint32_t)(b1 - b0) - pb;
+        if (jv.blocked && jv.blocked[j]) n = 0;
         Dp = jv.Dp[j];
         Wp = jv.Wp[j];
         ready = jv.ready[j];
@@ -167,7 +169,7 @@ __global__ void __launch_bounds__(256) commit_vote_kernel(const Award* __restric
     if (g == 0) *n_granted = 0;
     if (g >= G) return;
     const uint32_t j = awards[g].job;
-    if (j == 0xFFFFFFFFu) return;
+    if (j == 0xFFFFFFFFu || awards[g].granted) return;   // granted: settled in an earlier pass of this round
     const unsigned long long key = ((unsigned long long)awards[g].end_step << 32) | (0xFFFFFFFFu - g);
     atomicMax(jobwin + j, key);
 }
@@ -178,11 +180,11 @@ __global__ void __launch_bounds__(256) commit_apply_kernel(
     const unsigned long long* __restrict__ jobwin, const uint64_t* __restrict__ boff, const uint4* __restrict__ A,
     uint32_t* __restrict__ p, uint32_t* __restrict__ ready, uint32_t* __restrict__ pb, uint32_t* __restrict__ Dp,
     uint64_t* __restrict__ Wp, uint32_t* __restrict__ winners, uint32_t* __restrict__ n_granted,
-    uint32_t* __restrict__ flags) {
+    uint32_t* __restrict__ flags, uint32_t* __restrict__ blocked) {
     const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= G) return;
     Award a = awards[g];
-    if (a.job == 0xFFFFFFFFu) return;
+    if (a.job == 0xFFFFFFFFu || a.granted) return;   // granted: settled in an earlier pass of this round
     const unsigned long long key = ((unsigned long long)a.end_step << 32) | (0xFFFFFFFFu - g);
     if (jobwin[a.job] != key) { awards[g].granted = 0; return; }
     const uint32_t j = a.job;
@@ -196,6 +198,7 @@ __global__ void __launch_bounds__(256) commit_apply_kernel(
     pb[j] = row_rel + 1;
     Dp[j] = r.x;
     Wp[j] = pack64(r.z, r.w);
+    if (blocked) blocked[j] = 1u;   // re-auction: one subjob per job and round
     winners[atomicAdd(n_granted, 1u)] = j;
 }
 
@@ -314,6 +317,50 @@ __global__ void __launch_bounds__(256) copy_gaps_kernel(const Gap* __restrict__ 
 }
 
 // ---------------------------------------------------------------------------------------
+// Re-auction: keep, in their advertised order, the gaps that had a winner but were not
+// granted (their winner accepted another gap).  One CTA walks the ordered list in tiles of
+// 1024 with a block-wide exclusive count; *n_out receives the number of gaps kept.
+__global__ void __launch_bounds__(1024) collect_orphans_kernel(const Gap* __restrict__ sgaps_in, uint32_t G_in,
+                                                               const Award* __restrict__ awards,
+                                                               Gap* __restrict__ sgaps_out,
+                                                               uint32_t* __restrict__ n_out) {
+    __shared__ uint32_t warp_cnt[32];
+    __shared__ uint32_t tile_total;
+    const uint32_t t = threadIdx.x, lane = t & 31u, wid = t >> 5;
+    uint32_t carry = 0;
+    for (uint32_t base = 0; base < G_in; base += 1024) {
+        const uint32_t i = base + t;
+        Gap g;
+        bool keep = false;
+        if (i < G_in) {
+            g = sgaps_in[i];
+            const Award a = awards[g.slice];
+            keep = a.job != 0xFFFFFFFFu && a.granted == 0u;
+        }
+        const uint32_t ball = __ballot_sync(0xFFFFFFFFu, keep);
+        const uint32_t before = __popc(ball & ((1u << lane) - 1u));
+        if (lane == 0) warp_cnt[wid] = __popc(ball);
+        __syncthreads();
+        if (wid == 0) {
+            const uint32_t v = warp_cnt[lane];
+            uint32_t inc = v;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+                if (lane >= (uint32_t)o) inc += y;
+            }
+            warp_cnt[lane] = inc - v;
+            if (lane == 31) tile_total = inc;
+        }
+        __syncthreads();
+        if (keep) sgaps_out[carry + warp_cnt[wid] + before] = g;
+        carry += tile_total;
+        __syncthreads();
+    }
+    if (t == 0) *n_out = carry;
+}
+
+// ---------------------------------------------------------------------------------------
 // Merge kernel.  Each lane owns MERGE_R jobs and walks the gaps of its CTA's range in the
 // advertised order (capacity class, then T ascending).  Per job it keeps a cursor into the
 // job's boundary rows above the progress point: the number w of rows that satisfy both
@@ -409,6 +456,7 @@ __global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_me
             const uint32_t pb = jv.pb[j];
             row0[r] = jv.A + b0 + pb;
             n[r] = (uint32_t)(b1 - b0) - pb;
+            if (jv.blocked && jv.blocked[j]) n[r] = 0;
             Dp[r] = jv.Dp[j];
             Wp[r] = jv.Wp[j];
             ready[r] = jv.ready[j];
