@@ -30,9 +30,9 @@ from paper_2509_19086_b200 import workloads as wl  # noqa: E402
 METRIC = "job-gap pairs evaluated/s"
 UNIT = "pairs/s"
 POLICY_NAMES = {0: "efficiency", 1: "fairness", 2: "sla"}
-# kernels launched per step: count_boundaries, cta_offsets, row_offsets, scan_profiles | rank_gaps,
+# kernels launched per step: count_boundaries, cta_offsets, row_offsets, init_state, scan_profiles | rank_gaps,
 # place_gaps | select_merge (or select_search), finalize_awards | commit_vote, commit_apply, commit_refresh
-KERNELS_PER_STEP = 11
+KERNELS_PER_STEP = 12
 FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the scan kernel from its ncu capture on the 8192-job case (profiles/
 # scan_profiles_kernel_cfg2-jobs8192.md): dram__bytes_read.sum + dram__bytes_write.sum over 33 554 432 steps.
@@ -287,7 +287,7 @@ def main():
         ctx.advertise(dev_gaps)
         if args.reauction:
             _, passes = ctx.round_reauction(my_spec.policy, flags=args.flags)
-            launches[0] += 6 + 6 * passes      # per pass: select, finalize, 3 commit kernels, orphan compaction
+            launches[0] += 7 + 6 * passes      # per pass: select, finalize, 3 commit kernels, orphan compaction
         else:
             ctx.select(my_spec.policy, flags=args.flags)
             ctx.commit(want_count=False)

@@ -459,15 +459,20 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
     DeviceGuard guard(c->device);
     if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
 
-    // N = off[J]
+    // N = off[J].  Host arrays: read it here.  Device arrays: the kernels read it themselves and the
+    // host learns it together with the validation result, so no extra wait is needed -- unless a
+    // profile pointer is NULL, which is only legal for N = 0 and must be known before any launch.
     uint64_t N = 0;
+    bool n_known = true;
     if (where == SJA_MEM_HOST) {
         if (off[0] != 0) return fail(c, SJA_ERR_BAD_PROFILE, "off[0] != 0");
         N = off[J];
-    } else {
+    } else if (!dur_ms || !mem_MiB || !safe_bits) {
         CU(cudaMemcpyAsync(c->h_words, off + J, 8, cudaMemcpyDeviceToHost, c->stream));
         CU(cudaStreamSynchronize(c->stream));
         memcpy(&N, c->h_words, 8);
+    } else {
+        n_known = false;
     }
     if (N >= (1ull << 40)) return fail(c, SJA_ERR_BAD_PROFILE, "off[J] = %llu is implausible", (unsigned long long)N);
     if (N > 0 && (!dur_ms || !mem_MiB || !safe_bits))
@@ -489,7 +494,7 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
         d_d = c->st_d.as<uint32_t>();
         d_m = c->st_m.as<uint32_t>();
         d_s = c->st_s.as<uint32_t>();
-    } else if (N > 0 && (!aligned16(dur_ms) || !aligned16(mem_MiB) || !aligned16(safe_bits))) {
+    } else if ((!n_known || N > 0) && (!aligned16(dur_ms) || !aligned16(mem_MiB) || !aligned16(safe_bits))) {
         return fail(c, SJA_ERR_INVALID_ARG, "sja_load_profiles: device profile arrays must be 16-byte aligned");
     }
     TRY(reserve(c, c->st_p, (size_t)J * 4));
@@ -506,7 +511,7 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
     {
         ProfScope ps(c, CAT_PREP);
         count_boundaries_kernel<<<n_count_ctas, 256, 0, c->stream>>>(
-            d_off, d_s, c->st_p.as<uint32_t>(), J, N, c->nbj.as<uint64_t>(), c->cta_tot.as<uint64_t>(),
+            d_off, d_s, c->st_p.as<uint32_t>(), J, c->nbj.as<uint64_t>(), c->cta_tot.as<uint64_t>(),
             c->flags.as<uint32_t>());
         cta_offsets_kernel<<<1, 1024, 0, c->stream>>>(c->cta_tot.as<uint64_t>(), n_count_ctas,
                                                       c->cta_base.as<uint64_t>());
@@ -516,7 +521,13 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
     CU(cudaGetLastError());
     CU(cudaMemcpyAsync(c->h_words, c->flags.p, 4, cudaMemcpyDeviceToHost, c->stream));
     CU(cudaMemcpyAsync(c->h_words + 2, c->boff_next.as<uint64_t>() + J, 8, cudaMemcpyDeviceToHost, c->stream));
+    if (!n_known) CU(cudaMemcpyAsync(c->h_words + 4, d_off + J, 8, cudaMemcpyDeviceToHost, c->stream));
     CU(cudaStreamSynchronize(c->stream));
+    if (!n_known) {
+        memcpy(&N, c->h_words + 4, 8);
+        if (N >= (1ull << 40) && !(c->h_words[0] & FLAG_BAD_PROFILE))
+            return fail(c, SJA_ERR_BAD_PROFILE, "off[J] = %llu is implausible", (unsigned long long)N);
+    }
     if (c->h_words[0] & FLAG_BAD_PROFILE)
         return fail(c, SJA_ERR_BAD_PROFILE, "profile CSR invalid (offsets not monotone, job too long, or progress > len)");
     uint64_t n_rows = 0;
@@ -538,15 +549,17 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
     std::swap(c->boff, c->boff_next);
     {
         ProfScope ps(c, CAT_PREP);
-        CU(cudaMemcpyAsync(c->p.p, c->st_p.p, (size_t)J * 4, cudaMemcpyDeviceToDevice, c->stream));
-        TRY(copy_in(c, c->ready.p, ready_ms, (size_t)J * 4, where));
-        if (wait_ms) TRY(copy_in(c, c->wait.p, wait_ms, (size_t)J * 4, where));
-        if (prio) TRY(copy_in(c, c->prio.p, prio, (size_t)J, where));
-        CU(cudaMemsetAsync(c->pb.p, 0, (size_t)J * 4, c->stream));
-        CU(cudaMemsetAsync(c->Dp.p, 0, (size_t)J * 4, c->stream));
-        CU(cudaMemsetAsync(c->Wp.p, 0, (size_t)J * 8, c->stream));
-        CU(cudaMemsetAsync(c->jobwin.p, 0, (size_t)J * 8, c->stream));
-        CU(cudaMemsetAsync(c->counter.p, 0, 4, c->stream));
+        const bool dev = where == SJA_MEM_DEVICE;
+        if (!dev) {
+            TRY(copy_in(c, c->ready.p, ready_ms, (size_t)J * 4, where));
+            if (wait_ms) TRY(copy_in(c, c->wait.p, wait_ms, (size_t)J * 4, where));
+            if (prio) TRY(copy_in(c, c->prio.p, prio, (size_t)J, where));
+        }
+        init_state_kernel<<<(J + 255) / 256, 256, 0, c->stream>>>(
+            J, c->st_p.as<uint32_t>(), dev ? ready_ms : nullptr, dev ? wait_ms : nullptr, dev ? prio : nullptr,
+            c->p.as<uint32_t>(), c->ready.as<uint32_t>(), c->wait.as<uint32_t>(), c->prio.as<uint8_t>(),
+            c->pb.as<uint32_t>(), c->Dp.as<uint32_t>(), c->Wp.as<uint64_t>(), c->jobwin.as<unsigned long long>(),
+            c->counter.as<uint32_t>());
     }
     c->J = J;
     c->N = N;
@@ -562,7 +575,7 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
     a.boff = c->boff.as<uint64_t>();
     a.A = c->A.as<uint4>();
     a.B = c->B.as<uint2>();
-    a.N = N; a.J = J;
+    a.J = J;
     a.counter = c->counter.as<uint32_t>();
     a.flags = c->flags.as<uint32_t>();
     if (N > 0) {

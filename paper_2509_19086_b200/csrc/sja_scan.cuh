@@ -43,8 +43,7 @@ struct ScanArgs {
     const uint64_t* boff;    // [J+1] row offsets
     uint4* A;                // rows {D, M, W_lo, W_hi}
     uint2* B;                // rows {k, S}
-    uint64_t N;
-    uint32_t J;
+    uint32_t J;              // N = off[J] is read by the kernel
     uint32_t* counter;       // job hand-out counter (zeroed before launch)
     uint32_t* flags;
 };
@@ -77,9 +76,10 @@ constexpr int COUNT_JOBS_PER_CTA = 256;
 
 __global__ void __launch_bounds__(256) count_boundaries_kernel(
     const uint64_t* __restrict__ off, const uint32_t* __restrict__ sbits,
-    const uint32_t* __restrict__ p0, uint32_t J, uint64_t N, uint64_t* __restrict__ local_off,
+    const uint32_t* __restrict__ p0, uint32_t J, uint64_t* __restrict__ local_off,
     uint64_t* __restrict__ cta_total, uint32_t* __restrict__ flags) {
     __shared__ uint64_t warp_sums[8];
+    const uint64_t N = __ldg(off + J);   // total step count
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
     const uint32_t jbase = blockIdx.x * COUNT_JOBS_PER_CTA + wid * 32u;
     uint32_t mine = 0;   // row count of job jbase + lane
@@ -189,6 +189,28 @@ __global__ void __launch_bounds__(256) row_offsets_kernel(const uint64_t* __rest
     if (j == 0) boff[J] = cta_base[P];
 }
 
+// Per-job state of a fresh load in one launch: progress and attributes copied, cursors and
+// commit votes cleared, the scan's job counter reset.  Source pointers may be nullptr (then
+// the destination was filled by a host-to-device copy, or is not used).
+__global__ void __launch_bounds__(256) init_state_kernel(
+    uint32_t J, const uint32_t* __restrict__ p_src, const uint32_t* __restrict__ ready_src,
+    const uint32_t* __restrict__ wait_src, const uint8_t* __restrict__ prio_src, uint32_t* __restrict__ p,
+    uint32_t* __restrict__ ready, uint32_t* __restrict__ wait, uint8_t* __restrict__ prio, uint32_t* __restrict__ pb,
+    uint32_t* __restrict__ Dp, uint64_t* __restrict__ Wp, unsigned long long* __restrict__ jobwin,
+    uint32_t* __restrict__ counter) {
+    const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j == 0) *counter = 0;
+    if (j >= J) return;
+    p[j] = p_src[j];
+    if (ready_src) ready[j] = ready_src[j];
+    if (wait_src) wait[j] = wait_src[j];
+    if (prio_src) prio[j] = prio_src[j];
+    pb[j] = 0;
+    Dp[j] = 0;
+    Wp[j] = 0;
+    jobwin[j] = 0ull;
+}
+
 // ---------------------------------------------------------------------------------------
 // The scan proper.
 //
@@ -209,6 +231,7 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32, SCAN_CTAS_PER_SM) scan_profil
     const uint32_t wid = threadIdx.x >> 5;
     unsigned char* wbase = smem_raw + (size_t)wid * SCAN_STAGES * SCAN_STAGE_BYTES;
     const uint32_t wbase_s = (uint32_t)__cvta_generic_to_shared(wbase);
+    const uint64_t N_total = __ldg(a.off + a.J);
     const uint32_t lane_sw = (lane ^ ((lane >> 3) & 3u)) * 16u;   // swz(32 r + lane) * 16 - 512 r
     const uint32_t rd_x = (lane >> 1) & 3u;                        // swz(4 lane + r) = 4 lane + (r ^ rd_x)
 
@@ -250,7 +273,7 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32, SCAN_CTAS_PER_SM) scan_profil
                         const uint64_t step = bs + 4ull * c;
                         uint32_t bytes = 0;
                         if (step + 4 > s && step < e) {
-                            const uint64_t left = (a.N - step) * 4ull;
+                            const uint64_t left = (N_total - step) * 4ull;
                             bytes = left < 16 ? (uint32_t)left : 16u;
                         }
                         const uint64_t src = bytes ? step : 0ull;
