@@ -38,8 +38,37 @@ FALLBACK_HBM_GBS = 6650.0
 # scan_profiles_kernel_cfg2-jobs8192.md): dram__bytes_read.sum + dram__bytes_write.sum over 33 554 432 steps.
 # Traffic grows in proportion to the step count, so a full launch is this figure times N.  It is only reported
 # while csrc/sja_scan.cuh is the file the counters were taken from (first 16 hex digits of its sha256).
-NCU_SCAN_TRAFFIC_BYTES_PER_STEP = (273.046784e6 + 59.959040e6) / 33554432
-NCU_SCAN_SOURCE_SHA = "ad34fcb17e56902c"
+NCU_SCAN_TRAFFIC_BYTES_PER_STEP = (273.077248e6 + 62.033664e6) / 33554432
+NCU_SCAN_SOURCE_SHA = "4aeb21ec75c564b0"
+
+
+# Issue-slot roofline of the select kernel (it is bound by instruction issue, not HBM): warp instructions per
+# pair from its ncu capture (profiles/select_merge_kernel_cfg2-jobs32768.md), peak = SMs x 4 schedulers x SM clock.
+NCU_MERGE_WARP_INSTR_PER_PAIR = 163228366 / (32768 * 4096)
+NCU_MERGE_SOURCE_SHA = "87193c0c356ba439"
+N_SM, SCHEDULERS_PER_SM = 148, 4
+
+
+def _source_sha(name: str):
+    import hashlib
+    path = os.path.join(ROOT, "paper_2509_19086_b200", "csrc", name)
+    try:
+        return hashlib.sha256(open(path, "rb").read()).hexdigest()[:16]
+    except OSError:
+        return None
+
+
+def select_roofline(pairs_per_s, sm_mhz):
+    """Issue rate of the select kernel against the GPU's warp-instruction issue peak."""
+    if not pairs_per_s or _source_sha("sja_round.cuh") != NCU_MERGE_SOURCE_SHA:
+        return None
+    mhz = sm_mhz or 1965.0
+    peak = N_SM * SCHEDULERS_PER_SM * mhz * 1e6
+    achieved = pairs_per_s * NCU_MERGE_WARP_INSTR_PER_PAIR
+    return {"kernel": "select_merge_kernel", "bound": "alu", "achieved": achieved / 1e9, "peak": peak / 1e9,
+            "unit": "G warp-instructions/s", "frac": achieved / peak,
+            "peak_kind": f"{N_SM} SMs x {SCHEDULERS_PER_SM} issue slots x {mhz:.0f} MHz",
+            "warp_instr_per_pair": NCU_MERGE_WARP_INSTR_PER_PAIR}
 
 
 def scan_traffic(n_steps: int):
@@ -375,6 +404,7 @@ def main():
                 "ms_per_step": e2e_ms / max(1, args.e2e_steps), "steps": args.e2e_steps},
         "gpu_launches": timed_launches,
         "roofline": roofline,
+        "select_roofline": select_roofline(pairs / (select_ms * 1e-3) if select_ms > 0 else None, clocks.get("sm_mhz")),
         "kernel_ms_per_step": breakdown,
         "select_pairs_per_s": pairs / (select_ms * 1e-3) if select_ms > 0 else None,
         "profile_gb_per_s": prof.raw_bytes() / (scan_ms * 1e-3) / 1e9 if scan_ms > 0 else None,
