@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # Traffic grows in proportion to the step count, so a full launch is this figure times N.  It is only reported
 # while csrc/sja_scan.cuh is the file the counters were taken from (first 16 hex digits of its sha256).
 NCU_SCAN_TRAFFIC_BYTES_PER_STEP = (273.077248e6 + 62.033664e6) / 33554432
-NCU_SCAN_SOURCE_SHA = "4aeb21ec75c564b0"
+NCU_SCAN_SOURCE_SHA = "93addd443eb42e34"
 
 
 # Issue-slot roofline of the select kernel (it is bound by instruction issue, not HBM): warp instructions per

@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "sja_common.cuh"
+#include "sja_prep.cuh"
 #include "sja_round.cuh"
 #include "sja_scan.cuh"
 

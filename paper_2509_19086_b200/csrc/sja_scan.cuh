@@ -67,151 +67,6 @@ __device__ __forceinline__ void cp_async_wait() {
 __device__ __forceinline__ uint32_t swz(uint32_t c) { return c ^ ((c >> 3) & 3u); }
 
 // ---------------------------------------------------------------------------------------
-// Pass 0: validate the CSR and count the boundary rows of every job (popcount of its safe
-// bits above the progress point; the end of a job always counts).  A CTA owns 256
-// consecutive jobs: each warp counts 32 of them one after the other (lanes stride over the
-// job's safe words), the CTA scans the 256 counts and writes each job's offset relative to
-// the CTA plus the CTA total.  Two tiny kernels then turn CTA totals into global offsets.
-constexpr int COUNT_JOBS_PER_CTA = 256;
-
-__global__ void __launch_bounds__(256) count_boundaries_kernel(
-    const uint64_t* __restrict__ off, const uint32_t* __restrict__ sbits,
-    const uint32_t* __restrict__ p0, uint32_t J, uint64_t* __restrict__ local_off,
-    uint64_t* __restrict__ cta_total, uint32_t* __restrict__ flags) {
-    __shared__ uint64_t warp_sums[8];
-    const uint64_t N = __ldg(off + J);   // total step count
-    const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
-    const uint32_t jbase = blockIdx.x * COUNT_JOBS_PER_CTA + wid * 32u;
-    uint32_t mine = 0;   // row count of job jbase + lane
-    for (uint32_t i = 0; i < 32; ++i) {
-        const uint32_t j = jbase + i;
-        if (j >= J) break;
-        const uint64_t js = __ldg(off + j), je = __ldg(off + j + 1);
-        const uint32_t p = __ldg(p0 + j);
-        bool bad = (je < js) || (je > N) || (je - js > 0xFFFFFFFFull) || ((uint64_t)p > je - js);
-        if (j == 0 && js != 0) bad = true;
-        uint32_t cnt = 0;
-        if (bad) {
-            if (lane == 0) atomicOr(flags, FLAG_BAD_PROFILE);
-        } else {
-            const uint64_t s = js + p, e = je;
-            if (s < e) {
-                const uint64_t w0 = s >> 5, w1 = (e - 1) >> 5;
-                for (uint64_t w = w0 + lane; w <= w1; w += 32) {
-                    uint32_t x = __ldg(sbits + w);
-                    if (w == w0) x &= 0xFFFFFFFFu << (uint32_t)(s & 31);
-                    if (w == w1) x &= 0xFFFFFFFFu >> (31u - (uint32_t)((e - 1) & 31));
-                    cnt += __popc(x);
-                }
-                cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
-                const uint32_t lastbit = (__ldg(sbits + w1) >> (uint32_t)((e - 1) & 31)) & 1u;
-                cnt += 1u - lastbit;
-            }
-        }
-        if (lane == i) mine = cnt;
-    }
-    uint64_t inc = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint64_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-        if (lane >= (uint32_t)o) inc += y;
-    }
-    if (lane == 31) warp_sums[wid] = inc;
-    __syncthreads();
-    uint64_t before = 0, total = 0;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) {
-        const uint64_t v = warp_sums[w];
-        if ((uint32_t)w < wid) before += v;
-        total += v;
-    }
-    const uint32_t j = jbase + lane;
-    if (j < J) local_off[j] = before + inc - mine;
-    if (threadIdx.x == 0) cta_total[blockIdx.x] = total;
-}
-
-// Exclusive prefix sum of the per-CTA totals -> base[P+1].  One CTA of 1024 threads walks the
-// array in tiles of 8192 with a running carry.
-__global__ void __launch_bounds__(1024) cta_offsets_kernel(const uint64_t* __restrict__ totals, uint32_t P,
-                                                           uint64_t* __restrict__ base_out) {
-    __shared__ uint64_t warp_sums[32];
-    __shared__ uint64_t warp_excl[32];
-    __shared__ uint64_t tile_total;
-    const uint32_t t = threadIdx.x, lane = t & 31u, wid = t >> 5;
-    uint64_t carry = 0;  // same value in every thread
-    for (uint64_t base = 0; base < P; base += 8192) {
-        uint64_t v[8];
-        uint64_t local = 0;
-        const uint64_t i0 = base + (uint64_t)t * 8;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            v[i] = (i0 + i < P) ? totals[i0 + i] : 0ull;
-            local += v[i];
-        }
-        uint64_t inc = local;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint64_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-            if (lane >= (uint32_t)o) inc += y;
-        }
-        if (lane == 31) warp_sums[wid] = inc;
-        __syncthreads();
-        if (wid == 0) {
-            const uint64_t ws = warp_sums[lane];
-            uint64_t wi = ws;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint64_t y = __shfl_up_sync(0xFFFFFFFFu, wi, o);
-                if (lane >= (uint32_t)o) wi += y;
-            }
-            warp_excl[lane] = wi - ws;
-            if (lane == 31) tile_total = wi;
-        }
-        __syncthreads();
-        uint64_t run = carry + warp_excl[wid] + (inc - local);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            if (i0 + i < P) base_out[i0 + i] = run;
-            run += v[i];
-        }
-        carry += tile_total;
-        __syncthreads();  // warp_sums / tile_total are rewritten by the next tile
-    }
-    if (t == 0) base_out[P] = carry;
-}
-
-// boff[j] = base of the job's CTA + offset inside the CTA; boff[J] = total row count.
-__global__ void __launch_bounds__(256) row_offsets_kernel(const uint64_t* __restrict__ local_off,
-                                                          const uint64_t* __restrict__ cta_base, uint32_t J,
-                                                          uint32_t P, uint64_t* __restrict__ boff) {
-    const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j < J) boff[j] = cta_base[j / COUNT_JOBS_PER_CTA] + local_off[j];
-    if (j == 0) boff[J] = cta_base[P];
-}
-
-// Per-job state of a fresh load in one launch: progress and attributes copied, cursors and
-// commit votes cleared, the scan's job counter reset.  Source pointers may be nullptr (then
-// the destination was filled by a host-to-device copy, or is not used).
-__global__ void __launch_bounds__(256) init_state_kernel(
-    uint32_t J, const uint32_t* __restrict__ p_src, const uint32_t* __restrict__ ready_src,
-    const uint32_t* __restrict__ wait_src, const uint8_t* __restrict__ prio_src, uint32_t* __restrict__ p,
-    uint32_t* __restrict__ ready, uint32_t* __restrict__ wait, uint8_t* __restrict__ prio, uint32_t* __restrict__ pb,
-    uint32_t* __restrict__ Dp, uint64_t* __restrict__ Wp, unsigned long long* __restrict__ jobwin,
-    uint32_t* __restrict__ counter) {
-    const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j == 0) *counter = 0;
-    if (j >= J) return;
-    p[j] = p_src[j];
-    if (ready_src) ready[j] = ready_src[j];
-    if (wait_src) wait[j] = wait_src[j];
-    if (prio_src) prio[j] = prio_src[j];
-    pb[j] = 0;
-    Dp[j] = 0;
-    Wp[j] = 0;
-    jobwin[j] = 0ull;
-}
-
-// ---------------------------------------------------------------------------------------
 // The scan proper.
 //
 // Per 512-step block a warp knows, after one popcount scan, how many rows the block emits.
