@@ -51,10 +51,10 @@ def _load():
     lib.orc_pair.restype = ctypes.c_int
     lib.orc_pair.argtypes = [vp, vp, vp, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint32,
                              ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
-                             u32p, u32p, u64p]
+                             ctypes.c_uint32, ctypes.c_uint32, u32p, u32p, u64p]
     lib.orc_select.restype = ctypes.c_int
     lib.orc_select.argtypes = [ctypes.c_uint32, vp, vp, vp, vp, vp, vp, vp, vp,
-                               ctypes.c_uint32, vp, ctypes.c_uint32, vp]
+                               ctypes.c_uint32, vp, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, vp]
     lib.orc_commit.restype = ctypes.c_int64
     lib.orc_commit.argtypes = [ctypes.c_uint32, vp, vp, ctypes.c_uint32, vp, vp]
     lib.orc_num_threads.restype = ctypes.c_int
@@ -79,8 +79,13 @@ def num_threads() -> int:
     return int(_load().orc_num_threads())
 
 
-def pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: int):
-    """R1-R3 for one (gap, job) pair: ``None`` for decline, else ``(k, dur, work)``."""
+U32MAX = 0xFFFFFFFF
+
+
+def pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: int,
+         tau_min_ms: int = 0, tau_max_ms: int = U32MAX):
+    """R1-R3 (with the duration thresholds of R2') for one (gap, job) pair: ``None`` for decline,
+    else ``(k, dur, work)``."""
     lib = _load()
     k = ctypes.c_uint32()
     dur = ctypes.c_uint32()
@@ -88,14 +93,14 @@ def pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: i
     ok = lib.orc_pair(prof.dur_ms.ctypes.data, prof.mem_MiB.ctypes.data,
                       prof.safe_bits.ctypes.data, int(prof.off[j]), int(prof.off[j + 1]),
                       int(p), int(ready_ms), int(start_ms), int(T_ms), int(C_MiB),
-                      ctypes.byref(k), ctypes.byref(dur), ctypes.byref(work))
+                      int(tau_min_ms), int(tau_max_ms), ctypes.byref(k), ctypes.byref(dur), ctypes.byref(work))
     if not ok:
         return None
     return int(k.value), int(dur.value), int(work.value)
 
 
 def select(prof, progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray,
-           policy: int) -> np.ndarray:
+           policy: int, tau_min_ms: int = 0, tau_max_ms: int = U32MAX) -> np.ndarray:
     """R1-R5 for a batch of gaps; returns ``AWARD_DTYPE[G]`` (``granted`` all zero)."""
     lib = _load()
     off = _as(prof.off, np.uint64)
@@ -110,7 +115,8 @@ def select(prof, progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray,
     awards = np.zeros(gaps.shape[0], dtype=AWARD_DTYPE)
     rc = lib.orc_select(off.shape[0] - 1, _ptr(off), _ptr(d), _ptr(m), _ptr(s),
                         _ptr(progress), _ptr(ready_ms), _ptr(wait), _ptr(prio),
-                        gaps.shape[0], _ptr(gaps), int(policy), _ptr(awards))
+                        gaps.shape[0], _ptr(gaps), int(policy), int(tau_min_ms), int(tau_max_ms),
+                        _ptr(awards))
     if rc != 0:
         raise ValueError("oracle select: unknown policy or missing attribute array")
     return awards

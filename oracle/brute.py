@@ -15,7 +15,8 @@ def _safe(bits, i: int) -> bool:
     return bool((int(bits[i >> 5]) >> (i & 31)) & 1)
 
 
-def brute_pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: int):
+def brute_pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: int,
+               tau_min_ms: int = 0, tau_max_ms: int = 0xFFFFFFFF):
     """``None`` (decline) or ``(k, dur, work)`` of the longest feasible subjob."""
     s, e = int(prof.off[j]), int(prof.off[j + 1])
     length = e - s
@@ -31,6 +32,8 @@ def brute_pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_
         if not ends_safe:
             continue
         if sum(d[p:k]) > T_ms:
+            continue
+        if not (tau_min_ms <= sum(d[p:k]) <= tau_max_ms):      # Section 4.3 (5) thresholds
             continue
         if max(m[p:k]) > C_MiB:
             continue

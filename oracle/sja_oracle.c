@@ -32,6 +32,10 @@
  *                    SLA         lexicographic (prio_j, work), larger prio = more urgent.
  *   R5 select      : per gap, the interested job with the largest key; ties go to the
  *                    lowest job id; no interested job -> SJA_NO_JOB and zeros.
+ *   R2' bounds     : optional subjob duration thresholds (Section 4.3, item 5: minimum and maximum
+ *                    subjob duration enforced at the framework level): a candidate also needs
+ *                    tau_min <= sum d[p_j..k) <= tau_max.  tau_min = 0 and tau_max = 2^32-1 switch
+ *                    them off.
  *   R6 commit      : a job that won several gaps accepts the one with the largest k*,
  *                    ties to the lowest gap id; that gap is granted, the others are not;
  *                    then p_j = k*, ready_j = start_g + dur.
@@ -78,6 +82,7 @@ static int step_is_safe(const uint32_t *safe_bits, uint64_t i)
 int orc_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *safe_bits,
              uint64_t s, uint64_t e, uint32_t p, uint32_t ready_ms,
              uint32_t start_ms, uint32_t T_ms, uint32_t C_MiB,
+             uint32_t tau_min_ms, uint32_t tau_max_ms,
              uint32_t *k_out, uint32_t *dur_out, uint64_t *work_out)
 {
     uint64_t len = e - s;
@@ -94,7 +99,9 @@ int orc_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *sa
         if (mem_MiB[i] > peak) peak = mem_MiB[i];
         work += (uint64_t)dur_ms[i] * (uint64_t)mem_MiB[i];
         if (acc > (uint64_t)T_ms || peak > C_MiB) break;   /* R2: window or capacity broken */
-        if (step_is_safe(safe_bits, i) || i + 1 == e) {    /* R2: safe boundary after step i */
+        if (acc > (uint64_t)tau_max_ms) break;             /* R2': longer than the maximum subjob */
+        if ((step_is_safe(safe_bits, i) || i + 1 == e)     /* R2: safe boundary after step i */
+            && acc >= (uint64_t)tau_min_ms) {              /* R2': not shorter than the minimum subjob */
             found = 1;
             best_k = (uint32_t)(i + 1 - s);
             best_dur = (uint32_t)acc;
@@ -132,6 +139,7 @@ int orc_select(uint32_t n_jobs, const uint64_t *off,
                const uint32_t *progress, const uint32_t *ready_ms,
                const uint32_t *wait_ms, const uint8_t *prio,
                uint32_t n_gaps, const orc_gap *gaps, uint32_t policy,
+               uint32_t tau_min_ms, uint32_t tau_max_ms,
                orc_award *awards)
 {
     if (policy > ORC_SLA) return -1;
@@ -148,7 +156,8 @@ int orc_select(uint32_t n_jobs, const uint64_t *off,
             uint32_t k, dur;
             uint64_t work;
             if (!orc_pair(dur_ms, mem_MiB, safe_bits, off[j], off[j + 1], progress[j],
-                          ready_ms[j], gap.start_ms, gap.T_ms, gap.C_MiB, &k, &dur, &work))
+                          ready_ms[j], gap.start_ms, gap.T_ms, gap.C_MiB, tau_min_ms, tau_max_ms,
+                          &k, &dur, &work))
                 continue;                                      /* decline */
             uint32_t cls;
             uint64_t score;
