@@ -194,6 +194,15 @@ sja_status sja_select_static(sja_ctx* ctx, const sja_policy* policy, sja_award* 
 sja_status sja_commit(sja_ctx* ctx, uint32_t* n_granted);
 
 /*
+ * sja_commit for a round in which some grants are not taken up: a subjob that failed or was
+ * never started affects only itself, its parent job stays at the last completed fragment
+ * (Section 3.10).  accept is u8[G] in the order the gaps were advertised; a gap with
+ * accept[g] = 0 takes no part in the commit (its award keeps granted = 0, and a job that also
+ * won an accepted gap is granted that one).  Otherwise identical to sja_commit.
+ */
+sja_status sja_commit_masked(sja_ctx* ctx, const uint8_t* accept, sja_memspace where, uint32_t* n_granted);
+
+/*
  * One whole round with re-auction of orphaned gaps: sja_select + sja_commit, then again for
  * the gaps that had a winner but were not granted because that winner accepted another
  * gap, until no such gap is left, a pass grants nothing, or max_passes passes ran
@@ -208,6 +217,16 @@ sja_status sja_commit(sja_ctx* ctx, uint32_t* n_granted);
  */
 sja_status sja_round_reauction(sja_ctx* ctx, const sja_policy* policy, uint32_t max_passes, uint32_t* n_granted,
                                uint32_t* n_passes);
+
+/*
+ * Subjob granularity guard (Section 4.3, item 5: minimum and maximum subjob duration thresholds
+ * enforced at the framework level).  From the next select on, a subjob is a candidate only if
+ * tau_min_ms <= its duration <= tau_max_ms, on top of the window and capacity bounds: the
+ * longest subjob with duration <= min(T, tau_max) is taken, and the job declines if that one
+ * is shorter than tau_min.  Defaults 0 and 0xFFFFFFFF switch the guard off.  Stays in force
+ * until changed; tau_min_ms > tau_max_ms is SJA_ERR_INVALID_ARG.
+ */
+sja_status sja_set_duration_bounds(sja_ctx* ctx, uint32_t tau_min_ms, uint32_t tau_max_ms);
 
 /* Copy the G awards of the last select (with `granted` set if it was committed). */
 sja_status sja_get_awards(sja_ctx* ctx, sja_award* out, sja_memspace where);

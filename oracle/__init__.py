@@ -17,6 +17,7 @@ from .api import (  # noqa: F401
     NO_JOB,
     build,
     commit,
+    commit_masked,
     num_threads,
     pair,
     select,

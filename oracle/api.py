@@ -135,3 +135,19 @@ def commit(progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray,
     if n < 0:
         raise OverflowError("oracle commit: start + dur does not fit in 32 bits")
     return int(n)
+
+
+def commit_masked(progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray, awards: np.ndarray,
+                  accept: np.ndarray) -> int:
+    """R6 restricted to the gaps with ``accept[g] != 0``.
+
+    A subjob that failed or was never started leaves its parent job at the last completed
+    fragment (Section 3.10): such a grant is simply not committed.  Gaps that are not accepted take
+    no part in R6 (a job that also won an accepted gap is granted that one) and stay ungranted.
+    """
+    accept = np.asarray(accept).astype(bool)
+    visible = awards.copy()
+    visible["job"][~accept] = NO_JOB
+    n = commit(progress, ready_ms, gaps, visible)
+    awards["granted"] = visible["granted"]
+    return n

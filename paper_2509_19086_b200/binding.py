@@ -28,7 +28,7 @@ AWARD_DTYPE = np.dtype([("job", "<u4"), ("end_step", "<u4"), ("dur_ms", "<u4"), 
                         ("score", "<u8")])
 
 EXPORTS = [
-    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit", "sja_round_reauction",
+    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit", "sja_commit_masked", "sja_round_reauction", "sja_set_duration_bounds",
     "sja_get_awards", "sja_get_state", "sja_scan_size", "sja_get_scan", "sja_profile_enable",
     "sja_profile_read", "sja_last_error",
 ]
@@ -75,6 +75,8 @@ def load_library() -> ctypes.CDLL:
     lib.sja_select_static.argtypes = [vp, ctypes.POINTER(SjaPolicy), vp, i32]
     lib.sja_commit.argtypes = [vp, ctypes.POINTER(u32)]
     lib.sja_round_reauction.argtypes = [vp, ctypes.POINTER(SjaPolicy), u32, ctypes.POINTER(u32), ctypes.POINTER(u32)]
+    lib.sja_set_duration_bounds.argtypes = [vp, u32, u32]
+    lib.sja_commit_masked.argtypes = [vp, vp, i32, ctypes.POINTER(u32)]
     lib.sja_get_awards.argtypes = [vp, vp, i32]
     lib.sja_get_state.argtypes = [vp, vp, vp, i32]
     lib.sja_scan_size.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64)]
@@ -217,6 +219,14 @@ class Sja:
         self._check(self._lib.sja_commit(self._h, None))
         return None
 
+    # -- sja_commit_masked
+    def commit_masked(self, accept) -> int:
+        """sja_commit_masked: ``accept`` is a u8 array (numpy or CUDA tensor) with one entry per gap."""
+        p, space, _keep = _ptr_space(accept, None, np.uint8)
+        n = ctypes.c_uint32()
+        self._check(self._lib.sja_commit_masked(self._h, p, space, ctypes.byref(n)))
+        return int(n.value)
+
     # -- sja_round_reauction
     def round_reauction(self, policy: int, flags: int = 0, max_passes: int = 0):
         """select + commit, repeated for gaps orphaned by multi-winners; returns (n_granted, n_passes)."""
@@ -225,6 +235,10 @@ class Sja:
         self._check(self._lib.sja_round_reauction(self._h, ctypes.byref(pol), int(max_passes),
                                                   ctypes.byref(n), ctypes.byref(k)))
         return int(n.value), int(k.value)
+
+    # -- sja_set_duration_bounds
+    def set_duration_bounds(self, tau_min_ms: int = 0, tau_max_ms: int = 0xFFFFFFFF) -> None:
+        self._check(self._lib.sja_set_duration_bounds(self._h, int(tau_min_ms), int(tau_max_ms)))
 
     # -- sja_get_awards / sja_get_state
     def get_awards(self) -> np.ndarray:

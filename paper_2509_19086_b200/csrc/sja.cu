@@ -55,10 +55,11 @@ struct sja_ctx {
     // gaps / awards
     bool advertised = false, selected = false, committed = false;
     uint32_t G = 0, last_policy = 0;
+    uint32_t tau_min = 0, tau_max = 0xFFFFFFFFu;   // subjob duration thresholds for select
     bool gaps_sorted = false;          // sgaps is ordered by (C, T); else it is the caller's order
     uint32_t n_classes = 0;            // distinct capacities of the batch (valid when sorted)
     DevBuf gaps, sgaps, gap_info, gap_rank, awards, widx, partial, winners;
-    DevBuf sgaps_alt, blocked, n_active;   // re-auction: second ordered gap list, per-job block flags, gap counter
+    DevBuf sgaps_alt, blocked, n_active, accept;   // re-auction: second ordered gap list, per-job block flags, gap counter
 
     // profiling
     bool prof = false;
@@ -223,6 +224,8 @@ JobView job_view(const sja_ctx* c) {
     v.A = c->A.as<uint4>();
     v.B = c->B.as<uint2>();
     v.blocked = nullptr;
+    v.tau_min = c->tau_min;
+    v.tau_max = c->tau_max;
     v.J = c->J;
     return v;
 }
@@ -308,17 +311,17 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
 }
 
 // Launch the three commit kernels over all G awards.  `blocked` may be nullptr.
-void run_commit(sja_ctx* c, uint32_t* blocked) {
+void run_commit(sja_ctx* c, uint32_t* blocked, const uint8_t* accept = nullptr) {
     const uint32_t G = c->G;
     ProfScope ps(c, CAT_COMMIT);
     const uint32_t gb = (G + 255) / 256;
     commit_vote_kernel<<<gb, 256, 0, c->stream>>>(c->awards.as<Award>(), G, c->jobwin.as<unsigned long long>(),
-                                                  c->n_granted.as<uint32_t>());
+                                                  c->n_granted.as<uint32_t>(), accept);
     commit_apply_kernel<<<gb, 256, 0, c->stream>>>(
         c->awards.as<Award>(), c->gaps.as<Gap>(), c->widx.as<uint32_t>(), G, c->jobwin.as<unsigned long long>(),
         c->boff.as<uint64_t>(), c->A.as<uint4>(), c->p.as<uint32_t>(), c->ready.as<uint32_t>(), c->pb.as<uint32_t>(),
         c->Dp.as<uint32_t>(), c->Wp.as<uint64_t>(), c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(),
-        c->flags.as<uint32_t>(), blocked);
+        c->flags.as<uint32_t>(), blocked, accept);
     commit_refresh_kernel<<<(G * 32 + 255) / 256, 256, 0, c->stream>>>(
         c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(), G, c->boff.as<uint64_t>(), c->pb.as<uint32_t>(),
         c->A.as<uint4>(), c->B.as<uint2>(), c->jobwin.as<unsigned long long>());
@@ -407,7 +410,7 @@ sja_status sja_destroy(sja_ctx* c) {
     cudaStreamSynchronize(c->stream);
     DevBuf* bufs[] = {&c->st_off, &c->st_d, &c->st_m, &c->st_s, &c->st_p, &c->p, &c->ready, &c->pb, &c->Dp,
                       &c->Wp, &c->wait, &c->prio, &c->nbj, &c->cta_tot, &c->cta_base, &c->boff, &c->boff_next, &c->A, &c->B, &c->jobwin,
-                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->awards, &c->widx, &c->partial,
+                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->awards, &c->widx, &c->partial,
                       &c->winners};
     for (DevBuf* b : bufs) release(*b);
     for (ProfSpan& s : c->spans) { cudaEventDestroy(s.a); cudaEventDestroy(s.b); }
@@ -735,12 +738,10 @@ sja_status sja_select_static(sja_ctx* c, const sja_policy* policy, sja_award* ou
 }
 
 // ---------------------------------------------------------------------------------------
-sja_status sja_commit(sja_ctx* c, uint32_t* n_granted) {
-    TRY(check_ctx(c));
-    if (!c->selected) return fail(c, SJA_ERR_STATE, "sja_commit without a preceding sja_select");
-    if (c->committed) return fail(c, SJA_ERR_STATE, "sja_commit called twice for one select");
-    DeviceGuard guard(c->device);
-    run_commit(c, nullptr);
+static sja_status commit_impl(sja_ctx* c, const uint8_t* accept, uint32_t* n_granted, const char* who) {
+    if (!c->selected) return fail(c, SJA_ERR_STATE, "%s without a preceding sja_select", who);
+    if (c->committed) return fail(c, SJA_ERR_STATE, "%s: this select was already committed", who);
+    run_commit(c, nullptr, accept);
     CU(cudaGetLastError());
     c->committed = true;
     c->selected = false;
@@ -756,6 +757,26 @@ sja_status sja_commit(sja_ctx* c, uint32_t* n_granted) {
         }
     }
     return SJA_OK;
+}
+
+sja_status sja_commit(sja_ctx* c, uint32_t* n_granted) {
+    TRY(check_ctx(c));
+    DeviceGuard guard(c->device);
+    return commit_impl(c, nullptr, n_granted, "sja_commit");
+}
+
+sja_status sja_commit_masked(sja_ctx* c, const uint8_t* accept, sja_memspace where, uint32_t* n_granted) {
+    TRY(check_ctx(c));
+    if (!accept) return fail(c, SJA_ERR_INVALID_ARG, "sja_commit_masked: accept is NULL");
+    if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_commit_masked: bad memspace");
+    if (!c->selected) return fail(c, SJA_ERR_STATE, "sja_commit_masked without a preceding sja_select");
+    DeviceGuard guard(c->device);
+    TRY(reserve(c, c->accept, c->G));
+    TRY(copy_in(c, c->accept.p, accept, c->G, where));
+    const sja_status st = commit_impl(c, c->accept.as<uint8_t>(), n_granted, "sja_commit_masked");
+    if (st == SJA_OK && where == SJA_MEM_HOST && !n_granted) CU(cudaStreamSynchronize(c->stream));
+    return st;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -803,6 +824,16 @@ sja_status sja_round_reauction(sja_ctx* c, const sja_policy* policy, uint32_t ma
         CU(cudaMemsetAsync(c->flags.p, 0, 4, c->stream));
         return fail(c, SJA_ERR_OVERFLOW, "start + dur does not fit in 32 bits for a granted job (ready time saturated)");
     }
+    return SJA_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+sja_status sja_set_duration_bounds(sja_ctx* c, uint32_t tau_min_ms, uint32_t tau_max_ms) {
+    TRY(check_ctx(c));
+    if (tau_min_ms > tau_max_ms)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_set_duration_bounds: tau_min %u > tau_max %u", tau_min_ms, tau_max_ms);
+    c->tau_min = tau_min_ms;
+    c->tau_max = tau_max_ms;
     return SJA_OK;
 }
 

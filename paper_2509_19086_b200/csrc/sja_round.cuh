@@ -19,6 +19,7 @@ struct JobView {
     const uint4* A;
     const uint2* B;
     const uint32_t* blocked;  // may be nullptr; jobs with a non-zero entry decline every gap
+    uint32_t tau_min, tau_max;  // subjob duration thresholds (Section 4.3, item 5); 0 / 0xFFFFFFFF = off
     uint32_t J;
 };
 
@@ -68,7 +69,7 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
         const uint32_t gt = min((uint32_t)SEARCH_GT, g_end - g0);
         for (uint32_t gi = 0; gi < gt; ++gi) {
             const uint4 gq = __ldg(reinterpret_cast<const uint4*>(gaps) + g0 + gi);
-            const uint32_t start = gq.y, T = gq.z, C = gq.w;
+            const uint32_t start = gq.y, T = min(gq.z, jv.tau_max), C = gq.w;
             uint32_t cnt = 0;
             uint64_t key = 0;
             if (n != 0 && start >= ready) {
@@ -87,7 +88,8 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
                 cnt = lo;
                 if (cnt) {
                     const uint4 r = __ldg(jv.A + base + cnt - 1);
-                    key = policy_key(kind, pack64(r.z, r.w) - Wp, factor);
+                    if (r.x - Dp >= jv.tau_min) key = policy_key(kind, pack64(r.z, r.w) - Wp, factor);
+                    else cnt = 0;   // the longest fitting subjob is shorter than the minimum: decline
                 }
             }
             const uint64_t mk = warp_max_u64(key);
@@ -164,10 +166,12 @@ __global__ void __launch_bounds__(256) finalize_awards_kernel(
 // lowest gap id (one atomicMax on a packed key; the order of the atomics does not matter).
 __global__ void __launch_bounds__(256) commit_vote_kernel(const Award* __restrict__ awards, uint32_t G,
                                                           unsigned long long* __restrict__ jobwin,
-                                                          uint32_t* __restrict__ n_granted) {
+                                                          uint32_t* __restrict__ n_granted,
+                                                          const uint8_t* __restrict__ accept) {
     const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g == 0) *n_granted = 0;
     if (g >= G) return;
+    if (accept && !accept[g]) return;   // grant not taken up (failed subjob): no part in the commit
     const uint32_t j = awards[g].job;
     if (j == 0xFFFFFFFFu || awards[g].granted) return;   // granted: settled in an earlier pass of this round
     const unsigned long long key = ((unsigned long long)awards[g].end_step << 32) | (0xFFFFFFFFu - g);
@@ -180,9 +184,10 @@ __global__ void __launch_bounds__(256) commit_apply_kernel(
     const unsigned long long* __restrict__ jobwin, const uint64_t* __restrict__ boff, const uint4* __restrict__ A,
     uint32_t* __restrict__ p, uint32_t* __restrict__ ready, uint32_t* __restrict__ pb, uint32_t* __restrict__ Dp,
     uint64_t* __restrict__ Wp, uint32_t* __restrict__ winners, uint32_t* __restrict__ n_granted,
-    uint32_t* __restrict__ flags, uint32_t* __restrict__ blocked) {
+    uint32_t* __restrict__ flags, uint32_t* __restrict__ blocked, const uint8_t* __restrict__ accept) {
     const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= G) return;
+    if (accept && !accept[g]) return;
     Award a = awards[g];
     if (a.job == 0xFFFFFFFFu || a.granted) return;   // granted: settled in an earlier pass of this round
     const unsigned long long key = ((unsigned long long)a.end_step << 32) | (0xFFFFFFFFu - g);
@@ -470,7 +475,7 @@ __global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_me
 
     // Cursor update and lane-local best candidate for one gap.
     auto eval_gap = [&](const uint4 gq, uint64_t& best, uint32_t& best_r, uint32_t& best_cnt) {
-        const uint32_t start = gq.y, T = gq.z, C = gq.w;
+        const uint32_t start = gq.y, T = min(gq.z, jv.tau_max), C = gq.w;
         if (first || C != curC) {
             // new capacity class: T restarts from its smallest value, so do the cursors
             first = false;
@@ -508,7 +513,8 @@ __global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_me
             for (int r = 0; r < MERGE_R; ++r) {
                 while (((open >> r) & 1u) && T >= thr[r]) {
                     // row w qualifies: it becomes the candidate; fetch row w + 1 from the ring
-                    curKey[r] = policy_key(KIND, nextW[r] - Wp[r], factor[r]);
+                    // (a subjob shorter than the minimum duration is no candidate; longer rows may be)
+                    curKey[r] = thr[r] >= jv.tau_min ? policy_key(KIND, nextW[r] - Wp[r], factor[r]) : 0ull;
                     if (w[r] + MERGE_RING < n[r])
                         mg_cp_async16(ring_s[r] + (w[r] & (MERGE_RING - 1)) * 32 * 16, next_row[r]);
                     mg_commit();
