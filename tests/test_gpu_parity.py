@@ -308,3 +308,25 @@ def test_empty_and_degenerate_inputs(sja_mod, oracle_mod):
         want = oracle_mod.select(prof2, progress, prof2.ready_ms, gaps_from_lists([(0, 0, 0, 7), (0, 0, 0, 6)]), 0)
         _assert_awards_equal(got, want)
         assert got["job"].tolist() == [1, 1] and got["end_step"].tolist() == [2, 1]   # zero-work interest
+
+
+def test_select_very_large_gap_batch_unsorted_path(sja_mod, oracle_mod):
+    """More gaps than the ranking kernel orders (65 536): the batch stays in the caller's order and
+    the per-pair search kernel serves it."""
+    spec = wl.scaled(wl.SPECS[1], n_jobs=300, fixed_len=200, n_gaps=70000)
+    prof = wl.make_profiles(spec, threads=2)
+    gaps = wl.make_gaps(spec)
+    progress = np.zeros(prof.n_jobs, np.uint32)
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof)
+        ctx.advertise(gaps)
+        got = ctx.select(spec.policy, out="host")
+        want = oracle_mod.select(prof, progress, prof.ready_ms, gaps, spec.policy)
+        _assert_awards_equal(got, want)
+        assert ctx.commit() == oracle_mod.commit(progress, prof.ready_ms.copy(), gaps, want)
+        _assert_awards_equal(ctx.get_awards(), want, fields=("job", "end_step", "dur_ms", "score", "granted"))
+        # exactly at the limit the ordered path runs
+        ctx.load_profiles(prof.off, prof.dur_ms, prof.mem_MiB, prof.safe_bits, prof.ready_ms)
+        ctx.advertise(gaps[:65536])
+        got = ctx.select(spec.policy, out="host")
+        _assert_awards_equal(got, want[:65536])
