@@ -36,7 +36,9 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
             if (j == 0 && js != 0) bad = true;
             if (!bad) {
                 const uint64_t s = js + p, e = je;
-                if (s < e) {
+                if (s < e && ((e - 1) >> 5) - (s >> 5) >= 256) {
+                    cnt = 0x80000000u;   // long job: counted by the whole warp below
+                } else if (s < e) {
                     const uint64_t w0 = s >> 5, w1 = (e - 1) >> 5;
                     for (uint64_t w = w0 + sub; w <= w1; w += 8) {
                         uint32_t x = __ldg(sbits + w);
@@ -49,12 +51,33 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
             }
         }
         if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(flags, FLAG_BAD_PROFILE);
-        cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, 1);
-        cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, 2);
-        cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, 4);
+        if (cnt != 0x80000000u) {   // (uniform within the eight lanes of a job)
+            cnt += __shfl_xor_sync(0xFFu << (lane & 24u), cnt, 1);
+            cnt += __shfl_xor_sync(0xFFu << (lane & 24u), cnt, 2);
+            cnt += __shfl_xor_sync(0xFFu << (lane & 24u), cnt, 4);
+        }
         // job i's count sits in lanes 8*grp .. 8*grp+7; hand it to lane i
         const uint32_t got = __shfl_sync(0xFFFFFFFFu, cnt, (lane & 3u) * 8u);
         if ((lane >> 2) == it) mine = got;
+    }
+    // long jobs (more than 256 safe words): all 32 lanes stride over the words of one job
+    uint32_t pending = __ballot_sync(0xFFFFFFFFu, mine == 0x80000000u);
+    while (pending) {
+        const uint32_t i = (uint32_t)__ffs((int)pending) - 1u;
+        pending &= pending - 1u;
+        const uint32_t j = jbase + i;
+        const uint64_t s = __ldg(off + j) + __ldg(p0 + j), e = __ldg(off + j + 1);
+        const uint64_t w0 = s >> 5, w1 = (e - 1) >> 5;
+        uint32_t cnt = 0;
+        for (uint64_t w = w0 + lane; w <= w1; w += 32) {
+            uint32_t x = __ldg(sbits + w);
+            if (w == w0) x &= 0xFFFFFFFFu << (uint32_t)(s & 31);
+            if (w == w1) x &= 0xFFFFFFFFu >> (31u - (uint32_t)((e - 1) & 31));
+            cnt += __popc(x);
+        }
+        cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+        cnt += 1u - ((__ldg(sbits + w1) >> (uint32_t)((e - 1) & 31)) & 1u);
+        if (lane == i) mine = cnt;
     }
     uint64_t inc = mine;
 #pragma unroll
