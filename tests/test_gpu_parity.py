@@ -330,3 +330,29 @@ def test_select_very_large_gap_batch_unsorted_path(sja_mod, oracle_mod):
         ctx.advertise(gaps[:65536])
         got = ctx.select(spec.policy, out="host")
         _assert_awards_equal(got, want[:65536])
+
+
+def test_select_is_deterministic_and_device_outputs_match(sja_mod):
+    """The cross-CTA reduction is on a totally ordered key, so repeated selects give identical bytes;
+    a device output buffer receives the same awards as a host buffer."""
+    import torch
+    spec = wl.scaled(wl.SPECS[2], n_jobs=5000, fixed_len=600, n_gaps=700)
+    prof = wl.make_profiles(spec, threads=2)
+    gaps = wl.make_gaps(spec)
+    stream = torch.cuda.Stream()
+    with sja_mod.Sja(stream=stream.cuda_stream) as ctx:
+        _load(ctx, prof)
+        ctx.advertise(gaps)
+        first = ctx.select(spec.policy, out="host")
+        for flags in (0, 1, 0, 1, 0):
+            assert ctx.select(spec.policy, flags=flags, out="host").tobytes() == first.tobytes()
+        dev = torch.zeros(24 * gaps.shape[0], dtype=torch.uint8, device="cuda")
+        ctx.select(spec.policy, out=dev)
+        stream.synchronize()
+        assert dev.cpu().numpy().tobytes() == first.tobytes()
+        t = ctx.profile_read()
+        assert t["select_launches"] == 0          # profiling is off unless enabled
+        ctx.profile_enable(True)
+        ctx.select(spec.policy)
+        t = ctx.profile_read()
+        assert t["select_launches"] == 1 and t["select_ms"] > 0
