@@ -277,17 +277,32 @@ sja_status check_policy(sja_ctx* c, const sja_policy* policy, const char* who) {
 
 // Launch signal + score + select for the first G_act entries of `sgaps` (ordered or not);
 // awards and widx are written at the gaps' original indices.  `blocked` may be nullptr.
-sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sgaps, uint32_t G_act,
-                      const uint32_t* blocked) {
-    const uint32_t J = c->J;
+struct SelectPlan { bool use_merge; uint32_t jobs_per_cta, tile, n_chunks; };
+
+SelectPlan plan_select(const sja_ctx* c, uint32_t pflags) {
+    SelectPlan p;
     // The merge kernel pays one restart per capacity class; with very many classes (or an
     // unsorted batch) the per-pair search is the better tool.
-    const bool use_merge = !(pflags & SJA_FLAG_FORCE_SEARCH) && c->gaps_sorted &&
-                           c->n_classes <= std::max<uint32_t>(64u, c->G / 16u);
-    const uint32_t jobs_per_cta = use_merge ? (uint32_t)MERGE_JOBS : (uint32_t)SEARCH_THREADS;
-    const uint32_t tile = use_merge ? (uint32_t)MERGE_GT : (uint32_t)SEARCH_GT;
-    const uint32_t n_chunks = (J + jobs_per_cta - 1) / jobs_per_cta;
-    TRY(reserve(c, c->partial, (size_t)n_chunks * c->G * sizeof(Partial)));
+    p.use_merge = !(pflags & SJA_FLAG_FORCE_SEARCH) && c->gaps_sorted &&
+                  c->n_classes <= std::max<uint32_t>(64u, c->G / 16u);
+    p.jobs_per_cta = p.use_merge ? (uint32_t)MERGE_JOBS : (uint32_t)SEARCH_THREADS;
+    p.tile = p.use_merge ? (uint32_t)MERGE_GT : (uint32_t)SEARCH_GT;
+    p.n_chunks = (c->J + p.jobs_per_cta - 1) / p.jobs_per_cta;
+    return p;
+}
+
+// `scratch`: candidate rows (n_chunks x G entries); nullptr = the context's own buffer, grown on demand.
+// `timed`: record profiling events (creates CUDA events on first use).
+sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sgaps, uint32_t G_act,
+                      const uint32_t* blocked, Partial* scratch = nullptr, bool timed = true) {
+    const SelectPlan pl = plan_select(c, pflags);
+    const bool use_merge = pl.use_merge;
+    const uint32_t tile = pl.tile, n_chunks = pl.n_chunks;
+    Partial* partial = scratch;
+    if (!partial) {
+        TRY(reserve(c, c->partial, (size_t)n_chunks * c->G * sizeof(Partial)));
+        partial = c->partial.as<Partial>();
+    }
     // split the gaps so that the grid covers the SMs several times over
     uint32_t splits = (uint32_t)((8ull * c->n_sm + n_chunks - 1) / n_chunks);
     const uint32_t max_splits = (G_act + tile - 1) / tile;
@@ -296,17 +311,22 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
     uint32_t per_split = (G_act + splits - 1) / splits;
     per_split = ((per_split + tile - 1) / tile) * tile;
     splits = (G_act + per_split - 1) / per_split;
-    ProfScope ps(c, CAT_SELECT);
-    JobView jv = job_view(c);
-    jv.blocked = blocked;
-    if (use_merge) {
-        launch_merge(kind, dim3(n_chunks, splits), c->stream, jv, sgaps, G_act, per_split, c->partial.as<Partial>());
-    } else {
-        select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, 0, c->stream>>>(
-            jv, sgaps, G_act, per_split, kind, nullptr, 0, c->partial.as<Partial>());
+    const bool was_on = c->prof;
+    if (!timed) c->prof = false;
+    {
+        ProfScope ps(c, CAT_SELECT);
+        JobView jv = job_view(c);
+        jv.blocked = blocked;
+        if (use_merge) {
+            launch_merge(kind, dim3(n_chunks, splits), c->stream, jv, sgaps, G_act, per_split, partial);
+        } else {
+            select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, 0, c->stream>>>(
+                jv, sgaps, G_act, per_split, kind, nullptr, 0, partial);
+        }
+        finalize_awards_kernel<<<(uint32_t)(((uint64_t)G_act * FINALIZE_LANES + 255) / 256), 256, 0, c->stream>>>(
+            jv, partial, n_chunks, sgaps, G_act, kind, c->awards.as<Award>(), c->widx.as<uint32_t>());
     }
-    finalize_awards_kernel<<<(uint32_t)(((uint64_t)G_act * FINALIZE_LANES + 255) / 256), 256, 0, c->stream>>>(
-        jv, c->partial.as<Partial>(), n_chunks, sgaps, G_act, kind, c->awards.as<Award>(), c->widx.as<uint32_t>());
+    c->prof = was_on;
     return SJA_OK;
 }
 
@@ -322,7 +342,7 @@ void run_commit(sja_ctx* c, uint32_t* blocked, const uint8_t* accept = nullptr) 
         c->boff.as<uint64_t>(), c->A.as<uint4>(), c->p.as<uint32_t>(), c->ready.as<uint32_t>(), c->pb.as<uint32_t>(),
         c->Dp.as<uint32_t>(), c->Wp.as<uint64_t>(), c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(),
         c->flags.as<uint32_t>(), blocked, accept);
-    commit_refresh_kernel<<<(G * 32 + 255) / 256, 256, 0, c->stream>>>(
+    commit_refresh_kernel<<<(uint32_t)(((uint64_t)G * 32 + 255) / 256), 256, 0, c->stream>>>(
         c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(), G, c->boff.as<uint64_t>(), c->pb.as<uint32_t>(),
         c->A.as<uint4>(), c->B.as<uint2>(), c->jobwin.as<unsigned long long>());
 }
@@ -674,58 +694,27 @@ sja_status sja_select(sja_ctx* c, const sja_policy* policy, sja_award* out, sja_
 // no cudaFree, no event creation (kernel timing is therefore not recorded here).
 sja_status sja_select_static(sja_ctx* c, const sja_policy* policy, sja_award* out, sja_memspace where) {
     TRY(check_ctx(c));
-    if (!policy) return fail(c, SJA_ERR_INVALID_ARG, "sja_select_static: policy is NULL");
     if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE)
         return fail(c, SJA_ERR_INVALID_ARG, "sja_select_static: bad memspace");
-    const uint32_t kind = policy->kind;
-    if (kind > SJA_POLICY_SLA) return fail(c, SJA_ERR_INVALID_ARG, "sja_select_static: unknown policy %u", kind);
-    if (!c->loaded || !c->advertised) return fail(c, SJA_ERR_STATE, "sja_select_static before load / advertise");
-    if (kind == SJA_POLICY_FAIRNESS && !c->have_wait)
-        return fail(c, SJA_ERR_INVALID_ARG, "fairness policy needs wait_ms at load");
-    if (kind == SJA_POLICY_SLA && !c->have_prio) return fail(c, SJA_ERR_INVALID_ARG, "SLA policy needs prio at load");
-    if (kind == SJA_POLICY_FAIRNESS && (c->load_flags & FLAG_OVF_FAIR))
-        return fail(c, SJA_ERR_OVERFLOW, "fairness score may reach 2^63 for some job");
-    if (kind == SJA_POLICY_SLA && (c->load_flags & FLAG_OVF_SLA))
-        return fail(c, SJA_ERR_OVERFLOW, "SLA key needs work < 2^55 for every job");
+    TRY(check_policy(c, policy, "sja_select_static"));
     DeviceGuard guard(c->device);
     if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
 
-    const uint32_t G = c->G, J = c->J;
-    const bool use_merge = !(policy->flags & SJA_FLAG_FORCE_SEARCH) && c->gaps_sorted &&
-                           c->n_classes <= std::max<uint32_t>(64u, G / 16u);
-    const uint32_t jobs_per_cta = use_merge ? (uint32_t)MERGE_JOBS : (uint32_t)SEARCH_THREADS;
-    const uint32_t tile = use_merge ? (uint32_t)MERGE_GT : (uint32_t)SEARCH_GT;
-    const uint32_t n_chunks = (J + jobs_per_cta - 1) / jobs_per_cta;
-    const uint64_t need = (uint64_t)n_chunks * G;   // candidate slots: one per (CTA job chunk, gap)
+    const uint32_t kind = policy->kind, G = c->G, J = c->J;
+    const SelectPlan pl = plan_select(c, policy->flags);
+    const uint64_t need = (uint64_t)pl.n_chunks * G;   // candidate slots: one per (CTA job chunk, gap)
     const uint64_t have = (uint64_t)SJA_STATIC_SCRATCH_BYTES / sizeof(Partial);
     if (need > have)
         return fail(c, SJA_ERR_INVALID_ARG,
                     "sja_select_static: %u jobs x %u gaps need %llu candidate slots (ceil(J/%u) x G), the fixed "
                     "scratch holds %llu; use sja_select for this size",
-                    J, G, (unsigned long long)need, jobs_per_cta, (unsigned long long)have);
+                    J, G, (unsigned long long)need, pl.jobs_per_cta, (unsigned long long)have);
     Partial* scratch = nullptr;
     TRY(static_scratch_for(c, c->device, &scratch));
-
-    uint32_t splits = (uint32_t)((8ull * c->n_sm + n_chunks - 1) / n_chunks);
-    const uint32_t max_splits = (G + tile - 1) / tile;
-    if (splits > max_splits) splits = max_splits;
-    if (splits < 1) splits = 1;
-    uint32_t per_split = (G + splits - 1) / splits;
-    per_split = ((per_split + tile - 1) / tile) * tile;
-    splits = (G + per_split - 1) / per_split;
     // Every slot that finalize_awards_kernel reads is written by the select kernel of this
     // same call (all chunks x all gaps), so nothing left over from an earlier call is ever
-    // read and nothing has to be cleared first.
-    const JobView jv = job_view(c);
-    if (use_merge) {
-        launch_merge(kind, dim3(n_chunks, splits), c->stream, jv, c->sgaps.as<Gap>(), G, per_split, scratch);
-    } else {
-        select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, 0, c->stream>>>(
-            jv, c->sgaps.as<Gap>(), G, per_split, kind, nullptr, 0, scratch);
-    }
-    finalize_awards_kernel<<<(uint32_t)(((uint64_t)G * FINALIZE_LANES + 255) / 256), 256, 0, c->stream>>>(jv, scratch, n_chunks, c->sgaps.as<Gap>(), G,
-                                                                     kind, c->awards.as<Award>(),
-                                                                     c->widx.as<uint32_t>());
+    // read and nothing has to be cleared first.  No profiling events on this path.
+    TRY(run_select(c, kind, policy->flags, c->sgaps.as<Gap>(), G, nullptr, scratch, /*timed=*/false));
     CU(cudaGetLastError());
     c->selected = true;
     c->committed = false;
