@@ -326,7 +326,9 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32, SCAN_CTAS_PER_SM) scan_profil
                 uint32_t D = baseD;
                 uint64_t W = baseW;
                 uint32_t seg = seg_in;
-                uint64_t pos = out0 + (incC - cnt);
+                // finished rows: the first SCAN_STAGE_ROWS go through the row buffer and leave with
+                // coalesced stores, the rest is stored directly
+                uint32_t lpos = incC - cnt;
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     D += dv[i];
@@ -334,12 +336,24 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32, SCAN_CTAS_PER_SM) scan_profil
                     seg = max(seg, mv[i]);
                     run = max(run, mv[i]);
                     if ((bits >> i) & 1u) {
-                        if (pos < out_end) {
-                            a.A[pos] = make_uint4(D, run, (uint32_t)W, (uint32_t)(W >> 32));
-                            a.B[pos] = make_uint2(k0 + (uint32_t)i + 1u, seg);
+                        const uint4 ra = make_uint4(D, run, (uint32_t)W, (uint32_t)(W >> 32));
+                        const uint2 rb = make_uint2(k0 + (uint32_t)i + 1u, seg);
+                        if (lpos < (uint32_t)SCAN_STAGE_ROWS) {
+                            rowA[lpos] = ra;
+                            rowB[lpos] = rb;
+                        } else if (out0 + lpos < out_end) {
+                            a.A[out0 + lpos] = ra;
+                            a.B[out0 + lpos] = rb;
                         }
-                        ++pos;
+                        ++lpos;
                         seg = 0;
+                    }
+                }
+                __syncwarp();
+                for (uint32_t idx = lane; idx < (uint32_t)SCAN_STAGE_ROWS; idx += 32) {
+                    if (out0 + idx < out_end) {
+                        a.A[out0 + idx] = rowA[idx];
+                        a.B[out0 + idx] = rowB[idx];
                     }
                 }
                 carryRun = max(before, __shfl_sync(0xFFFFFFFFu, incR, 31));
