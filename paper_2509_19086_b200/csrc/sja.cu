@@ -244,15 +244,30 @@ __global__ void export_rows_kernel(const uint4* __restrict__ A, const uint2* __r
     if (W) W[i] = pack64(a.z, a.w);
 }
 
-void launch_merge(uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& jv, const Gap* sgaps, uint32_t G,
-                  uint32_t per_split, Partial* partial) {
+template <bool BOUNDED>
+void launch_merge_b(uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& jv, const Gap* sgaps, uint32_t G,
+                    uint32_t per_split, Partial* partial) {
     const int threads = MERGE_WARPS * 32;
     if (kind == SJA_POLICY_FAIRNESS)
-        select_merge_kernel<1><<<grid, threads, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split, partial);
+        select_merge_kernel<1, BOUNDED><<<grid, threads, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split, partial);
     else if (kind == SJA_POLICY_SLA)
-        select_merge_kernel<2><<<grid, threads, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split, partial);
+        select_merge_kernel<2, BOUNDED><<<grid, threads, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split, partial);
     else
-        select_merge_kernel<0><<<grid, threads, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split, partial);
+        select_merge_kernel<0, BOUNDED><<<grid, threads, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split, partial);
+}
+
+void launch_merge(uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& jv, const Gap* sgaps, uint32_t G,
+                  uint32_t per_split, Partial* partial) {
+    if (jv.tau_min != 0u || jv.tau_max != 0xFFFFFFFFu)
+        launch_merge_b<true>(kind, grid, stream, jv, sgaps, G, per_split, partial);
+    else
+        launch_merge_b<false>(kind, grid, stream, jv, sgaps, G, per_split, partial);
+}
+
+template <uint32_t KIND, bool BOUNDED>
+cudaError_t merge_smem_attr() {
+    return cudaFuncSetAttribute(select_merge_kernel<KIND, BOUNDED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                MERGE_SMEM_BYTES);
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -407,12 +422,12 @@ sja_status sja_create(sja_ctx** out, int device, void* cuda_stream) {
         if (cudaMemsetAsync(c->flags.p, 0, 4, c->stream) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         if (cudaFuncSetAttribute(scan_profiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  SCAN_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
-        if (cudaFuncSetAttribute(select_merge_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 MERGE_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
-        if (cudaFuncSetAttribute(select_merge_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 MERGE_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
-        if (cudaFuncSetAttribute(select_merge_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 MERGE_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
+        if (merge_smem_attr<0, false>() != cudaSuccess || merge_smem_attr<1, false>() != cudaSuccess ||
+            merge_smem_attr<2, false>() != cudaSuccess || merge_smem_attr<0, true>() != cudaSuccess ||
+            merge_smem_attr<1, true>() != cudaSuccess || merge_smem_attr<2, true>() != cudaSuccess) {
+            st = SJA_ERR_CUDA;
+            break;
+        }
         if ((st = reserve(c, c->gap_info, sizeof(GapInfo))) != SJA_OK) break;
     } while (0);
     if (st != SJA_OK) {

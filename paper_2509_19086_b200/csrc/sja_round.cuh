@@ -430,7 +430,8 @@ __device__ __forceinline__ WarpBest warp_argmax_lowest_lane(uint64_t best, uint3
     return o;
 }
 
-template <uint32_t KIND>
+// BOUNDED: the subjob duration thresholds are in force (off by default, and then compiled out).
+template <uint32_t KIND, bool BOUNDED>
 __global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_merge_kernel(
     JobView jv, const Gap* __restrict__ sgaps, uint32_t G, uint32_t gaps_per_split, Partial* __restrict__ partial_out) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -475,7 +476,7 @@ __global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_me
 
     // Cursor update and lane-local best candidate for one gap.
     auto eval_gap = [&](const uint4 gq, uint64_t& best, uint32_t& best_r, uint32_t& best_cnt) {
-        const uint32_t start = gq.y, T = min(gq.z, jv.tau_max), C = gq.w;
+        const uint32_t start = gq.y, T = BOUNDED ? min(gq.z, jv.tau_max) : gq.z, C = gq.w;
         if (first || C != curC) {
             // new capacity class: T restarts from its smallest value, so do the cursors
             first = false;
@@ -514,7 +515,7 @@ __global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_me
                 while (((open >> r) & 1u) && T >= thr[r]) {
                     // row w qualifies: it becomes the candidate; fetch row w + 1 from the ring
                     // (a subjob shorter than the minimum duration is no candidate; longer rows may be)
-                    curKey[r] = thr[r] >= jv.tau_min ? policy_key(KIND, nextW[r] - Wp[r], factor[r]) : 0ull;
+                    curKey[r] = (!BOUNDED || thr[r] >= jv.tau_min) ? policy_key(KIND, nextW[r] - Wp[r], factor[r]) : 0ull;
                     if (w[r] + MERGE_RING < n[r])
                         mg_cp_async16(ring_s[r] + (w[r] & (MERGE_RING - 1)) * 32 * 16, next_row[r]);
                     mg_commit();
