@@ -38,14 +38,14 @@ FALLBACK_HBM_GBS = 6650.0
 # scan_profiles_kernel_cfg2-jobs8192.md): dram__bytes_read.sum + dram__bytes_write.sum over 33 554 432 steps.
 # Traffic grows in proportion to the step count, so a full launch is this figure times N.  It is only reported
 # while csrc/sja_scan.cuh is the file the counters were taken from (first 16 hex digits of its sha256).
-NCU_SCAN_TRAFFIC_BYTES_PER_STEP = (273.077248e6 + 62.033664e6) / 33554432
-NCU_SCAN_SOURCE_SHA = "93addd443eb42e34"
+NCU_SCAN_TRAFFIC_BYTES_PER_STEP = (273.048064e6 + 59.769344e6) / 33554432
+NCU_SCAN_SOURCE_SHA = "8bd8a77590ca9c38"
 
 
 # Issue-slot roofline of the select kernel (it is bound by instruction issue, not HBM): warp instructions per
 # pair from its ncu capture (profiles/select_merge_kernel_cfg2-jobs32768.md), peak = SMs x 4 schedulers x SM clock.
 NCU_MERGE_WARP_INSTR_PER_PAIR = 163228366 / (32768 * 4096)
-NCU_MERGE_SOURCE_SHA = "87193c0c356ba439"
+NCU_MERGE_SOURCE_SHA = "f21050b3c2d531d2"
 N_SM, SCHEDULERS_PER_SM = 148, 4
 
 
