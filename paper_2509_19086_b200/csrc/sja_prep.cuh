@@ -40,10 +40,21 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
                     cnt = 0x80000000u;   // long job: counted by the whole warp below
                 } else if (s < e) {
                     const uint64_t w0 = s >> 5, w1 = (e - 1) >> 5;
-                    for (uint64_t w = w0 + sub; w <= w1; w += 8) {
+                    const uint32_t m0 = 0xFFFFFFFFu << (uint32_t)(s & 31);
+                    const uint32_t m1 = 0xFFFFFFFFu >> (31u - (uint32_t)((e - 1) & 31));
+                    uint64_t w = w0 + sub;
+                    // four independent loads in flight per lane
+                    for (; w + 24 <= w1; w += 32) {
+                        uint32_t x0 = __ldg(sbits + w), x1 = __ldg(sbits + w + 8);
+                        uint32_t x2 = __ldg(sbits + w + 16), x3 = __ldg(sbits + w + 24);
+                        if (w == w0) x0 &= m0;
+                        if (w + 24 == w1) x3 &= m1;
+                        cnt += __popc(x0) + __popc(x1) + __popc(x2) + __popc(x3);
+                    }
+                    for (; w <= w1; w += 8) {
                         uint32_t x = __ldg(sbits + w);
-                        if (w == w0) x &= 0xFFFFFFFFu << (uint32_t)(s & 31);
-                        if (w == w1) x &= 0xFFFFFFFFu >> (31u - (uint32_t)((e - 1) & 31));
+                        if (w == w0) x &= m0;
+                        if (w == w1) x &= m1;
                         cnt += __popc(x);
                     }
                     if (sub == 0) cnt += 1u - ((__ldg(sbits + w1) >> (uint32_t)((e - 1) & 31)) & 1u);
