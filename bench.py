@@ -404,7 +404,9 @@ def main():
                 "ms_per_step": e2e_ms / max(1, args.e2e_steps), "steps": args.e2e_steps},
         "gpu_launches": timed_launches,
         "roofline": roofline,
-        "select_roofline": select_roofline(pairs / (select_ms * 1e-3) if select_ms > 0 else None, clocks.get("sm_mhz")),
+        # the instruction count per pair was captured on the large uniform workload only
+        "select_roofline": select_roofline(pairs / (select_ms * 1e-3) if select_ms > 0 else None, clocks.get("sm_mhz"))
+        if spec.index == 2 and not args.flags and not args.reauction else None,
         "kernel_ms_per_step": breakdown,
         "select_pairs_per_s": pairs / (select_ms * 1e-3) if select_ms > 0 else None,
         "profile_gb_per_s": prof.raw_bytes() / (scan_ms * 1e-3) / 1e9 if scan_ms > 0 else None,
