@@ -77,9 +77,12 @@ typedef enum {
     SJA_POLICY_SLA = 2         /* key = (prio, work); needs prio at load; reported score = work */
 } sja_policy_kind;
 
-/* Bit 0 of sja_policy.flags: evaluate every pair with the per-pair binary search over the
- * boundary table instead of the windowed merge kernel (same results; for testing). */
+/* sja_policy.flags.  By default select runs the tile-sweep kernel over the gaps ordered by
+ * (capacity, T).  Bit 0: evaluate every pair with the per-pair binary search over the boundary
+ * table instead.  Bit 1: use the per-gap merge kernel instead.  Same results on every path;
+ * the bits exist for testing and comparison. */
 #define SJA_FLAG_FORCE_SEARCH 1u
+#define SJA_FLAG_FORCE_MERGE 2u
 
 typedef struct {
     uint32_t kind;  /* sja_policy_kind */
@@ -169,9 +172,10 @@ sja_status sja_select(sja_ctx* ctx, const sja_policy* policy, sja_award* out, sj
  * cudaFree or other allocating routine and records no profiling events.
  *
  * Cost and limit: every GPU on which the library is used holds the array until the process
- * exits.  The call needs ceil(J / 1024) * G candidate slots of 16 bytes (ceil(J / 256) * G
- * with SJA_FLAG_FORCE_SEARCH or an unsorted / many-capacity batch); if that exceeds the
- * array it returns SJA_ERR_INVALID_ARG with the numbers in sja_last_error() and does nothing.
+ * exits.  The call needs ceil(J / 512) * G candidate slots of 16 bytes (ceil(J / 1024) * G
+ * with SJA_FLAG_FORCE_MERGE; ceil(J / 256) * G with SJA_FLAG_FORCE_SEARCH or an unsorted /
+ * many-capacity batch); if that exceeds the array it returns SJA_ERR_INVALID_ARG with the
+ * numbers in sja_last_error() and does nothing.
  *
  * The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
  * the context's device current); make that first call before starting any stream capture.

@@ -16,6 +16,7 @@
 #include "sja_prep.cuh"
 #include "sja_round.cuh"
 #include "sja_scan.cuh"
+#include "sja_tile.cuh"
 
 using namespace sja;
 
@@ -244,30 +245,47 @@ __global__ void export_rows_kernel(const uint4* __restrict__ A, const uint2* __r
     if (W) W[i] = pack64(a.z, a.w);
 }
 
-template <bool BOUNDED>
-void launch_merge_b(uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& jv, const Gap* sgaps, uint32_t G,
-                    uint32_t per_split, Partial* partial) {
-    const int threads = MERGE_WARPS * 32;
-    if (kind == SJA_POLICY_FAIRNESS)
-        select_merge_kernel<1, BOUNDED><<<grid, threads, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split, partial);
-    else if (kind == SJA_POLICY_SLA)
-        select_merge_kernel<2, BOUNDED><<<grid, threads, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split, partial);
+// The merge and tile kernels are templated on the policy and on whether the subjob duration
+// thresholds are in force; these helpers pick the instance.
+enum SelectKernel { SEL_TILE = 0, SEL_MERGE = 1, SEL_SEARCH = 2 };
+
+template <uint32_t KIND, bool BOUNDED>
+void launch_sorted_kb(SelectKernel which, dim3 grid, cudaStream_t stream, const JobView& jv, const Gap* sgaps,
+                      uint32_t G, uint32_t per_split, Partial* partial) {
+    if (which == SEL_TILE)
+        select_tile_kernel<KIND, BOUNDED><<<grid, TILE_WARPS * 32, TILE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split,
+                                                                                             partial);
     else
-        select_merge_kernel<0, BOUNDED><<<grid, threads, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split, partial);
+        select_merge_kernel<KIND, BOUNDED><<<grid, MERGE_WARPS * 32, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G,
+                                                                                                per_split, partial);
 }
 
-void launch_merge(uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& jv, const Gap* sgaps, uint32_t G,
-                  uint32_t per_split, Partial* partial) {
-    if (jv.tau_min != 0u || jv.tau_max != 0xFFFFFFFFu)
-        launch_merge_b<true>(kind, grid, stream, jv, sgaps, G, per_split, partial);
+template <bool BOUNDED>
+void launch_sorted_b(SelectKernel which, uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& jv,
+                     const Gap* sgaps, uint32_t G, uint32_t per_split, Partial* partial) {
+    if (kind == SJA_POLICY_FAIRNESS)
+        launch_sorted_kb<1, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial);
+    else if (kind == SJA_POLICY_SLA)
+        launch_sorted_kb<2, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial);
     else
-        launch_merge_b<false>(kind, grid, stream, jv, sgaps, G, per_split, partial);
+        launch_sorted_kb<0, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial);
+}
+
+void launch_sorted(SelectKernel which, uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& jv,
+                   const Gap* sgaps, uint32_t G, uint32_t per_split, Partial* partial) {
+    if (jv.tau_min != 0u || jv.tau_max != 0xFFFFFFFFu)
+        launch_sorted_b<true>(which, kind, grid, stream, jv, sgaps, G, per_split, partial);
+    else
+        launch_sorted_b<false>(which, kind, grid, stream, jv, sgaps, G, per_split, partial);
 }
 
 template <uint32_t KIND, bool BOUNDED>
-cudaError_t merge_smem_attr() {
-    return cudaFuncSetAttribute(select_merge_kernel<KIND, BOUNDED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                MERGE_SMEM_BYTES);
+cudaError_t sorted_smem_attr() {
+    cudaError_t e = cudaFuncSetAttribute(select_merge_kernel<KIND, BOUNDED>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, MERGE_SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(select_tile_kernel<KIND, BOUNDED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                TILE_SMEM_BYTES);
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -292,16 +310,18 @@ sja_status check_policy(sja_ctx* c, const sja_policy* policy, const char* who) {
 
 // Launch signal + score + select for the first G_act entries of `sgaps` (ordered or not);
 // awards and widx are written at the gaps' original indices.  `blocked` may be nullptr.
-struct SelectPlan { bool use_merge; uint32_t jobs_per_cta, tile, n_chunks; };
+struct SelectPlan { SelectKernel kernel; uint32_t jobs_per_cta, tile, n_chunks; };
 
 SelectPlan plan_select(const sja_ctx* c, uint32_t pflags) {
     SelectPlan p;
-    // The merge kernel pays one restart per capacity class; with very many classes (or an
-    // unsorted batch) the per-pair search is the better tool.
-    p.use_merge = !(pflags & SJA_FLAG_FORCE_SEARCH) && c->gaps_sorted &&
-                  c->n_classes <= std::max<uint32_t>(64u, c->G / 16u);
-    p.jobs_per_cta = p.use_merge ? (uint32_t)MERGE_JOBS : (uint32_t)SEARCH_THREADS;
-    p.tile = p.use_merge ? (uint32_t)MERGE_GT : (uint32_t)SEARCH_GT;
+    // The tile and merge kernels need the (capacity, T) order and pay one restart per capacity
+    // class; with very many classes (or an unsorted batch) the per-pair search is the better tool.
+    const bool sorted_ok = !(pflags & SJA_FLAG_FORCE_SEARCH) && c->gaps_sorted &&
+                           c->n_classes <= std::max<uint32_t>(64u, c->G / 16u);
+    p.kernel = !sorted_ok ? SEL_SEARCH : (pflags & SJA_FLAG_FORCE_MERGE) ? SEL_MERGE : SEL_TILE;
+    p.jobs_per_cta = p.kernel == SEL_TILE ? (uint32_t)TILE_JOBS
+                                          : p.kernel == SEL_MERGE ? (uint32_t)MERGE_JOBS : (uint32_t)SEARCH_THREADS;
+    p.tile = p.kernel == SEL_TILE ? (uint32_t)TILE_GT : p.kernel == SEL_MERGE ? (uint32_t)MERGE_GT : (uint32_t)SEARCH_GT;
     p.n_chunks = (c->J + p.jobs_per_cta - 1) / p.jobs_per_cta;
     return p;
 }
@@ -311,7 +331,6 @@ SelectPlan plan_select(const sja_ctx* c, uint32_t pflags) {
 sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sgaps, uint32_t G_act,
                       const uint32_t* blocked, Partial* scratch = nullptr, bool timed = true) {
     const SelectPlan pl = plan_select(c, pflags);
-    const bool use_merge = pl.use_merge;
     const uint32_t tile = pl.tile, n_chunks = pl.n_chunks;
     Partial* partial = scratch;
     if (!partial) {
@@ -332,8 +351,8 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
         ProfScope ps(c, CAT_SELECT);
         JobView jv = job_view(c);
         jv.blocked = blocked;
-        if (use_merge) {
-            launch_merge(kind, dim3(n_chunks, splits), c->stream, jv, sgaps, G_act, per_split, partial);
+        if (pl.kernel != SEL_SEARCH) {
+            launch_sorted(pl.kernel, kind, dim3(n_chunks, splits), c->stream, jv, sgaps, G_act, per_split, partial);
         } else {
             select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, 0, c->stream>>>(
                 jv, sgaps, G_act, per_split, kind, nullptr, 0, partial);
@@ -422,9 +441,9 @@ sja_status sja_create(sja_ctx** out, int device, void* cuda_stream) {
         if (cudaMemsetAsync(c->flags.p, 0, 4, c->stream) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         if (cudaFuncSetAttribute(scan_profiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  SCAN_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
-        if (merge_smem_attr<0, false>() != cudaSuccess || merge_smem_attr<1, false>() != cudaSuccess ||
-            merge_smem_attr<2, false>() != cudaSuccess || merge_smem_attr<0, true>() != cudaSuccess ||
-            merge_smem_attr<1, true>() != cudaSuccess || merge_smem_attr<2, true>() != cudaSuccess) {
+        if (sorted_smem_attr<0, false>() != cudaSuccess || sorted_smem_attr<1, false>() != cudaSuccess ||
+            sorted_smem_attr<2, false>() != cudaSuccess || sorted_smem_attr<0, true>() != cudaSuccess ||
+            sorted_smem_attr<1, true>() != cudaSuccess || sorted_smem_attr<2, true>() != cudaSuccess) {
             st = SJA_ERR_CUDA;
             break;
         }

@@ -106,7 +106,7 @@ def test_scan_cfg1_sampled_jobs(sja_mod, oracle_mod):
 
 
 # ------------------------------------------------------------------ select (a2-a5)
-@pytest.mark.parametrize("flags", [0, 1])
+@pytest.mark.parametrize("flags", [0, 1, 2])
 @pytest.mark.parametrize("policy", [0, 1, 2])
 def test_select_tiny_random_vs_oracle(sja_mod, oracle_mod, policy, flags):
     rng = np.random.default_rng(200 + policy)
@@ -140,7 +140,7 @@ def test_select_published_small_configs(sja_mod, oracle_mod, cfg):
         _load(ctx, prof)
         ctx.advertise(gaps)
         want = oracle_mod.select(prof, progress, prof.ready_ms, gaps, spec.policy)
-        for flags in (0, 1):
+        for flags in (0, 1, 2):
             got = ctx.select(spec.policy, flags=flags, out="host")
             _assert_awards_equal(got, want)
         assert (got["job"] != U32MAX).sum() > 0
@@ -162,7 +162,7 @@ def test_select_fairness_and_sla_scaled_configs(sja_mod, oracle_mod):
             _load(ctx, prof)
             ctx.advertise(gaps)
             want = oracle_mod.select(prof, progress, prof.ready_ms, gaps, spec.policy)
-            for flags in (0, 1):
+            for flags in (0, 1, 2):
                 got = ctx.select(spec.policy, flags=flags, out="host")
                 _assert_awards_equal(got, want)
 
@@ -182,13 +182,43 @@ def test_select_long_windows_and_many_capacity_classes(sja_mod, oracle_mod):
         _load(ctx, prof, progress)
         ctx.advertise(gaps)
         want = oracle_mod.select(prof, progress, prof.ready_ms, gaps, 0)
-        for flags in (0, 1):
+        for flags in (0, 1, 2):
             got = ctx.select(0, flags=flags, out="host")
             _assert_awards_equal(got, want)
 
 
+@pytest.mark.parametrize("policy", [0, 1, 2])
+def test_select_ties_duplicate_jobs_and_ready_boundaries(sja_mod, oracle_mod, policy):
+    """Many exact ties (copies of the same profile), zero-work segments (a longer subjob with the
+    same score), few distinct ready times met exactly by the gap starts, repeated T values, and
+    job / gap counts that are not multiples of 32: every kernel against the oracle."""
+    rng = np.random.default_rng(4100 + policy)
+    base = random_small_profiles(rng, 9, 60, p_safe=0.4, dmax=12, mmax=50, allow_zero=True)
+    jobs = [base[int(rng.integers(0, len(base)))] for _ in range(173)]
+    J = len(jobs)
+    prof = profiles_from_lists(jobs, ready=rng.choice([0, 5, 5, 10, 4000000000], J),
+                               wait=rng.choice([0, 999, 1000, 2000], J), prio=rng.choice([0, 1, 1, 2], J))
+    progress = np.zeros(J, np.uint32)
+    rows = [(int(rng.integers(0, 7)), int(rng.choice([0, 4, 5, 9, 10, 11, 3999999999, 4000000000])),
+             int(rng.choice([0, 3, 17, 17, 40, 90, 90, 250, U32MAX])), int(rng.choice([7, 25, 50])))
+            for _ in range(77)]
+    gaps = gaps_from_lists(rows)
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof, progress)
+        for rnd in range(4):
+            ctx.advertise(gaps)
+            want = oracle_mod.select(prof, progress, prof.ready_ms, gaps, policy)
+            assert (want["job"] != U32MAX).any()
+            for flags in (0, 1, 2):
+                _assert_awards_equal(ctx.select(policy, flags=flags, out="host"), want)
+            ctx.commit()
+            oracle_mod.commit(progress, prof.ready_ms, gaps, want)
+            p, r = ctx.get_state()
+            assert np.array_equal(p, progress) and np.array_equal(r, prof.ready_ms)
+
+
 # ------------------------------------------------------------------ commit (a6), multi-round
-@pytest.mark.parametrize("flags", [0, 1])
+@pytest.mark.parametrize("flags", [0, 1, 2])
 def test_streaming_rounds_bit_exact(sja_mod, oracle_mod, flags):
     """Scaled streaming workload: per-round awards (with grants) and final state match the oracle."""
     spec = wl.scaled(wl.SPECS[4], n_jobs=1500, fixed_len=300, n_gaps=200, n_rounds=60)
@@ -344,7 +374,7 @@ def test_select_is_deterministic_and_device_outputs_match(sja_mod):
         _load(ctx, prof)
         ctx.advertise(gaps)
         first = ctx.select(spec.policy, out="host")
-        for flags in (0, 1, 0, 1, 0):
+        for flags in (0, 1, 2, 0, 1, 2, 0):
             assert ctx.select(spec.policy, flags=flags, out="host").tobytes() == first.tobytes()
         dev = torch.zeros(24 * gaps.shape[0], dtype=torch.uint8, device="cuda")
         ctx.select(spec.policy, out=dev)

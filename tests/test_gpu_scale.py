@@ -52,9 +52,10 @@ def test_cfg2_large_uniform_all_awards(oracle_mod):
         # the per-pair search kernel on a sample of the gaps
         sub = gaps[::16]
         ctx.advertise(sub)
-        got = ctx.select(spec.policy, flags=binding.FLAG_FORCE_SEARCH, out="host")
         want = oracle_mod.select(prof, progress, ready, sub, spec.policy)
-        _assert_equal(got, want)
+        _assert_equal(ctx.select(spec.policy, flags=binding.FLAG_FORCE_SEARCH, out="host"), want)
+        # and the per-gap merge kernel
+        _assert_equal(ctx.select(spec.policy, flags=binding.FLAG_FORCE_MERGE, out="host"), want)
 
 
 def test_cfg3_heavy_tailed_sampled_gaps(oracle_mod):
@@ -74,6 +75,8 @@ def test_cfg3_heavy_tailed_sampled_gaps(oracle_mod):
         sample = np.sort(rng.choice(gaps.shape[0], 4096, replace=False))
         want = oracle_mod.select(prof, progress, prof.ready_ms, gaps[sample], spec.policy)
         _assert_equal(got[sample], want)
+        # the three select kernels agree on every gap (the sampled ones are pinned by the oracle above)
+        assert ctx.select(spec.policy, flags=binding.FLAG_FORCE_MERGE, out="host").tobytes() == got.tobytes()
         # every award: winner eligible, subjob inside the job, ends on a boundary, fits T
         win = got["job"] != U32MAX
         assert win.mean() > 0.9
@@ -116,6 +119,11 @@ def test_cfg4_streaming_1000_rounds(oracle_mod):
             gaps = wl.make_gaps(spec, r)
             ctx.advertise(gaps)
             ctx.select(spec.policy)
+            if r % 100 == 50:
+                # late rounds (jobs partly consumed, ready times spread out): both ordered-gap kernels agree
+                a = ctx.select(spec.policy, flags=binding.FLAG_FORCE_MERGE, out="host")
+                b = ctx.select(spec.policy, out="host")
+                assert a.tobytes() == b.tobytes(), r
             n = ctx.commit()
             aw = ctx.get_awards()
             if r < 3:
