@@ -20,6 +20,11 @@
 
 using namespace sja;
 
+// Select grids aim at this many CTAs per SM (several waves even out the tail).
+#ifndef SJA_SELECT_CTAS_PER_SM
+#define SJA_SELECT_CTAS_PER_SM 8
+#endif
+
 namespace {
 
 struct DevBuf {
@@ -338,7 +343,7 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
         partial = c->partial.as<Partial>();
     }
     // split the gaps so that the grid covers the SMs several times over
-    uint32_t splits = (uint32_t)((8ull * c->n_sm + n_chunks - 1) / n_chunks);
+    uint32_t splits = (uint32_t)(((uint64_t)SJA_SELECT_CTAS_PER_SM * c->n_sm + n_chunks - 1) / n_chunks);
     const uint32_t max_splits = (G_act + tile - 1) / tile;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;

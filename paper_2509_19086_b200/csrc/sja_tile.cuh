@@ -12,13 +12,18 @@
 //    window must not begin before the job can) are a prefix of that order, so its base
 //    answer is ONE lookup, PM[#eligible - 1] -- no per-job work at all.
 //  * events: rows whose duration lies in (T_lo, T_hi].  The owning lanes step their
-//    cursors (all lanes that have one step together) and post (duration, ready, key) to
-//    shared memory; every gap lane tests each posted event with two compares and a key
-//    comparison.  An event is looked at once, by one warp instruction stream.
+//    cursors, all lanes that have steps to do at once.  A step can only matter if its key
+//    beats the PM entry at the job's own rank as it stood at the start of the run: every gap
+//    that may take the job (rank < #eligible) already holds at least that entry.  Such steps
+//    (few: the prefix maxima of a random order of 32 are about 4 jobs) are posted to shared
+//    memory as (duration, rank, key); the others are silent.  Every lane then looks at each
+//    posted event twice over: as a gap (is the row within my window, is the job among my
+//    eligible ones, does it beat my best) and as PM entry (does it raise the prefix maximum
+//    at my rank), which leaves the PM ready for the next 32 gaps.
 //
-// The cost is therefore per (warp, 32 gaps) a fixed part (PM rebuild, lookup) plus a part
-// proportional to the number of boundary rows the windows actually reach, not to the
-// number of pairs.
+// The cost is therefore per (warp, 32 gaps) a small fixed part (the lookup) plus the cursor
+// steps, not the number of pairs.  The PM is rebuilt by a warp scan only after a restart of
+// the cursors (a new capacity class, or the start of a CTA's gap range).
 #pragma once
 #include "sja_round.cuh"
 
@@ -46,15 +51,20 @@ constexpr int TILE_STAGE_BYTES = TILE_WARPS * TILE_GT * 16;
 constexpr int TILE_GAP_BYTES = TILE_GT * 16;
 constexpr int TILE_EVENT_BYTES = TILE_WARPS * 32 * 16;   // posted events, one slot per lane
 constexpr int TILE_ECNT_BYTES = TILE_WARPS * 32 * 4;     // their row counts
-constexpr int TILE_PM_BYTES = TILE_WARPS * 32 * 16;      // rank-ordered candidates before the scan
-constexpr int TILE_SMEM_BYTES =
-    TILE_RING_BYTES + TILE_STAGE_BYTES + TILE_GAP_BYTES + TILE_EVENT_BYTES + TILE_ECNT_BYTES + TILE_PM_BYTES;
+constexpr int TILE_SMEM_BYTES = TILE_RING_BYTES + TILE_STAGE_BYTES + TILE_GAP_BYTES + TILE_EVENT_BYTES + TILE_ECNT_BYTES;
 static_assert((TILE_RING & (TILE_RING - 1)) == 0, "ring size must be a power of two");
 static_assert(TILE_GT % 32 == 0 && TILE_GT <= TILE_JOBS, "one thread per gap of a staging tile");
 
 // Candidate order: larger key first, then the lower job id.
 __device__ __forceinline__ bool cand_better(uint64_t ka, uint32_t ja, uint64_t kb, uint32_t jb) {
     return ka > kb || (ka == kb && ja < jb);
+}
+
+// Inside a warp a candidate is (key, inv) with inv = 31 - owning lane: the larger pair wins
+// (larger key, then the lower lane = lower job id).  An equal pair is a later row of the job
+// that already leads: it wins too (same score, longer subjob).
+__device__ __forceinline__ bool pair_ge(uint64_t ka, uint32_t ia, uint64_t kb, uint32_t ib) {
+    return ka > kb || (ka == kb && ia >= ib);
 }
 
 template <uint32_t KIND, bool BOUNDED>
@@ -69,8 +79,6 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
     uint4* ev = reinterpret_cast<uint4*>(smem_raw + TILE_RING_BYTES + TILE_STAGE_BYTES + TILE_GAP_BYTES) + wid * 32;
     uint32_t* evc = reinterpret_cast<uint32_t*>(smem_raw + TILE_RING_BYTES + TILE_STAGE_BYTES + TILE_GAP_BYTES +
                                                 TILE_EVENT_BYTES) + wid * 32;
-    uint4* pm_s = reinterpret_cast<uint4*>(smem_raw + TILE_RING_BYTES + TILE_STAGE_BYTES + TILE_GAP_BYTES +
-                                           TILE_EVENT_BYTES + TILE_ECNT_BYTES) + wid * 32;
     const uint32_t ring_s = smem_s + (wid * TILE_RING * 32 + lane) * 16;   // slot i of the ring: + i * 512
 
     // ---- the lane's job
@@ -102,14 +110,15 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
         const uint32_t rl = __shfl_sync(0xFFFFFFFFu, ready, l);
         rank += (rl < ready || (rl == ready && l < lane)) ? 1u : 0u;
     }
-    pm_s[rank] = make_uint4(ready, j, 0u, 0u);
+    evc[rank] = lane;
+    ev[rank].x = ready;
     __syncwarp();
-    const uint32_t sready = pm_s[lane].x;   // ready time of the job of rank `lane`
-    const uint32_t sjob = pm_s[lane].y;     // and its id
+    const uint32_t sready = ev[lane].x;     // ready time of the job of rank `lane`
+    const uint32_t slane = evc[lane];       // and the lane that owns it
     __syncwarp();
     const uint32_t sready_last = __shfl_sync(0xFFFFFFFFu, sready, 31);
-    uint64_t pk = 0;                 // PM entry of rank `lane`: key, job, row count
-    uint32_t pj = 0xFFFFFFFFu, pc = 0;
+    uint64_t pk = 0;                 // PM entry of rank `lane`: key and 31 - owning lane
+    uint32_t pi = 0;
 
     const uint32_t g_begin = blockIdx.y * gaps_per_split;
     const uint32_t g_end = min(G, g_begin + gaps_per_split);
@@ -143,8 +152,16 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
             if (in) gq = sg[sub + lane];
             const uint32_t start = gq.y, C = gq.w;
             const uint32_t T = BOUNDED ? min(gq.z, jv.tau_max) : gq.z;
-            uint64_t bk = 0;                 // this gap's best candidate of the warp
-            uint32_t bj = 0xFFFFFFFFu, bc = 0;
+            // number of jobs of the warp that are ready by this gap's start (they are ranks 0 .. e-1)
+            uint32_t e = 0;
+#pragma unroll
+            for (uint32_t s = 16; s >= 1; s >>= 1) {
+                const uint32_t v = __shfl_sync(0xFFFFFFFFu, sready, (e + s - 1u) & 31u);
+                if (v <= start) e += s;
+            }
+            if (e == 31u && sready_last <= start) e = 32u;
+            uint64_t bk = 0;                 // this gap's best candidate of the warp: key, 31 - lane, rows
+            uint32_t bi = 0, bc = 0;
             uint32_t todo = __ballot_sync(0xFFFFFFFFu, in);
             while (todo) {
                 // the next run of gaps of one capacity (the list is ordered by capacity, then T)
@@ -177,71 +194,69 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
                     }
                     dirty = true;
                 }
-                // catch up: rows no longer than T_lo qualify for every gap of the run
-                while (__any_sync(0xFFFFFFFFu, open && thr <= T_lo)) {
-                    if (open && thr <= T_lo) step_cursor(Cc);
-                    dirty = true;
-                }
                 if (dirty) {
-                    // PM: candidates in ready order, inclusive prefix maximum
-                    __syncwarp();
-                    pm_s[rank] = make_uint4((uint32_t)curKey, (uint32_t)(curKey >> 32), w, 0u);
-                    __syncwarp();
-                    const uint4 v = pm_s[lane];
-                    pk = pack64(v.x, v.y); pc = v.z; pj = sjob;
+                    // after a restart: catch up without posting (rows no longer than T_lo qualify for
+                    // every gap of the run), then PM by a warp scan over the candidates in ready order
+                    while (__any_sync(0xFFFFFFFFu, open && thr <= T_lo)) {
+                        if (open && thr <= T_lo) step_cursor(Cc);
+                    }
+                    pk = __shfl_sync(0xFFFFFFFFu, curKey, slane);
+                    pi = 31u - slane;
 #pragma unroll
                     for (int o = 1; o < 32; o <<= 1) {
                         const uint64_t k2 = __shfl_up_sync(0xFFFFFFFFu, pk, o);
-                        const uint32_t j2 = __shfl_up_sync(0xFFFFFFFFu, pj, o);
-                        const uint32_t c2 = __shfl_up_sync(0xFFFFFFFFu, pc, o);
-                        if (lane >= (uint32_t)o && cand_better(k2, j2, pk, pj)) { pk = k2; pj = j2; pc = c2; }
+                        const uint32_t i2 = __shfl_up_sync(0xFFFFFFFFu, pi, o);
+                        if (lane >= (uint32_t)o && pair_ge(k2, i2, pk, pi)) { pk = k2; pi = i2; }
                     }
                     dirty = false;
                 }
-                // base answer: number of jobs of the warp that are ready by this gap's start
-                uint32_t e = 0;
-#pragma unroll
-                for (uint32_t s = 16; s >= 1; s >>= 1) {
-                    const uint32_t v = __shfl_sync(0xFFFFFFFFu, sready, (e + s - 1u) & 31u);
-                    if (v <= start) e += s;
-                }
-                if (e == 31u && sready_last <= start) e = 32u;
+                // PM entry at my job's rank as the run starts: what a step of my job has to beat
+                const uint64_t pmr_k = __shfl_sync(0xFFFFFFFFu, pk, rank);
+                const uint32_t pmr_i = __shfl_sync(0xFFFFFFFFu, pi, rank);
+                // base answer: PM[e - 1]; its row count is the owner's current cursor
                 {
                     const uint32_t src = (e ? e - 1u : 0u) & 31u;
                     const uint64_t k0 = __shfl_sync(0xFFFFFFFFu, pk, src);
-                    const uint32_t j0 = __shfl_sync(0xFFFFFFFFu, pj, src);
-                    const uint32_t c0 = __shfl_sync(0xFFFFFFFFu, pc, src);
-                    if (mine && e) { bk = k0; bj = j0; bc = c0; }
+                    const uint32_t i0 = __shfl_sync(0xFFFFFFFFu, pi, src);
+                    const uint32_t c0 = __shfl_sync(0xFFFFFFFFu, w, 31u - i0);
+                    if (mine && e) { bk = k0; bi = i0; bc = c0; }
                 }
-                // events: rows with a duration in (T_lo, T_hi]
-                uint32_t pending;
-                while ((pending = __ballot_sync(0xFFFFFFFFu, open && thr <= T_hi)) != 0u) {
+                // events: rows with a duration up to T_hi
+                while (__any_sync(0xFFFFFFFFu, open && thr <= T_hi)) {
+                    bool post = false;
                     if (open && thr <= T_hi) {
-                        const uint32_t thr_e = thr;
-                        step_cursor(Cc);
-                        ev[lane] = make_uint4(thr_e, ready, (uint32_t)curKey, (uint32_t)(curKey >> 32));
-                        evc[lane] = w;
+                        uint32_t thr_e;
+                        do {
+                            thr_e = thr;
+                            step_cursor(Cc);
+                            post = pair_ge(curKey, 31u - lane, pmr_k, pmr_i);
+                        } while (!post && open && thr <= T_hi);
+                        if (post) {
+                            ev[lane] = make_uint4(thr_e, rank, (uint32_t)curKey, (uint32_t)(curKey >> 32));
+                            evc[lane] = w;
+                        }
                     }
-                    dirty = true;
+                    uint32_t m = __ballot_sync(0xFFFFFFFFu, post);
+                    if (m == 0u) continue;
                     __syncwarp();
-                    uint32_t m = pending;
                     while (m) {
                         const uint32_t b = (uint32_t)__ffs((int)m) - 1u;
                         m &= m - 1u;
-                        const uint4 q = ev[b];
+                        const uint4 q = ev[b];           // duration, rank of the job, key
                         const uint32_t c = evc[b];
                         const uint64_t k = pack64(q.z, q.w);
-                        const uint32_t jb = job0 + b;
-                        // a later row of the job that already leads replaces it (jb == bj): the longest subjob
-                        const bool take = mine && T >= q.x && start >= q.y && (k > bk || (k == bk && jb <= bj));
-                        if (take) { bk = k; bj = jb; bc = c; }
+                        const uint32_t ib = 31u - b;
+                        // as a gap: row within my window, job among my eligible ones, beats my best
+                        if (mine && T >= q.x && q.y < e && pair_ge(k, ib, bk, bi)) { bk = k; bi = ib; bc = c; }
+                        // as PM entry `lane`: the job is among the first lane + 1 by ready time
+                        if (lane >= q.y && pair_ge(k, ib, pk, pi)) { pk = k; pi = ib; }
                     }
                     __syncwarp();
                 }
             }
             if (in) {
                 Partial pr;
-                pr.key = bk; pr.job = bk ? bj : 0xFFFFFFFFu; pr.cnt = bk ? bc : 0u;
+                pr.key = bk; pr.job = bk ? job0 + 31u - bi : 0xFFFFFFFFu; pr.cnt = bk ? bc : 0u;
                 stage[wid * TILE_GT + sub + lane] = pr;
             }
         }
