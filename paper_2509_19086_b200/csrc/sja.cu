@@ -336,7 +336,12 @@ SelectPlan plan_select(const sja_ctx* c, uint32_t pflags) {
 sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sgaps, uint32_t G_act,
                       const uint32_t* blocked, Partial* scratch = nullptr, bool timed = true) {
     const SelectPlan pl = plan_select(c, pflags);
-    const uint32_t tile = pl.tile, n_chunks = pl.n_chunks;
+    const uint32_t n_chunks = pl.n_chunks;
+    // granularity of a gap split: a staging tile; the tile kernel also works in 32-gap steps, which a
+    // small problem needs to put enough CTAs on the GPU
+    uint32_t tile = pl.tile;
+    if (pl.kernel == SEL_TILE && (uint64_t)n_chunks * ((G_act + tile - 1) / tile) < (uint64_t)SJA_SELECT_CTAS_PER_SM * c->n_sm)
+        tile = 32u;
     Partial* partial = scratch;
     if (!partial) {
         TRY(reserve(c, c->partial, (size_t)n_chunks * c->G * sizeof(Partial)));

@@ -7,24 +7,29 @@ namespace sja {
 
 // ---------------------------------------------------------------------------------------
 // Pass 0: validate the CSR and count the boundary rows of every job (popcount of its safe
-// bits above the progress point; the end of a job always counts).  A CTA owns 256
-// consecutive jobs: each warp counts 32 of them one after the other (lanes stride over the
-// job's safe words), the CTA scans the 256 counts and writes each job's offset relative to
-// the CTA plus the CTA total.  Two tiny kernels then turn CTA totals into global offsets.
-constexpr int COUNT_JOBS_PER_CTA = 256;
+// bits above the progress point; the end of a job always counts).  The kernel is bound by
+// memory latency, so it wants many warps with several loads in flight each: a CTA of 8
+// warps owns 64 consecutive jobs, a warp counts 8 of them, four at a time with eight lanes
+// per job (lanes stride over the job's safe words, four independent loads per lane).  The
+// CTA scans its 64 counts and writes each job's offset relative to the CTA plus the CTA
+// total.  Two tiny kernels then turn CTA totals into global offsets.
+constexpr int COUNT_JOBS_PER_CTA = 64;
+constexpr int COUNT_JOBS_PER_WARP = 8;
+constexpr uint32_t COUNT_LONG = 0x80000000u;   // marker: job left to the whole-warp pass
 
 __global__ void __launch_bounds__(256) count_boundaries_kernel(
     const uint64_t* __restrict__ off, const uint32_t* __restrict__ sbits,
     const uint32_t* __restrict__ p0, uint32_t J, uint64_t* __restrict__ local_off,
     uint64_t* __restrict__ cta_total, uint32_t* __restrict__ flags) {
-    __shared__ uint64_t warp_sums[8];
+    __shared__ uint32_t cnts[COUNT_JOBS_PER_CTA];
+    __shared__ uint64_t warp_sums[COUNT_JOBS_PER_CTA / 32];
     const uint64_t N = __ldg(off + J);   // total step count
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
-    const uint32_t jbase = blockIdx.x * COUNT_JOBS_PER_CTA + wid * 32u;
-    uint32_t mine = 0;   // row count of job jbase + lane
-    // four jobs at a time, eight lanes per job (more loads in flight than one job per warp pass)
+    const uint32_t slot0 = wid * COUNT_JOBS_PER_WARP;              // first job slot of this warp in the CTA
+    const uint32_t jbase = blockIdx.x * COUNT_JOBS_PER_CTA + slot0;
     const uint32_t grp = lane >> 3, sub = lane & 7u;
-    for (uint32_t it = 0; it < 8; ++it) {
+#pragma unroll
+    for (uint32_t it = 0; it < COUNT_JOBS_PER_WARP / 4; ++it) {
         const uint32_t i = it * 4u + grp;
         const uint32_t j = jbase + i;
         uint32_t cnt = 0;
@@ -37,7 +42,7 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
             if (!bad) {
                 const uint64_t s = js + p, e = je;
                 if (s < e && ((e - 1) >> 5) - (s >> 5) >= 256) {
-                    cnt = 0x80000000u;   // long job: counted by the whole warp below
+                    cnt = COUNT_LONG;   // long job: counted by the whole warp below
                 } else if (s < e) {
                     const uint64_t w0 = s >> 5, w1 = (e - 1) >> 5;
                     const uint32_t m0 = 0xFFFFFFFFu << (uint32_t)(s & 31);
@@ -62,20 +67,17 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
             }
         }
         if (__any_sync(0xFFFFFFFFu, bad) && lane == 0) atomicOr(flags, FLAG_BAD_PROFILE);
-        if (cnt != 0x80000000u) {   // (uniform within the eight lanes of a job)
+        if (cnt != COUNT_LONG) {   // (uniform within the eight lanes of a job)
             cnt += __shfl_xor_sync(0xFFu << (lane & 24u), cnt, 1);
             cnt += __shfl_xor_sync(0xFFu << (lane & 24u), cnt, 2);
             cnt += __shfl_xor_sync(0xFFu << (lane & 24u), cnt, 4);
         }
-        // job i's count sits in lanes 8*grp .. 8*grp+7; hand it to lane i
-        const uint32_t got = __shfl_sync(0xFFFFFFFFu, cnt, (lane & 3u) * 8u);
-        if ((lane >> 2) == it) mine = got;
+        if (sub == 0) cnts[slot0 + i] = cnt;
     }
+    __syncwarp();
     // long jobs (more than 256 safe words): all 32 lanes stride over the words of one job
-    uint32_t pending = __ballot_sync(0xFFFFFFFFu, mine == 0x80000000u);
-    while (pending) {
-        const uint32_t i = (uint32_t)__ffs((int)pending) - 1u;
-        pending &= pending - 1u;
+    for (uint32_t i = 0; i < COUNT_JOBS_PER_WARP; ++i) {
+        if (cnts[slot0 + i] != COUNT_LONG) continue;   // same value in every lane
         const uint32_t j = jbase + i;
         const uint64_t s = __ldg(off + j) + __ldg(p0 + j), e = __ldg(off + j + 1);
         const uint64_t w0 = s >> 5, w1 = (e - 1) >> 5;
@@ -88,26 +90,37 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
         }
         cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
         cnt += 1u - ((__ldg(sbits + w1) >> (uint32_t)((e - 1) & 31)) & 1u);
-        if (lane == i) mine = cnt;
+        __syncwarp();
+        if (lane == 0) cnts[slot0 + i] = cnt;
+        __syncwarp();
     }
-    uint64_t inc = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint64_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-        if (lane >= (uint32_t)o) inc += y;
-    }
-    if (lane == 31) warp_sums[wid] = inc;
     __syncthreads();
-    uint64_t before = 0, total = 0;
+    // exclusive scan of the CTA's counts by its first warps, one job per thread
+    uint32_t mine = 0;
+    uint64_t inc = 0;
+    if (threadIdx.x < COUNT_JOBS_PER_CTA) {
+        mine = cnts[threadIdx.x];
+        inc = mine;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) {
-        const uint64_t v = warp_sums[w];
-        if ((uint32_t)w < wid) before += v;
-        total += v;
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint64_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= (uint32_t)o) inc += y;
+        }
+        if (lane == 31) warp_sums[wid] = inc;
     }
-    const uint32_t j = jbase + lane;
-    if (j < J) local_off[j] = before + inc - mine;
-    if (threadIdx.x == 0) cta_total[blockIdx.x] = total;
+    __syncthreads();
+    if (threadIdx.x < COUNT_JOBS_PER_CTA) {
+        uint64_t before = 0, total = 0;
+#pragma unroll
+        for (int w = 0; w < COUNT_JOBS_PER_CTA / 32; ++w) {
+            const uint64_t v = warp_sums[w];
+            if ((uint32_t)w < wid) before += v;
+            total += v;
+        }
+        const uint32_t j = blockIdx.x * COUNT_JOBS_PER_CTA + threadIdx.x;
+        if (j < J) local_off[j] = before + inc - mine;
+        if (threadIdx.x == 0) cta_total[blockIdx.x] = total;
+    }
 }
 
 // Exclusive prefix sum of the per-CTA totals -> base[P+1].  One CTA of 1024 threads walks the

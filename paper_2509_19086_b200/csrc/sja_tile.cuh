@@ -39,7 +39,7 @@ namespace sja {
 #define SJA_TILE_RING 4
 #endif
 #ifndef SJA_TILE_GT
-#define SJA_TILE_GT 128
+#define SJA_TILE_GT 256
 #endif
 constexpr int TILE_WARPS = SJA_TILE_WARPS;
 constexpr int TILE_CTAS_PER_SM = SJA_TILE_CTAS_PER_SM;
