@@ -31,7 +31,7 @@ METRIC = "job-gap pairs evaluated/s"
 UNIT = "pairs/s"
 POLICY_NAMES = {0: "efficiency", 1: "fairness", 2: "sla"}
 # kernels launched per step: count_boundaries, cta_offsets, row_offsets, init_state, scan_profiles | rank_gaps,
-# place_gaps | select_merge (or select_search), finalize_awards | commit_vote, commit_apply, commit_refresh
+# place_gaps | select_tile (or select_merge / select_search), finalize_awards | commit_vote, commit_apply, commit_refresh
 KERNELS_PER_STEP = 12
 FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the scan kernel from its ncu capture on the 8192-job case (profiles/
@@ -42,10 +42,13 @@ NCU_SCAN_TRAFFIC_BYTES_PER_STEP = (273.048064e6 + 59.769344e6) / 33554432
 NCU_SCAN_SOURCE_SHA = "8bd8a77590ca9c38"
 
 
-# Issue-slot roofline of the select kernel (it is bound by instruction issue, not HBM): warp instructions per
-# pair from its ncu capture (profiles/select_merge_kernel_cfg2-jobs32768.md), peak = SMs x 4 schedulers x SM clock.
-NCU_MERGE_WARP_INSTR_PER_PAIR = 163228366 / (32768 * 4096)
-NCU_MERGE_SOURCE_SHA = "f21050b3c2d531d2"
+# Issue-slot roofline of the select kernel (it is bound by instruction issue, not HBM): warp instructions of one
+# launch on the large uniform workload from ncu (profiles/select_tile_kernel_cfg2-jobs32768.md, full-size line),
+# peak = SMs x 4 schedulers x SM clock.  The kernel's work is not proportional to the pair count, so the figure
+# holds for that workload only; it is reported while csrc/sja_tile.cuh is the file the counters were taken from.
+NCU_TILE_WARP_INSTR_PER_LAUNCH = 100790035
+NCU_TILE_PAIRS = 65536 * 4096
+NCU_TILE_SOURCE_SHA = "fcfa235eeb8ecc2b"
 N_SM, SCHEDULERS_PER_SM = 148, 4
 
 
@@ -58,17 +61,18 @@ def _source_sha(name: str):
         return None
 
 
-def select_roofline(pairs_per_s, sm_mhz):
-    """Issue rate of the select kernel against the GPU's warp-instruction issue peak."""
-    if not pairs_per_s or _source_sha("sja_round.cuh") != NCU_MERGE_SOURCE_SHA:
+def select_roofline(pairs, select_ms, sm_mhz):
+    """Issue rate of the select kernel against the GPU's warp-instruction issue peak (select_ms also holds the
+    few microseconds of finalize_awards_kernel, so the rate is slightly understated)."""
+    if not select_ms or pairs != NCU_TILE_PAIRS or _source_sha("sja_tile.cuh") != NCU_TILE_SOURCE_SHA:
         return None
     mhz = sm_mhz or 1965.0
     peak = N_SM * SCHEDULERS_PER_SM * mhz * 1e6
-    achieved = pairs_per_s * NCU_MERGE_WARP_INSTR_PER_PAIR
-    return {"kernel": "select_merge_kernel", "bound": "alu", "achieved": achieved / 1e9, "peak": peak / 1e9,
+    achieved = NCU_TILE_WARP_INSTR_PER_LAUNCH / (select_ms * 1e-3)
+    return {"kernel": "select_tile_kernel", "bound": "alu", "achieved": achieved / 1e9, "peak": peak / 1e9,
             "unit": "G warp-instructions/s", "frac": achieved / peak,
             "peak_kind": f"{N_SM} SMs x {SCHEDULERS_PER_SM} issue slots x {mhz:.0f} MHz",
-            "warp_instr_per_pair": NCU_MERGE_WARP_INSTR_PER_PAIR}
+            "warp_instr_per_pair": NCU_TILE_WARP_INSTR_PER_LAUNCH / NCU_TILE_PAIRS}
 
 
 def scan_traffic(n_steps: int):
@@ -250,7 +254,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--flags", type=int, default=0, help="sja_policy.flags (1 = per-pair search kernel)")
+    ap.add_argument("--flags", type=int, default=0, help="sja_policy.flags (1 = per-pair search kernel, 2 = per-gap merge kernel, 4 = tile kernel at any size)")
     ap.add_argument("--reauction", action="store_true",
                     help="time sja_round_reauction (select + commit repeated for orphaned gaps) instead of one select + commit")
     ap.add_argument("--jobs", type=int, default=0, help="override the job count (profiling captures)")
@@ -405,7 +409,7 @@ def main():
         "gpu_launches": timed_launches,
         "roofline": roofline,
         # the instruction count per pair was captured on the large uniform workload only
-        "select_roofline": select_roofline(pairs / (select_ms * 1e-3) if select_ms > 0 else None, clocks.get("sm_mhz"))
+        "select_roofline": select_roofline(pairs, select_ms, clocks.get("sm_mhz"))
         if spec.index == 2 and not args.flags and not args.reauction else None,
         "kernel_ms_per_step": breakdown,
         "select_pairs_per_s": pairs / (select_ms * 1e-3) if select_ms > 0 else None,

@@ -78,11 +78,14 @@ typedef enum {
 } sja_policy_kind;
 
 /* sja_policy.flags.  By default select runs the tile-sweep kernel over the gaps ordered by
- * (capacity, T).  Bit 0: evaluate every pair with the per-pair binary search over the boundary
- * table instead.  Bit 1: use the per-gap merge kernel instead.  Same results on every path;
- * the bits exist for testing and comparison. */
+ * (capacity, T), or the per-pair search for rounds of fewer than 65 536 pairs.  Bit 0:
+ * evaluate every pair with the per-pair binary search over the boundary table.  Bit 1: use
+ * the per-gap merge kernel.  Bit 2: use the tile-sweep kernel whatever the size.  Same
+ * results on every path; the bits exist for testing and comparison (bit 0 wins over the
+ * others, and an unsorted or many-capacity batch always takes the search). */
 #define SJA_FLAG_FORCE_SEARCH 1u
 #define SJA_FLAG_FORCE_MERGE 2u
+#define SJA_FLAG_FORCE_TILE 4u
 
 typedef struct {
     uint32_t kind;  /* sja_policy_kind */
@@ -173,8 +176,7 @@ sja_status sja_select(sja_ctx* ctx, const sja_policy* policy, sja_award* out, sj
  *
  * Cost and limit: every GPU on which the library is used holds the array until the process
  * exits.  The call needs ceil(J / 512) * G candidate slots of 16 bytes (ceil(J / 1024) * G
- * with SJA_FLAG_FORCE_MERGE; ceil(J / 256) * G with SJA_FLAG_FORCE_SEARCH or an unsorted /
- * many-capacity batch); if that exceeds the array it returns SJA_ERR_INVALID_ARG with the
+ * with SJA_FLAG_FORCE_MERGE; ceil(J / 256) * G where the per-pair search runs, see the flags); if that exceeds the array it returns SJA_ERR_INVALID_ARG with the
  * numbers in sja_last_error() and does nothing.
  *
  * The first call on a device looks up the array's device address (cudaGetSymbolAddress, with

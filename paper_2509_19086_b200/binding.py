@@ -22,6 +22,7 @@ MEM_HOST, MEM_DEVICE = 0, 1
 POLICY_EFFICIENCY, POLICY_FAIRNESS, POLICY_SLA = 0, 1, 2
 FLAG_FORCE_SEARCH = 1
 FLAG_FORCE_MERGE = 2
+FLAG_FORCE_TILE = 4
 NO_JOB = 0xFFFFFFFF
 
 GAP_DTYPE = np.dtype([("slice", "<u4"), ("start_ms", "<u4"), ("T_ms", "<u4"), ("C_MiB", "<u4")])

@@ -321,7 +321,11 @@ SelectPlan plan_select(const sja_ctx* c, uint32_t pflags) {
     SelectPlan p;
     // The tile and merge kernels need the (capacity, T) order and pay one restart per capacity
     // class; with very many classes (or an unsorted batch) the per-pair search is the better tool.
-    const bool sorted_ok = !(pflags & SJA_FLAG_FORCE_SEARCH) && c->gaps_sorted &&
+    const bool forced = (pflags & (SJA_FLAG_FORCE_MERGE | SJA_FLAG_FORCE_TILE)) != 0;
+    // A round of a few thousand pairs cannot fill the GPU either way; there the cursors' sequential walk
+    // through each capacity class is pure latency and the independent per-pair searches finish sooner.
+    const bool tiny = (uint64_t)c->J * c->G < (1ull << 16);
+    const bool sorted_ok = !(pflags & SJA_FLAG_FORCE_SEARCH) && c->gaps_sorted && (forced || !tiny) &&
                            c->n_classes <= std::max<uint32_t>(64u, c->G / 16u);
     p.kernel = !sorted_ok ? SEL_SEARCH : (pflags & SJA_FLAG_FORCE_MERGE) ? SEL_MERGE : SEL_TILE;
     p.jobs_per_cta = p.kernel == SEL_TILE ? (uint32_t)TILE_JOBS

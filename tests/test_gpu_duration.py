@@ -32,7 +32,7 @@ def test_duration_bounds_match_oracle(oracle_mod, base, changes):
             ctx.set_duration_bounds(lo, hi)
             for rnd in range(2):                      # second round starts from committed state
                 want = oracle_mod.select(prof, progress, ready, gaps, spec.policy, lo, hi)
-                for flags in (0, 1, 2):
+                for flags in (0, 1, 2, 4):
                     ctx.advertise(gaps)
                     got = ctx.select(spec.policy, flags=flags, out="host")
                     for f in FIELDS[:4]:

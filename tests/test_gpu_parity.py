@@ -106,7 +106,7 @@ def test_scan_cfg1_sampled_jobs(sja_mod, oracle_mod):
 
 
 # ------------------------------------------------------------------ select (a2-a5)
-@pytest.mark.parametrize("flags", [0, 1, 2])
+@pytest.mark.parametrize("flags", [0, 1, 2, 4])
 @pytest.mark.parametrize("policy", [0, 1, 2])
 def test_select_tiny_random_vs_oracle(sja_mod, oracle_mod, policy, flags):
     rng = np.random.default_rng(200 + policy)
@@ -140,7 +140,7 @@ def test_select_published_small_configs(sja_mod, oracle_mod, cfg):
         _load(ctx, prof)
         ctx.advertise(gaps)
         want = oracle_mod.select(prof, progress, prof.ready_ms, gaps, spec.policy)
-        for flags in (0, 1, 2):
+        for flags in (0, 1, 2, 4):
             got = ctx.select(spec.policy, flags=flags, out="host")
             _assert_awards_equal(got, want)
         assert (got["job"] != U32MAX).sum() > 0
@@ -162,7 +162,7 @@ def test_select_fairness_and_sla_scaled_configs(sja_mod, oracle_mod):
             _load(ctx, prof)
             ctx.advertise(gaps)
             want = oracle_mod.select(prof, progress, prof.ready_ms, gaps, spec.policy)
-            for flags in (0, 1, 2):
+            for flags in (0, 1, 2, 4):
                 got = ctx.select(spec.policy, flags=flags, out="host")
                 _assert_awards_equal(got, want)
 
@@ -182,7 +182,7 @@ def test_select_long_windows_and_many_capacity_classes(sja_mod, oracle_mod):
         _load(ctx, prof, progress)
         ctx.advertise(gaps)
         want = oracle_mod.select(prof, progress, prof.ready_ms, gaps, 0)
-        for flags in (0, 1, 2):
+        for flags in (0, 1, 2, 4):
             got = ctx.select(0, flags=flags, out="host")
             _assert_awards_equal(got, want)
 
@@ -209,7 +209,7 @@ def test_select_ties_duplicate_jobs_and_ready_boundaries(sja_mod, oracle_mod, po
             ctx.advertise(gaps)
             want = oracle_mod.select(prof, progress, prof.ready_ms, gaps, policy)
             assert (want["job"] != U32MAX).any()
-            for flags in (0, 1, 2):
+            for flags in (0, 1, 2, 4):
                 _assert_awards_equal(ctx.select(policy, flags=flags, out="host"), want)
             ctx.commit()
             oracle_mod.commit(progress, prof.ready_ms, gaps, want)
@@ -218,7 +218,7 @@ def test_select_ties_duplicate_jobs_and_ready_boundaries(sja_mod, oracle_mod, po
 
 
 # ------------------------------------------------------------------ commit (a6), multi-round
-@pytest.mark.parametrize("flags", [0, 1, 2])
+@pytest.mark.parametrize("flags", [0, 1, 2, 4])
 def test_streaming_rounds_bit_exact(sja_mod, oracle_mod, flags):
     """Scaled streaming workload: per-round awards (with grants) and final state match the oracle."""
     spec = wl.scaled(wl.SPECS[4], n_jobs=1500, fixed_len=300, n_gaps=200, n_rounds=60)
@@ -374,7 +374,7 @@ def test_select_is_deterministic_and_device_outputs_match(sja_mod):
         _load(ctx, prof)
         ctx.advertise(gaps)
         first = ctx.select(spec.policy, out="host")
-        for flags in (0, 1, 2, 0, 1, 2, 0):
+        for flags in (0, 1, 2, 4, 0, 1, 2, 4, 0):
             assert ctx.select(spec.policy, flags=flags, out="host").tobytes() == first.tobytes()
         dev = torch.zeros(24 * gaps.shape[0], dtype=torch.uint8, device="cuda")
         ctx.select(spec.policy, out=dev)

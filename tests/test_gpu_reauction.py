@@ -19,7 +19,7 @@ def _assert_equal(got, want):
         assert bad.size == 0, (f, bad[:5], got[bad[:5]], want[bad[:5]])
 
 
-@pytest.mark.parametrize("flags", [0, 1, 2])
+@pytest.mark.parametrize("flags", [0, 1, 2, 4])
 @pytest.mark.parametrize("base,changes", [
     (1, dict(n_jobs=900, fixed_len=300, n_gaps=300)),
     (2, dict(n_jobs=1500, fixed_len=400, n_gaps=257)),
