@@ -51,12 +51,13 @@ def _load():
     lib.orc_pair.restype = ctypes.c_int
     lib.orc_pair.argtypes = [vp, vp, vp, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint32,
                              ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
-                             ctypes.c_uint32, ctypes.c_uint32, u32p, u32p, u64p]
+                             ctypes.c_uint32, ctypes.c_uint32, ctypes.c_int, ctypes.c_uint32, u32p, u32p, u64p]
     lib.orc_select.restype = ctypes.c_int
     lib.orc_select.argtypes = [ctypes.c_uint32, vp, vp, vp, vp, vp, vp, vp, vp,
-                               ctypes.c_uint32, vp, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, vp]
+                               ctypes.c_uint32, vp, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
+                               ctypes.c_int, vp, vp]
     lib.orc_commit.restype = ctypes.c_int64
-    lib.orc_commit.argtypes = [ctypes.c_uint32, vp, vp, ctypes.c_uint32, vp, vp]
+    lib.orc_commit.argtypes = [ctypes.c_uint32, vp, vp, ctypes.c_uint32, vp, vp, ctypes.c_int]
     lib.orc_num_threads.restype = ctypes.c_int
     lib.orc_num_threads.argtypes = []
     del u8p
@@ -83,9 +84,9 @@ U32MAX = 0xFFFFFFFF
 
 
 def pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: int,
-         tau_min_ms: int = 0, tau_max_ms: int = U32MAX):
-    """R1-R3 (with the duration thresholds of R2') for one (gap, job) pair: ``None`` for decline,
-    else ``(k, dur, work)``."""
+         tau_min_ms: int = 0, tau_max_ms: int = U32MAX, late_start: bool = False, deadline_ms: int = U32MAX):
+    """R1-R3 (with the duration thresholds of R2' and the window options of R1'') for one (gap, job)
+    pair: ``None`` for decline, else ``(k, dur, work)``."""
     lib = _load()
     k = ctypes.c_uint32()
     dur = ctypes.c_uint32()
@@ -93,15 +94,18 @@ def pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: i
     ok = lib.orc_pair(prof.dur_ms.ctypes.data, prof.mem_MiB.ctypes.data,
                       prof.safe_bits.ctypes.data, int(prof.off[j]), int(prof.off[j + 1]),
                       int(p), int(ready_ms), int(start_ms), int(T_ms), int(C_MiB),
-                      int(tau_min_ms), int(tau_max_ms), ctypes.byref(k), ctypes.byref(dur), ctypes.byref(work))
+                      int(tau_min_ms), int(tau_max_ms), int(bool(late_start)), int(deadline_ms),
+                      ctypes.byref(k), ctypes.byref(dur), ctypes.byref(work))
     if not ok:
         return None
     return int(k.value), int(dur.value), int(work.value)
 
 
 def select(prof, progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray,
-           policy: int, tau_min_ms: int = 0, tau_max_ms: int = U32MAX) -> np.ndarray:
-    """R1-R5 for a batch of gaps; returns ``AWARD_DTYPE[G]`` (``granted`` all zero)."""
+           policy: int, tau_min_ms: int = 0, tau_max_ms: int = U32MAX, late_start: bool = False,
+           deadline_ms: Optional[np.ndarray] = None) -> np.ndarray:
+    """R1-R5 for a batch of gaps; returns ``AWARD_DTYPE[G]`` (``granted`` all zero).
+    ``late_start`` / ``deadline_ms`` (u32 per job) switch on the window options of R1''."""
     lib = _load()
     off = _as(prof.off, np.uint64)
     d = _as(prof.dur_ms, np.uint32)
@@ -113,32 +117,35 @@ def select(prof, progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray,
     prio = _as(prof.prio, np.uint8)
     gaps = np.ascontiguousarray(gaps, dtype=GAP_DTYPE)
     awards = np.zeros(gaps.shape[0], dtype=AWARD_DTYPE)
+    deadline = _as(deadline_ms, np.uint32)
+    assert deadline is None or deadline.shape[0] == off.shape[0] - 1
     rc = lib.orc_select(off.shape[0] - 1, _ptr(off), _ptr(d), _ptr(m), _ptr(s),
                         _ptr(progress), _ptr(ready_ms), _ptr(wait), _ptr(prio),
                         gaps.shape[0], _ptr(gaps), int(policy), int(tau_min_ms), int(tau_max_ms),
-                        _ptr(awards))
+                        int(bool(late_start)), _ptr(deadline), _ptr(awards))
     if rc != 0:
         raise ValueError("oracle select: unknown policy or missing attribute array")
     return awards
 
 
 def commit(progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray,
-           awards: np.ndarray) -> int:
-    """R6, in place on ``progress``, ``ready_ms`` and ``awards['granted']``."""
+           awards: np.ndarray, late_start: bool = False) -> int:
+    """R6, in place on ``progress``, ``ready_ms`` and ``awards['granted']``.  With ``late_start`` a granted
+    subjob began at ``max(start, ready)`` (R1''), so that is what the new ready time counts from."""
     lib = _load()
     assert progress.dtype == np.uint32 and progress.flags.c_contiguous
     assert ready_ms.dtype == np.uint32 and ready_ms.flags.c_contiguous
     assert awards.dtype == AWARD_DTYPE and awards.flags.c_contiguous
     gaps = np.ascontiguousarray(gaps, dtype=GAP_DTYPE)
     n = lib.orc_commit(progress.shape[0], _ptr(progress), _ptr(ready_ms),
-                       gaps.shape[0], _ptr(gaps), _ptr(awards))
+                       gaps.shape[0], _ptr(gaps), _ptr(awards), int(bool(late_start)))
     if n < 0:
-        raise OverflowError("oracle commit: start + dur does not fit in 32 bits")
+        raise OverflowError("oracle commit: begin + dur does not fit in 32 bits")
     return int(n)
 
 
 def commit_masked(progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray, awards: np.ndarray,
-                  accept: np.ndarray) -> int:
+                  accept: np.ndarray, late_start: bool = False) -> int:
     """R6 restricted to the gaps with ``accept[g] != 0``.
 
     A subjob that failed or was never started leaves its parent job at the last completed
@@ -148,6 +155,6 @@ def commit_masked(progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray, 
     accept = np.asarray(accept).astype(bool)
     visible = awards.copy()
     visible["job"][~accept] = NO_JOB
-    n = commit(progress, ready_ms, gaps, visible)
+    n = commit(progress, ready_ms, gaps, visible, late_start)
     awards["granted"] = visible["granted"]
     return n

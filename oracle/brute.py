@@ -16,14 +16,20 @@ def _safe(bits, i: int) -> bool:
 
 
 def brute_pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: int,
-               tau_min_ms: int = 0, tau_max_ms: int = 0xFFFFFFFF):
-    """``None`` (decline) or ``(k, dur, work)`` of the longest feasible subjob."""
+               tau_min_ms: int = 0, tau_max_ms: int = 0xFFFFFFFF, late_start: bool = False,
+               deadline_ms: int = 0xFFFFFFFF):
+    """``None`` (decline) or ``(k, dur, work)`` of the longest feasible subjob.
+
+    Window options: with ``late_start`` the subjob occupies ``[begin, begin + dur)`` with
+    ``begin = max(start, ready)`` and has to lie inside the gap ``[start, start + T]``; without it the
+    job must be ready when the gap opens.  It has to be over by ``deadline_ms``."""
     s, e = int(prof.off[j]), int(prof.off[j + 1])
     length = e - s
     if p >= length:
         return None
-    if start_ms < ready_ms:
+    if start_ms < ready_ms and not late_start:
         return None
+    begin = max(start_ms, ready_ms)
     d = [int(x) for x in prof.dur_ms[s:e]]
     m = [int(x) for x in prof.mem_MiB[s:e]]
     candidates = []
@@ -31,7 +37,9 @@ def brute_pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_
         ends_safe = _safe(prof.safe_bits, s + k - 1) or k == length
         if not ends_safe:
             continue
-        if sum(d[p:k]) > T_ms:
+        if begin + sum(d[p:k]) > start_ms + T_ms:               # ends inside the gap
+            continue
+        if deadline_ms != 0xFFFFFFFF and begin + sum(d[p:k]) > deadline_ms:   # Section 4.4 (2): done by the deadline
             continue
         if not (tau_min_ms <= sum(d[p:k]) <= tau_max_ms):      # Section 4.3 (5) thresholds
             continue

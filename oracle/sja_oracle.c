@@ -39,6 +39,14 @@
  *   R6 commit      : a job that won several gaps accepts the one with the largest k*,
  *                    ties to the lowest gap id; that gap is granted, the others are not;
  *                    then p_j = k*, ready_j = start_g + dur.
+ *   R1'' options   : two optional refinements of the window a pair sees, both off by default.
+ *                    Late start: a job that becomes ready inside the window may begin then, so
+ *                    begin = max(start_g, ready_j), eligible iff begin <= start_g + T_g, and only
+ *                    the rest of the window counts: sum d <= T_g - (begin - start_g); the commit
+ *                    sets ready_j = begin + dur.  Deadline (Section 4.4, item 2: admit only
+ *                    subjobs that complete by their deadline; the risk margin lives in the
+ *                    durations, as it does in the memory envelope): a candidate also needs
+ *                    begin + sum d <= deadline_j; 2^32-1 means no deadline.
  *
  * The walk below visits one step at a time, exactly in that order: no prefix arrays,
  * no search, no blocking.  OpenMP only spreads independent gaps over host threads.
@@ -83,11 +91,20 @@ int orc_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *sa
              uint64_t s, uint64_t e, uint32_t p, uint32_t ready_ms,
              uint32_t start_ms, uint32_t T_ms, uint32_t C_MiB,
              uint32_t tau_min_ms, uint32_t tau_max_ms,
+             int late_start, uint32_t deadline_ms,
              uint32_t *k_out, uint32_t *dur_out, uint64_t *work_out)
 {
     uint64_t len = e - s;
     if ((uint64_t)p >= len) return 0;            /* R1: finished job */
-    if (start_ms < ready_ms) return 0;           /* R1: gap opens before the job is ready */
+    uint64_t begin = start_ms;                   /* when the subjob would start running */
+    if (start_ms < ready_ms) {
+        if (!late_start) return 0;               /* R1: gap opens before the job is ready */
+        begin = ready_ms;                        /* R1'': start inside the window */
+    }
+    uint64_t window_end = (uint64_t)start_ms + (uint64_t)T_ms;
+    if (begin > window_end) return 0;            /* R1'': ready only after the window has closed */
+    const int has_deadline = deadline_ms != 0xFFFFFFFFu;          /* 2^32-1: no deadline */
+    if (has_deadline && begin > (uint64_t)deadline_ms) return 0; /* R1'': deadline already passed */
 
     uint64_t acc = 0, work = 0;
     uint32_t peak = 0;
@@ -98,7 +115,8 @@ int orc_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *sa
         acc += dur_ms[i];
         if (mem_MiB[i] > peak) peak = mem_MiB[i];
         work += (uint64_t)dur_ms[i] * (uint64_t)mem_MiB[i];
-        if (acc > (uint64_t)T_ms || peak > C_MiB) break;   /* R2: window or capacity broken */
+        if (begin + acc > window_end || peak > C_MiB) break;   /* R2: window or capacity broken */
+        if (has_deadline && begin + acc > (uint64_t)deadline_ms) break;   /* R1'': would finish after the deadline */
         if (acc > (uint64_t)tau_max_ms) break;             /* R2': longer than the maximum subjob */
         if ((step_is_safe(safe_bits, i) || i + 1 == e)     /* R2: safe boundary after step i */
             && acc >= (uint64_t)tau_min_ms) {              /* R2': not shorter than the minimum subjob */
@@ -140,6 +158,7 @@ int orc_select(uint32_t n_jobs, const uint64_t *off,
                const uint32_t *wait_ms, const uint8_t *prio,
                uint32_t n_gaps, const orc_gap *gaps, uint32_t policy,
                uint32_t tau_min_ms, uint32_t tau_max_ms,
+               int late_start, const uint32_t *deadline_ms /* per job, or NULL = none */,
                orc_award *awards)
 {
     if (policy > ORC_SLA) return -1;
@@ -157,6 +176,7 @@ int orc_select(uint32_t n_jobs, const uint64_t *off,
             uint64_t work;
             if (!orc_pair(dur_ms, mem_MiB, safe_bits, off[j], off[j + 1], progress[j],
                           ready_ms[j], gap.start_ms, gap.T_ms, gap.C_MiB, tau_min_ms, tau_max_ms,
+                          late_start, deadline_ms ? deadline_ms[j] : 0xFFFFFFFFu,
                           &k, &dur, &work))
                 continue;                                      /* decline */
             uint32_t cls;
@@ -185,10 +205,10 @@ int orc_select(uint32_t n_jobs, const uint64_t *off,
 
 /*
  * R6.  Marks granted gaps in awards[], advances progress / ready_ms of the granted
- * jobs, returns the number of grants (or -1 if start + dur does not fit in 32 bits).
+ * jobs, returns the number of grants (or -1 if begin + dur does not fit in 32 bits).
  */
 int64_t orc_commit(uint32_t n_jobs, uint32_t *progress, uint32_t *ready_ms,
-                   uint32_t n_gaps, const orc_gap *gaps, orc_award *awards)
+                   uint32_t n_gaps, const orc_gap *gaps, orc_award *awards, int late_start)
 {
     int64_t granted = 0;
     for (uint32_t g = 0; g < n_gaps; ++g) awards[g].granted = 0;
@@ -210,7 +230,9 @@ int64_t orc_commit(uint32_t n_jobs, uint32_t *progress, uint32_t *ready_ms,
     for (uint32_t g = 0; g < n_gaps; ++g) {
         if (!awards[g].granted) continue;
         uint32_t j = awards[g].job;
-        uint64_t new_ready = (uint64_t)gaps[g].start_ms + (uint64_t)awards[g].dur_ms;
+        uint64_t begin = gaps[g].start_ms;
+        if (late_start && ready_ms[j] > gaps[g].start_ms) begin = ready_ms[j];   /* R1'': began inside the window */
+        uint64_t new_ready = begin + (uint64_t)awards[g].dur_ms;
         if (new_ready > 0xFFFFFFFFull) return -1;
         progress[j] = awards[g].end_step;
         ready_ms[j] = (uint32_t)new_ready;
