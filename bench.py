@@ -257,6 +257,8 @@ def main():
     ap.add_argument("--flags", type=int, default=0, help="sja_policy.flags (1 = per-pair search kernel, 2 = per-gap merge kernel, 4 = tile kernel at any size)")
     ap.add_argument("--reauction", action="store_true",
                     help="time sja_round_reauction (select + commit repeated for orphaned gaps) instead of one select + commit")
+    ap.add_argument("--window-options", action="store_true",
+                    help="late start inside a gap and per-job deadlines (ready + 2000..8000 ms): per-pair search path")
     ap.add_argument("--jobs", type=int, default=0, help="override the job count (profiling captures)")
     ap.add_argument("--gaps", type=int, default=0, help="override the gap count (profiling captures)")
     args = ap.parse_args()
@@ -310,6 +312,12 @@ def main():
     gaps_pinned = gaps_pinned.view(wl.GAP_DTYPE)
     dev = {k: _to_device(a, device) for k, a in host_arrays.items()}
     dev_gaps = _to_device(gaps, device)
+    dev_deadline = None
+    if args.window_options:
+        rng = np.random.default_rng(my_spec.seed + 77)
+        deadline = (prof.ready_ms.astype(np.uint64) + rng.integers(2000, 8001, J).astype(np.uint64)).astype(np.uint32)
+        dev_deadline = _to_device(deadline, device)
+        pinned_keep["deadline"], pinned["deadline"] = _pinned(deadline)
     torch.cuda.synchronize()
 
     launches = [0]
@@ -317,6 +325,8 @@ def main():
     def step_device():
         ctx.load_profiles(dev["off"], dev["d"], dev["m"], dev["s"], dev["ready"],
                           wait_ms=dev.get("wait"), prio=dev.get("prio"))
+        if args.window_options:
+            ctx.set_window_options(True, dev_deadline)
         ctx.advertise(dev_gaps)
         if args.reauction:
             _, passes = ctx.round_reauction(my_spec.policy, flags=args.flags)
@@ -329,6 +339,8 @@ def main():
     def step_e2e():
         ctx.load_profiles(pinned["off"], pinned["d"], pinned["m"], pinned["s"], pinned["ready"],
                           wait_ms=pinned.get("wait"), prio=pinned.get("prio"))
+        if args.window_options:
+            ctx.set_window_options(True, pinned["deadline"])
         ctx.advertise(gaps_pinned)
         aw = ctx.select(my_spec.policy, flags=args.flags, out="host")
         n = ctx.commit(want_count=True)
@@ -379,7 +391,7 @@ def main():
     ms_per_step = ms_total / args.steps
     value = replicas.throughput(total_pairs, args.steps, ms_total)
     e2e_value = replicas.throughput(total_pairs, args.e2e_steps, e2e_ms) if e2e_ms > 0 else None
-    h2d = sum(int(a.nbytes) for a in host_arrays.values()) + int(gaps.nbytes)
+    h2d = sum(int(a.nbytes) for a in host_arrays.values()) + int(gaps.nbytes) + (4 * J if args.window_options else 0)
     d2h = 24 * G + 4
 
     peak, peak_kind = measured_peak()
@@ -402,7 +414,8 @@ def main():
                    "boundary_rows": n_rows, "policy": POLICY_NAMES[spec.policy], "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2 (profile arrays re-read from HBM every step)"
                    if prof.raw_bytes() > 200e6 else "inputs smaller than L2",
-                   "flags": args.flags, "reauction": bool(args.reauction)},
+                   "flags": args.flags, "reauction": bool(args.reauction),
+                   "window_options": bool(args.window_options)},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / max(1, args.e2e_steps), "steps": args.e2e_steps},
@@ -410,7 +423,7 @@ def main():
         "roofline": roofline,
         # the instruction count per pair was captured on the large uniform workload only
         "select_roofline": select_roofline(pairs, select_ms, clocks.get("sm_mhz"))
-        if spec.index == 2 and not args.flags and not args.reauction else None,
+        if spec.index == 2 and not args.flags and not args.reauction and not args.window_options else None,
         "kernel_ms_per_step": breakdown,
         "select_pairs_per_s": pairs / (select_ms * 1e-3) if select_ms > 0 else None,
         "profile_gb_per_s": prof.raw_bytes() / (scan_ms * 1e-3) / 1e9 if scan_ms > 0 else None,

@@ -234,6 +234,29 @@ sja_status sja_round_reauction(sja_ctx* ctx, const sja_policy* policy, uint32_t 
  */
 sja_status sja_set_duration_bounds(sja_ctx* ctx, uint32_t tau_min_ms, uint32_t tau_max_ms);
 
+/*
+ * Window options: two refinements of the window a (gap, job) pair sees, both off by default.
+ *
+ * late_start = 1: a job that becomes ready inside an advertised window may begin then instead
+ * of declining: the subjob begins at max(start, ready_j), the job is eligible iff that is not
+ * later than start + T, only the rest of the window counts (sum d <= T - (begin - start)),
+ * and the commit sets ready_j = begin + dur.  (The paper leaves open whether a window has to
+ * be taken from its first millisecond; the default is the strict reading.)
+ *
+ * deadline_ms (u32[J], or NULL for none; an entry of 0xFFFFFFFF means no deadline for that
+ * job): deadline- and SLO-aware admission (Section 4.4, item 2: admit only subjobs whose
+ * completion time stays below their deadline).  A candidate also needs
+ * begin + sum d <= deadline_j; the tolerated risk of a violation lives in the per-step
+ * durations, as the memory risk lives in the envelope.  The array is copied.
+ *
+ * With either option on, every select runs the per-pair search kernel (the usable window
+ * then differs from pair to pair, which the ordered-gap kernels cannot follow); results obey
+ * the same rules otherwise and sja_round_reauction / sja_commit_masked work unchanged.
+ * Call after sja_load_profiles (a new load clears the deadlines and keeps late_start).  A
+ * select that has not been committed yet is discarded by the call: select again before commit.
+ */
+sja_status sja_set_window_options(sja_ctx* ctx, uint32_t late_start, const uint32_t* deadline_ms, sja_memspace where);
+
 /* Copy the G awards of the last select (with `granted` set if it was committed). */
 sja_status sja_get_awards(sja_ctx* ctx, sja_award* out, sja_memspace where);
 

@@ -30,7 +30,7 @@ AWARD_DTYPE = np.dtype([("job", "<u4"), ("end_step", "<u4"), ("dur_ms", "<u4"), 
                         ("score", "<u8")])
 
 EXPORTS = [
-    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit", "sja_commit_masked", "sja_round_reauction", "sja_set_duration_bounds",
+    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit", "sja_commit_masked", "sja_round_reauction", "sja_set_duration_bounds", "sja_set_window_options",
     "sja_get_awards", "sja_get_state", "sja_scan_size", "sja_get_scan", "sja_profile_enable",
     "sja_profile_read", "sja_last_error",
 ]
@@ -78,6 +78,7 @@ def load_library() -> ctypes.CDLL:
     lib.sja_commit.argtypes = [vp, ctypes.POINTER(u32)]
     lib.sja_round_reauction.argtypes = [vp, ctypes.POINTER(SjaPolicy), u32, ctypes.POINTER(u32), ctypes.POINTER(u32)]
     lib.sja_set_duration_bounds.argtypes = [vp, u32, u32]
+    lib.sja_set_window_options.argtypes = [vp, u32, vp, i32]
     lib.sja_commit_masked.argtypes = [vp, vp, i32, ctypes.POINTER(u32)]
     lib.sja_get_awards.argtypes = [vp, vp, i32]
     lib.sja_get_state.argtypes = [vp, vp, vp, i32]
@@ -241,6 +242,15 @@ class Sja:
     # -- sja_set_duration_bounds
     def set_duration_bounds(self, tau_min_ms: int = 0, tau_max_ms: int = 0xFFFFFFFF) -> None:
         self._check(self._lib.sja_set_duration_bounds(self._h, int(tau_min_ms), int(tau_max_ms)))
+
+    # -- sja_set_window_options
+    def set_window_options(self, late_start: bool = False, deadline_ms=None) -> None:
+        """``deadline_ms``: u32 per job (numpy or CUDA tensor) or None."""
+        p, space, _keep = _ptr_space(deadline_ms, None, np.uint32)
+        if deadline_ms is not None and int(_keep.shape[0]) != self.n_jobs:
+            raise ValueError("deadline_ms needs one entry per loaded job")
+        self._check(self._lib.sja_set_window_options(self._h, 1 if late_start else 0, p,
+                                                     MEM_HOST if space is None else space))
 
     # -- sja_get_awards / sja_get_state
     def get_awards(self) -> np.ndarray:

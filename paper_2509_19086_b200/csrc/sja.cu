@@ -62,6 +62,8 @@ struct sja_ctx {
     bool advertised = false, selected = false, committed = false;
     uint32_t G = 0, last_policy = 0;
     uint32_t tau_min = 0, tau_max = 0xFFFFFFFFu;   // subjob duration thresholds for select
+    bool late_start = false, have_deadline = false;   // window options (sja_set_window_options)
+    DevBuf deadline;
     bool gaps_sorted = false;          // sgaps is ordered by (C, T); else it is the caller's order
     uint32_t n_classes = 0;            // distinct capacities of the batch (valid when sorted)
     DevBuf gaps, sgaps, gap_info, gap_rank, awards, widx, partial, winners;
@@ -232,6 +234,8 @@ JobView job_view(const sja_ctx* c) {
     v.blocked = nullptr;
     v.tau_min = c->tau_min;
     v.tau_max = c->tau_max;
+    v.deadline = c->have_deadline ? c->deadline.as<uint32_t>() : nullptr;
+    v.late_start = c->late_start ? 1u : 0u;
     v.J = c->J;
     return v;
 }
@@ -325,7 +329,9 @@ SelectPlan plan_select(const sja_ctx* c, uint32_t pflags) {
     // A round of a few thousand pairs cannot fill the GPU either way; there the cursors' sequential walk
     // through each capacity class is pure latency and the independent per-pair searches finish sooner.
     const bool tiny = (uint64_t)c->J * c->G < (1ull << 16);
-    const bool sorted_ok = !(pflags & SJA_FLAG_FORCE_SEARCH) && c->gaps_sorted && (forced || !tiny) &&
+    // with a window option the usable window differs from pair to pair: only the search kernel does that
+    const bool per_pair_window = c->late_start || c->have_deadline;
+    const bool sorted_ok = !(pflags & SJA_FLAG_FORCE_SEARCH) && !per_pair_window && c->gaps_sorted && (forced || !tiny) &&
                            c->n_classes <= std::max<uint32_t>(64u, c->G / 16u);
     p.kernel = !sorted_ok ? SEL_SEARCH : (pflags & SJA_FLAG_FORCE_MERGE) ? SEL_MERGE : SEL_TILE;
     p.jobs_per_cta = p.kernel == SEL_TILE ? (uint32_t)TILE_JOBS
@@ -389,7 +395,7 @@ void run_commit(sja_ctx* c, uint32_t* blocked, const uint8_t* accept = nullptr) 
         c->awards.as<Award>(), c->gaps.as<Gap>(), c->widx.as<uint32_t>(), G, c->jobwin.as<unsigned long long>(),
         c->boff.as<uint64_t>(), c->A.as<uint4>(), c->p.as<uint32_t>(), c->ready.as<uint32_t>(), c->pb.as<uint32_t>(),
         c->Dp.as<uint32_t>(), c->Wp.as<uint64_t>(), c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(),
-        c->flags.as<uint32_t>(), blocked, accept);
+        c->flags.as<uint32_t>(), blocked, accept, c->late_start ? 1u : 0u);
     commit_refresh_kernel<<<(uint32_t)(((uint64_t)G * 32 + 255) / 256), 256, 0, c->stream>>>(
         c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(), G, c->boff.as<uint64_t>(), c->pb.as<uint32_t>(),
         c->A.as<uint4>(), c->B.as<uint2>(), c->jobwin.as<unsigned long long>());
@@ -478,7 +484,7 @@ sja_status sja_destroy(sja_ctx* c) {
     cudaStreamSynchronize(c->stream);
     DevBuf* bufs[] = {&c->st_off, &c->st_d, &c->st_m, &c->st_s, &c->st_p, &c->p, &c->ready, &c->pb, &c->Dp,
                       &c->Wp, &c->wait, &c->prio, &c->nbj, &c->cta_tot, &c->cta_base, &c->boff, &c->boff_next, &c->A, &c->B, &c->jobwin,
-                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->awards, &c->widx, &c->partial,
+                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->deadline, &c->awards, &c->widx, &c->partial,
                       &c->winners};
     for (DevBuf* b : bufs) release(*b);
     for (ProfSpan& s : c->spans) { cudaEventDestroy(s.a); cudaEventDestroy(s.b); }
@@ -607,6 +613,7 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
 
     // from here on the previous load is replaced
     c->loaded = false;
+    c->have_deadline = false;   // deadlines belong to the jobs of a load
     c->advertised = c->selected = c->committed = false;
     TRY(reserve(c, c->A, (size_t)n_rows * 16 + 16));
     TRY(reserve(c, c->B, (size_t)n_rows * 8 + 16));
@@ -871,6 +878,24 @@ sja_status sja_set_duration_bounds(sja_ctx* c, uint32_t tau_min_ms, uint32_t tau
         return fail(c, SJA_ERR_INVALID_ARG, "sja_set_duration_bounds: tau_min %u > tau_max %u", tau_min_ms, tau_max_ms);
     c->tau_min = tau_min_ms;
     c->tau_max = tau_max_ms;
+    return SJA_OK;
+}
+
+sja_status sja_set_window_options(sja_ctx* c, uint32_t late_start, const uint32_t* deadline_ms, sja_memspace where) {
+    TRY(check_ctx(c));
+    if (late_start > 1u) return fail(c, SJA_ERR_INVALID_ARG, "sja_set_window_options: late_start must be 0 or 1");
+    if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_set_window_options: bad memspace");
+    if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_set_window_options before sja_load_profiles");
+    DeviceGuard guard(c->device);
+    if (deadline_ms) {
+        TRY(reserve(c, c->deadline, (size_t)c->J * 4));
+        TRY(copy_in(c, c->deadline.p, deadline_ms, (size_t)c->J * 4, where));
+        if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));   // the caller may reuse its buffer
+    }
+    c->have_deadline = deadline_ms != nullptr;
+    c->late_start = late_start != 0u;
+    c->selected = false;   // awards chosen under the old options must not be committed under the new ones
     return SJA_OK;
 }
 

@@ -20,6 +20,8 @@ struct JobView {
     const uint2* B;
     const uint32_t* blocked;  // may be nullptr; jobs with a non-zero entry decline every gap
     uint32_t tau_min, tau_max;  // subjob duration thresholds (Section 4.3, item 5); 0 / 0xFFFFFFFF = off
+    const uint32_t* deadline;   // may be nullptr; per job, 0xFFFFFFFF = none (Section 4.4, item 2)
+    uint32_t late_start;        // non-zero: a job that turns ready inside a window may begin then
     uint32_t J;
 };
 
@@ -34,7 +36,11 @@ __device__ __forceinline__ uint32_t policy_factor(const JobView& jv, uint32_t ki
 // for each pair it finds the number of boundary rows that satisfy both monotone bounds
 // (D - Dp <= T and running max <= C) with a galloping + binary search over the rows above
 // the progress point, turns the last such row into a policy key, and the warp reduces the
-// 32 keys to one candidate per gap (largest key, then lowest job id).
+// 32 keys to one candidate per gap (largest key, then lowest job id).  Because every pair
+// is searched on its own, this is also the kernel for the window options, where the usable
+// window differs from pair to pair: with a late start the subjob begins at
+// max(start, ready) and only the rest of the window counts; with a deadline it must be over
+// by then.
 constexpr int SEARCH_THREADS = 256;
 constexpr int SEARCH_GT = 64;   // gaps per staging tile
 
@@ -50,7 +56,7 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
     if (slot < n_jobs) j = job_list ? job_list[slot] : slot;
 
     uint64_t base = 0, Wp = 0;
-    uint32_t n = 0, Dp = 0, ready = 0, factor = 0;
+    uint32_t n = 0, Dp = 0, ready = 0, factor = 0, deadline = 0xFFFFFFFFu;
     if (j != SJA_NO_JOB_DEV) {
         const uint64_t b0 = jv.boff[j], b1 = jv.boff[j + 1];
         const uint32_t pb = jv.pb[j];
@@ -61,7 +67,9 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
         Wp = jv.Wp[j];
         ready = jv.ready[j];
         factor = policy_factor(jv, kind, j);
+        if (jv.deadline) deadline = jv.deadline[j];
     }
+    const bool late = jv.late_start != 0u;
     const uint32_t g_begin = blockIdx.y * gaps_per_split;
     const uint32_t g_end = min(G, g_begin + gaps_per_split);
 
@@ -69,10 +77,24 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
         const uint32_t gt = min((uint32_t)SEARCH_GT, g_end - g0);
         for (uint32_t gi = 0; gi < gt; ++gi) {
             const uint4 gq = __ldg(reinterpret_cast<const uint4*>(gaps) + g0 + gi);
-            const uint32_t start = gq.y, T = min(gq.z, jv.tau_max), C = gq.w;
+            const uint32_t start = gq.y, C = gq.w;
+            // the window this pair sees: what is left of the gap once the job can begin, cut at its deadline
+            uint32_t T = gq.z, begin = start;
+            bool eligible = n != 0;
+            if (start < ready) {
+                const uint32_t late_by = ready - start;
+                if (!late || late_by > T) eligible = false;
+                begin = ready;
+                T -= min(late_by, T);
+            }
+            if (deadline != 0xFFFFFFFFu) {
+                if (begin > deadline) eligible = false;
+                T = min(T, deadline - min(begin, deadline));
+            }
+            T = min(T, jv.tau_max);
             uint32_t cnt = 0;
             uint64_t key = 0;
-            if (n != 0 && start >= ready) {
+            if (eligible) {
                 uint32_t lo = 0, hi = n, idx = 0;
                 for (;;) {   // gallop over rows 0, 1, 3, 7, ...
                     if (idx >= n) { hi = n; break; }
@@ -184,7 +206,8 @@ __global__ void __launch_bounds__(256) commit_apply_kernel(
     const unsigned long long* __restrict__ jobwin, const uint64_t* __restrict__ boff, const uint4* __restrict__ A,
     uint32_t* __restrict__ p, uint32_t* __restrict__ ready, uint32_t* __restrict__ pb, uint32_t* __restrict__ Dp,
     uint64_t* __restrict__ Wp, uint32_t* __restrict__ winners, uint32_t* __restrict__ n_granted,
-    uint32_t* __restrict__ flags, uint32_t* __restrict__ blocked, const uint8_t* __restrict__ accept) {
+    uint32_t* __restrict__ flags, uint32_t* __restrict__ blocked, const uint8_t* __restrict__ accept,
+    uint32_t late_start) {
     const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= G) return;
     if (accept && !accept[g]) return;
@@ -195,7 +218,9 @@ __global__ void __launch_bounds__(256) commit_apply_kernel(
     const uint32_t j = a.job;
     const uint32_t row_rel = pb[j] + widx[g] - 1;
     const uint4 r = A[boff[j] + row_rel];
-    const uint64_t new_ready = (uint64_t)gaps[g].start + (uint64_t)a.dur;
+    // the subjob began when the gap opened, or when the job turned ready inside it (late start)
+    const uint32_t begin = late_start ? max(gaps[g].start, ready[j]) : gaps[g].start;
+    const uint64_t new_ready = (uint64_t)begin + (uint64_t)a.dur;
     if (new_ready > 0xFFFFFFFFull) atomicOr(flags, FLAG_OVF_READY);
     awards[g].granted = 1;
     p[j] = a.end_step;
