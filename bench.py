@@ -259,6 +259,9 @@ def main():
                     help="time sja_round_reauction (select + commit repeated for orphaned gaps) instead of one select + commit")
     ap.add_argument("--window-options", action="store_true",
                     help="late start inside a gap and per-job deadlines (ready + 2000..8000 ms): per-pair search path")
+    ap.add_argument("--streaming", action="store_true",
+                    help="multi-round workloads only: load once, then every step is one advertise/select/commit round "
+                         "with that round's gap batch (use --steps 1000 for the published streaming configuration)")
     ap.add_argument("--jobs", type=int, default=0, help="override the job count (profiling captures)")
     ap.add_argument("--gaps", type=int, default=0, help="override the gap count (profiling captures)")
     args = ap.parse_args()
@@ -273,6 +276,8 @@ def main():
     if args.impl == "reference":
         run_reference(args, spec)
         return
+    if args.streaming and (spec.n_rounds <= 1 or args.reauction):
+        raise SystemExit("--streaming needs a multi-round workload (--workload 4) and no --reauction")
 
     import torch
     from paper_2509_19086_b200 import binding
@@ -321,6 +326,34 @@ def main():
     torch.cuda.synchronize()
 
     launches = [0]
+    round_gaps_dev, round_gaps_pinned = [], []
+    if args.streaming:
+        # one gap batch per round, resident on the device (and pinned on the host for the end-to-end leg)
+        for r in range(max(args.steps, args.warmup, args.e2e_steps)):
+            gr = wl.make_gaps(my_spec, r)
+            round_gaps_dev.append(_to_device(gr, device))
+            if r < args.e2e_steps:
+                keep, pin = _pinned(gr.view(np.uint8))
+                pinned_keep[f"gaps{r}"] = keep
+                round_gaps_pinned.append(pin.view(wl.GAP_DTYPE))
+        torch.cuda.synchronize()
+
+    def load_device():
+        ctx.load_profiles(dev["off"], dev["d"], dev["m"], dev["s"], dev["ready"],
+                          wait_ms=dev.get("wait"), prio=dev.get("prio"))
+        if args.window_options:
+            ctx.set_window_options(True, dev_deadline)
+
+    def round_device(r):
+        ctx.advertise(round_gaps_dev[r])
+        ctx.select(my_spec.policy, flags=args.flags)
+        ctx.commit(want_count=False)
+        launches[0] += KERNELS_PER_STEP - 5       # no load: the five load kernels do not run
+
+    def round_e2e(r):
+        ctx.advertise(round_gaps_pinned[r])
+        aw = ctx.select(my_spec.policy, flags=args.flags, out="host")
+        return aw, ctx.commit(want_count=True)
 
     def step_device():
         ctx.load_profiles(dev["off"], dev["d"], dev["m"], dev["s"], dev["ready"],
@@ -353,8 +386,14 @@ def main():
         torch.cuda.synchronize()
 
     with torch.cuda.stream(stream):
-        for _ in range(args.warmup):
-            step_device()
+        if args.streaming:
+            load_device()
+            for r in range(args.warmup):
+                round_device(r)
+            load_device()                      # back to the state before round 0 (untimed)
+        else:
+            for _ in range(args.warmup):
+                step_device()
         n_rows = ctx.scan_size()
         ctx.profile_enable(True)
         sampler = ClockSampler(local_rank)
@@ -365,8 +404,11 @@ def main():
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         launches[0] = 0
-        for _ in range(args.steps):
-            step_device()
+        for r in range(args.steps):
+            if args.streaming:
+                round_device(r)
+            else:
+                step_device()
         e1.record(stream)
         timed_launches = launches[0]
         barrier()
@@ -378,7 +420,15 @@ def main():
 
         # end to end: pinned host inputs in, awards + grant count out, every step
         e2e_s = 0.0
-        if args.e2e_steps > 0:
+        if args.e2e_steps > 0 and args.streaming:
+            load_device()
+            barrier()
+            t0 = time.perf_counter()
+            for r in range(args.e2e_steps):
+                aw, n_granted = round_e2e(r)
+            torch.cuda.synchronize()
+            e2e_s = time.perf_counter() - t0
+        elif args.e2e_steps > 0:
             step_e2e()
             barrier()
             t0 = time.perf_counter()
@@ -392,10 +442,14 @@ def main():
     value = replicas.throughput(total_pairs, args.steps, ms_total)
     e2e_value = replicas.throughput(total_pairs, args.e2e_steps, e2e_ms) if e2e_ms > 0 else None
     h2d = sum(int(a.nbytes) for a in host_arrays.values()) + int(gaps.nbytes) + (4 * J if args.window_options else 0)
+    if args.streaming:
+        h2d = int(gaps.nbytes)                 # a round moves only its gap batch to the device
     d2h = 24 * G + 4
 
     peak, peak_kind = measured_peak()
-    scan_ms = timing["scan_ms"] / max(1, timing["scan_launches"])
+    if args.streaming:
+        timing["scan_launches"] = 0            # the scan ran before the timed region
+    scan_ms = timing["scan_ms"] / max(1, timing["scan_launches"]) if timing["scan_launches"] else 0.0
     scan_bytes = prof.raw_bytes() + 24 * n_rows
     achieved = scan_bytes / (scan_ms * 1e-3) / 1e9 if scan_ms > 0 else 0.0
     roofline = {
@@ -403,6 +457,8 @@ def main():
         "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": scan_traffic(N),
         "bytes_per_launch": scan_bytes, "ms_per_launch": scan_ms,
     }
+    if args.streaming:
+        roofline = None                        # no scan in the timed region; the rounds are bound by instruction issue
     breakdown = {k: timing[k] / args.steps for k in ("scan_ms", "prep_ms", "advertise_ms", "select_ms", "commit_ms")}
     select_ms = breakdown["select_ms"]
 
@@ -415,7 +471,8 @@ def main():
                    "l2": "inputs larger than L2 (profile arrays re-read from HBM every step)"
                    if prof.raw_bytes() > 200e6 else "inputs smaller than L2",
                    "flags": args.flags, "reauction": bool(args.reauction),
-                   "window_options": bool(args.window_options)},
+                   "window_options": bool(args.window_options),
+                   "streaming": "load once, one advertise/select/commit round per step" if args.streaming else False},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / max(1, args.e2e_steps), "steps": args.e2e_steps},
