@@ -685,7 +685,9 @@ sja_status sja_advertise(sja_ctx* c, uint32_t G, const sja_gap* gaps, sja_memspa
     DeviceGuard guard(c->device);
     TRY(reserve(c, c->gaps, (size_t)G * sizeof(sja_gap)));
     TRY(reserve(c, c->sgaps, (size_t)G * sizeof(sja_gap)));
-    TRY(reserve(c, c->gap_rank, (size_t)G * 8));
+    // u32 rank[G] (rounded up to 16 bytes), then u64 tile_key and u32 tile_idx, both padded to whole sort tiles
+    const size_t rank_bytes = (((size_t)G * 4 + 15) / 16) * 16;
+    TRY(reserve(c, c->gap_rank, rank_bytes + (size_t)((G + SORT_TILE - 1) / SORT_TILE) * SORT_TILE * 12));
     TRY(reserve(c, c->awards, (size_t)G * sizeof(sja_award)));
     TRY(reserve(c, c->widx, (size_t)G * 4));
     TRY(reserve(c, c->winners, (size_t)G * 4));
@@ -694,19 +696,22 @@ sja_status sja_advertise(sja_ctx* c, uint32_t G, const sja_gap* gaps, sja_memspa
         ProfScope ps(c, CAT_ADVERTISE);
         TRY(copy_in(c, c->gaps.p, gaps, (size_t)G * sizeof(sja_gap), where));
         if (sortable) {
-            // rank[G] and not_leader[G] share one buffer; both and the class counter start at zero
+            // sorted tiles live behind the ranks in one buffer; the sort kernel clears the ranks and the class counter
+            const uint32_t n_tiles = (G + SORT_TILE - 1) / SORT_TILE;
             uint32_t* rank = c->gap_rank.as<uint32_t>();
-            CU(cudaMemsetAsync(rank, 0, (size_t)G * 8, c->stream));
-            CU(cudaMemsetAsync(c->gap_info.p, 0, sizeof(GapInfo), c->stream));
-            const uint32_t i_blocks = (G + RANK_THREADS - 1) / RANK_THREADS;
-            uint32_t slices = (uint32_t)((16ull * c->n_sm + i_blocks - 1) / i_blocks);   // enough CTAs to fill the GPU
-            slices = std::max(1u, std::min(slices, (G + 63u) / 64u));
-            const uint32_t slice_len = (G + slices - 1) / slices;
-            slices = (G + slice_len - 1) / slice_len;
-            rank_gaps_kernel<<<dim3(i_blocks, slices), RANK_THREADS, 0, c->stream>>>(c->gaps.as<Gap>(), G, slice_len,
-                                                                                      rank, rank + G);
-            place_gaps_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(c->gaps.as<Gap>(), G, rank, rank + G,
-                                                                      c->sgaps.as<Gap>(), c->gap_info.as<GapInfo>());
+            uint64_t* tile_key = reinterpret_cast<uint64_t*>(c->gap_rank.as<unsigned char>() + rank_bytes);
+            uint32_t* tile_idx = reinterpret_cast<uint32_t*>(tile_key + (size_t)n_tiles * SORT_TILE);
+            const bool one_tile = n_tiles == 1;
+            sort_gap_tiles_kernel<<<n_tiles, SORT_TILE, 0, c->stream>>>(c->gaps.as<Gap>(), G, tile_key, tile_idx, rank,
+                                                                        c->gap_info.as<GapInfo>(),
+                                                                        one_tile ? c->sgaps.as<Gap>() : nullptr);
+            if (!one_tile) {
+                rank_gap_tiles_kernel<<<dim3(n_tiles, n_tiles), SORT_TILE, 0, c->stream>>>(tile_key, tile_idx, rank);
+                place_gaps_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(c->gaps.as<Gap>(), G, rank,
+                                                                          c->sgaps.as<Gap>());
+                count_classes_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(c->sgaps.as<Gap>(), G,
+                                                                            c->gap_info.as<GapInfo>());
+            }
             CU(cudaMemcpyAsync(c->h_words + 4, c->gap_info.p, sizeof(GapInfo), cudaMemcpyDeviceToHost, c->stream));
         } else {
             copy_gaps_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(c->gaps.as<Gap>(), G, c->sgaps.as<Gap>());

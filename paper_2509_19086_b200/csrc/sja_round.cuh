@@ -273,65 +273,112 @@ __global__ void __launch_bounds__(256) commit_refresh_kernel(
 namespace sja {
 
 // ---------------------------------------------------------------------------------------
-// Advertise: order the gaps by (capacity, window length).  Gaps of one capacity form a
-// "class" (the finite capacity set of Section 3.9); inside a class T ascends, so every job's
-// answer moves monotonically along its boundary rows and the select kernel can merge
-// instead of search.  The order is found by ranking: gap i goes to position
-// #{j : (C_j, T_j, j) < (C_i, T_i, i)}.  That is G^2 comparisons, but they are independent
-// (no barriers, no passes): thread (i, slice) counts over one slice of j held in shared
-// memory and adds its partial rank with one atomic; for the batch sizes of a scheduling
-// round (thousands of gaps) this takes a few microseconds.  The same sweep marks every gap
-// that has a predecessor of equal capacity, so the unmarked ones count the classes.
+// Advertise: order the gaps by (capacity, window length, index).  Gaps of one capacity form
+// a "class" (the finite capacity set of Section 3.9); inside a class T ascends, so every
+// job's answer moves monotonically along its boundary rows and the select kernels can walk
+// instead of search.  The order is found by ranking against sorted tiles:
+//   1. sort_gap_tiles_kernel: every CTA sorts one tile of 1024 keys in shared memory
+//      (bitonic network; key = capacity:T, ties by index);
+//   2. rank_gap_tiles_kernel: CTA (q, t) holds sorted tile t in shared memory and adds, for
+//      each key of tile q, the number of smaller keys in tile t (a 10-probe binary search)
+//      to that gap's rank -- G * G/1024 searches instead of G * G comparisons, no pass
+//      waits on another;
+//   3. place_gaps_kernel writes gap i to position rank[i];
+//   4. count_classes_kernel counts the positions whose predecessor has another capacity.
 constexpr uint32_t SORT_MAX_GAPS = 65536;
-constexpr int RANK_THREADS = 128;
-constexpr int RANK_TILE = 1024;   // keys per shared-memory tile
+constexpr int SORT_TILE = 1024;
 
 struct GapInfo { uint32_t n_classes; uint32_t pad[3]; };
 
-__global__ void __launch_bounds__(RANK_THREADS) rank_gaps_kernel(const Gap* __restrict__ gaps, uint32_t G,
-                                                                 uint32_t slice_len, uint32_t* __restrict__ rank,
-                                                                 uint32_t* __restrict__ not_leader) {
-    __shared__ uint64_t skey[RANK_TILE];
-    const uint32_t i = blockIdx.x * RANK_THREADS + threadIdx.x;
-    uint64_t ki = 0;
-    if (i < G) { const Gap g = gaps[i]; ki = ((uint64_t)g.C << 32) | g.T; }
-    const uint32_t j_begin = blockIdx.y * slice_len;
-    const uint32_t j_end = min(G, j_begin + slice_len);
-    uint32_t cnt = 0, same = 0;
-    for (uint32_t t0 = j_begin; t0 < j_end; t0 += RANK_TILE) {
-        const uint32_t tn = min((uint32_t)RANK_TILE, j_end - t0);
-        __syncthreads();
-        for (uint32_t q = threadIdx.x; q < tn; q += RANK_THREADS) {
-            const Gap g = gaps[t0 + q];
-            skey[q] = ((uint64_t)g.C << 32) | g.T;
-        }
-        __syncthreads();
-        for (uint32_t q = 0; q < tn; ++q) {
-            const uint64_t kj = skey[q];
-            const bool less = kj < ki || (kj == ki && t0 + q < i);
-            cnt += less ? 1u : 0u;
-            same |= (less && (uint32_t)(kj >> 32) == (uint32_t)(ki >> 32)) ? 1u : 0u;
+__device__ __forceinline__ bool gap_key_less(uint64_t ka, uint32_t ia, uint64_t kb, uint32_t ib) {
+    return ka < kb || (ka == kb && ia < ib);
+}
+
+// With `sorted_out` set (a batch of one tile) the kernel finishes the job alone: it writes the ordered gaps and
+// the class count.  Otherwise it stores the sorted tile for the ranking pass and clears the ranks and the counter.
+__global__ void __launch_bounds__(SORT_TILE) sort_gap_tiles_kernel(const Gap* __restrict__ gaps, uint32_t G,
+                                                                   uint64_t* __restrict__ tile_key,
+                                                                   uint32_t* __restrict__ tile_idx,
+                                                                   uint32_t* __restrict__ rank, GapInfo* __restrict__ info,
+                                                                   Gap* __restrict__ sorted_out) {
+    __shared__ uint64_t sk[SORT_TILE];
+    __shared__ uint32_t si[SORT_TILE];
+    const uint32_t t = threadIdx.x;
+    const uint32_t i = blockIdx.x * SORT_TILE + t;
+    uint64_t k = ~0ull;          // padding sorts last and is never smaller than a real key
+    uint32_t x = 0xFFFFFFFFu;
+    if (i < G) { const Gap g = gaps[i]; k = ((uint64_t)g.C << 32) | g.T; x = i; }
+    sk[t] = k; si[t] = x;
+    if (i == 0) info->n_classes = 0;
+    __syncthreads();
+    for (uint32_t size = 2; size <= SORT_TILE; size <<= 1) {
+        for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
+            const uint32_t p = t ^ stride;
+            if (p > t) {
+                const uint64_t ka = sk[t], kb = sk[p];
+                const uint32_t ia = si[t], ib = si[p];
+                const bool ascending = (t & size) == 0;
+                if (gap_key_less(kb, ib, ka, ia) == ascending) { sk[t] = kb; si[t] = ib; sk[p] = ka; si[p] = ia; }
+            }
+            __syncthreads();
         }
     }
-    if (i < G) {
-        if (cnt) atomicAdd(rank + i, cnt);
-        if (same) atomicOr(not_leader + i, 1u);
+    if (sorted_out) {            // one tile: position t is final
+        const uint32_t src = si[t];
+        const bool real = src != 0xFFFFFFFFu;
+        if (real) {
+            const Gap g = gaps[src];
+            Gap o;
+            o.slice = src;       // the original position travels in the slice field
+            o.start = g.start; o.T = g.T; o.C = g.C;
+            sorted_out[t] = o;
+        }
+        const bool leader = real && (t == 0 || (uint32_t)(sk[t - 1] >> 32) != (uint32_t)(sk[t] >> 32));
+        const uint32_t n = __syncthreads_count(leader);
+        if (t == 0) info->n_classes = n;
+        return;
     }
+    tile_key[i] = sk[t];         // the arrays are padded to whole tiles
+    tile_idx[i] = si[t];
+    if (i < G) rank[i] = 0;
+}
+
+__global__ void __launch_bounds__(SORT_TILE) rank_gap_tiles_kernel(const uint64_t* __restrict__ tile_key,
+                                                                   const uint32_t* __restrict__ tile_idx,
+                                                                   uint32_t* __restrict__ rank) {
+    __shared__ uint64_t sk[SORT_TILE];
+    __shared__ uint32_t si[SORT_TILE];
+    const uint32_t t = threadIdx.x;
+    sk[t] = tile_key[blockIdx.y * SORT_TILE + t];
+    si[t] = tile_idx[blockIdx.y * SORT_TILE + t];
+    const uint64_t k = tile_key[blockIdx.x * SORT_TILE + t];
+    const uint32_t x = tile_idx[blockIdx.x * SORT_TILE + t];
+    __syncthreads();
+    if (x == 0xFFFFFFFFu) return;   // padding
+    uint32_t pos = 0;               // number of keys of tile blockIdx.y below (k, x)
+#pragma unroll
+    for (uint32_t s = SORT_TILE / 2; s > 0; s >>= 1) {
+        if (gap_key_less(sk[pos + s - 1], si[pos + s - 1], k, x)) pos += s;
+    }
+    if (gap_key_less(sk[pos], si[pos], k, x)) pos += 1;
+    if (pos) atomicAdd(rank + x, pos);
 }
 
 __global__ void __launch_bounds__(256) place_gaps_kernel(const Gap* __restrict__ gaps, uint32_t G,
-                                                         const uint32_t* __restrict__ rank,
-                                                         const uint32_t* __restrict__ not_leader,
-                                                         Gap* __restrict__ sorted, GapInfo* __restrict__ info) {
+                                                         const uint32_t* __restrict__ rank, Gap* __restrict__ sorted) {
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    const bool leader = i < G && not_leader[i] == 0u;
-    if (i < G) {
-        const Gap g = gaps[i];
-        Gap o;
-        o.slice = i;   // the original position travels in the slice field
-        o.start = g.start; o.T = g.T; o.C = g.C;
-        sorted[rank[i]] = o;
-    }
+    if (i >= G) return;
+    const Gap g = gaps[i];
+    Gap o;
+    o.slice = i;   // the original position travels in the slice field
+    o.start = g.start; o.T = g.T; o.C = g.C;
+    sorted[rank[i]] = o;
+}
+
+__global__ void __launch_bounds__(256) count_classes_kernel(const Gap* __restrict__ sorted, uint32_t G,
+                                                            GapInfo* __restrict__ info) {
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool leader = i < G && (i == 0 || sorted[i - 1].C != sorted[i].C);
     const uint32_t n = __popc(__ballot_sync(0xFFFFFFFFu, leader));
     if ((threadIdx.x & 31u) == 0 && n) atomicAdd(&info->n_classes, n);
 }
