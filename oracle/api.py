@@ -51,7 +51,8 @@ def _load():
     lib.orc_pair.restype = ctypes.c_int
     lib.orc_pair.argtypes = [vp, vp, vp, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint32,
                              ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
-                             ctypes.c_uint32, ctypes.c_uint32, ctypes.c_int, ctypes.c_uint32, u32p, u32p, u64p]
+                             ctypes.c_uint32, ctypes.c_uint32, ctypes.c_int, ctypes.c_uint32, u32p, u32p, u64p,
+                             u32p]
     lib.orc_select.restype = ctypes.c_int
     lib.orc_select.argtypes = [ctypes.c_uint32, vp, vp, vp, vp, vp, vp, vp, vp,
                                ctypes.c_uint32, vp, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
@@ -84,20 +85,24 @@ U32MAX = 0xFFFFFFFF
 
 
 def pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: int,
-         tau_min_ms: int = 0, tau_max_ms: int = U32MAX, late_start: bool = False, deadline_ms: int = U32MAX):
+         tau_min_ms: int = 0, tau_max_ms: int = U32MAX, late_start: bool = False, deadline_ms: int = U32MAX,
+         want_peak: bool = False):
     """R1-R3 (with the duration thresholds of R2' and the window options of R1'') for one (gap, job)
-    pair: ``None`` for decline, else ``(k, dur, work)``."""
+    pair: ``None`` for decline, else ``(k, dur, work)`` (``(k, dur, work, peak)`` with ``want_peak``)."""
     lib = _load()
     k = ctypes.c_uint32()
     dur = ctypes.c_uint32()
     work = ctypes.c_uint64()
+    peak = ctypes.c_uint32()
     ok = lib.orc_pair(prof.dur_ms.ctypes.data, prof.mem_MiB.ctypes.data,
                       prof.safe_bits.ctypes.data, int(prof.off[j]), int(prof.off[j + 1]),
                       int(p), int(ready_ms), int(start_ms), int(T_ms), int(C_MiB),
                       int(tau_min_ms), int(tau_max_ms), int(bool(late_start)), int(deadline_ms),
-                      ctypes.byref(k), ctypes.byref(dur), ctypes.byref(work))
+                      ctypes.byref(k), ctypes.byref(dur), ctypes.byref(work), ctypes.byref(peak))
     if not ok:
         return None
+    if want_peak:
+        return int(k.value), int(dur.value), int(work.value), int(peak.value)
     return int(k.value), int(dur.value), int(work.value)
 
 

@@ -72,6 +72,9 @@ def brute_select(prof, progress, ready_ms, gaps, policy: int):
                 score = (work * (1 + int(prof.wait_ms[j]) // 1000)) & _MASK64
             elif policy == 2:
                 cls = int(prof.prio[j])
+            elif policy == 3:
+                s0 = int(prof.off[j])
+                score = max(int(x) for x in prof.mem_MiB[s0 + int(progress[j]):s0 + k])   # peak of the subjob
             # larger class, then larger score, then smaller job id
             entries.append((-cls, -score, j, k, dur, score))
         if not entries:

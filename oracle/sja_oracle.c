@@ -29,7 +29,10 @@
  *                    longest one, k* = max candidates; dur = sum d, work = sum d*m (u64).
  *   R4 score       : efficiency  work;
  *                    fairness    work * (1 + wait_j/1000), truncating division, u64;
- *                    SLA         lexicographic (prio_j, work), larger prio = more urgent.
+ *                    SLA         lexicographic (prio_j, work), larger prio = more urgent;
+ *                    tight fit   peak = max m over the subjob: the job that leaves the least slack
+ *                                C_g - peak on the slice wins (the slack-minimising principle of
+ *                                Section 3.9, applied by the scheduler across jobs).
  *   R5 select      : per gap, the interested job with the largest key; ties go to the
  *                    lowest job id; no interested job -> SJA_NO_JOB and zeros.
  *   R2' bounds     : optional subjob duration thresholds (Section 4.3, item 5: minimum and maximum
@@ -76,7 +79,7 @@ typedef struct {
     uint64_t score;
 } orc_award;
 
-enum { ORC_EFFICIENCY = 0, ORC_FAIRNESS = 1, ORC_SLA = 2 };
+enum { ORC_EFFICIENCY = 0, ORC_FAIRNESS = 1, ORC_SLA = 2, ORC_TIGHT_FIT = 3 };
 
 static int step_is_safe(const uint32_t *safe_bits, uint64_t i)
 {
@@ -92,7 +95,7 @@ int orc_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *sa
              uint32_t start_ms, uint32_t T_ms, uint32_t C_MiB,
              uint32_t tau_min_ms, uint32_t tau_max_ms,
              int late_start, uint32_t deadline_ms,
-             uint32_t *k_out, uint32_t *dur_out, uint64_t *work_out)
+             uint32_t *k_out, uint32_t *dur_out, uint64_t *work_out, uint32_t *peak_out /* may be NULL */)
 {
     uint64_t len = e - s;
     if ((uint64_t)p >= len) return 0;            /* R1: finished job */
@@ -109,7 +112,7 @@ int orc_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *sa
     uint64_t acc = 0, work = 0;
     uint32_t peak = 0;
     int found = 0;
-    uint32_t best_k = 0, best_dur = 0;
+    uint32_t best_k = 0, best_dur = 0, best_peak = 0;
     uint64_t best_work = 0;
     for (uint64_t i = s + p; i < e; ++i) {
         acc += dur_ms[i];
@@ -124,17 +127,19 @@ int orc_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *sa
             best_k = (uint32_t)(i + 1 - s);
             best_dur = (uint32_t)acc;
             best_work = work;
+            best_peak = peak;
         }
     }
     if (!found) return 0;
     *k_out = best_k;
     *dur_out = best_dur;
     *work_out = best_work;
+    if (peak_out) *peak_out = best_peak;
     return 1;
 }
 
 /* R4: the policy key of an interested job, as (class, score). */
-static void policy_key(uint32_t policy, uint64_t work, uint32_t j,
+static void policy_key(uint32_t policy, uint64_t work, uint32_t peak, uint32_t j,
                        const uint32_t *wait_ms, const uint8_t *prio,
                        uint32_t *cls_out, uint64_t *score_out)
 {
@@ -144,6 +149,8 @@ static void policy_key(uint32_t policy, uint64_t work, uint32_t j,
         *score_out = work * (uint64_t)(1u + wait_ms[j] / 1000u);
     } else if (policy == ORC_SLA) {
         *cls_out = prio[j];
+    } else if (policy == ORC_TIGHT_FIT) {
+        *score_out = peak;      /* largest peak <=> least slack C_g - peak */
     }
 }
 
@@ -161,7 +168,7 @@ int orc_select(uint32_t n_jobs, const uint64_t *off,
                int late_start, const uint32_t *deadline_ms /* per job, or NULL = none */,
                orc_award *awards)
 {
-    if (policy > ORC_SLA) return -1;
+    if (policy > ORC_TIGHT_FIT) return -1;
     if (policy == ORC_FAIRNESS && !wait_ms) return -1;
     if (policy == ORC_SLA && !prio) return -1;
 
@@ -172,16 +179,16 @@ int orc_select(uint32_t n_jobs, const uint64_t *off,
         uint32_t best_cls = 0, best_job = ORC_NO_JOB, best_k = 0, best_dur = 0;
         uint64_t best_score = 0;
         for (uint32_t j = 0; j < n_jobs; ++j) {
-            uint32_t k, dur;
+            uint32_t k, dur, peak;
             uint64_t work;
             if (!orc_pair(dur_ms, mem_MiB, safe_bits, off[j], off[j + 1], progress[j],
                           ready_ms[j], gap.start_ms, gap.T_ms, gap.C_MiB, tau_min_ms, tau_max_ms,
                           late_start, deadline_ms ? deadline_ms[j] : 0xFFFFFFFFu,
-                          &k, &dur, &work))
+                          &k, &dur, &work, &peak))
                 continue;                                      /* decline */
             uint32_t cls;
             uint64_t score;
-            policy_key(policy, work, j, wait_ms, prio, &cls, &score);
+            policy_key(policy, work, peak, j, wait_ms, prio, &cls, &score);
             /* jobs are visited in ascending id, so a strict ">" keeps the lowest id on ties */
             if (!have || cls > best_cls || (cls == best_cls && score > best_score)) {
                 have = 1;

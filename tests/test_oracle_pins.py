@@ -60,7 +60,7 @@ def test_p1_random_tiny_select(oracle_mod):
         gaps = gaps_from_lists([(int(rng.integers(0, 7)), int(rng.integers(0, 8)),
                                  int(rng.integers(0, 40)), int(rng.integers(0, 22)))
                                 for _ in range(6)])
-        for policy in (0, 1, 2):
+        for policy in (0, 1, 2, 3):
             aw = oracle.select(prof, progress, prof.ready_ms, gaps, policy)
             ref = oracle.brute_select(prof, progress, prof.ready_ms, gaps, policy)
             for g in range(len(gaps)):
@@ -300,7 +300,7 @@ def test_p6_duplicate_job_and_permutations(oracle_mod):
     prof = profiles_from_lists(jobs_dup, wait=wait, prio=prio)
     gaps = gaps_from_lists([(0, 0, int(rng.integers(10, 300)), int(rng.integers(20, 110)))
                             for _ in range(30)])
-    for policy in (0, 1, 2):
+    for policy in (0, 1, 2, 3):
         aw = _select_all(oracle, prof, gaps, policy)
         assert not (aw["job"] == 12).any()            # the copy never beats the lower id
         # permuting the gaps permutes the awards
@@ -310,11 +310,39 @@ def test_p6_duplicate_job_and_permutations(oracle_mod):
     # reversing job order: same scores; winners differ only through ties
     rev = list(reversed(jobs_dup))
     prof_r = profiles_from_lists(rev, wait=wait[::-1], prio=prio[::-1])
-    for policy in (0, 1, 2):
+    for policy in (0, 1, 2, 3):
         a = _select_all(oracle, prof, gaps, policy)
         b = _select_all(oracle, prof_r, gaps, policy)
         assert (a["score"] == b["score"]).all()
         assert ((a["job"] == U32MAX) == (b["job"] == U32MAX)).all()
+
+
+def test_tight_fit_winner_leaves_the_least_slack(oracle_mod):
+    """Policy 3 (Section 3.9, slack-minimising): no interested job would leave less slack C - peak on the
+    slice than the winner, the winner's subjob is still its longest one, and the score is its peak."""
+    oracle = oracle_mod
+    rng = np.random.default_rng(88)
+    jobs = random_small_profiles(rng, 40, 30, p_safe=0.3, dmax=9, mmax=60)
+    prof = profiles_from_lists(jobs, ready=rng.integers(0, 5, 40))
+    gaps = gaps_from_lists([(0, int(rng.integers(0, 8)), int(rng.integers(5, 120)), int(rng.integers(5, 70)))
+                            for _ in range(40)])
+    z = np.zeros(40, np.uint32)
+    aw = oracle.select(prof, z, prof.ready_ms, gaps, 3)
+    won = 0
+    for g in range(len(gaps)):
+        start, T, C = int(gaps["start_ms"][g]), int(gaps["T_ms"][g]), int(gaps["C_MiB"][g])
+        pairs = [oracle.brute_pair(prof, j, 0, int(prof.ready_ms[j]), start, T, C) for j in range(40)]
+        peaks = [None if r is None else max(jobs[j][1][:r[0]]) for j, r in enumerate(pairs)]
+        interested = [j for j in range(40) if pairs[j] is not None]
+        if not interested:
+            assert int(aw["job"][g]) == U32MAX
+            continue
+        w = int(aw["job"][g])
+        won += 1
+        assert w in interested and int(aw["end_step"][g]) == pairs[w][0] and int(aw["score"][g]) == peaks[w]
+        assert all(C - peaks[w] <= C - peaks[j] for j in interested)
+        assert all(peaks[j] < peaks[w] for j in interested if j < w)     # lowest id among the tightest
+    assert won > 20
 
 
 def test_ready_time_and_finished_jobs(oracle_mod):
