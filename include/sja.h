@@ -20,7 +20,8 @@
  *                max m[p_j..k) <= C_g (all bounds inclusive).  Its subjob is the longest
  *                such k; dur = sum d, work = sum d*m over [p_j, k).
  *   score        EFFICIENCY work; FAIRNESS work * (1 + wait_j/1000) (truncating division);
- *                SLA (prio_j, work) compared lexicographically, larger prio more urgent.
+ *                SLA (prio_j, work) compared lexicographically, larger prio more urgent;
+ *                TIGHT_FIT max m over [p_j, k).
  *   select       per gap the interested job with the largest score, ties to the lowest job id.
  *   commit       a job that won several gaps accepts the one with the largest k, ties to
  *                the lowest gap id; p_j = k, ready_j = start_g + dur.
@@ -74,7 +75,10 @@ typedef struct {
 typedef enum {
     SJA_POLICY_EFFICIENCY = 0, /* score = work */
     SJA_POLICY_FAIRNESS = 1,   /* score = work * (1 + wait_ms/1000); needs wait_ms at load */
-    SJA_POLICY_SLA = 2         /* key = (prio, work); needs prio at load; reported score = work */
+    SJA_POLICY_SLA = 2,        /* key = (prio, work); needs prio at load; reported score = work */
+    SJA_POLICY_TIGHT_FIT = 3   /* score = peak memory (MiB) of the subjob: the job that leaves the least slack
+                                  C - peak on the slice wins (slack-minimising principle of Section 3.9, applied
+                                  by the scheduler across jobs); ties to the lowest job id */
 } sja_policy_kind;
 
 /* sja_policy.flags.  By default select runs the tile-sweep kernel over the gaps ordered by

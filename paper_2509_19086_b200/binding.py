@@ -19,7 +19,7 @@ STATUS_NAMES = {
     4: "SJA_ERR_STATE", 5: "SJA_ERR_OOM", 6: "SJA_ERR_CUDA", 7: "SJA_ERR_TIMEOUT",
 }
 MEM_HOST, MEM_DEVICE = 0, 1
-POLICY_EFFICIENCY, POLICY_FAIRNESS, POLICY_SLA = 0, 1, 2
+POLICY_EFFICIENCY, POLICY_FAIRNESS, POLICY_SLA, POLICY_TIGHT_FIT = 0, 1, 2, 3
 FLAG_FORCE_SEARCH = 1
 FLAG_FORCE_MERGE = 2
 FLAG_FORCE_TILE = 4

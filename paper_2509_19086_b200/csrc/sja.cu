@@ -276,6 +276,8 @@ void launch_sorted_b(SelectKernel which, uint32_t kind, dim3 grid, cudaStream_t 
         launch_sorted_kb<1, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial);
     else if (kind == SJA_POLICY_SLA)
         launch_sorted_kb<2, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial);
+    else if (kind == SJA_POLICY_TIGHT_FIT)
+        launch_sorted_kb<3, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial);
     else
         launch_sorted_kb<0, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial);
 }
@@ -305,7 +307,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 sja_status check_policy(sja_ctx* c, const sja_policy* policy, const char* who) {
     if (!policy) return fail(c, SJA_ERR_INVALID_ARG, "%s: policy is NULL", who);
     const uint32_t kind = policy->kind;
-    if (kind > SJA_POLICY_SLA) return fail(c, SJA_ERR_INVALID_ARG, "%s: unknown policy %u", who, kind);
+    if (kind > SJA_POLICY_TIGHT_FIT) return fail(c, SJA_ERR_INVALID_ARG, "%s: unknown policy %u", who, kind);
     if (!c->loaded || !c->advertised) return fail(c, SJA_ERR_STATE, "%s before load / advertise", who);
     if (kind == SJA_POLICY_FAIRNESS && !c->have_wait)
         return fail(c, SJA_ERR_INVALID_ARG, "fairness policy needs wait_ms at load");
@@ -462,8 +464,9 @@ sja_status sja_create(sja_ctx** out, int device, void* cuda_stream) {
         if (cudaFuncSetAttribute(scan_profiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  SCAN_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         if (sorted_smem_attr<0, false>() != cudaSuccess || sorted_smem_attr<1, false>() != cudaSuccess ||
-            sorted_smem_attr<2, false>() != cudaSuccess || sorted_smem_attr<0, true>() != cudaSuccess ||
-            sorted_smem_attr<1, true>() != cudaSuccess || sorted_smem_attr<2, true>() != cudaSuccess) {
+            sorted_smem_attr<2, false>() != cudaSuccess || sorted_smem_attr<3, false>() != cudaSuccess ||
+            sorted_smem_attr<0, true>() != cudaSuccess || sorted_smem_attr<1, true>() != cudaSuccess ||
+            sorted_smem_attr<2, true>() != cudaSuccess || sorted_smem_attr<3, true>() != cudaSuccess) {
             st = SJA_ERR_CUDA;
             break;
         }

@@ -39,11 +39,17 @@ __device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {
 constexpr uint64_t KEY_SLA_SHIFT = 55;  // SLA key = 1 + (prio << 55) + work, work < 2^55
 
 // Policy key of an interested job: 0 is reserved for "no candidate".
-// kind 0 efficiency, 1 fairness (factor = 1 + wait/1000), 2 SLA (factor = prio).
-__device__ __forceinline__ uint64_t policy_key(uint32_t kind, uint64_t work, uint32_t factor) {
-    if (kind == 1) return work * (uint64_t)factor + 1ull;
-    if (kind == 2) return ((uint64_t)factor << KEY_SLA_SHIFT) + work + 1ull;
-    return work + 1ull;
+// kind 0 efficiency, 1 fairness (factor = 1 + wait/1000), 2 SLA (factor = prio): payload = work of the subjob;
+// kind 3 tight fit: payload = peak memory of the subjob (the running maximum of its last row).
+__device__ __forceinline__ uint64_t policy_key(uint32_t kind, uint64_t payload, uint32_t factor) {
+    if (kind == 1) return payload * (uint64_t)factor + 1ull;
+    if (kind == 2) return ((uint64_t)factor << KEY_SLA_SHIFT) + payload + 1ull;
+    return payload + 1ull;
+}
+
+// What policy_key wants from a boundary row {D, M, W_lo, W_hi}: the work above the progress point, or the peak.
+__device__ __forceinline__ uint64_t policy_payload(uint32_t kind, const uint4& row, uint64_t Wp) {
+    return kind == 3 ? (uint64_t)row.y : pack64(row.z, row.w) - Wp;
 }
 
 __device__ __forceinline__ uint64_t key_to_score(uint32_t kind, uint64_t key) {

@@ -110,7 +110,7 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
                 cnt = lo;
                 if (cnt) {
                     const uint4 r = __ldg(jv.A + base + cnt - 1);
-                    if (r.x - Dp >= jv.tau_min) key = policy_key(kind, pack64(r.z, r.w) - Wp, factor);
+                    if (r.x - Dp >= jv.tau_min) key = policy_key(kind, policy_payload(kind, r, Wp), factor);
                     else cnt = 0;   // the longest fitting subjob is shorter than the minimum: decline
                 }
             }
@@ -572,7 +572,7 @@ __global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_me
                 thr[r] = 0xFFFFFFFFu;
                 if (n[r]) {
                     const uint4 row = mg_lds128(ring_s[r]);
-                    nextW[r] = pack64(row.z, row.w);
+                    nextW[r] = policy_payload(KIND, row, Wp[r]);
                     if (row.y <= C) { open |= 1u << r; thr[r] = row.x - Dp[r]; }
                 }
             }
@@ -587,7 +587,7 @@ __global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_me
                 while (((open >> r) & 1u) && T >= thr[r]) {
                     // row w qualifies: it becomes the candidate; fetch row w + 1 from the ring
                     // (a subjob shorter than the minimum duration is no candidate; longer rows may be)
-                    curKey[r] = (!BOUNDED || thr[r] >= jv.tau_min) ? policy_key(KIND, nextW[r] - Wp[r], factor[r]) : 0ull;
+                    curKey[r] = (!BOUNDED || thr[r] >= jv.tau_min) ? policy_key(KIND, nextW[r], factor[r]) : 0ull;
                     if (w[r] + MERGE_RING < n[r])
                         mg_cp_async16(ring_s[r] + (w[r] & (MERGE_RING - 1)) * 32 * 16, next_row[r]);
                     mg_commit();
@@ -598,7 +598,7 @@ __global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_me
                     if (w[r] < n[r]) {
                         mg_wait<MERGE_RING - 1>();
                         const uint4 row = mg_lds128(ring_s[r] + (w[r] & (MERGE_RING - 1)) * 32 * 16);
-                        nextW[r] = pack64(row.z, row.w);
+                        nextW[r] = policy_payload(KIND, row, Wp[r]);
                         if (row.y <= C) { open |= 1u << r; thr[r] = row.x - Dp[r]; }
                     }
                 }

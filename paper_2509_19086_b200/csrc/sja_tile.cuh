@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
 
     // One cursor step of this lane: row w becomes the job's candidate, row w + 1 is fetched.
     auto step_cursor = [&](uint32_t C) {
-        curKey = (!BOUNDED || thr >= jv.tau_min) ? policy_key(KIND, nextW - Wp, factor) : 0ull;
+        curKey = (!BOUNDED || thr >= jv.tau_min) ? policy_key(KIND, nextW, factor) : 0ull;
         if (w + TILE_RING < n) mg_cp_async16(ring_s + (w & (TILE_RING - 1)) * 512, next_row);
         mg_commit();
         ++next_row;
@@ -137,7 +137,7 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
         if (w < n) {
             mg_wait<TILE_RING - 1>();
             const uint4 row = mg_lds128(ring_s + (w & (TILE_RING - 1)) * 512);
-            nextW = pack64(row.z, row.w);
+            nextW = policy_payload(KIND, row, Wp);
             if (row.y <= C) { open = true; thr = row.x - Dp; }
         }
     };
@@ -189,7 +189,7 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
                     w = 0; curKey = 0; open = false; thr = 0xFFFFFFFFu;
                     if (n) {
                         const uint4 row = mg_lds128(ring_s);
-                        nextW = pack64(row.z, row.w);
+                        nextW = policy_payload(KIND, row, Wp);
                         if (row.y <= Cc) { open = true; thr = row.x - Dp; }
                     }
                     dirty = true;

@@ -107,7 +107,7 @@ def test_scan_cfg1_sampled_jobs(sja_mod, oracle_mod):
 
 # ------------------------------------------------------------------ select (a2-a5)
 @pytest.mark.parametrize("flags", [0, 1, 2, 4])
-@pytest.mark.parametrize("policy", [0, 1, 2])
+@pytest.mark.parametrize("policy", [0, 1, 2, 3])
 def test_select_tiny_random_vs_oracle(sja_mod, oracle_mod, policy, flags):
     rng = np.random.default_rng(200 + policy)
     with sja_mod.Sja() as ctx:
@@ -187,7 +187,7 @@ def test_select_long_windows_and_many_capacity_classes(sja_mod, oracle_mod):
             _assert_awards_equal(got, want)
 
 
-@pytest.mark.parametrize("policy", [0, 1, 2])
+@pytest.mark.parametrize("policy", [0, 1, 2, 3])
 def test_select_ties_duplicate_jobs_and_ready_boundaries(sja_mod, oracle_mod, policy):
     """Many exact ties (copies of the same profile), zero-work segments (a longer subjob with the
     same score), few distinct ready times met exactly by the gap starts, repeated T values, and
@@ -215,6 +215,27 @@ def test_select_ties_duplicate_jobs_and_ready_boundaries(sja_mod, oracle_mod, po
             oracle_mod.commit(progress, prof.ready_ms, gaps, want)
             p, r = ctx.get_state()
             assert np.array_equal(p, progress) and np.array_equal(r, prof.ready_ms)
+
+
+def test_tight_fit_policy_committed_rounds_all_kernels(sja_mod, oracle_mod):
+    """Policy 3 (least slack on the slice) at a size where the tile kernel is the default: awards of every
+    kernel, grants and job state over committed rounds.  Many jobs share a peak, so ties are frequent."""
+    spec = wl.scaled(wl.SPECS[4], n_jobs=3000, fixed_len=700, n_gaps=384)
+    prof = wl.make_profiles(spec, threads=2)
+    progress = np.zeros(prof.n_jobs, np.uint32)
+    ready = prof.ready_ms.copy()
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof)
+        for rnd in range(5):
+            gaps = wl.make_gaps(spec, rnd)
+            ctx.advertise(gaps)
+            want = oracle_mod.select(prof, progress, ready, gaps, 3)
+            assert (want["job"] != U32MAX).mean() > 0.5
+            for flags in (0, 1, 2, 4):
+                _assert_awards_equal(ctx.select(3, flags=flags, out="host"), want)
+            assert ctx.commit() == oracle_mod.commit(progress, ready, gaps, want)
+            p, r = ctx.get_state()
+            assert np.array_equal(p, progress) and np.array_equal(r, ready)
 
 
 # ------------------------------------------------------------------ commit (a6), multi-round

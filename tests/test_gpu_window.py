@@ -22,7 +22,7 @@ def _same(got, want, fields=FIELDS):
         assert bad.size == 0, (f, bad[:5], got[bad[:5]], want[bad[:5]])
 
 
-@pytest.mark.parametrize("policy", [0, 1, 2])
+@pytest.mark.parametrize("policy", [0, 1, 2, 3])
 def test_window_options_tiny_random(oracle_mod, policy):
     from paper_2509_19086_b200 import binding
     rng = np.random.default_rng(900 + policy)
