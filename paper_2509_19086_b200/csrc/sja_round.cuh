@@ -40,14 +40,21 @@ __device__ __forceinline__ uint32_t policy_factor(const JobView& jv, uint32_t ki
 // is searched on its own, this is also the kernel for the window options, where the usable
 // window differs from pair to pair: with a late start the subjob begins at
 // max(start, ready) and only the rest of the window counts; with a deadline it must be over
-// by then.
+// by then.  The first SEARCH_ROWS rows of every job are staged in shared memory once per CTA
+// (most windows end inside them), so the usual pair is a five-probe search in shared memory;
+// only longer answers continue in global memory.
 constexpr int SEARCH_THREADS = 256;
 constexpr int SEARCH_GT = 64;   // gaps per staging tile
+constexpr int SEARCH_ROWS = 16; // boundary rows staged per job
+constexpr int SEARCH_SMEM_BYTES = 2 * SEARCH_ROWS * SEARCH_THREADS * 8;   // {D - Dp, M} and payload, [row][thread]
 
 __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
     JobView jv, const Gap* __restrict__ gaps, uint32_t G, uint32_t gaps_per_split, uint32_t kind,
     const uint32_t* __restrict__ job_list, uint32_t n_list, Partial* __restrict__ partial_out) {
     __shared__ Partial stage[SEARCH_GT][SEARCH_THREADS / 32];
+    extern __shared__ __align__(16) uint2 search_rows[];
+    uint2* sDM = search_rows + threadIdx.x;                                     // row r of this thread: sDM[r * THREADS]
+    uint2* sPay = search_rows + SEARCH_ROWS * SEARCH_THREADS + threadIdx.x;     // its policy payload (work or peak)
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
     const uint32_t slot = blockIdx.x * SEARCH_THREADS + threadIdx.x;
     // the jobs of this launch: either all jobs (job_list == nullptr) or a list of job ids
@@ -72,6 +79,14 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
     const bool late = jv.late_start != 0u;
     const uint32_t g_begin = blockIdx.y * gaps_per_split;
     const uint32_t g_end = min(G, g_begin + gaps_per_split);
+    const uint32_t ns = min(n, (uint32_t)SEARCH_ROWS);   // rows of this job held in shared memory
+    for (uint32_t r = 0; r < ns; ++r) {
+        const uint4 row = __ldg(jv.A + base + r);
+        const uint64_t pay = policy_payload(kind, row, Wp);
+        sDM[r * SEARCH_THREADS] = make_uint2(row.x - Dp, row.y);
+        sPay[r * SEARCH_THREADS] = make_uint2((uint32_t)pay, (uint32_t)(pay >> 32));
+    }
+    // (each thread reads back only what it wrote: no barrier needed)
 
     for (uint32_t g0 = g_begin; g0 < g_end; g0 += SEARCH_GT) {
         const uint32_t gt = min((uint32_t)SEARCH_GT, g_end - g0);
@@ -95,22 +110,43 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
             uint32_t cnt = 0;
             uint64_t key = 0;
             if (eligible) {
-                uint32_t lo = 0, hi = n, idx = 0;
-                for (;;) {   // gallop over rows 0, 1, 3, 7, ...
-                    if (idx >= n) { hi = n; break; }
-                    const uint4 r = __ldg(jv.A + base + idx);
-                    if (r.x - Dp <= T && r.y <= C) { lo = idx + 1; idx = idx * 2 + 1; }
-                    else { hi = idx; break; }
-                }
+                // the staged rows first
+                uint32_t lo = 0, hi = ns;
                 while (lo < hi) {
-                    const uint32_t mid = lo + ((hi - lo) >> 1);
-                    const uint4 r = __ldg(jv.A + base + mid);
-                    if (r.x - Dp <= T && r.y <= C) lo = mid + 1; else hi = mid;
+                    const uint32_t mid = (lo + hi) >> 1;
+                    const uint2 r = sDM[mid * SEARCH_THREADS];
+                    if (r.x <= T && r.y <= C) lo = mid + 1; else hi = mid;
+                }
+                if (lo == ns && ns < n) {
+                    // every staged row fits: gallop on through global memory (rows ns, ns + 1, ns + 3, ...)
+                    hi = n;
+                    uint32_t step = 1;
+                    for (uint32_t idx = ns;;) {
+                        if (idx >= n) { hi = n; break; }
+                        const uint4 r = __ldg(jv.A + base + idx);
+                        if (r.x - Dp <= T && r.y <= C) { lo = idx + 1; idx += step; step <<= 1; }
+                        else { hi = idx; break; }
+                    }
+                    while (lo < hi) {
+                        const uint32_t mid = lo + ((hi - lo) >> 1);
+                        const uint4 r = __ldg(jv.A + base + mid);
+                        if (r.x - Dp <= T && r.y <= C) lo = mid + 1; else hi = mid;
+                    }
                 }
                 cnt = lo;
                 if (cnt) {
-                    const uint4 r = __ldg(jv.A + base + cnt - 1);
-                    if (r.x - Dp >= jv.tau_min) key = policy_key(kind, policy_payload(kind, r, Wp), factor);
+                    uint32_t dur;
+                    uint64_t pay;
+                    if (cnt <= ns) {
+                        dur = sDM[(cnt - 1) * SEARCH_THREADS].x;
+                        const uint2 pw = sPay[(cnt - 1) * SEARCH_THREADS];
+                        pay = pack64(pw.x, pw.y);
+                    } else {
+                        const uint4 r = __ldg(jv.A + base + cnt - 1);
+                        dur = r.x - Dp;
+                        pay = policy_payload(kind, r, Wp);
+                    }
+                    if (dur >= jv.tau_min) key = policy_key(kind, pay, factor);
                     else cnt = 0;   // the longest fitting subjob is shorter than the minimum: decline
                 }
             }
