@@ -281,7 +281,8 @@ sja_status sja_scan_size(sja_ctx* ctx, uint64_t* n_boundaries);
 sja_status sja_get_scan(sja_ctx* ctx, uint64_t* boff, uint32_t* k, uint32_t* D, uint32_t* M,
                         uint32_t* S, uint64_t* W, sja_memspace where);
 
-/* Switch per-kernel CUDA-event timing on (1) or off (0); resets the counters. */
+/* Per-kernel CUDA-event timing: 0 off, 1 every phase, 2 the scan kernel only (two event records per load
+ * instead of about fourteen per round, for timing a whole step with little disturbance).  Resets the counters. */
 sja_status sja_profile_enable(sja_ctx* ctx, int on);
 
 /* Wait for the stream and read the accumulated kernel times. */

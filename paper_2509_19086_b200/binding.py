@@ -283,8 +283,9 @@ class Sja:
         return dict(boff=boff, k=k, D=D, M=M, S=S, W=W)
 
     # -- profiling
-    def profile_enable(self, on: bool = True) -> None:
-        self._check(self._lib.sja_profile_enable(self._h, 1 if on else 0))
+    def profile_enable(self, on=True) -> None:
+        """``on``: False / 0 off, True / 1 every phase, 2 the scan kernel only."""
+        self._check(self._lib.sja_profile_enable(self._h, int(on)))
 
     def profile_read(self) -> dict:
         t = SjaTiming()

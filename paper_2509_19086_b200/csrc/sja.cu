@@ -70,7 +70,7 @@ struct sja_ctx {
     DevBuf sgaps_alt, blocked, n_active, accept;   // re-auction: second ordered gap list, per-job block flags, gap counter
 
     // profiling
-    bool prof = false;
+    int prof = 0;                      // 0 off, 1 every phase, 2 the scan kernel only
     std::vector<ProfSpan> spans;
     std::vector<cudaEvent_t> free_events;
     float acc_ms[CAT_COUNT] = {0};
@@ -149,7 +149,7 @@ struct ProfScope {
     sja_ctx* c;
     ProfSpan sp;
     bool on;
-    ProfScope(sja_ctx* ctx, int cat) : c(ctx), on(ctx->prof) {
+    ProfScope(sja_ctx* ctx, int cat) : c(ctx), on(ctx->prof == 1 || (ctx->prof == 2 && cat == CAT_SCAN)) {
         if (!on) return;
         sp.cat = cat;
         sp.a = take();
@@ -367,8 +367,8 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
     uint32_t per_split = (G_act + splits - 1) / splits;
     per_split = ((per_split + tile - 1) / tile) * tile;
     splits = (G_act + per_split - 1) / per_split;
-    const bool was_on = c->prof;
-    if (!timed) c->prof = false;
+    const int was_on = c->prof;
+    if (!timed) c->prof = 0;
     {
         ProfScope ps(c, CAT_SELECT);
         JobView jv = job_view(c);
@@ -507,7 +507,8 @@ sja_status sja_profile_enable(sja_ctx* c, int on) {
     DeviceGuard guard(c->device);
     TRY(collect_spans(c));
     for (int i = 0; i < CAT_COUNT; ++i) { c->acc_ms[i] = 0.f; c->acc_n[i] = 0; }
-    c->prof = on != 0;
+    if (on < 0 || on > 2) return fail(c, SJA_ERR_INVALID_ARG, "sja_profile_enable: mode must be 0, 1 or 2");
+    c->prof = on;
     return SJA_OK;
 }
 
@@ -589,6 +590,17 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
     if (progress) TRY(copy_in(c, c->st_p.p, progress, (size_t)J * 4, where));
     else CU(cudaMemsetAsync(c->st_p.p, 0, (size_t)J * 4, c->stream));
 
+    // Device inputs and buffers of an earlier load at hand: the state kernel and the scan are launched right
+    // behind the validation pass and check its verdict on the device (they do nothing for a rejected load or
+    // one whose table outgrows the buffers), so the host waits once per load instead of twice.  Otherwise
+    // the host waits for the verdict and the row count first, as it must to size the table.
+    const size_t need4 = (size_t)J * 4, need8 = (size_t)J * 8;
+    const bool perjob_ready = c->p.cap >= need4 && c->ready.cap >= need4 && c->pb.cap >= need4 && c->Dp.cap >= need4 &&
+                              c->Wp.cap >= need8 && c->jobwin.cap >= need8 && (!wait_ms || c->wait.cap >= need4) &&
+                              (!prio || c->prio.cap >= (size_t)J);
+    const bool speculate = where == SJA_MEM_DEVICE && !n_known && perjob_ready && c->A.cap >= 32 && c->B.cap >= 24;
+    const uint64_t cap_rows = speculate ? std::min<uint64_t>(c->A.cap / 16 - 1, c->B.cap / 8 - 2) : ~0ull;
+
     // pass 0: validate + count rows, then row offsets; nothing of the loaded state is touched yet
     CU(cudaMemsetAsync(c->flags.p, 0, 4, c->stream));
     {
@@ -599,79 +611,113 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
         cta_offsets_kernel<<<1, 1024, 0, c->stream>>>(c->cta_tot.as<uint64_t>(), n_count_ctas,
                                                       c->cta_base.as<uint64_t>());
         row_offsets_kernel<<<(J + 255) / 256, 256, 0, c->stream>>>(c->nbj.as<uint64_t>(), c->cta_base.as<uint64_t>(),
-                                                                   J, n_count_ctas, c->boff_next.as<uint64_t>());
+                                                                   J, n_count_ctas, c->boff_next.as<uint64_t>(),
+                                                                   cap_rows, c->flags.as<uint32_t>());
     }
     CU(cudaGetLastError());
-    CU(cudaMemcpyAsync(c->h_words, c->flags.p, 4, cudaMemcpyDeviceToHost, c->stream));
-    CU(cudaMemcpyAsync(c->h_words + 2, c->boff_next.as<uint64_t>() + J, 8, cudaMemcpyDeviceToHost, c->stream));
-    if (!n_known) CU(cudaMemcpyAsync(c->h_words + 4, d_off + J, 8, cudaMemcpyDeviceToHost, c->stream));
-    CU(cudaStreamSynchronize(c->stream));
-    if (!n_known) {
-        memcpy(&N, c->h_words + 4, 8);
-        if (N >= (1ull << 40) && !(c->h_words[0] & FLAG_BAD_PROFILE))
-            return fail(c, SJA_ERR_BAD_PROFILE, "off[J] = %llu is implausible", (unsigned long long)N);
-    }
-    if (c->h_words[0] & FLAG_BAD_PROFILE)
-        return fail(c, SJA_ERR_BAD_PROFILE, "profile CSR invalid (offsets not monotone, job too long, or progress > len)");
-    uint64_t n_rows = 0;
-    memcpy(&n_rows, c->h_words + 2, 8);
 
-    // from here on the previous load is replaced
-    c->loaded = false;
-    c->have_deadline = false;   // deadlines belong to the jobs of a load
-    c->advertised = c->selected = c->committed = false;
-    TRY(reserve(c, c->A, (size_t)n_rows * 16 + 16));
-    TRY(reserve(c, c->B, (size_t)n_rows * 8 + 16));
-    TRY(reserve(c, c->p, (size_t)J * 4));
-    TRY(reserve(c, c->ready, (size_t)J * 4));
-    TRY(reserve(c, c->pb, (size_t)J * 4));
-    TRY(reserve(c, c->Dp, (size_t)J * 4));
-    TRY(reserve(c, c->Wp, (size_t)J * 8));
-    TRY(reserve(c, c->jobwin, (size_t)J * 8));
-    if (wait_ms) TRY(reserve(c, c->wait, (size_t)J * 4));
-    if (prio) TRY(reserve(c, c->prio, (size_t)J));
-    std::swap(c->boff, c->boff_next);
-    {
-        ProfScope ps(c, CAT_PREP);
-        const bool dev = where == SJA_MEM_DEVICE;
-        if (!dev) {
-            TRY(copy_in(c, c->ready.p, ready_ms, (size_t)J * 4, where));
-            if (wait_ms) TRY(copy_in(c, c->wait.p, wait_ms, (size_t)J * 4, where));
-            if (prio) TRY(copy_in(c, c->prio.p, prio, (size_t)J, where));
+    // verdict of pass 0 (waits for the stream): flags, row count and, if not known yet, N
+    uint64_t n_rows = 0;
+    uint32_t flags = 0;
+    bool n_resolved = n_known;
+    auto read_verdict = [&]() -> sja_status {
+        CU(cudaMemcpyAsync(c->h_words, c->flags.p, 4, cudaMemcpyDeviceToHost, c->stream));
+        CU(cudaMemcpyAsync(c->h_words + 2, c->boff_next.as<uint64_t>() + J, 8, cudaMemcpyDeviceToHost, c->stream));
+        if (!n_known) CU(cudaMemcpyAsync(c->h_words + 4, d_off + J, 8, cudaMemcpyDeviceToHost, c->stream));
+        CU(cudaStreamSynchronize(c->stream));
+        flags = c->h_words[0];
+        if (!n_known) {
+            memcpy(&N, c->h_words + 4, 8);
+            n_resolved = true;
+            if (N >= (1ull << 40) && !(flags & FLAG_BAD_PROFILE))
+                return fail(c, SJA_ERR_BAD_PROFILE, "off[J] = %llu is implausible", (unsigned long long)N);
         }
-        init_state_kernel<<<(J + 255) / 256, 256, 0, c->stream>>>(
-            J, c->st_p.as<uint32_t>(), dev ? ready_ms : nullptr, dev ? wait_ms : nullptr, dev ? prio : nullptr,
-            c->p.as<uint32_t>(), c->ready.as<uint32_t>(), c->wait.as<uint32_t>(), c->prio.as<uint8_t>(),
-            c->pb.as<uint32_t>(), c->Dp.as<uint32_t>(), c->Wp.as<uint64_t>(), c->jobwin.as<unsigned long long>(),
-            c->counter.as<uint32_t>());
+        if (flags & FLAG_BAD_PROFILE)
+            return fail(c, SJA_ERR_BAD_PROFILE,
+                        "profile CSR invalid (offsets not monotone, job too long, or progress > len)");
+        memcpy(&n_rows, c->h_words + 2, 8);
+        return SJA_OK;
+    };
+    // per-job state and the scan, reading the row offsets from boff_next (it becomes boff once the load stands)
+    auto launch_state_and_scan = [&]() -> sja_status {
+        {
+            ProfScope ps(c, CAT_PREP);
+            const bool dev = where == SJA_MEM_DEVICE;
+            if (!dev) {
+                TRY(copy_in(c, c->ready.p, ready_ms, (size_t)J * 4, where));
+                if (wait_ms) TRY(copy_in(c, c->wait.p, wait_ms, (size_t)J * 4, where));
+                if (prio) TRY(copy_in(c, c->prio.p, prio, (size_t)J, where));
+            }
+            init_state_kernel<<<(J + 255) / 256, 256, 0, c->stream>>>(
+                J, c->st_p.as<uint32_t>(), dev ? ready_ms : nullptr, dev ? wait_ms : nullptr, dev ? prio : nullptr,
+                c->p.as<uint32_t>(), c->ready.as<uint32_t>(), c->wait.as<uint32_t>(), c->prio.as<uint8_t>(),
+                c->pb.as<uint32_t>(), c->Dp.as<uint32_t>(), c->Wp.as<uint64_t>(),
+                c->jobwin.as<unsigned long long>(), c->counter.as<uint32_t>(), c->flags.as<uint32_t>());
+        }
+        ScanArgs a;
+        a.off = d_off; a.d = d_d; a.m = d_m; a.sbits = d_s;
+        a.p0 = c->st_p.as<uint32_t>();
+        a.wait = wait_ms ? c->wait.as<uint32_t>() : nullptr;
+        a.prio = prio ? c->prio.as<uint8_t>() : nullptr;
+        a.boff = c->boff_next.as<uint64_t>();
+        a.A = c->A.as<uint4>();
+        a.B = c->B.as<uint2>();
+        a.J = J;
+        a.counter = c->counter.as<uint32_t>();
+        a.flags = c->flags.as<uint32_t>();
+        if (!n_resolved || N > 0) {
+            ProfScope ps(c, CAT_SCAN);
+            const uint32_t ctas_per_sm = SCAN_CTAS_PER_SM;
+            const uint32_t want = (J + SCAN_WARPS - 1) / SCAN_WARPS;
+            const uint32_t grid = std::min<uint32_t>(want, (uint32_t)c->n_sm * ctas_per_sm);
+            scan_profiles_kernel<<<grid, SCAN_WARPS * 32, SCAN_SMEM_BYTES, c->stream>>>(a);
+        }
+        CU(cudaGetLastError());
+        return SJA_OK;
+    };
+    auto reserve_state = [&]() -> sja_status {
+        TRY(reserve(c, c->A, (size_t)n_rows * 16 + 16));
+        TRY(reserve(c, c->B, (size_t)n_rows * 8 + 16));
+        TRY(reserve(c, c->p, need4));
+        TRY(reserve(c, c->ready, need4));
+        TRY(reserve(c, c->pb, need4));
+        TRY(reserve(c, c->Dp, need4));
+        TRY(reserve(c, c->Wp, need8));
+        TRY(reserve(c, c->jobwin, need8));
+        if (wait_ms) TRY(reserve(c, c->wait, need4));
+        if (prio) TRY(reserve(c, c->prio, (size_t)J));
+        return SJA_OK;
+    };
+
+    if (speculate) {
+        TRY(launch_state_and_scan());
+        TRY(read_verdict());                     // a rejected load has touched nothing of the previous one
+        // from here on the previous load is replaced
+        c->loaded = false;
+        c->have_deadline = false;                // deadlines belong to the jobs of a load
+        c->advertised = c->selected = c->committed = false;
+        if (flags & FLAG_NEED_ROWS) {
+            // the table outgrew the buffers and the kernels stood still: size them and run again
+            TRY(reserve_state());
+            CU(cudaMemsetAsync(c->flags.p, 0, 4, c->stream));
+            TRY(launch_state_and_scan());
+            TRY(read_flags(c, &flags));
+        }
+    } else {
+        TRY(read_verdict());
+        c->loaded = false;
+        c->have_deadline = false;
+        c->advertised = c->selected = c->committed = false;
+        TRY(reserve_state());
+        TRY(launch_state_and_scan());
+        TRY(read_flags(c, &flags));
     }
+    std::swap(c->boff, c->boff_next);
     c->J = J;
     c->N = N;
     c->n_rows = n_rows;
     c->have_wait = wait_ms != nullptr;
     c->have_prio = prio != nullptr;
-
-    ScanArgs a;
-    a.off = d_off; a.d = d_d; a.m = d_m; a.sbits = d_s;
-    a.p0 = c->st_p.as<uint32_t>();
-    a.wait = c->have_wait ? c->wait.as<uint32_t>() : nullptr;
-    a.prio = c->have_prio ? c->prio.as<uint8_t>() : nullptr;
-    a.boff = c->boff.as<uint64_t>();
-    a.A = c->A.as<uint4>();
-    a.B = c->B.as<uint2>();
-    a.J = J;
-    a.counter = c->counter.as<uint32_t>();
-    a.flags = c->flags.as<uint32_t>();
-    if (N > 0) {
-        ProfScope ps(c, CAT_SCAN);
-        const uint32_t ctas_per_sm = SCAN_CTAS_PER_SM;
-        const uint32_t want = (J + SCAN_WARPS - 1) / SCAN_WARPS;
-        const uint32_t grid = std::min<uint32_t>(want, (uint32_t)c->n_sm * ctas_per_sm);
-        scan_profiles_kernel<<<grid, SCAN_WARPS * 32, SCAN_SMEM_BYTES, c->stream>>>(a);
-    }
-    CU(cudaGetLastError());
-    uint32_t flags = 0;
-    TRY(read_flags(c, &flags));
     if (flags & FLAG_INTERNAL) return fail(c, SJA_ERR_CUDA, "scan self-check failed (row count mismatch)");
     if (flags & FLAG_OVF_DURATION) return fail(c, SJA_ERR_OVERFLOW, "a job's total duration does not fit in 32 bits");
     if (flags & FLAG_OVF_WORK) return fail(c, SJA_ERR_OVERFLOW, "a job's total work is >= 2^63");

@@ -14,6 +14,7 @@ enum : uint32_t {
     FLAG_OVF_SLA = 1u << 4,       // total work >= 2^55 for some job (SLA key packing)
     FLAG_OVF_READY = 1u << 5,     // start + dur >= 2^32 at commit
     FLAG_INTERNAL = 1u << 6,      // self-check failed (boundary count mismatch)
+    FLAG_NEED_ROWS = 1u << 7,     // the boundary table of this load needs more rows than the buffers given hold
 };
 
 constexpr uint32_t SJA_NO_JOB_DEV = 0xFFFFFFFFu;

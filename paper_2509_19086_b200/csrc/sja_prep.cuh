@@ -173,24 +173,32 @@ __global__ void __launch_bounds__(1024) cta_offsets_kernel(const uint64_t* __res
     if (t == 0) base_out[P] = carry;
 }
 
-// boff[j] = base of the job's CTA + offset inside the CTA; boff[J] = total row count.
+// boff[j] = base of the job's CTA + offset inside the CTA; boff[J] = total row count.  A total above
+// `cap_rows` (what the table buffers handed to the following kernels can hold) raises FLAG_NEED_ROWS.
 __global__ void __launch_bounds__(256) row_offsets_kernel(const uint64_t* __restrict__ local_off,
                                                           const uint64_t* __restrict__ cta_base, uint32_t J,
-                                                          uint32_t P, uint64_t* __restrict__ boff) {
+                                                          uint32_t P, uint64_t* __restrict__ boff, uint64_t cap_rows,
+                                                          uint32_t* __restrict__ flags) {
     const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j < J) boff[j] = cta_base[j / COUNT_JOBS_PER_CTA] + local_off[j];
-    if (j == 0) boff[J] = cta_base[P];
+    if (j == 0) {
+        const uint64_t total = cta_base[P];
+        boff[J] = total;
+        if (total > cap_rows) atomicOr(flags, FLAG_NEED_ROWS);
+    }
 }
 
 // Per-job state of a fresh load in one launch: progress and attributes copied, cursors and
 // commit votes cleared, the scan's job counter reset.  Source pointers may be nullptr (then
-// the destination was filled by a host-to-device copy, or is not used).
+// the destination was filled by a host-to-device copy, or is not used).  Does nothing when the
+// validation pass rejected the load or the table buffers are too small (see sja_load_profiles).
 __global__ void __launch_bounds__(256) init_state_kernel(
     uint32_t J, const uint32_t* __restrict__ p_src, const uint32_t* __restrict__ ready_src,
     const uint32_t* __restrict__ wait_src, const uint8_t* __restrict__ prio_src, uint32_t* __restrict__ p,
     uint32_t* __restrict__ ready, uint32_t* __restrict__ wait, uint8_t* __restrict__ prio, uint32_t* __restrict__ pb,
     uint32_t* __restrict__ Dp, uint64_t* __restrict__ Wp, unsigned long long* __restrict__ jobwin,
-    uint32_t* __restrict__ counter) {
+    uint32_t* __restrict__ counter, const uint32_t* __restrict__ flags) {
+    if (*flags & (FLAG_BAD_PROFILE | FLAG_NEED_ROWS)) return;
     const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j == 0) *counter = 0;
     if (j >= J) return;

@@ -86,6 +86,8 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32, SCAN_CTAS_PER_SM) scan_profil
     const uint32_t wid = threadIdx.x >> 5;
     unsigned char* wbase = smem_raw + (size_t)wid * SCAN_STAGES * SCAN_STAGE_BYTES;
     const uint32_t wbase_s = (uint32_t)__cvta_generic_to_shared(wbase);
+    // a load that was rejected by the validation pass, or whose table does not fit the buffers, is not scanned
+    if (*reinterpret_cast<volatile const uint32_t*>(a.flags) & (FLAG_BAD_PROFILE | FLAG_NEED_ROWS)) return;
     const uint64_t N_total = __ldg(a.off + a.J);
     const uint32_t lane_sw = (lane ^ ((lane >> 3) & 3u)) * 16u;   // swz(32 r + lane) * 16 - 512 r
     const uint32_t rd_x = (lane >> 1) & 3u;                        // swz(4 lane + r) = 4 lane + (r ^ rd_x)

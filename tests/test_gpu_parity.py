@@ -383,6 +383,55 @@ def test_select_very_large_gap_batch_unsorted_path(sja_mod, oracle_mod):
         _assert_awards_equal(got, want[:65536])
 
 
+def test_reloads_from_device_arrays(sja_mod, oracle_mod):
+    """Loads from device-resident arrays into a context that already holds a load take the path with a
+    single host wait (the validation verdict is checked on the device).  Covered here: a same-size reload,
+    a rejected CSR (the previous load must stay usable, bit for bit), a larger load (the table outgrows
+    the buffers and the scan is run again), a smaller one, and scan rows against the oracle after each."""
+    import torch
+    dev = torch.device("cuda", 0)
+
+    def to_dev(prof, off=None):
+        t = lambda a, dt: None if a is None else torch.from_numpy(np.ascontiguousarray(a).view(dt)).to(dev)
+        return dict(off=t(prof.off if off is None else off, np.int64), d=t(prof.dur_ms, np.int32),
+                    m=t(prof.mem_MiB, np.int32), s=t(prof.safe_bits, np.int32), ready=t(prof.ready_ms, np.int32),
+                    wait=t(prof.wait_ms, np.int32), prio=t(prof.prio, np.uint8))
+
+    def load_dev(ctx, d):
+        ctx.load_profiles(d["off"], d["d"], d["m"], d["s"], d["ready"], wait_ms=d["wait"], prio=d["prio"])
+
+    def check(ctx, prof, spec):
+        gaps = wl.make_gaps(spec)
+        ctx.advertise(gaps)
+        z = np.zeros(prof.n_jobs, np.uint32)
+        want = oracle_mod.select(prof, z, prof.ready_ms, gaps, spec.policy)
+        _assert_awards_equal(ctx.select(spec.policy, out="host"), want)
+        assert ctx.scan_size() == int(wl.unpack_safe_bits(prof.safe_bits, prof.n_steps).sum())
+        return want
+
+    small = wl.scaled(wl.SPECS[3], n_jobs=900, zipf_max=3000, n_gaps=300)
+    large = wl.scaled(wl.SPECS[3], n_jobs=900, zipf_max=60000, n_gaps=300)     # same J, far more rows
+    p_small, p_large = wl.make_profiles(small, threads=2), wl.make_profiles(large, threads=2)
+    assert p_large.n_steps > 2 * p_small.n_steps
+    with sja_mod.Sja() as ctx:
+        d_small, d_large = to_dev(p_small), to_dev(p_large)
+        load_dev(ctx, d_small)                      # first load: nothing to reuse yet
+        check(ctx, p_small, small)
+        load_dev(ctx, d_small)                      # reload: single-wait path
+        want = check(ctx, p_small, small)
+        bad = p_small.off.copy()
+        bad[5], bad[6] = bad[6], bad[5]             # offsets not monotone
+        with pytest.raises(sja_mod.SjaError) as e:
+            load_dev(ctx, to_dev(p_small, off=bad))
+        assert e.value.status == 2
+        _assert_awards_equal(ctx.select(small.policy, out="host"), want)     # the old load still stands
+        assert ctx.commit() > 0
+        load_dev(ctx, d_large)                      # more rows than the table buffers hold
+        check(ctx, p_large, large)
+        load_dev(ctx, d_small)                      # and back
+        check(ctx, p_small, small)
+
+
 def test_select_is_deterministic_and_device_outputs_match(sja_mod):
     """The cross-CTA reduction is on a totally ordered key, so repeated selects give identical bytes;
     a device output buffer receives the same awards as a host buffer."""
