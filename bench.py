@@ -39,17 +39,17 @@ FALLBACK_HBM_GBS = 6650.0
 # scan_profiles_kernel_cfg2-jobs8192.md): dram__bytes_read.sum + dram__bytes_write.sum over 33 554 432 steps.
 # Traffic grows in proportion to the step count, so a full launch is this figure times N.  It is only reported
 # while csrc/sja_scan.cuh is the file the counters were taken from (first 16 hex digits of its sha256).
-NCU_SCAN_TRAFFIC_BYTES_PER_STEP = (273.048064e6 + 59.769344e6) / 33554432
-NCU_SCAN_SOURCE_SHA = "8bd8a77590ca9c38"
+NCU_SCAN_TRAFFIC_BYTES_PER_STEP = (273.041664e6 + 59.891712e6) / 33554432
+NCU_SCAN_SOURCE_SHA = "45fc1da5bae387db"
 
 
 # Issue-slot roofline of the select kernel (it is bound by instruction issue, not HBM): warp instructions of one
 # launch on the large uniform workload from ncu (profiles/select_tile_kernel_cfg2-jobs32768.md, full-size line),
 # peak = SMs x 4 schedulers x SM clock.  The kernel's work is not proportional to the pair count, so the figure
 # holds for that workload only; it is reported while csrc/sja_tile.cuh is the file the counters were taken from.
-NCU_TILE_WARP_INSTR_PER_LAUNCH = 100790035
+NCU_TILE_WARP_INSTR_PER_LAUNCH = 101670675
 NCU_TILE_PAIRS = 65536 * 4096
-NCU_TILE_SOURCE_SHA = "fcfa235eeb8ecc2b"
+NCU_TILE_SOURCE_SHA = "2c15766b184311a3"
 N_SM, SCHEDULERS_PER_SM = 148, 4
 
 
