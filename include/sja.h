@@ -261,6 +261,20 @@ sja_status sja_set_duration_bounds(sja_ctx* ctx, uint32_t tau_min_ms, uint32_t t
  */
 sja_status sja_set_window_options(sja_ctx* ctx, uint32_t late_start, const uint32_t* deadline_ms, sja_memspace where);
 
+/*
+ * Re-profile one job.  Segmentation is on demand because the envelope U(t) "may evolve as runtime
+ * predictions are refined" (Section 3.9): this call replaces the per-step durations and memory values of
+ * the steps job `job` has not been granted yet, steps p_job .. len_job - 1, n_steps = len_job - p_job of
+ * them (SJA_ERR_BAD_PROFILE otherwise).  The job's safe boundaries stay where they are (a refined
+ * prediction changes how long and how large a phase is, not where the checkpoints are), so only the
+ * contents of the job's boundary rows are recomputed; no other job is touched and nothing is rescanned.
+ * dur_ms / mem_MiB are u32[n_steps], host or device as `where` says, copied before the call returns.
+ * SJA_ERR_OVERFLOW (total duration >= 2^32 ms or total work >= 2^63) leaves the job as it was.
+ * Waits for completion.  A select that has not been committed yet is discarded: select again.
+ */
+sja_status sja_update_profile(sja_ctx* ctx, uint32_t job, uint32_t n_steps, const uint32_t* dur_ms,
+                              const uint32_t* mem_MiB, sja_memspace where);
+
 /* Copy the G awards of the last select (with `granted` set if it was committed). */
 sja_status sja_get_awards(sja_ctx* ctx, sja_award* out, sja_memspace where);
 

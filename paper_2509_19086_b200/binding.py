@@ -30,7 +30,7 @@ AWARD_DTYPE = np.dtype([("job", "<u4"), ("end_step", "<u4"), ("dur_ms", "<u4"), 
                         ("score", "<u8")])
 
 EXPORTS = [
-    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit", "sja_commit_masked", "sja_round_reauction", "sja_set_duration_bounds", "sja_set_window_options",
+    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit", "sja_commit_masked", "sja_round_reauction", "sja_set_duration_bounds", "sja_set_window_options", "sja_update_profile",
     "sja_get_awards", "sja_get_state", "sja_scan_size", "sja_get_scan", "sja_profile_enable",
     "sja_profile_read", "sja_last_error",
 ]
@@ -79,6 +79,7 @@ def load_library() -> ctypes.CDLL:
     lib.sja_round_reauction.argtypes = [vp, ctypes.POINTER(SjaPolicy), u32, ctypes.POINTER(u32), ctypes.POINTER(u32)]
     lib.sja_set_duration_bounds.argtypes = [vp, u32, u32]
     lib.sja_set_window_options.argtypes = [vp, u32, vp, i32]
+    lib.sja_update_profile.argtypes = [vp, u32, u32, vp, vp, i32]
     lib.sja_commit_masked.argtypes = [vp, vp, i32, ctypes.POINTER(u32)]
     lib.sja_get_awards.argtypes = [vp, vp, i32]
     lib.sja_get_state.argtypes = [vp, vp, vp, i32]
@@ -251,6 +252,16 @@ class Sja:
             raise ValueError("deadline_ms needs one entry per loaded job")
         self._check(self._lib.sja_set_window_options(self._h, 1 if late_start else 0, p,
                                                      MEM_HOST if space is None else space))
+
+    # -- sja_update_profile
+    def update_profile(self, job: int, dur_ms, mem_MiB) -> None:
+        """New durations / memory values (u32, numpy or CUDA tensors) for the steps ``job`` has left."""
+        pd, space, keep_d = _ptr_space(dur_ms, None, np.uint32)
+        pm, space, keep_m = _ptr_space(mem_MiB, space, np.uint32)
+        n = int(keep_d.shape[0]) if keep_d is not None else 0
+        if keep_m is not None and int(keep_m.shape[0]) != n:
+            raise ValueError("dur_ms and mem_MiB must have the same length")
+        self._check(self._lib.sja_update_profile(self._h, int(job), n, pd, pm, MEM_HOST if space is None else space))
 
     # -- sja_get_awards / sja_get_state
     def get_awards(self) -> np.ndarray:

@@ -17,6 +17,7 @@
 #include "sja_round.cuh"
 #include "sja_scan.cuh"
 #include "sja_tile.cuh"
+#include "sja_update.cuh"
 
 using namespace sja;
 
@@ -64,6 +65,7 @@ struct sja_ctx {
     uint32_t tau_min = 0, tau_max = 0xFFFFFFFFu;   // subjob duration thresholds for select
     bool late_start = false, have_deadline = false;   // window options (sja_set_window_options)
     DevBuf deadline;
+    DevBuf upd_d, upd_m, upd_scratch, upd_status;   // sja_update_profile: staged inputs, segment values, verdict
     bool gaps_sorted = false;          // sgaps is ordered by (C, T); else it is the caller's order
     uint32_t n_classes = 0;            // distinct capacities of the batch (valid when sorted)
     DevBuf gaps, sgaps, gap_info, gap_rank, awards, widx, partial, winners;
@@ -489,7 +491,7 @@ sja_status sja_destroy(sja_ctx* c) {
     cudaStreamSynchronize(c->stream);
     DevBuf* bufs[] = {&c->st_off, &c->st_d, &c->st_m, &c->st_s, &c->st_p, &c->p, &c->ready, &c->pb, &c->Dp,
                       &c->Wp, &c->wait, &c->prio, &c->nbj, &c->cta_tot, &c->cta_base, &c->boff, &c->boff_next, &c->A, &c->B, &c->jobwin,
-                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->deadline, &c->awards, &c->widx, &c->partial,
+                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->deadline, &c->upd_d, &c->upd_m, &c->upd_scratch, &c->upd_status, &c->awards, &c->widx, &c->partial,
                       &c->winners};
     for (DevBuf* b : bufs) release(*b);
     for (ProfSpan& s : c->spans) { cudaEventDestroy(s.a); cudaEventDestroy(s.b); }
@@ -934,6 +936,51 @@ sja_status sja_set_duration_bounds(sja_ctx* c, uint32_t tau_min_ms, uint32_t tau
         return fail(c, SJA_ERR_INVALID_ARG, "sja_set_duration_bounds: tau_min %u > tau_max %u", tau_min_ms, tau_max_ms);
     c->tau_min = tau_min_ms;
     c->tau_max = tau_max_ms;
+    return SJA_OK;
+}
+
+sja_status sja_update_profile(sja_ctx* c, uint32_t job, uint32_t n_steps, const uint32_t* dur_ms,
+                              const uint32_t* mem_MiB, sja_memspace where) {
+    TRY(check_ctx(c));
+    if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_update_profile: bad memspace");
+    if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_update_profile before sja_load_profiles");
+    if (job >= c->J) return fail(c, SJA_ERR_INVALID_ARG, "sja_update_profile: job %u of %u", job, c->J);
+    if (n_steps && (!dur_ms || !mem_MiB)) return fail(c, SJA_ERR_INVALID_ARG, "sja_update_profile: array is NULL");
+    DeviceGuard guard(c->device);
+    const uint32_t *d_d = dur_ms, *d_m = mem_MiB;
+    if (where == SJA_MEM_HOST && n_steps) {
+        TRY(reserve(c, c->upd_d, (size_t)n_steps * 4));
+        TRY(reserve(c, c->upd_m, (size_t)n_steps * 4));
+        TRY(copy_in(c, c->upd_d.p, dur_ms, (size_t)n_steps * 4, where));
+        TRY(copy_in(c, c->upd_m.p, mem_MiB, (size_t)n_steps * 4, where));
+        d_d = c->upd_d.as<uint32_t>();
+        d_m = c->upd_m.as<uint32_t>();
+    }
+    TRY(reserve(c, c->upd_scratch, (size_t)std::max<uint32_t>(n_steps, 1u) * 16));   // a job has at most one row per step
+    TRY(reserve(c, c->upd_status, 4));
+    CU(cudaMemsetAsync(c->upd_status.p, 0, 4, c->stream));
+    UpdateArgs a;
+    a.j = job; a.n = n_steps; a.d = d_d; a.m = d_m;
+    a.boff = c->boff.as<uint64_t>(); a.pb = c->pb.as<uint32_t>(); a.p = c->p.as<uint32_t>();
+    a.Dp = c->Dp.as<uint32_t>(); a.Wp = c->Wp.as<uint64_t>();
+    a.wait = c->have_wait ? c->wait.as<uint32_t>() : nullptr;
+    a.A = c->A.as<uint4>(); a.B = c->B.as<uint2>();
+    a.scratch = c->upd_scratch.as<uint4>();
+    a.flags = c->flags.as<uint32_t>();
+    a.status = c->upd_status.as<uint32_t>();
+    update_profile_kernel<<<1, UPDATE_THREADS, 0, c->stream>>>(a);
+    CU(cudaGetLastError());
+    CU(cudaMemcpyAsync(c->h_words, c->upd_status.p, 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaMemcpyAsync(c->h_words + 1, c->flags.p, 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaStreamSynchronize(c->stream));
+    if (c->h_words[0] == UPD_BAD_SIZE)
+        return fail(c, SJA_ERR_BAD_PROFILE, "sja_update_profile: n_steps = %u is not the number of steps job %u has left",
+                    n_steps, job);
+    if (c->h_words[0] == UPD_OVERFLOW)
+        return fail(c, SJA_ERR_OVERFLOW, "sja_update_profile: total duration >= 2^32 ms or total work >= 2^63 for job %u", job);
+    c->load_flags |= c->h_words[1] & (FLAG_OVF_FAIR | FLAG_OVF_SLA);
+    c->selected = false;   // awards chosen from the old profile must not be committed
     return SJA_OK;
 }
 
