@@ -157,3 +157,43 @@ def test_cfg4_streaming_1000_rounds(oracle_mod):
         assert np.array_equal(rd.astype(np.int64), replay_r)
         print("cfg4 grants over 1000 rounds:", total)
         assert total > 50_000
+
+
+@pytest.mark.parametrize("case", ["many_classes", "equal_T", "equal_ready_and_start", "unbounded_T", "late_progress",
+                                  "ragged_counts"])
+def test_select_kernels_agree_on_structured_batches(oracle_mod, case):
+    """Batches built to stress the ordered-gap kernels (runs of one gap, a single run, one eligibility prefix for
+    everybody, windows longer than any job, cursors that start deep inside the jobs, counts that are not multiples
+    of anything): tile, merge and search kernels give identical awards, and 200 sampled gaps match the oracle."""
+    from paper_2509_19086_b200 import binding
+    rng = np.random.default_rng(7000 + sum(map(ord, case)))
+    n_jobs, n_gaps = (20011, 1999) if case == "ragged_counts" else (20000, 2000)
+    spec = wl.scaled(wl.SPECS[3], n_jobs=n_jobs, zipf_max=4000, n_gaps=n_gaps)
+    prof = wl.make_profiles(spec, threads=8)
+    gaps = wl.make_gaps(spec)
+    progress = np.zeros(prof.n_jobs, np.uint32)
+    ready = prof.ready_ms.copy()
+    if case == "many_classes":
+        gaps["C_MiB"] = rng.choice(np.arange(2000, 82000, 700), n_gaps)          # 115 capacities, runs of ~17 gaps
+    elif case == "equal_T":
+        gaps["T_ms"] = 1234
+    elif case == "equal_ready_and_start":
+        ready[:] = 500
+        gaps["start_ms"] = rng.choice([499, 500], n_gaps)
+    elif case == "unbounded_T":
+        gaps["T_ms"] = U32MAX
+        gaps["start_ms"] = 1000
+    elif case == "late_progress":
+        lens = np.diff(prof.off).astype(np.int64)
+        progress = (lens * rng.uniform(0.0, 1.0, prof.n_jobs)).astype(np.uint32)
+    with binding.Sja() as ctx:
+        ctx.load_profiles(prof.off, prof.dur_ms, prof.mem_MiB, prof.safe_bits, ready,
+                          progress=progress, wait_ms=prof.wait_ms, prio=prof.prio)
+        ctx.advertise(gaps)
+        for policy in (0, 2, 3):
+            tile = ctx.select(policy, flags=binding.FLAG_FORCE_TILE, out="host")
+            assert ctx.select(policy, flags=binding.FLAG_FORCE_MERGE, out="host").tobytes() == tile.tobytes(), policy
+            assert ctx.select(policy, flags=binding.FLAG_FORCE_SEARCH, out="host").tobytes() == tile.tobytes(), policy
+            sample = np.sort(rng.choice(n_gaps, 200, replace=False))
+            want = oracle_mod.select(prof, progress, ready, gaps[sample], policy)
+            _assert_equal(tile[sample], want)
