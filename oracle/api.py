@@ -51,12 +51,12 @@ def _load():
     lib.orc_pair.restype = ctypes.c_int
     lib.orc_pair.argtypes = [vp, vp, vp, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint32,
                              ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
-                             ctypes.c_uint32, ctypes.c_uint32, ctypes.c_int, ctypes.c_uint32, u32p, u32p, u64p,
-                             u32p]
+                             ctypes.c_uint32, ctypes.c_uint32, ctypes.c_int, ctypes.c_uint32, vp, ctypes.c_uint32,
+                             u32p, u32p, u64p, u32p]
     lib.orc_select.restype = ctypes.c_int
     lib.orc_select.argtypes = [ctypes.c_uint32, vp, vp, vp, vp, vp, vp, vp, vp,
                                ctypes.c_uint32, vp, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
-                               ctypes.c_int, vp, vp]
+                               ctypes.c_int, vp, vp, vp, vp]
     lib.orc_commit.restype = ctypes.c_int64
     lib.orc_commit.argtypes = [ctypes.c_uint32, vp, vp, ctypes.c_uint32, vp, vp, ctypes.c_int]
     lib.orc_num_threads.restype = ctypes.c_int
@@ -86,9 +86,10 @@ U32MAX = 0xFFFFFFFF
 
 def pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: int,
          tau_min_ms: int = 0, tau_max_ms: int = U32MAX, late_start: bool = False, deadline_ms: int = U32MAX,
-         want_peak: bool = False):
+         want_peak: bool = False, power_W: Optional[np.ndarray] = None, power_cap_W: int = U32MAX):
     """R1-R3 (with the duration thresholds of R2' and the window options of R1'') for one (gap, job)
-    pair: ``None`` for decline, else ``(k, dur, work)`` (``(k, dur, work, peak)`` with ``want_peak``)."""
+    pair: ``None`` for decline, else ``(k, dur, work)`` (``(k, dur, work, peak)`` with ``want_peak``).
+    ``power_W`` (u32 per step, aligned with the profile arrays) and ``power_cap_W`` switch on R2''."""
     lib = _load()
     k = ctypes.c_uint32()
     dur = ctypes.c_uint32()
@@ -98,6 +99,7 @@ def pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: i
                       prof.safe_bits.ctypes.data, int(prof.off[j]), int(prof.off[j + 1]),
                       int(p), int(ready_ms), int(start_ms), int(T_ms), int(C_MiB),
                       int(tau_min_ms), int(tau_max_ms), int(bool(late_start)), int(deadline_ms),
+                      _ptr(_as(power_W, np.uint32)), int(power_cap_W),
                       ctypes.byref(k), ctypes.byref(dur), ctypes.byref(work), ctypes.byref(peak))
     if not ok:
         return None
@@ -108,9 +110,11 @@ def pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: i
 
 def select(prof, progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray,
            policy: int, tau_min_ms: int = 0, tau_max_ms: int = U32MAX, late_start: bool = False,
-           deadline_ms: Optional[np.ndarray] = None) -> np.ndarray:
+           deadline_ms: Optional[np.ndarray] = None, power_W: Optional[np.ndarray] = None,
+           power_cap_W: Optional[np.ndarray] = None) -> np.ndarray:
     """R1-R5 for a batch of gaps; returns ``AWARD_DTYPE[G]`` (``granted`` all zero).
-    ``late_start`` / ``deadline_ms`` (u32 per job) switch on the window options of R1''."""
+    ``late_start`` / ``deadline_ms`` (u32 per job) switch on the window options of R1''; ``power_W`` (u32 per
+    step) with ``power_cap_W`` (u32 per gap) the power envelope of R2''."""
     lib = _load()
     off = _as(prof.off, np.uint64)
     d = _as(prof.dur_ms, np.uint32)
@@ -124,10 +128,14 @@ def select(prof, progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray,
     awards = np.zeros(gaps.shape[0], dtype=AWARD_DTYPE)
     deadline = _as(deadline_ms, np.uint32)
     assert deadline is None or deadline.shape[0] == off.shape[0] - 1
+    power = _as(power_W, np.uint32)
+    caps = _as(power_cap_W, np.uint32)
+    assert power is None or power.shape[0] == d.shape[0]
+    assert caps is None or caps.shape[0] == gaps.shape[0]
     rc = lib.orc_select(off.shape[0] - 1, _ptr(off), _ptr(d), _ptr(m), _ptr(s),
                         _ptr(progress), _ptr(ready_ms), _ptr(wait), _ptr(prio),
                         gaps.shape[0], _ptr(gaps), int(policy), int(tau_min_ms), int(tau_max_ms),
-                        int(bool(late_start)), _ptr(deadline), _ptr(awards))
+                        int(bool(late_start)), _ptr(deadline), _ptr(power), _ptr(caps), _ptr(awards))
     if rc != 0:
         raise ValueError("oracle select: unknown policy or missing attribute array")
     return awards

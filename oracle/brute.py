@@ -17,12 +17,13 @@ def _safe(bits, i: int) -> bool:
 
 def brute_pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: int,
                tau_min_ms: int = 0, tau_max_ms: int = 0xFFFFFFFF, late_start: bool = False,
-               deadline_ms: int = 0xFFFFFFFF):
+               deadline_ms: int = 0xFFFFFFFF, power_W=None, power_cap_W: int = 0xFFFFFFFF):
     """``None`` (decline) or ``(k, dur, work)`` of the longest feasible subjob.
 
     Window options: with ``late_start`` the subjob occupies ``[begin, begin + dur)`` with
     ``begin = max(start, ready)`` and has to lie inside the gap ``[start, start + T]``; without it the
-    job must be ready when the gap opens.  It has to be over by ``deadline_ms``."""
+    job must be ready when the gap opens.  It has to be over by ``deadline_ms``.  With a per-step power trace
+    and a cap, no step of the subjob may draw more than the cap (Section 4.4, item 1)."""
     s, e = int(prof.off[j]), int(prof.off[j + 1])
     length = e - s
     if p >= length:
@@ -44,6 +45,9 @@ def brute_pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_
         if not (tau_min_ms <= sum(d[p:k]) <= tau_max_ms):      # Section 4.3 (5) thresholds
             continue
         if max(m[p:k]) > C_MiB:
+            continue
+        if power_W is not None and power_cap_W != 0xFFFFFFFF and \
+                max(int(x) for x in power_W[s + p:s + k]) > power_cap_W:
             continue
         candidates.append(k)
     if not candidates:

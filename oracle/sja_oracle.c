@@ -50,6 +50,11 @@
  *                    subjobs that complete by their deadline; the risk margin lives in the
  *                    durations, as it does in the memory envelope): a candidate also needs
  *                    begin + sum d <= deadline_j; 2^32-1 means no deadline.
+ *   R2'' power     : optional second resource envelope (Section 4.4, item 1: offers carry a power
+ *                    cap, subjobs answer with a predicted power trace, admission keeps
+ *                    max_t P(t) <= power_cap with the risk margin in the trace): with a per-step
+ *                    power_W array and a per-gap cap, a candidate also needs
+ *                    max power_W[p_j..k) <= cap_g; a cap of 2^32-1 means none.
  *
  * The walk below visits one step at a time, exactly in that order: no prefix arrays,
  * no search, no blocking.  OpenMP only spreads independent gaps over host threads.
@@ -95,6 +100,7 @@ int orc_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *sa
              uint32_t start_ms, uint32_t T_ms, uint32_t C_MiB,
              uint32_t tau_min_ms, uint32_t tau_max_ms,
              int late_start, uint32_t deadline_ms,
+             const uint32_t *power_W /* per step like mem_MiB, or NULL */, uint32_t power_cap_W,
              uint32_t *k_out, uint32_t *dur_out, uint64_t *work_out, uint32_t *peak_out /* may be NULL */)
 {
     uint64_t len = e - s;
@@ -110,7 +116,8 @@ int orc_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *sa
     if (has_deadline && begin > (uint64_t)deadline_ms) return 0; /* R1'': deadline already passed */
 
     uint64_t acc = 0, work = 0;
-    uint32_t peak = 0;
+    uint32_t peak = 0, power_peak = 0;
+    const int has_cap = power_W != NULL && power_cap_W != 0xFFFFFFFFu;
     int found = 0;
     uint32_t best_k = 0, best_dur = 0, best_peak = 0;
     uint64_t best_work = 0;
@@ -119,6 +126,10 @@ int orc_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *sa
         if (mem_MiB[i] > peak) peak = mem_MiB[i];
         work += (uint64_t)dur_ms[i] * (uint64_t)mem_MiB[i];
         if (begin + acc > window_end || peak > C_MiB) break;   /* R2: window or capacity broken */
+        if (has_cap) {
+            if (power_W[i] > power_peak) power_peak = power_W[i];
+            if (power_peak > power_cap_W) break;               /* R2'': above the power cap of the offer */
+        }
         if (has_deadline && begin + acc > (uint64_t)deadline_ms) break;   /* R1'': would finish after the deadline */
         if (acc > (uint64_t)tau_max_ms) break;             /* R2': longer than the maximum subjob */
         if ((step_is_safe(safe_bits, i) || i + 1 == e)     /* R2: safe boundary after step i */
@@ -166,6 +177,7 @@ int orc_select(uint32_t n_jobs, const uint64_t *off,
                uint32_t n_gaps, const orc_gap *gaps, uint32_t policy,
                uint32_t tau_min_ms, uint32_t tau_max_ms,
                int late_start, const uint32_t *deadline_ms /* per job, or NULL = none */,
+               const uint32_t *power_W /* per step, or NULL */, const uint32_t *power_cap_W /* per gap, or NULL */,
                orc_award *awards)
 {
     if (policy > ORC_TIGHT_FIT) return -1;
@@ -184,6 +196,7 @@ int orc_select(uint32_t n_jobs, const uint64_t *off,
             if (!orc_pair(dur_ms, mem_MiB, safe_bits, off[j], off[j + 1], progress[j],
                           ready_ms[j], gap.start_ms, gap.T_ms, gap.C_MiB, tau_min_ms, tau_max_ms,
                           late_start, deadline_ms ? deadline_ms[j] : 0xFFFFFFFFu,
+                          power_W, power_cap_W ? power_cap_W[g] : 0xFFFFFFFFu,
                           &k, &dur, &work, &peak))
                 continue;                                      /* decline */
             uint32_t cls;
