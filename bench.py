@@ -260,6 +260,9 @@ def main():
                     help="time sja_round_reauction (select + commit repeated for orphaned gaps) instead of one select + commit")
     ap.add_argument("--window-options", action="store_true",
                     help="late start inside a gap and per-job deadlines (ready + 2000..8000 ms): per-pair search path")
+    ap.add_argument("--power-caps", action="store_true",
+                    help="second resource envelope: a per-step power trace (50 W + 350 W x mem / 80 GiB + noise) loaded "
+                         "with every load and a cap of 100..400 W per gap: per-pair search path")
     ap.add_argument("--streaming", action="store_true",
                     help="multi-round workloads only: load once, then every step is one advertise/select/commit round "
                          "with that round's gap batch (use --steps 1000 for the published streaming configuration)")
@@ -277,6 +280,8 @@ def main():
     if args.impl == "reference":
         run_reference(args, spec)
         return
+    if args.power_caps:
+        args.e2e_steps = 0          # the end-to-end leg moves the four input arrays of the boundary only
     if args.streaming and (spec.n_rounds <= 1 or args.reauction):
         raise SystemExit("--streaming needs a multi-round workload (--workload 4) and no --reauction")
 
@@ -318,6 +323,13 @@ def main():
     gaps_pinned = gaps_pinned.view(wl.GAP_DTYPE)
     dev = {k: _to_device(a, device) for k, a in host_arrays.items()}
     dev_gaps = _to_device(gaps, device)
+    dev_power = dev_caps = None
+    if args.power_caps:
+        rng = np.random.default_rng(my_spec.seed + 78)
+        power = (50 + prof.mem_MiB.astype(np.int64) * 350 // 81920 + rng.integers(0, 120, N)).astype(np.uint32)
+        dev_power = _to_device(power, device)
+        dev_caps = _to_device(rng.integers(100, 401, G).astype(np.uint32), device)
+        del power
     dev_deadline = None
     if args.window_options:
         rng = np.random.default_rng(my_spec.seed + 77)
@@ -345,9 +357,13 @@ def main():
                           wait_ms=dev.get("wait"), prio=dev.get("prio"))
         if args.window_options:
             ctx.set_window_options(True, dev_deadline)
+        if args.power_caps:
+            ctx.load_power(dev["off"], dev_power)
 
     def round_device(r):
         ctx.advertise(round_gaps_dev[r])
+        if args.power_caps:
+            ctx.advertise_power_caps(dev_caps)
         ctx.select(my_spec.policy, flags=args.flags)
         ctx.commit(want_count=False)
         launches[0] += KERNELS_PER_STEP - 5 - one_tile_saving   # no load: the five load kernels do not run
@@ -362,14 +378,18 @@ def main():
                           wait_ms=dev.get("wait"), prio=dev.get("prio"))
         if args.window_options:
             ctx.set_window_options(True, dev_deadline)
+        if args.power_caps:
+            ctx.load_power(dev["off"], dev_power)
         ctx.advertise(dev_gaps)
+        if args.power_caps:
+            ctx.advertise_power_caps(dev_caps)
         if args.reauction:
             _, passes = ctx.round_reauction(my_spec.policy, flags=args.flags)
             launches[0] += 7 + 6 * passes      # per pass: select, finalize, 3 commit kernels, orphan compaction
         else:
             ctx.select(my_spec.policy, flags=args.flags)
             ctx.commit(want_count=False)
-            launches[0] += KERNELS_PER_STEP - one_tile_saving
+            launches[0] += KERNELS_PER_STEP - one_tile_saving + (1 if args.power_caps else 0)
 
     def step_e2e():
         ctx.load_profiles(pinned["off"], pinned["d"], pinned["m"], pinned["s"], pinned["ready"],
@@ -489,7 +509,7 @@ def main():
                    "l2": "inputs larger than L2 (profile arrays re-read from HBM every step)"
                    if prof.raw_bytes() > 200e6 else "inputs smaller than L2",
                    "flags": args.flags, "reauction": bool(args.reauction),
-                   "window_options": bool(args.window_options),
+                   "window_options": bool(args.window_options), "power_caps": bool(args.power_caps),
                    "streaming": "load once, one advertise/select/commit round per step" if args.streaming else False},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -498,7 +518,8 @@ def main():
         "roofline": roofline,
         # the instruction count per pair was captured on the large uniform workload only
         "select_roofline": select_roofline(pairs, select_ms, clocks.get("sm_mhz"))
-        if spec.index == 2 and not args.flags and not args.reauction and not args.window_options else None,
+        if spec.index == 2 and not args.flags and not args.reauction and not args.window_options
+        and not args.power_caps else None,
         "kernel_ms_per_step": breakdown,
         "select_pairs_per_s": pairs / (select_ms * 1e-3) if select_ms > 0 else None,
         "profile_gb_per_s": prof.raw_bytes() / (scan_ms * 1e-3) / 1e9 if scan_ms > 0 else None,

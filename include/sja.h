@@ -262,6 +262,27 @@ sja_status sja_set_duration_bounds(sja_ctx* ctx, uint32_t tau_min_ms, uint32_t t
 sja_status sja_set_window_options(sja_ctx* ctx, uint32_t late_start, const uint32_t* deadline_ms, sja_memspace where);
 
 /*
+ * Power envelope, a second resource channel beside memory (Section 4.4, item 1: offers carry power caps,
+ * subjobs answer with predicted power traces, and admission keeps max_t P(t) <= power_cap; as with memory,
+ * the tolerated risk lives in the trace, which is a risk-adjusted envelope).
+ *
+ * sja_load_power: per-step predicted power in watts, u32[N], aligned step for step with the arrays given to
+ * sja_load_profiles; `off` is the same CSR offset array again (the library does not keep it; a different
+ * job length is SJA_ERR_BAD_PROFILE).  Builds, for every boundary row above the jobs' progress points, the
+ * running maximum of the trace.  Call after sja_load_profiles, at any time between rounds; a new load
+ * drops the trace.  Waits for completion.
+ *
+ * sja_advertise_power_caps: cap_W u32[G] for the batch just advertised, in the order of its gaps; an entry
+ * of 0xFFFFFFFF, or cap_W = NULL, means no cap.  A new sja_advertise drops the caps.  With a trace loaded
+ * and caps advertised, a candidate subjob also needs max power_W[p_j..k) <= cap_g, and every select runs
+ * the per-pair search kernel (the cap differs from gap to gap inside a capacity class, which the
+ * ordered-gap kernels cannot follow).  sja_commit keeps the running maximum current for granted jobs.
+ * Both calls discard a select that has not been committed yet.
+ */
+sja_status sja_load_power(sja_ctx* ctx, const uint64_t* off, const uint32_t* power_W, sja_memspace where);
+sja_status sja_advertise_power_caps(sja_ctx* ctx, const uint32_t* cap_W, sja_memspace where);
+
+/*
  * Re-profile one job.  Segmentation is on demand because the envelope U(t) "may evolve as runtime
  * predictions are refined" (Section 3.9): this call replaces the per-step durations and memory values of
  * the steps job `job` has not been granted yet, steps p_job .. len_job - 1, n_steps = len_job - p_job of

@@ -30,7 +30,7 @@ AWARD_DTYPE = np.dtype([("job", "<u4"), ("end_step", "<u4"), ("dur_ms", "<u4"), 
                         ("score", "<u8")])
 
 EXPORTS = [
-    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit", "sja_commit_masked", "sja_round_reauction", "sja_set_duration_bounds", "sja_set_window_options", "sja_update_profile",
+    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit", "sja_commit_masked", "sja_round_reauction", "sja_set_duration_bounds", "sja_set_window_options", "sja_update_profile", "sja_load_power", "sja_advertise_power_caps",
     "sja_get_awards", "sja_get_state", "sja_scan_size", "sja_get_scan", "sja_profile_enable",
     "sja_profile_read", "sja_last_error",
 ]
@@ -80,6 +80,8 @@ def load_library() -> ctypes.CDLL:
     lib.sja_set_duration_bounds.argtypes = [vp, u32, u32]
     lib.sja_set_window_options.argtypes = [vp, u32, vp, i32]
     lib.sja_update_profile.argtypes = [vp, u32, u32, vp, vp, i32]
+    lib.sja_load_power.argtypes = [vp, vp, vp, i32]
+    lib.sja_advertise_power_caps.argtypes = [vp, vp, i32]
     lib.sja_commit_masked.argtypes = [vp, vp, i32, ctypes.POINTER(u32)]
     lib.sja_get_awards.argtypes = [vp, vp, i32]
     lib.sja_get_state.argtypes = [vp, vp, vp, i32]
@@ -252,6 +254,20 @@ class Sja:
             raise ValueError("deadline_ms needs one entry per loaded job")
         self._check(self._lib.sja_set_window_options(self._h, 1 if late_start else 0, p,
                                                      MEM_HOST if space is None else space))
+
+    # -- sja_load_power / sja_advertise_power_caps
+    def load_power(self, off, power_W) -> None:
+        """Per-step power trace (u32, aligned with the loaded profile arrays) and the CSR offsets again."""
+        po, space, _k0 = _ptr_space(off, None, np.uint64)
+        pp, space, _k1 = _ptr_space(power_W, space, np.uint32)
+        self._check(self._lib.sja_load_power(self._h, po, pp, space))
+
+    def advertise_power_caps(self, cap_W) -> None:
+        """One cap per gap of the advertised batch (u32, numpy or CUDA tensor), or None."""
+        p, space, keep = _ptr_space(cap_W, None, np.uint32)
+        if keep is not None and int(keep.shape[0]) != self.n_gaps:
+            raise ValueError("cap_W needs one entry per advertised gap")
+        self._check(self._lib.sja_advertise_power_caps(self._h, p, MEM_HOST if space is None else space))
 
     # -- sja_update_profile
     def update_profile(self, job: int, dur_ms, mem_MiB) -> None:

@@ -18,6 +18,7 @@
 #include "sja_scan.cuh"
 #include "sja_tile.cuh"
 #include "sja_update.cuh"
+#include "sja_power.cuh"
 
 using namespace sja;
 
@@ -65,6 +66,8 @@ struct sja_ctx {
     uint32_t tau_min = 0, tau_max = 0xFFFFFFFFu;   // subjob duration thresholds for select
     bool late_start = false, have_deadline = false;   // window options (sja_set_window_options)
     DevBuf deadline;
+    bool have_power = false, have_caps = false;        // power envelope (sja_load_power, sja_advertise_power_caps)
+    DevBuf PW, caps, st_power;
     DevBuf upd_d, upd_m, upd_scratch, upd_status;   // sja_update_profile: staged inputs, segment values, verdict
     bool gaps_sorted = false;          // sgaps is ordered by (C, T); else it is the caller's order
     uint32_t n_classes = 0;            // distinct capacities of the batch (valid when sorted)
@@ -238,6 +241,8 @@ JobView job_view(const sja_ctx* c) {
     v.tau_max = c->tau_max;
     v.deadline = c->have_deadline ? c->deadline.as<uint32_t>() : nullptr;
     v.late_start = c->late_start ? 1u : 0u;
+    v.PW = (c->have_power && c->have_caps) ? c->PW.as<uint2>() : nullptr;
+    v.caps = (c->have_power && c->have_caps) ? c->caps.as<uint32_t>() : nullptr;
     v.J = c->J;
     return v;
 }
@@ -334,7 +339,7 @@ SelectPlan plan_select(const sja_ctx* c, uint32_t pflags) {
     // through each capacity class is pure latency and the independent per-pair searches finish sooner.
     const bool tiny = (uint64_t)c->J * c->G < (1ull << 16);
     // with a window option the usable window differs from pair to pair: only the search kernel does that
-    const bool per_pair_window = c->late_start || c->have_deadline;
+    const bool per_pair_window = c->late_start || c->have_deadline || (c->have_power && c->have_caps);
     const bool sorted_ok = !(pflags & SJA_FLAG_FORCE_SEARCH) && !per_pair_window && c->gaps_sorted && (forced || !tiny) &&
                            c->n_classes <= std::max<uint32_t>(64u, c->G / 16u);
     p.kernel = !sorted_ok ? SEL_SEARCH : (pflags & SJA_FLAG_FORCE_MERGE) ? SEL_MERGE : SEL_TILE;
@@ -402,7 +407,8 @@ void run_commit(sja_ctx* c, uint32_t* blocked, const uint8_t* accept = nullptr) 
         c->flags.as<uint32_t>(), blocked, accept, c->late_start ? 1u : 0u);
     commit_refresh_kernel<<<(uint32_t)(((uint64_t)G * 32 + 255) / 256), 256, 0, c->stream>>>(
         c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(), G, c->boff.as<uint64_t>(), c->pb.as<uint32_t>(),
-        c->A.as<uint4>(), c->B.as<uint2>(), c->jobwin.as<unsigned long long>());
+        c->A.as<uint4>(), c->B.as<uint2>(), c->jobwin.as<unsigned long long>(),
+        c->have_power ? c->PW.as<uint2>() : nullptr);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -491,7 +497,7 @@ sja_status sja_destroy(sja_ctx* c) {
     cudaStreamSynchronize(c->stream);
     DevBuf* bufs[] = {&c->st_off, &c->st_d, &c->st_m, &c->st_s, &c->st_p, &c->p, &c->ready, &c->pb, &c->Dp,
                       &c->Wp, &c->wait, &c->prio, &c->nbj, &c->cta_tot, &c->cta_base, &c->boff, &c->boff_next, &c->A, &c->B, &c->jobwin,
-                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->deadline, &c->upd_d, &c->upd_m, &c->upd_scratch, &c->upd_status, &c->awards, &c->widx, &c->partial,
+                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->deadline, &c->PW, &c->caps, &c->st_power, &c->upd_d, &c->upd_m, &c->upd_scratch, &c->upd_status, &c->awards, &c->widx, &c->partial,
                       &c->winners};
     for (DevBuf* b : bufs) release(*b);
     for (ProfSpan& s : c->spans) { cudaEventDestroy(s.a); cudaEventDestroy(s.b); }
@@ -696,7 +702,8 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
         TRY(read_verdict());                     // a rejected load has touched nothing of the previous one
         // from here on the previous load is replaced
         c->loaded = false;
-        c->have_deadline = false;                // deadlines belong to the jobs of a load
+        c->have_deadline = false;                // deadlines and power traces belong to the jobs of a load
+        c->have_power = false;
         c->advertised = c->selected = c->committed = false;
         if (flags & FLAG_NEED_ROWS) {
             // the table outgrew the buffers and the kernels stood still: size them and run again
@@ -709,6 +716,7 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
         TRY(read_verdict());
         c->loaded = false;
         c->have_deadline = false;
+        c->have_power = false;
         c->advertised = c->selected = c->committed = false;
         TRY(reserve_state());
         TRY(launch_state_and_scan());
@@ -774,6 +782,7 @@ sja_status sja_advertise(sja_ctx* c, uint32_t G, const sja_gap* gaps, sja_memspa
     // the class count steers the kernel choice of sja_select, and a host buffer may be reused on return
     CU(cudaStreamSynchronize(c->stream));
     c->gaps_sorted = sortable;
+    c->have_caps = false;      // power caps belong to a batch
     c->n_classes = sortable ? c->h_words[4] : 0;
     c->G = G;
     c->advertised = true;
@@ -981,6 +990,58 @@ sja_status sja_update_profile(sja_ctx* c, uint32_t job, uint32_t n_steps, const 
         return fail(c, SJA_ERR_OVERFLOW, "sja_update_profile: total duration >= 2^32 ms or total work >= 2^63 for job %u", job);
     c->load_flags |= c->h_words[1] & (FLAG_OVF_FAIR | FLAG_OVF_SLA);
     c->selected = false;   // awards chosen from the old profile must not be committed
+    return SJA_OK;
+}
+
+sja_status sja_load_power(sja_ctx* c, const uint64_t* off, const uint32_t* power_W, sja_memspace where) {
+    TRY(check_ctx(c));
+    if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_load_power: bad memspace");
+    if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_load_power before sja_load_profiles");
+    if (!off || (c->N > 0 && !power_W)) return fail(c, SJA_ERR_INVALID_ARG, "sja_load_power: off / power_W is NULL");
+    DeviceGuard guard(c->device);
+    const uint64_t* d_off = off;
+    const uint32_t* d_pw = power_W;
+    if (where == SJA_MEM_HOST) {
+        if (off[0] != 0 || off[c->J] != c->N)
+            return fail(c, SJA_ERR_BAD_PROFILE, "sja_load_power: off does not describe the loaded profiles");
+        TRY(reserve(c, c->st_off, (size_t)(c->J + 1) * 8));
+        TRY(reserve(c, c->st_power, (size_t)c->N * 4 + 16));
+        TRY(copy_in(c, c->st_off.p, off, (size_t)(c->J + 1) * 8, where));
+        TRY(copy_in(c, c->st_power.p, power_W, (size_t)c->N * 4, where));
+        d_off = c->st_off.as<uint64_t>();
+        d_pw = c->st_power.as<uint32_t>();
+    }
+    TRY(reserve(c, c->PW, (size_t)c->n_rows * 8 + 16));
+    c->have_power = false;
+    c->selected = false;       // awards chosen without the trace must not be committed with it
+    scan_power_kernel<<<(uint32_t)(((uint64_t)c->J * 32 + 255) / 256), 256, 0, c->stream>>>(
+        d_off, d_pw, c->J, c->boff.as<uint64_t>(), c->pb.as<uint32_t>(), c->p.as<uint32_t>(), c->B.as<uint2>(),
+        c->PW.as<uint2>(), c->flags.as<uint32_t>());
+    CU(cudaGetLastError());
+    uint32_t flags = 0;
+    TRY(read_flags(c, &flags));
+    if (flags & FLAG_BAD_PROFILE) {
+        CU(cudaMemsetAsync(c->flags.p, 0, 4, c->stream));   // the bit is only ever set by a load and reported at once
+        return fail(c, SJA_ERR_BAD_PROFILE, "sja_load_power: off does not describe the loaded profiles");
+    }
+    c->have_power = true;
+    return SJA_OK;
+}
+
+sja_status sja_advertise_power_caps(sja_ctx* c, const uint32_t* cap_W, sja_memspace where) {
+    TRY(check_ctx(c));
+    if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_advertise_power_caps: bad memspace");
+    if (!c->advertised) return fail(c, SJA_ERR_STATE, "sja_advertise_power_caps before sja_advertise");
+    DeviceGuard guard(c->device);
+    if (cap_W) {
+        TRY(reserve(c, c->caps, (size_t)c->G * 4));
+        TRY(copy_in(c, c->caps.p, cap_W, (size_t)c->G * 4, where));
+        if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));   // the caller may reuse its buffer
+    }
+    c->have_caps = cap_W != nullptr;
+    c->selected = false;       // awards chosen under other caps must not be committed
     return SJA_OK;
 }
 

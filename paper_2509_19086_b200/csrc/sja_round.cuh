@@ -22,6 +22,8 @@ struct JobView {
     uint32_t tau_min, tau_max;  // subjob duration thresholds (Section 4.3, item 5); 0 / 0xFFFFFFFF = off
     const uint32_t* deadline;   // may be nullptr; per job, 0xFFFFFFFF = none (Section 4.4, item 2)
     uint32_t late_start;        // non-zero: a job that turns ready inside a window may begin then
+    const uint2* PW;            // may be nullptr; per row {running max, segment max} of the power trace (Section 4.4, item 1)
+    const uint32_t* caps;       // may be nullptr; per gap (caller's index) power cap, 0xFFFFFFFF = none
     uint32_t J;
 };
 
@@ -93,6 +95,9 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
         for (uint32_t gi = 0; gi < gt; ++gi) {
             const uint4 gq = __ldg(reinterpret_cast<const uint4*>(gaps) + g0 + gi);
             const uint32_t start = gq.y, C = gq.w;
+            // power cap of the offer (the caller's gap index travels in the slice field)
+            const uint32_t cap = (jv.PW && jv.caps) ? __ldg(jv.caps + gq.x) : 0xFFFFFFFFu;
+            const bool capped = cap != 0xFFFFFFFFu;
             // the window this pair sees: what is left of the gap once the job can begin, cut at its deadline
             uint32_t T = gq.z, begin = start;
             bool eligible = n != 0;
@@ -115,7 +120,9 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
                 while (lo < hi) {
                     const uint32_t mid = (lo + hi) >> 1;
                     const uint2 r = sDM[mid * SEARCH_THREADS];
-                    if (r.x <= T && r.y <= C) lo = mid + 1; else hi = mid;
+                    bool ok = r.x <= T && r.y <= C;
+                    if (ok && capped) ok = __ldg(&jv.PW[base + mid].x) <= cap;
+                    if (ok) lo = mid + 1; else hi = mid;
                 }
                 if (lo == ns && ns < n) {
                     // every staged row fits: gallop on through global memory (rows ns, ns + 1, ns + 3, ...)
@@ -124,13 +131,17 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
                     for (uint32_t idx = ns;;) {
                         if (idx >= n) { hi = n; break; }
                         const uint4 r = __ldg(jv.A + base + idx);
-                        if (r.x - Dp <= T && r.y <= C) { lo = idx + 1; idx += step; step <<= 1; }
+                        bool ok = r.x - Dp <= T && r.y <= C;
+                        if (ok && capped) ok = __ldg(&jv.PW[base + idx].x) <= cap;
+                        if (ok) { lo = idx + 1; idx += step; step <<= 1; }
                         else { hi = idx; break; }
                     }
                     while (lo < hi) {
                         const uint32_t mid = lo + ((hi - lo) >> 1);
                         const uint4 r = __ldg(jv.A + base + mid);
-                        if (r.x - Dp <= T && r.y <= C) lo = mid + 1; else hi = mid;
+                        bool ok = r.x - Dp <= T && r.y <= C;
+                        if (ok && capped) ok = __ldg(&jv.PW[base + mid].x) <= cap;
+                        if (ok) lo = mid + 1; else hi = mid;
                     }
                 }
                 cnt = lo;
@@ -274,7 +285,7 @@ __global__ void __launch_bounds__(256) commit_apply_kernel(
 __global__ void __launch_bounds__(256) commit_refresh_kernel(
     const uint32_t* __restrict__ winners, const uint32_t* __restrict__ n_granted, uint32_t G,
     const uint64_t* __restrict__ boff, const uint32_t* __restrict__ pb, uint4* __restrict__ A,
-    const uint2* __restrict__ B, unsigned long long* __restrict__ jobwin) {
+    const uint2* __restrict__ B, unsigned long long* __restrict__ jobwin, uint2* __restrict__ PW) {
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (w >= G || w >= *n_granted) return;
@@ -299,6 +310,27 @@ __global__ void __launch_bounds__(256) commit_refresh_kernel(
         const uint32_t last = min(31u, n - 1 - c);
         const uint32_t v_last = __shfl_sync(0xFFFFFFFFu, v, last);
         const uint32_t old_last = __shfl_sync(0xFFFFFFFFu, old, last);
+        if (v_last == old_last) break;
+        carry = v_last;
+    }
+    if (!PW) return;
+    // the same for the running maximum of the power trace
+    carry = 0;
+    for (uint32_t c = 0; c < n; c += 32) {
+        const uint32_t idx = c + lane;
+        const bool ok = idx < n;
+        const uint2 pw = ok ? PW[base + idx] : make_uint2(0u, 0u);
+        uint32_t v = pw.y;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, v, o);
+            if (lane >= (uint32_t)o) v = max(v, y);
+        }
+        v = max(v, carry);
+        if (ok && pw.x != v) PW[base + idx].x = v;
+        const uint32_t last = min(31u, n - 1 - c);
+        const uint32_t v_last = __shfl_sync(0xFFFFFFFFu, v, last);
+        const uint32_t old_last = __shfl_sync(0xFFFFFFFFu, pw.x, last);
         if (v_last == old_last) break;
         carry = v_last;
     }
