@@ -260,6 +260,9 @@ def main():
                     help="time sja_round_reauction (select + commit repeated for orphaned gaps) instead of one select + commit")
     ap.add_argument("--window-options", action="store_true",
                     help="late start inside a gap and per-job deadlines (ready + 2000..8000 ms): per-pair search path")
+    ap.add_argument("--sharded", action="store_true",
+                    help="with --gpus N: ONE scheduler over N GPUs (jobs sharded, gaps replicated, one all-gather of a "
+                         "32-byte bid per gap and GPU per round) instead of N independent replicas; strong scaling")
     ap.add_argument("--power-caps", action="store_true",
                     help="second resource envelope: a per-step power trace (50 W + 350 W x mem / 80 GiB + noise) loaded "
                          "with every load and a cap of 100..400 W per gap: per-pair search path")
@@ -301,10 +304,19 @@ def main():
         dist = dist_mod
         dist.init_process_group("nccl", device_id=device)
 
-    # replicas: every rank runs an independent scheduler instance on its own seeded workload
-    my_spec = replicas.replica_spec(spec, rank)
+    # replicas: every rank runs an independent scheduler instance on its own seeded workload;
+    # sharded: every rank holds a contiguous range of the jobs of the one published workload
+    my_spec = spec if args.sharded else replicas.replica_spec(spec, rank)
     prof = wl.make_profiles(my_spec, threads=max(1, (os.cpu_count() or 8) // max(1, world)))
     gaps = wl.make_gaps(my_spec)
+    shard_lo = 0
+    if args.sharded:
+        if args.reauction or args.streaming or args.window_options or args.power_caps:
+            raise SystemExit("--sharded times the plain round only")
+        from paper_2509_19086_b200 import sharded
+        global_jobs = prof.n_jobs
+        shard_lo, shard_hi = sharded.shard_bounds(global_jobs, world, rank)
+        prof = sharded.shard_profiles(prof, shard_lo, shard_hi)
     J, G, N = prof.n_jobs, int(gaps.shape[0]), prof.n_steps
     pairs = J * G
 
@@ -373,9 +385,18 @@ def main():
         aw = ctx.select(my_spec.policy, flags=args.flags, out="host")
         return aw, ctx.commit(want_count=True)
 
+    sched = None
+    if args.sharded:
+        sched = sharded.ShardedScheduler(ctx, shard_lo, rank, world, dist, device)
+
     def step_device():
         ctx.load_profiles(dev["off"], dev["d"], dev["m"], dev["s"], dev["ready"],
                           wait_ms=dev.get("wait"), prio=dev.get("prio"))
+        if sched is not None:
+            # advertise + select on the shard, one all-gather of the bids, fold, commit what this shard won
+            sched.round(dev_gaps, my_spec.policy, flags=args.flags)
+            launches[0] += KERNELS_PER_STEP - one_tile_saving + 2
+            return
         if args.window_options:
             ctx.set_window_options(True, dev_deadline)
         if args.power_caps:
@@ -394,6 +415,9 @@ def main():
     def step_e2e():
         ctx.load_profiles(pinned["off"], pinned["d"], pinned["m"], pinned["s"], pinned["ready"],
                           wait_ms=pinned.get("wait"), prio=pinned.get("prio"))
+        if sched is not None:
+            glob, n = sched.round(gaps_pinned, my_spec.policy, flags=args.flags, want_count=True)
+            return glob.cpu(), n
         if args.window_options:
             ctx.set_window_options(True, pinned["deadline"])
         ctx.advertise(gaps_pinned)
@@ -502,14 +526,16 @@ def main():
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "strong" if args.sharded else "weak",
         "vs_baseline": None, "dtype": "u32/u64", "data": "synthetic",
         "config": {"workload": my_spec.name if rank == 0 else spec.name, "jobs": J, "gaps": G, "steps_total": N,
-                   "boundary_rows": n_rows, "policy": POLICY_NAMES[spec.policy], "parallelism": f"replicas x{world}",
+                   "boundary_rows": n_rows, "policy": POLICY_NAMES[spec.policy], "parallelism": f"jobs sharded x{world}, one bid all-gather per round" if args.sharded else f"replicas x{world}",
                    "l2": "inputs larger than L2 (profile arrays re-read from HBM every step)"
                    if prof.raw_bytes() > 200e6 else "inputs smaller than L2",
                    "flags": args.flags, "reauction": bool(args.reauction),
                    "window_options": bool(args.window_options), "power_caps": bool(args.power_caps),
+                   "jobs_all_ranks": global_jobs if args.sharded else J * world,
                    "streaming": "load once, one advertise/select/commit round per step" if args.streaming else False},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

@@ -262,6 +262,34 @@ sja_status sja_set_duration_bounds(sja_ctx* ctx, uint32_t tau_min_ms, uint32_t t
 sja_status sja_set_window_options(sja_ctx* ctx, uint32_t late_start, const uint32_t* deadline_ms, sja_memspace where);
 
 /*
+ * One scheduler over several GPUs (the paper has no counterpart; the round itself is Section 3.5).  The jobs
+ * are sharded over the GPUs in contiguous id ranges, the gaps are advertised on every GPU, every GPU selects
+ * among its own jobs, and the only exchange of a round is one bid per gap and GPU:
+ *
+ *     sja_select(...)                                   on every GPU, over its shard
+ *     sja_get_bids(ctx, job_base, rank, bids, ...)      its winner per gap with the totally ordered policy key
+ *     all-gather of the G bids of every GPU             by the caller (e.g. NCCL), rank r at all[r * G]
+ *     sja_reduce_bids(ctx, n, rank, all, accept, ...)   global winner per gap: largest key, lowest global job id
+ *     sja_commit_masked(ctx, accept, ...)               the owner of a winner grants; the others grant nothing
+ *
+ * The result equals that of one GPU holding all jobs: the per-gap rule is the same argmax, and a job that won
+ * several gaps resolves them on its owner.  job_base is the global id of the shard's first job; `rank` is
+ * carried in the bids so that sja_reduce_bids can tell whose winner a gap's is.  sja_get_bids needs a select
+ * that has not been committed; sja_reduce_bids needs the advertised batch (G).  global_awards may be NULL;
+ * otherwise it receives the winning award per gap with global job ids (granted = 0).
+ */
+typedef struct {
+    uint64_t key;      /* 0 = no interested job in this shard; else larger wins */
+    uint32_t job;      /* global job id (job_base + local id), or SJA_NO_JOB */
+    uint32_t end_step, dur_ms;
+    uint32_t rank;     /* the GPU that made the bid */
+    uint64_t score;
+} sja_bid;             /* 32 bytes */
+sja_status sja_get_bids(sja_ctx* ctx, uint32_t job_base, uint32_t rank, sja_bid* out, sja_memspace where);
+sja_status sja_reduce_bids(sja_ctx* ctx, uint32_t n_ranks, uint32_t my_rank, const sja_bid* all, uint8_t* accept,
+                           sja_award* global_awards, sja_memspace where);
+
+/*
  * Power envelope, a second resource channel beside memory (Section 4.4, item 1: offers carry power caps,
  * subjobs answer with predicted power traces, and admission keeps max_t P(t) <= power_cap; as with memory,
  * the tolerated risk lives in the trace, which is a risk-adjusted envelope).

@@ -26,11 +26,13 @@ FLAG_FORCE_TILE = 4
 NO_JOB = 0xFFFFFFFF
 
 GAP_DTYPE = np.dtype([("slice", "<u4"), ("start_ms", "<u4"), ("T_ms", "<u4"), ("C_MiB", "<u4")])
+BID_DTYPE = np.dtype([("key", "<u8"), ("job", "<u4"), ("end_step", "<u4"), ("dur_ms", "<u4"), ("rank", "<u4"),
+                      ("score", "<u8")])
 AWARD_DTYPE = np.dtype([("job", "<u4"), ("end_step", "<u4"), ("dur_ms", "<u4"), ("granted", "<u4"),
                         ("score", "<u8")])
 
 EXPORTS = [
-    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit", "sja_commit_masked", "sja_round_reauction", "sja_set_duration_bounds", "sja_set_window_options", "sja_update_profile", "sja_load_power", "sja_advertise_power_caps",
+    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit", "sja_commit_masked", "sja_round_reauction", "sja_set_duration_bounds", "sja_set_window_options", "sja_update_profile", "sja_load_power", "sja_advertise_power_caps", "sja_get_bids", "sja_reduce_bids",
     "sja_get_awards", "sja_get_state", "sja_scan_size", "sja_get_scan", "sja_profile_enable",
     "sja_profile_read", "sja_last_error",
 ]
@@ -81,6 +83,8 @@ def load_library() -> ctypes.CDLL:
     lib.sja_set_window_options.argtypes = [vp, u32, vp, i32]
     lib.sja_update_profile.argtypes = [vp, u32, u32, vp, vp, i32]
     lib.sja_load_power.argtypes = [vp, vp, vp, i32]
+    lib.sja_get_bids.argtypes = [vp, u32, u32, vp, i32]
+    lib.sja_reduce_bids.argtypes = [vp, u32, u32, vp, vp, vp, i32]
     lib.sja_advertise_power_caps.argtypes = [vp, vp, i32]
     lib.sja_commit_masked.argtypes = [vp, vp, i32, ctypes.POINTER(u32)]
     lib.sja_get_awards.argtypes = [vp, vp, i32]
@@ -226,9 +230,13 @@ class Sja:
         return None
 
     # -- sja_commit_masked
-    def commit_masked(self, accept) -> int:
-        """sja_commit_masked: ``accept`` is a u8 array (numpy or CUDA tensor) with one entry per gap."""
+    def commit_masked(self, accept, want_count: bool = True) -> Optional[int]:
+        """sja_commit_masked: ``accept`` is a u8 array (numpy or CUDA tensor) with one entry per gap.
+        Without ``want_count`` the call does not wait for the GPU and returns None."""
         p, space, _keep = _ptr_space(accept, None, np.uint8)
+        if not want_count:
+            self._check(self._lib.sja_commit_masked(self._h, p, space, None))
+            return None
         n = ctypes.c_uint32()
         self._check(self._lib.sja_commit_masked(self._h, p, space, ctypes.byref(n)))
         return int(n.value)
@@ -254,6 +262,35 @@ class Sja:
             raise ValueError("deadline_ms needs one entry per loaded job")
         self._check(self._lib.sja_set_window_options(self._h, 1 if late_start else 0, p,
                                                      MEM_HOST if space is None else space))
+
+    # -- sja_get_bids / sja_reduce_bids (one scheduler over several GPUs)
+    def get_bids(self, job_base: int, rank: int, out=None):
+        """Bids of this shard for the advertised gaps: a numpy BID_DTYPE array, or written to the CUDA uint8
+        tensor ``out`` (32 * G bytes)."""
+        if out is None:
+            arr = np.empty(self.n_gaps, dtype=BID_DTYPE)
+            self._check(self._lib.sja_get_bids(self._h, int(job_base), int(rank), arr.ctypes.data, MEM_HOST))
+            return arr
+        p, space, _ = _ptr_space(out, None)
+        self._check(self._lib.sja_get_bids(self._h, int(job_base), int(rank), p, space))
+        return out
+
+    def reduce_bids(self, n_ranks: int, my_rank: int, all_bids, accept=None, global_awards=None):
+        """Fold the gathered bids (rank r at ``all_bids[r * G]``).  Host arrays in: returns ``(accept u8[G],
+        awards AWARD_DTYPE[G])``.  CUDA tensors in: ``accept`` (G bytes) and ``global_awards`` (24 * G bytes,
+        may be None) are CUDA uint8 tensors that receive the result."""
+        if _is_torch(all_bids):
+            p, space, _ = _ptr_space(all_bids, None)
+            pa, space, _ = _ptr_space(accept, space)
+            pg, space, _ = _ptr_space(global_awards, space)
+            self._check(self._lib.sja_reduce_bids(self._h, int(n_ranks), int(my_rank), p, pa, pg, space))
+            return accept, global_awards
+        all_bids = np.ascontiguousarray(all_bids, dtype=BID_DTYPE)
+        acc = np.empty(self.n_gaps, dtype=np.uint8)
+        aw = np.empty(self.n_gaps, dtype=AWARD_DTYPE)
+        self._check(self._lib.sja_reduce_bids(self._h, int(n_ranks), int(my_rank), all_bids.ctypes.data,
+                                              acc.ctypes.data, aw.ctypes.data, MEM_HOST))
+        return acc, aw
 
     # -- sja_load_power / sja_advertise_power_caps
     def load_power(self, off, power_W) -> None:

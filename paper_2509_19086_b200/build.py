@@ -8,7 +8,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libsja.so")
 SOURCES = ["sja.cu"]
-HEADERS = ["sja_common.cuh", "sja_prep.cuh", "sja_scan.cuh", "sja_round.cuh", "sja_tile.cuh", "sja_update.cuh", "sja_power.cuh", os.path.join("..", "..", "include", "sja.h")]
+HEADERS = ["sja_common.cuh", "sja_prep.cuh", "sja_scan.cuh", "sja_round.cuh", "sja_tile.cuh", "sja_update.cuh", "sja_power.cuh", "sja_shard.cuh", os.path.join("..", "..", "include", "sja.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -19,6 +19,7 @@
 #include "sja_tile.cuh"
 #include "sja_update.cuh"
 #include "sja_power.cuh"
+#include "sja_shard.cuh"
 
 using namespace sja;
 
@@ -68,6 +69,7 @@ struct sja_ctx {
     DevBuf deadline;
     bool have_power = false, have_caps = false;        // power envelope (sja_load_power, sja_advertise_power_caps)
     DevBuf PW, caps, st_power;
+    DevBuf st_bids, st_accept, st_global;              // sharded rounds: staging for host-side callers
     DevBuf upd_d, upd_m, upd_scratch, upd_status;   // sja_update_profile: staged inputs, segment values, verdict
     bool gaps_sorted = false;          // sgaps is ordered by (C, T); else it is the caller's order
     uint32_t n_classes = 0;            // distinct capacities of the batch (valid when sorted)
@@ -497,7 +499,7 @@ sja_status sja_destroy(sja_ctx* c) {
     cudaStreamSynchronize(c->stream);
     DevBuf* bufs[] = {&c->st_off, &c->st_d, &c->st_m, &c->st_s, &c->st_p, &c->p, &c->ready, &c->pb, &c->Dp,
                       &c->Wp, &c->wait, &c->prio, &c->nbj, &c->cta_tot, &c->cta_base, &c->boff, &c->boff_next, &c->A, &c->B, &c->jobwin,
-                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->deadline, &c->PW, &c->caps, &c->st_power, &c->upd_d, &c->upd_m, &c->upd_scratch, &c->upd_status, &c->awards, &c->widx, &c->partial,
+                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->deadline, &c->PW, &c->caps, &c->st_power, &c->st_bids, &c->st_accept, &c->st_global, &c->upd_d, &c->upd_m, &c->upd_scratch, &c->upd_status, &c->awards, &c->widx, &c->partial,
                       &c->winners};
     for (DevBuf* b : bufs) release(*b);
     for (ProfSpan& s : c->spans) { cudaEventDestroy(s.a); cudaEventDestroy(s.b); }
@@ -990,6 +992,66 @@ sja_status sja_update_profile(sja_ctx* c, uint32_t job, uint32_t n_steps, const 
         return fail(c, SJA_ERR_OVERFLOW, "sja_update_profile: total duration >= 2^32 ms or total work >= 2^63 for job %u", job);
     c->load_flags |= c->h_words[1] & (FLAG_OVF_FAIR | FLAG_OVF_SLA);
     c->selected = false;   // awards chosen from the old profile must not be committed
+    return SJA_OK;
+}
+
+static_assert(sizeof(sja_bid) == 32 && sizeof(Bid) == 32, "bid layout");
+
+sja_status sja_get_bids(sja_ctx* c, uint32_t job_base, uint32_t rank, sja_bid* out, sja_memspace where) {
+    TRY(check_ctx(c));
+    if (!out) return fail(c, SJA_ERR_INVALID_ARG, "sja_get_bids: out is NULL");
+    if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE) return fail(c, SJA_ERR_INVALID_ARG, "sja_get_bids: bad memspace");
+    if (!c->selected) return fail(c, SJA_ERR_STATE, "sja_get_bids without a preceding sja_select");
+    if ((uint64_t)job_base + c->J > 0xFFFFFFFFull)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_get_bids: job_base + J does not fit a 32-bit job id");
+    DeviceGuard guard(c->device);
+    Bid* d_out = reinterpret_cast<Bid*>(out);
+    if (where == SJA_MEM_HOST) {
+        TRY(reserve(c, c->st_bids, (size_t)c->G * sizeof(Bid)));
+        d_out = c->st_bids.as<Bid>();
+    }
+    make_bids_kernel<<<(c->G + 255) / 256, 256, 0, c->stream>>>(c->awards.as<Award>(), c->G, c->last_policy,
+                                                                c->have_prio ? c->prio.as<uint8_t>() : nullptr,
+                                                                job_base, rank, d_out);
+    CU(cudaGetLastError());
+    if (where == SJA_MEM_HOST) {
+        TRY(copy_out(c, out, d_out, (size_t)c->G * sizeof(Bid), where));
+        CU(cudaStreamSynchronize(c->stream));
+    }
+    return SJA_OK;
+}
+
+sja_status sja_reduce_bids(sja_ctx* c, uint32_t n_ranks, uint32_t my_rank, const sja_bid* all, uint8_t* accept,
+                           sja_award* global_awards, sja_memspace where) {
+    TRY(check_ctx(c));
+    if (!all || !accept || n_ranks == 0 || my_rank >= n_ranks)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_reduce_bids: bad arguments");
+    if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_reduce_bids: bad memspace");
+    if (!c->advertised) return fail(c, SJA_ERR_STATE, "sja_reduce_bids before sja_advertise");
+    DeviceGuard guard(c->device);
+    const uint32_t G = c->G;
+    const Bid* d_all = reinterpret_cast<const Bid*>(all);
+    uint8_t* d_accept = accept;
+    Award* d_global = reinterpret_cast<Award*>(global_awards);
+    if (where == SJA_MEM_HOST) {
+        TRY(reserve(c, c->st_bids, (size_t)n_ranks * G * sizeof(Bid)));
+        TRY(reserve(c, c->st_accept, G));
+        TRY(copy_in(c, c->st_bids.p, all, (size_t)n_ranks * G * sizeof(Bid), where));
+        d_all = c->st_bids.as<Bid>();
+        d_accept = c->st_accept.as<uint8_t>();
+        if (global_awards) {
+            TRY(reserve(c, c->st_global, (size_t)G * sizeof(Award)));
+            d_global = c->st_global.as<Award>();
+        }
+    }
+    reduce_bids_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(d_all, n_ranks, G, my_rank, d_accept, d_global);
+    CU(cudaGetLastError());
+    if (where == SJA_MEM_HOST) {
+        TRY(copy_out(c, accept, d_accept, G, where));
+        if (global_awards) TRY(copy_out(c, global_awards, d_global, (size_t)G * sizeof(Award), where));
+        CU(cudaStreamSynchronize(c->stream));
+    }
     return SJA_OK;
 }
 
