@@ -385,8 +385,13 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
         if (pl.kernel != SEL_SEARCH) {
             launch_sorted(pl.kernel, kind, dim3(n_chunks, splits), c->stream, jv, sgaps, G_act, per_split, partial);
         } else {
-            select_search_kernel<<<dim3(n_chunks, splits), SEARCH_THREADS, SEARCH_SMEM_BYTES, c->stream>>>(
-                jv, sgaps, G_act, per_split, kind, nullptr, 0, partial);
+            const bool opts = jv.late_start != 0u || jv.deadline != nullptr || jv.PW != nullptr;
+            if (opts)
+                select_search_kernel<true><<<dim3(n_chunks, splits), SEARCH_THREADS, SEARCH_SMEM_BYTES, c->stream>>>(
+                    jv, sgaps, G_act, per_split, kind, partial);
+            else
+                select_search_kernel<false><<<dim3(n_chunks, splits), SEARCH_THREADS, SEARCH_SMEM_BYTES, c->stream>>>(
+                    jv, sgaps, G_act, per_split, kind, partial);
         }
         finalize_awards_kernel<<<(uint32_t)(((uint64_t)G_act * FINALIZE_LANES + 255) / 256), 256, 0, c->stream>>>(
             jv, partial, n_chunks, sgaps, G_act, kind, c->awards.as<Award>(), c->widx.as<uint32_t>());
@@ -473,7 +478,9 @@ sja_status sja_create(sja_ctx** out, int device, void* cuda_stream) {
         if (cudaMemsetAsync(c->flags.p, 0, 4, c->stream) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         if (cudaFuncSetAttribute(scan_profiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  SCAN_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
-        if (cudaFuncSetAttribute(select_search_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(select_search_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 SEARCH_SMEM_BYTES) != cudaSuccess ||
+            cudaFuncSetAttribute(select_search_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  SEARCH_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         if (sorted_smem_attr<0, false>() != cudaSuccess || sorted_smem_attr<1, false>() != cudaSuccess ||
             sorted_smem_attr<2, false>() != cudaSuccess || sorted_smem_attr<3, false>() != cudaSuccess ||

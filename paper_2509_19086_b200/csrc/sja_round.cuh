@@ -47,26 +47,32 @@ __device__ __forceinline__ uint32_t policy_factor(const JobView& jv, uint32_t ki
 // only longer answers continue in global memory.
 constexpr int SEARCH_THREADS = 256;
 constexpr int SEARCH_GT = 64;   // gaps per staging tile
-constexpr int SEARCH_ROWS = 16; // boundary rows staged per job
-constexpr int SEARCH_SMEM_BYTES = 2 * SEARCH_ROWS * SEARCH_THREADS * 8;   // {D - Dp, M} and payload, [row][thread]
+#ifndef SJA_SEARCH_ROWS
+#define SJA_SEARCH_ROWS 16
+#endif
+#ifndef SJA_SEARCH_PAY_ROWS
+#define SJA_SEARCH_PAY_ROWS 16
+#endif
+constexpr int SEARCH_ROWS = SJA_SEARCH_ROWS;          // boundary rows staged per job as {D - Dp, M} (a power of two)
+constexpr int SEARCH_PAY_ROWS = SJA_SEARCH_PAY_ROWS;  // of which the first ones also with their policy payload
+constexpr int SEARCH_SMEM_BYTES = (SEARCH_ROWS + SEARCH_PAY_ROWS) * SEARCH_THREADS * 8;   // [row][thread]
+static_assert((SEARCH_ROWS & (SEARCH_ROWS - 1)) == 0 && SEARCH_PAY_ROWS <= SEARCH_ROWS, "staging shape");
 
+// OPTS: a window option or a power cap is in force (compiled out otherwise).
+template <bool OPTS>
 __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
     JobView jv, const Gap* __restrict__ gaps, uint32_t G, uint32_t gaps_per_split, uint32_t kind,
-    const uint32_t* __restrict__ job_list, uint32_t n_list, Partial* __restrict__ partial_out) {
+    Partial* __restrict__ partial_out) {
     __shared__ Partial stage[SEARCH_GT][SEARCH_THREADS / 32];
     extern __shared__ __align__(16) uint2 search_rows[];
     uint2* sDM = search_rows + threadIdx.x;                                     // row r of this thread: sDM[r * THREADS]
     uint2* sPay = search_rows + SEARCH_ROWS * SEARCH_THREADS + threadIdx.x;     // its policy payload (work or peak)
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
-    const uint32_t slot = blockIdx.x * SEARCH_THREADS + threadIdx.x;
-    // the jobs of this launch: either all jobs (job_list == nullptr) or a list of job ids
-    const uint32_t n_jobs = job_list ? n_list : jv.J;
-    uint32_t j = SJA_NO_JOB_DEV;
-    if (slot < n_jobs) j = job_list ? job_list[slot] : slot;
+    const uint32_t j = blockIdx.x * SEARCH_THREADS + threadIdx.x;
 
     uint64_t base = 0, Wp = 0;
-    uint32_t n = 0, Dp = 0, ready = 0, factor = 0, deadline = 0xFFFFFFFFu;
-    if (j != SJA_NO_JOB_DEV) {
+    uint32_t n = 0, Dp = 0, ready = 0xFFFFFFFFu, factor = 0, deadline = 0xFFFFFFFFu;
+    if (j < jv.J) {
         const uint64_t b0 = jv.boff[j], b1 = jv.boff[j + 1];
         const uint32_t pb = jv.pb[j];
         base = b0 + pb;
@@ -76,90 +82,101 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
         Wp = jv.Wp[j];
         ready = jv.ready[j];
         factor = policy_factor(jv, kind, j);
-        if (jv.deadline) deadline = jv.deadline[j];
+        if (OPTS && jv.deadline) deadline = jv.deadline[j];
     }
-    const bool late = jv.late_start != 0u;
+    const bool late = OPTS && jv.late_start != 0u;
     const uint32_t g_begin = blockIdx.y * gaps_per_split;
     const uint32_t g_end = min(G, g_begin + gaps_per_split);
-    const uint32_t ns = min(n, (uint32_t)SEARCH_ROWS);   // rows of this job held in shared memory
-    for (uint32_t r = 0; r < ns; ++r) {
-        const uint4 row = __ldg(jv.A + base + r);
-        const uint64_t pay = policy_payload(kind, row, Wp);
-        sDM[r * SEARCH_THREADS] = make_uint2(row.x - Dp, row.y);
-        sPay[r * SEARCH_THREADS] = make_uint2((uint32_t)pay, (uint32_t)(pay >> 32));
+    // The first rows of the job in shared memory; the slots beyond its last row hold a sentinel that no
+    // window admits (except T = C = 2^32-1, where the clamp below takes care), so every thread runs the
+    // same five probes.  Each thread reads back only what it wrote: no barrier needed.
+    const uint32_t ns = min(n, (uint32_t)SEARCH_ROWS);
+    for (uint32_t r = 0; r < (uint32_t)SEARCH_ROWS; ++r) {
+        uint2 dm = make_uint2(0xFFFFFFFFu, 0xFFFFFFFFu), pay = make_uint2(0u, 0u);
+        if (r < ns) {
+            const uint4 row = __ldg(jv.A + base + r);
+            const uint64_t pl = policy_payload(kind, row, Wp);
+            dm = make_uint2(row.x - Dp, row.y);
+            pay = make_uint2((uint32_t)pl, (uint32_t)(pl >> 32));
+        }
+        sDM[r * SEARCH_THREADS] = dm;
+        if (r < (uint32_t)SEARCH_PAY_ROWS) sPay[r * SEARCH_THREADS] = pay;
     }
-    // (each thread reads back only what it wrote: no barrier needed)
 
     for (uint32_t g0 = g_begin; g0 < g_end; g0 += SEARCH_GT) {
         const uint32_t gt = min((uint32_t)SEARCH_GT, g_end - g0);
         for (uint32_t gi = 0; gi < gt; ++gi) {
             const uint4 gq = __ldg(reinterpret_cast<const uint4*>(gaps) + g0 + gi);
             const uint32_t start = gq.y, C = gq.w;
-            // power cap of the offer (the caller's gap index travels in the slice field)
-            const uint32_t cap = (jv.PW && jv.caps) ? __ldg(jv.caps + gq.x) : 0xFFFFFFFFu;
-            const bool capped = cap != 0xFFFFFFFFu;
-            // the window this pair sees: what is left of the gap once the job can begin, cut at its deadline
-            uint32_t T = gq.z, begin = start;
+            uint32_t T = gq.z, cap = 0xFFFFFFFFu;
             bool eligible = n != 0;
-            if (start < ready) {
-                const uint32_t late_by = ready - start;
-                if (!late || late_by > T) eligible = false;
-                begin = ready;
-                T -= min(late_by, T);
-            }
-            if (deadline != 0xFFFFFFFFu) {
-                if (begin > deadline) eligible = false;
-                T = min(T, deadline - min(begin, deadline));
+            if (OPTS) {
+                // power cap of the offer (the caller's gap index travels in the slice field)
+                if (jv.PW && jv.caps) cap = __ldg(jv.caps + gq.x);
+                // the window this pair sees: what is left of the gap once the job can begin, cut at its deadline
+                uint32_t begin = start;
+                if (start < ready) {
+                    const uint32_t late_by = ready - start;
+                    if (!late || late_by > T) eligible = false;
+                    begin = ready;
+                    T -= min(late_by, T);
+                }
+                if (deadline != 0xFFFFFFFFu) {
+                    if (begin > deadline) eligible = false;
+                    T = min(T, deadline - min(begin, deadline));
+                }
+            } else {
+                eligible = eligible && start >= ready;
             }
             T = min(T, jv.tau_max);
-            uint32_t cnt = 0;
-            uint64_t key = 0;
-            if (eligible) {
-                // the staged rows first
-                uint32_t lo = 0, hi = ns;
+            const bool capped = OPTS && cap != 0xFFFFFFFFu;
+            // number of staged rows that satisfy all bounds (they form a prefix): five probes, no branches
+            auto fits = [&](uint32_t idx) -> bool {
+                const uint2 r = sDM[idx * SEARCH_THREADS];
+                bool ok = r.x <= T && r.y <= C;
+                if (OPTS && capped && ok && idx < ns) ok = __ldg(&jv.PW[base + idx].x) <= cap;
+                return ok;
+            };
+            uint32_t lo = 0;
+#pragma unroll
+            for (uint32_t s = SEARCH_ROWS / 2; s > 0; s >>= 1) lo += fits(lo + s - 1) ? s : 0u;
+            lo += fits(lo) ? 1u : 0u;
+            lo = eligible ? min(lo, ns) : 0u;
+            if (eligible && lo == ns && ns < n) {
+                // every staged row fits: gallop on through global memory (rows ns, ns + 1, ns + 3, ...)
+                uint32_t hi = n, step = 1;
+                for (uint32_t idx = ns;;) {
+                    if (idx >= n) { hi = n; break; }
+                    const uint4 r = __ldg(jv.A + base + idx);
+                    bool ok = r.x - Dp <= T && r.y <= C;
+                    if (OPTS && ok && capped) ok = __ldg(&jv.PW[base + idx].x) <= cap;
+                    if (ok) { lo = idx + 1; idx += step; step <<= 1; }
+                    else { hi = idx; break; }
+                }
                 while (lo < hi) {
-                    const uint32_t mid = (lo + hi) >> 1;
-                    const uint2 r = sDM[mid * SEARCH_THREADS];
-                    bool ok = r.x <= T && r.y <= C;
-                    if (ok && capped) ok = __ldg(&jv.PW[base + mid].x) <= cap;
+                    const uint32_t mid = lo + ((hi - lo) >> 1);
+                    const uint4 r = __ldg(jv.A + base + mid);
+                    bool ok = r.x - Dp <= T && r.y <= C;
+                    if (OPTS && ok && capped) ok = __ldg(&jv.PW[base + mid].x) <= cap;
                     if (ok) lo = mid + 1; else hi = mid;
                 }
-                if (lo == ns && ns < n) {
-                    // every staged row fits: gallop on through global memory (rows ns, ns + 1, ns + 3, ...)
-                    hi = n;
-                    uint32_t step = 1;
-                    for (uint32_t idx = ns;;) {
-                        if (idx >= n) { hi = n; break; }
-                        const uint4 r = __ldg(jv.A + base + idx);
-                        bool ok = r.x - Dp <= T && r.y <= C;
-                        if (ok && capped) ok = __ldg(&jv.PW[base + idx].x) <= cap;
-                        if (ok) { lo = idx + 1; idx += step; step <<= 1; }
-                        else { hi = idx; break; }
-                    }
-                    while (lo < hi) {
-                        const uint32_t mid = lo + ((hi - lo) >> 1);
-                        const uint4 r = __ldg(jv.A + base + mid);
-                        bool ok = r.x - Dp <= T && r.y <= C;
-                        if (ok && capped) ok = __ldg(&jv.PW[base + mid].x) <= cap;
-                        if (ok) lo = mid + 1; else hi = mid;
-                    }
+            }
+            uint32_t cnt = lo;
+            uint64_t key = 0;
+            if (cnt) {
+                uint32_t dur;
+                uint64_t pay;
+                if (cnt <= min(ns, (uint32_t)SEARCH_PAY_ROWS)) {
+                    dur = sDM[(cnt - 1) * SEARCH_THREADS].x;
+                    const uint2 pw = sPay[(cnt - 1) * SEARCH_THREADS];
+                    pay = pack64(pw.x, pw.y);
+                } else {
+                    const uint4 r = __ldg(jv.A + base + cnt - 1);
+                    dur = r.x - Dp;
+                    pay = policy_payload(kind, r, Wp);
                 }
-                cnt = lo;
-                if (cnt) {
-                    uint32_t dur;
-                    uint64_t pay;
-                    if (cnt <= ns) {
-                        dur = sDM[(cnt - 1) * SEARCH_THREADS].x;
-                        const uint2 pw = sPay[(cnt - 1) * SEARCH_THREADS];
-                        pay = pack64(pw.x, pw.y);
-                    } else {
-                        const uint4 r = __ldg(jv.A + base + cnt - 1);
-                        dur = r.x - Dp;
-                        pay = policy_payload(kind, r, Wp);
-                    }
-                    if (dur >= jv.tau_min) key = policy_key(kind, pay, factor);
-                    else cnt = 0;   // the longest fitting subjob is shorter than the minimum: decline
-                }
+                if (dur >= jv.tau_min) key = policy_key(kind, pay, factor);
+                else cnt = 0;   // the longest fitting subjob is shorter than the minimum: decline
             }
             const uint64_t mk = warp_max_u64(key);
             const uint32_t jmin = __reduce_min_sync(0xFFFFFFFFu, (key == mk && key != 0) ? j : 0xFFFFFFFFu);
