@@ -406,7 +406,9 @@ def main():
             ctx.advertise_power_caps(dev_caps)
         if args.reauction:
             _, passes = ctx.round_reauction(my_spec.policy, flags=args.flags)
-            launches[0] += 7 + 6 * passes      # per pass: select, finalize, 3 commit kernels, orphan compaction
+            # 5 load kernels, 4 advertise kernels (1 for a one-tile batch); per pass: select, finalize, 3 commit
+            # kernels, orphan compaction
+            launches[0] += 9 - one_tile_saving + 6 * passes
         else:
             ctx.select(my_spec.policy, flags=args.flags)
             ctx.commit(want_count=False)
