@@ -39,8 +39,8 @@ FALLBACK_HBM_GBS = 6650.0
 # scan_profiles_kernel_cfg2-jobs8192.md): dram__bytes_read.sum + dram__bytes_write.sum over 33 554 432 steps.
 # Traffic grows in proportion to the step count, so a full launch is this figure times N.  It is only reported
 # while csrc/sja_scan.cuh is the file the counters were taken from (first 16 hex digits of its sha256).
-NCU_SCAN_TRAFFIC_BYTES_PER_STEP = (273.041664e6 + 59.891712e6) / 33554432
-NCU_SCAN_SOURCE_SHA = "45fc1da5bae387db"
+NCU_SCAN_TRAFFIC_BYTES_PER_STEP = (273.045760e6 + 60.581120e6) / 33554432
+NCU_SCAN_SOURCE_SHA = "8b4aa85b4bb68d65"
 
 
 # Issue-slot roofline of the select kernel (it is bound by instruction issue, not HBM): warp instructions of one

@@ -59,6 +59,7 @@ struct sja_ctx {
     DevBuf p, ready, pb, Dp, Wp, wait, prio;          // per-job state and attributes
     DevBuf nbj, cta_tot, cta_base, boff, boff_next, A, B, jobwin;   // row counting scratch, boundary table
     DevBuf flags, counter, n_granted;                 // small device words
+    DevBuf long_list;                                 // jobs the scan of a load takes first
     uint32_t* h_words = nullptr;                      // pinned host scratch (8 x u64)
 
     // gaps / awards
@@ -472,10 +473,10 @@ sja_status sja_create(sja_ctx** out, int device, void* cuda_stream) {
         if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         c->n_sm = prop.multiProcessorCount;
         if (cudaMallocHost(reinterpret_cast<void**>(&c->h_words), 64) != cudaSuccess) { st = SJA_ERR_OOM; break; }
-        if ((st = reserve(c, c->flags, 4)) != SJA_OK) break;
+        if ((st = reserve(c, c->flags, 8)) != SJA_OK) break;   // [0] status bits, [1] long-job count of a load
         if ((st = reserve(c, c->counter, 4)) != SJA_OK) break;
         if ((st = reserve(c, c->n_granted, 4)) != SJA_OK) break;
-        if (cudaMemsetAsync(c->flags.p, 0, 4, c->stream) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
+        if (cudaMemsetAsync(c->flags.p, 0, 8, c->stream) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         if (cudaFuncSetAttribute(scan_profiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  SCAN_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         if (cudaFuncSetAttribute(select_search_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -506,7 +507,7 @@ sja_status sja_destroy(sja_ctx* c) {
     cudaStreamSynchronize(c->stream);
     DevBuf* bufs[] = {&c->st_off, &c->st_d, &c->st_m, &c->st_s, &c->st_p, &c->p, &c->ready, &c->pb, &c->Dp,
                       &c->Wp, &c->wait, &c->prio, &c->nbj, &c->cta_tot, &c->cta_base, &c->boff, &c->boff_next, &c->A, &c->B, &c->jobwin,
-                      &c->flags, &c->counter, &c->n_granted, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->deadline, &c->PW, &c->caps, &c->st_power, &c->st_bids, &c->st_accept, &c->st_global, &c->upd_d, &c->upd_m, &c->upd_scratch, &c->upd_status, &c->awards, &c->widx, &c->partial,
+                      &c->flags, &c->counter, &c->n_granted, &c->long_list, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->deadline, &c->PW, &c->caps, &c->st_power, &c->st_bids, &c->st_accept, &c->st_global, &c->upd_d, &c->upd_m, &c->upd_scratch, &c->upd_status, &c->awards, &c->widx, &c->partial,
                       &c->winners};
     for (DevBuf* b : bufs) release(*b);
     for (ProfSpan& s : c->spans) { cudaEventDestroy(s.a); cudaEventDestroy(s.b); }
@@ -619,12 +620,13 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
     const uint64_t cap_rows = speculate ? std::min<uint64_t>(c->A.cap / 16 - 1, c->B.cap / 8 - 2) : ~0ull;
 
     // pass 0: validate + count rows, then row offsets; nothing of the loaded state is touched yet
-    CU(cudaMemsetAsync(c->flags.p, 0, 4, c->stream));
+    TRY(reserve(c, c->long_list, (size_t)J * 4));
+    CU(cudaMemsetAsync(c->flags.p, 0, 8, c->stream));
     {
         ProfScope ps(c, CAT_PREP);
         count_boundaries_kernel<<<n_count_ctas, 256, 0, c->stream>>>(
             d_off, d_s, c->st_p.as<uint32_t>(), J, c->nbj.as<uint64_t>(), c->cta_tot.as<uint64_t>(),
-            c->flags.as<uint32_t>());
+            c->flags.as<uint32_t>(), c->long_list.as<uint32_t>());
         cta_offsets_kernel<<<1, 1024, 0, c->stream>>>(c->cta_tot.as<uint64_t>(), n_count_ctas,
                                                       c->cta_base.as<uint64_t>());
         row_offsets_kernel<<<(J + 255) / 256, 256, 0, c->stream>>>(c->nbj.as<uint64_t>(), c->cta_base.as<uint64_t>(),
@@ -682,6 +684,7 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
         a.J = J;
         a.counter = c->counter.as<uint32_t>();
         a.flags = c->flags.as<uint32_t>();
+        a.long_list = c->long_list.as<uint32_t>();
         if (!n_resolved || N > 0) {
             ProfScope ps(c, CAT_SCAN);
             const uint32_t ctas_per_sm = SCAN_CTAS_PER_SM;

@@ -19,6 +19,17 @@ enum : uint32_t {
 
 constexpr uint32_t SJA_NO_JOB_DEV = 0xFFFFFFFFu;
 
+// A job counts as "long" for the scan's hand-out order when it has more steps left than twice the
+// mean job length (and at least 8192): such jobs are scanned first, so that none of them starts late and
+// stretches the kernel's tail.  The row-counting kernel lists them, the scan kernel skips them later.
+#ifndef SJA_LONG_FACTOR
+#define SJA_LONG_FACTOR 2
+#endif
+__host__ __device__ inline uint64_t long_job_threshold(uint64_t n_steps, uint32_t n_jobs) {
+    const uint64_t above = (uint64_t)SJA_LONG_FACTOR * (n_steps / (n_jobs ? n_jobs : 1u));
+    return above > 8192ull ? above : 8192ull;
+}
+
 // One row of the boundary table, "search" half: everything a feasibility probe reads.
 // D = cumulative duration of [p_load, k), M = max m over [p_now, k), W = sum d*m over [p_load, k).
 // Stored as uint4 {D, M, W_lo, W_hi}.

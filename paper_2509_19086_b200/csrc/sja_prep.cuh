@@ -20,10 +20,11 @@ constexpr uint32_t COUNT_LONG = 0x80000000u;   // marker: job left to the whole-
 __global__ void __launch_bounds__(256) count_boundaries_kernel(
     const uint64_t* __restrict__ off, const uint32_t* __restrict__ sbits,
     const uint32_t* __restrict__ p0, uint32_t J, uint64_t* __restrict__ local_off,
-    uint64_t* __restrict__ cta_total, uint32_t* __restrict__ flags) {
+    uint64_t* __restrict__ cta_total, uint32_t* __restrict__ flags, uint32_t* __restrict__ long_list) {
     __shared__ uint32_t cnts[COUNT_JOBS_PER_CTA];
     __shared__ uint64_t warp_sums[COUNT_JOBS_PER_CTA / 32];
     const uint64_t N = __ldg(off + J);   // total step count
+    const uint64_t long_thresh = long_job_threshold(N, J);
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
     const uint32_t slot0 = wid * COUNT_JOBS_PER_WARP;              // first job slot of this warp in the CTA
     const uint32_t jbase = blockIdx.x * COUNT_JOBS_PER_CTA + slot0;
@@ -41,6 +42,8 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
             if (j == 0 && js != 0) bad = true;
             if (!bad) {
                 const uint64_t s = js + p, e = je;
+                // long jobs go on the list the scan works off first (flags[1] counts them)
+                if (sub == 0 && e - s > long_thresh) long_list[atomicAdd(flags + 1, 1u)] = j;
                 if (s < e && ((e - 1) >> 5) - (s >> 5) >= 256) {
                     cnt = COUNT_LONG;   // long job: counted by the whole warp below
                 } else if (s < e) {

@@ -45,7 +45,8 @@ struct ScanArgs {
     uint2* B;                // rows {k, S}
     uint32_t J;              // N = off[J] is read by the kernel
     uint32_t* counter;       // job hand-out counter (zeroed before launch)
-    uint32_t* flags;
+    uint32_t* flags;         // flags[0] status bits, flags[1] number of listed long jobs
+    const uint32_t* long_list;   // jobs to scan first (see long_job_threshold)
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
@@ -89,19 +90,30 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32, SCAN_CTAS_PER_SM) scan_profil
     // a load that was rejected by the validation pass, or whose table does not fit the buffers, is not scanned
     if (*reinterpret_cast<volatile const uint32_t*>(a.flags) & (FLAG_BAD_PROFILE | FLAG_NEED_ROWS)) return;
     const uint64_t N_total = __ldg(a.off + a.J);
+    const uint32_t n_long = a.flags[1];
+    const uint64_t long_thresh = long_job_threshold(N_total, a.J);
     const uint32_t lane_sw = (lane ^ ((lane >> 3) & 3u)) * 16u;   // swz(32 r + lane) * 16 - 512 r
     const uint32_t rd_x = (lane >> 1) & 3u;                        // swz(4 lane + r) = 4 lane + (r ^ rd_x)
 
     for (;;) {
-        uint32_t j = 0;
-        if (lane == 0) j = atomicAdd(a.counter, 1u);
-        j = __shfl_sync(0xFFFFFFFFu, j, 0);
-        if (j >= a.J) break;
+        // hand-out order: the listed long jobs first, then all jobs in id order (neighbouring warps stream
+        // neighbouring memory), the long ones skipped
+        uint32_t c = 0;
+        if (lane == 0) c = atomicAdd(a.counter, 1u);
+        c = __shfl_sync(0xFFFFFFFFu, c, 0);
+        uint32_t j;
+        if (c < n_long) {
+            j = __ldg(a.long_list + c);
+        } else {
+            j = c - n_long;
+            if (j >= a.J) break;
+        }
 
         const uint64_t js = __ldg(a.off + j), je = __ldg(a.off + j + 1);
         const uint32_t p = __ldg(a.p0 + j);
         const uint64_t s = js + p, e = je;
         if (s >= e) continue;
+        if (c >= n_long && e - s > long_thresh) continue;   // scanned in the first phase
         const uint64_t blk0 = s & ~31ull;
         const uint64_t nblk = (e - blk0 + (SCAN_BLK - 1)) / SCAN_BLK;
         const uint64_t out_base = __ldg(a.boff + j);
