@@ -104,7 +104,7 @@ typedef struct {
     uint32_t end_step; /* k: the subjob is steps [p_job, k) of the winner */
     uint32_t dur_ms;   /* its cumulative duration, <= T_ms */
     uint32_t granted;  /* 0 until sja_commit; then 1 iff the winner accepted this gap */
-    uint64_t score;    /* policy score of the winner (work for SLA) */
+    uint64_t score;    /* policy score of the winner (work for SLA, peak memory in MiB for TIGHT_FIT) */
 } sja_award;
 
 /* Device times (CUDA events on the context's stream) accumulated while profiling is on. */
@@ -130,7 +130,8 @@ sja_status sja_destroy(sja_ctx* ctx);
 /*
  * Load J job profiles (ragged CSR) and run the segmented scan (the "on demand"
  * segmentation of Section 3.9: the envelope may be refined, so the scan is re-runnable;
- * a new load replaces the previous one and clears any advertised gaps).
+ * a new load replaces the previous one and clears any advertised gaps, the deadlines of
+ * sja_set_window_options and the trace of sja_load_power).
  *   off        u64[J+1], off[0] = 0, non-decreasing; job j owns steps [off[j], off[j+1]).
  *   dur_ms     u32[N], N = off[J]         per-step duration
  *   mem_MiB    u32[N]                     per-step memory envelope
