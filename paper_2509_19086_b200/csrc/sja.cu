@@ -333,14 +333,16 @@ sja_status check_policy(sja_ctx* c, const sja_policy* policy, const char* who) {
 // awards and widx are written at the gaps' original indices.  `blocked` may be nullptr.
 struct SelectPlan { SelectKernel kernel; uint32_t jobs_per_cta, tile, n_chunks; };
 
-SelectPlan plan_select(const sja_ctx* c, uint32_t pflags) {
+SelectPlan plan_select(const sja_ctx* c, uint32_t pflags, uint32_t G_act) {
     SelectPlan p;
     // The tile and merge kernels need the (capacity, T) order and pay one restart per capacity
     // class; with very many classes (or an unsorted batch) the per-pair search is the better tool.
     const bool forced = (pflags & (SJA_FLAG_FORCE_MERGE | SJA_FLAG_FORCE_TILE)) != 0;
     // A round of a few thousand pairs cannot fill the GPU either way; there the cursors' sequential walk
     // through each capacity class is pure latency and the independent per-pair searches finish sooner.
-    const bool tiny = (uint64_t)c->J * c->G < (1ull << 16);
+    // (a later pass of a re-auction with a handful of gaps left is such a round too, whatever J is: below
+    // 2^21 pairs the fixed start-up of the ordered-gap kernels outweighs what they save)
+    const bool tiny = (uint64_t)c->J * c->G < (1ull << 16) || (G_act < c->G && (uint64_t)c->J * G_act < (1ull << 21));
     // with a window option the usable window differs from pair to pair: only the search kernel does that
     const bool per_pair_window = c->late_start || c->have_deadline || (c->have_power && c->have_caps);
     const bool sorted_ok = !(pflags & SJA_FLAG_FORCE_SEARCH) && !per_pair_window && c->gaps_sorted && (forced || !tiny) &&
@@ -357,7 +359,7 @@ SelectPlan plan_select(const sja_ctx* c, uint32_t pflags) {
 // `timed`: record profiling events (creates CUDA events on first use).
 sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sgaps, uint32_t G_act,
                       const uint32_t* blocked, Partial* scratch = nullptr, bool timed = true) {
-    const SelectPlan pl = plan_select(c, pflags);
+    const SelectPlan pl = plan_select(c, pflags, G_act);
     const uint32_t n_chunks = pl.n_chunks;
     // granularity of a gap split: a staging tile; the tile kernel also works in 32-gap steps, which a
     // small problem needs to put enough CTAs on the GPU
@@ -835,7 +837,7 @@ sja_status sja_select_static(sja_ctx* c, const sja_policy* policy, sja_award* ou
     if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
 
     const uint32_t kind = policy->kind, G = c->G, J = c->J;
-    const SelectPlan pl = plan_select(c, policy->flags);
+    const SelectPlan pl = plan_select(c, policy->flags, G);
     const uint64_t need = (uint64_t)pl.n_chunks * G;   // candidate slots: one per (CTA job chunk, gap)
     const uint64_t have = (uint64_t)SJA_STATIC_SCRATCH_BYTES / sizeof(Partial);
     if (need > have)
@@ -911,7 +913,7 @@ sja_status sja_round_reauction(sja_ctx* c, const sja_policy* policy, uint32_t ma
     const uint32_t kind = policy->kind, G = c->G, J = c->J;
     TRY(reserve(c, c->sgaps_alt, (size_t)G * sizeof(sja_gap)));
     TRY(reserve(c, c->blocked, (size_t)J * 4));
-    TRY(reserve(c, c->n_active, 4));
+    TRY(reserve(c, c->n_active, 16));   // per-pass report: orphans left, grants, flag word
     CU(cudaMemsetAsync(c->blocked.p, 0, (size_t)J * 4, c->stream));
 
     const Gap* cur = c->sgaps.as<Gap>();
@@ -923,17 +925,16 @@ sja_status sja_round_reauction(sja_ctx* c, const sja_policy* policy, uint32_t ma
         TRY(run_select(c, kind, policy->flags, cur, g_act, c->blocked.as<uint32_t>()));
         run_commit(c, c->blocked.as<uint32_t>());
         collect_orphans_kernel<<<1, 1024, 0, c->stream>>>(cur, g_act, c->awards.as<Award>(), spare,
+                                                          c->n_granted.as<uint32_t>(), c->flags.as<uint32_t>(),
                                                           c->n_active.as<uint32_t>());
         CU(cudaGetLastError());
-        CU(cudaMemcpyAsync(c->h_words, c->n_granted.p, 4, cudaMemcpyDeviceToHost, c->stream));
-        CU(cudaMemcpyAsync(c->h_words + 1, c->n_active.p, 4, cudaMemcpyDeviceToHost, c->stream));
-        CU(cudaMemcpyAsync(c->h_words + 2, c->flags.p, 4, cudaMemcpyDeviceToHost, c->stream));
+        CU(cudaMemcpyAsync(c->h_words, c->n_active.p, 12, cudaMemcpyDeviceToHost, c->stream));
         CU(cudaStreamSynchronize(c->stream));
         ++passes;
-        total += c->h_words[0];
+        total += c->h_words[1];
         if (c->h_words[2] & FLAG_OVF_READY) overflow = true;
-        if (c->h_words[0] == 0) break;          // nothing granted: the remaining gaps cannot be filled
-        g_act = c->h_words[1];
+        if (c->h_words[1] == 0) break;          // nothing granted: the remaining gaps cannot be filled
+        g_act = c->h_words[0];
         cur = spare;
         spare = (spare == c->sgaps_alt.as<Gap>()) ? own : c->sgaps_alt.as<Gap>();
     }

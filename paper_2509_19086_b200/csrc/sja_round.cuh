@@ -481,11 +481,14 @@ __global__ void __launch_bounds__(256) copy_gaps_kernel(const Gap* __restrict__ 
 // ---------------------------------------------------------------------------------------
 // Re-auction: keep, in their advertised order, the gaps that had a winner but were not
 // granted (their winner accepted another gap).  One CTA walks the ordered list in tiles of
-// 1024 with a block-wide exclusive count; *n_out receives the number of gaps kept.
+// 1024 with a block-wide exclusive count.  report[0] receives the number of gaps kept, report[1] the grants
+// of the pass and report[2] the status flag word, so that the host reads one record per pass.
 __global__ void __launch_bounds__(1024) collect_orphans_kernel(const Gap* __restrict__ sgaps_in, uint32_t G_in,
                                                                const Award* __restrict__ awards,
                                                                Gap* __restrict__ sgaps_out,
-                                                               uint32_t* __restrict__ n_out) {
+                                                               const uint32_t* __restrict__ n_granted,
+                                                               const uint32_t* __restrict__ flags,
+                                                               uint32_t* __restrict__ report) {
     __shared__ uint32_t warp_cnt[32];
     __shared__ uint32_t tile_total;
     const uint32_t t = threadIdx.x, lane = t & 31u, wid = t >> 5;
@@ -519,7 +522,7 @@ __global__ void __launch_bounds__(1024) collect_orphans_kernel(const Gap* __rest
         carry += tile_total;
         __syncthreads();
     }
-    if (t == 0) *n_out = carry;
+    if (t == 0) { report[0] = carry; report[1] = *n_granted; report[2] = *flags; }
 }
 
 // ---------------------------------------------------------------------------------------
