@@ -396,7 +396,7 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
                 select_search_kernel<false><<<dim3(n_chunks, splits), SEARCH_THREADS, SEARCH_SMEM_BYTES, c->stream>>>(
                     jv, sgaps, G_act, per_split, kind, partial);
         }
-        finalize_awards_kernel<<<(uint32_t)(((uint64_t)G_act * FINALIZE_LANES + 255) / 256), 256, 0, c->stream>>>(
+        finalize_awards_kernel<<<(G_act + 31) / 32, FINALIZE_WARPS * 32, 0, c->stream>>>(
             jv, partial, n_chunks, sgaps, G_act, kind, c->awards.as<Award>(), c->widx.as<uint32_t>());
     }
     c->prof = was_on;

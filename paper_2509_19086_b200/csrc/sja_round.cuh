@@ -203,32 +203,33 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
 }
 
 // ---------------------------------------------------------------------------------------
-// Final reduction: one thread per gap folds the candidate rows of all CTAs into the award.
-constexpr int FINALIZE_LANES = 8;   // lanes that share the candidate rows of one gap
+// Final reduction: fold the candidate rows of all CTAs into the award of every gap.  A CTA of 8 warps
+// owns 32 consecutive gaps, one per lane, so that a warp reads 512 contiguous bytes of a candidate row;
+// warp w folds rows w, w + 8, ..., then the 8 warps are folded through shared memory.
+constexpr int FINALIZE_WARPS = 8;
 
-__global__ void __launch_bounds__(256) finalize_awards_kernel(
+__global__ void __launch_bounds__(FINALIZE_WARPS * 32) finalize_awards_kernel(
     JobView jv, const Partial* __restrict__ partial, uint32_t n_rows, const Gap* __restrict__ sgaps, uint32_t G,
     uint32_t kind, Award* __restrict__ awards, uint32_t* __restrict__ widx) {
-    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
-    const uint32_t g = t / FINALIZE_LANES;     // position in the advertised (sorted) order
-    const uint32_t sub = t % FINALIZE_LANES;
+    __shared__ Partial fold[FINALIZE_WARPS][32];
+    const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
+    const uint32_t g = blockIdx.x * 32u + lane;     // position in the advertised (sorted) order
     Partial best;
     best.key = 0; best.job = 0xFFFFFFFFu; best.cnt = 0;
     if (g < G) {
-        for (uint32_t r = sub; r < n_rows; r += FINALIZE_LANES) {
+        for (uint32_t r = wid; r < n_rows; r += FINALIZE_WARPS) {
             const Partial c = partial[(size_t)r * G + g];
             if (c.key > best.key || (c.key == best.key && c.job < best.job)) best = c;
         }
     }
+    fold[wid][lane] = best;
+    __syncthreads();
+    if (wid != 0 || g >= G) return;
 #pragma unroll
-    for (int o = FINALIZE_LANES / 2; o > 0; o >>= 1) {
-        Partial c;
-        c.key = __shfl_xor_sync(0xFFFFFFFFu, best.key, o);
-        c.job = __shfl_xor_sync(0xFFFFFFFFu, best.job, o);
-        c.cnt = __shfl_xor_sync(0xFFFFFFFFu, best.cnt, o);
+    for (int w = 1; w < FINALIZE_WARPS; ++w) {
+        const Partial c = fold[w][lane];
         if (c.key > best.key || (c.key == best.key && c.job < best.job)) best = c;
     }
-    if (g >= G || sub != 0) return;
     const uint32_t orig = sgaps[g].slice;   // caller's gap index
     Award a;
     if (best.key == 0) {
@@ -393,21 +394,33 @@ __global__ void __launch_bounds__(SORT_TILE) sort_gap_tiles_kernel(const Gap* __
     uint64_t k = ~0ull;          // padding sorts last and is never smaller than a real key
     uint32_t x = 0xFFFFFFFFu;
     if (i < G) { const Gap g = gaps[i]; k = ((uint64_t)g.C << 32) | g.T; x = i; }
-    sk[t] = k; si[t] = x;
     if (i == 0) info->n_classes = 0;
-    __syncthreads();
+    // Bitonic network, one element per thread.  Partners less than 32 apart sit in the same warp and are
+    // exchanged by shuffles; only the wider strides go through shared memory (15 barrier stages, not 55).
     for (uint32_t size = 2; size <= SORT_TILE; size <<= 1) {
-        for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
-            const uint32_t p = t ^ stride;
-            if (p > t) {
-                const uint64_t ka = sk[t], kb = sk[p];
-                const uint32_t ia = si[t], ib = si[p];
-                const bool ascending = (t & size) == 0;
-                if (gap_key_less(kb, ib, ka, ia) == ascending) { sk[t] = kb; si[t] = ib; sk[p] = ka; si[p] = ia; }
-            }
+        const bool ascending = (t & size) == 0;
+        for (uint32_t stride = size >> 1; stride >= 32; stride >>= 1) {
+            sk[t] = k; si[t] = x;
             __syncthreads();
+            const uint32_t p = t ^ stride;
+            const uint64_t kp = sk[p];
+            const uint32_t xp = si[p];
+            // the lower position keeps the smaller key when ascending, the upper one the larger
+            const bool partner_less = gap_key_less(kp, xp, k, x);
+            const bool take = ((t & stride) == 0) == ascending ? partner_less : !partner_less;
+            __syncthreads();
+            if (take) { k = kp; x = xp; }
+        }
+        for (uint32_t stride = min(size >> 1, 16u); stride > 0; stride >>= 1) {
+            const uint64_t kp = __shfl_xor_sync(0xFFFFFFFFu, k, stride);
+            const uint32_t xp = __shfl_xor_sync(0xFFFFFFFFu, x, stride);
+            const bool partner_less = gap_key_less(kp, xp, k, x);
+            const bool take = ((t & stride) == 0) == ascending ? partner_less : !partner_less;
+            if (take) { k = kp; x = xp; }
         }
     }
+    sk[t] = k; si[t] = x;
+    __syncthreads();
     if (sorted_out) {            // one tile: position t is final
         const uint32_t src = si[t];
         const bool real = src != 0xFFFFFFFFu;
