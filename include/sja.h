@@ -223,7 +223,7 @@ sja_status sja_commit_masked(sja_ctx* ctx, const uint8_t* accept, sja_memspace w
  * it from wasting windows that further jobs had signalled interest in.
  * A pass-0-only call (max_passes = 1) equals sja_select followed by sja_commit.
  * The award of a gap (sja_get_awards) is the one of the last pass the gap took part in.
- * n_granted / n_passes are HOST pointers or NULL.  Waits for completion after every pass.
+ * n_granted / n_passes are HOST pointers or NULL.  Waits for the GPU after every batch of up to 16 passes.
  * Uses up the advertised batch like sja_commit.
  */
 sja_status sja_round_reauction(sja_ctx* ctx, const sja_policy* policy, uint32_t max_passes, uint32_t* n_granted,

@@ -23,6 +23,10 @@
 
 using namespace sja;
 
+// Passes of a re-auction queued between two host waits (four words of the pinned read-back area each).
+#ifndef REAUCTION_BATCH
+#define REAUCTION_BATCH 16
+#endif
 // Select grids aim at this many CTAs per SM (several waves even out the tail).
 #ifndef SJA_SELECT_CTAS_PER_SM
 #define SJA_SELECT_CTAS_PER_SM 8
@@ -60,7 +64,7 @@ struct sja_ctx {
     DevBuf nbj, cta_tot, cta_base, boff, boff_next, A, B, jobwin;   // row counting scratch, boundary table
     DevBuf flags, counter, n_granted;                 // small device words
     DevBuf long_list;                                 // jobs the scan of a load takes first
-    uint32_t* h_words = nullptr;                      // pinned host scratch (8 x u64)
+    uint32_t* h_words = nullptr;                      // pinned host scratch (128 words)
 
     // gaps / awards
     bool advertised = false, selected = false, committed = false;
@@ -270,10 +274,10 @@ enum SelectKernel { SEL_TILE = 0, SEL_MERGE = 1, SEL_SEARCH = 2 };
 
 template <uint32_t KIND, bool BOUNDED>
 void launch_sorted_kb(SelectKernel which, dim3 grid, cudaStream_t stream, const JobView& jv, const Gap* sgaps,
-                      uint32_t G, uint32_t per_split, Partial* partial) {
+                      uint32_t G, uint32_t per_split, Partial* partial, const uint32_t* G_dev) {
     if (which == SEL_TILE)
         select_tile_kernel<KIND, BOUNDED><<<grid, TILE_WARPS * 32, TILE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split,
-                                                                                             partial);
+                                                                                             partial, G_dev);
     else
         select_merge_kernel<KIND, BOUNDED><<<grid, MERGE_WARPS * 32, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G,
                                                                                                 per_split, partial);
@@ -281,23 +285,23 @@ void launch_sorted_kb(SelectKernel which, dim3 grid, cudaStream_t stream, const 
 
 template <bool BOUNDED>
 void launch_sorted_b(SelectKernel which, uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& jv,
-                     const Gap* sgaps, uint32_t G, uint32_t per_split, Partial* partial) {
+                     const Gap* sgaps, uint32_t G, uint32_t per_split, Partial* partial, const uint32_t* G_dev) {
     if (kind == SJA_POLICY_FAIRNESS)
-        launch_sorted_kb<1, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial);
+        launch_sorted_kb<1, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
     else if (kind == SJA_POLICY_SLA)
-        launch_sorted_kb<2, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial);
+        launch_sorted_kb<2, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
     else if (kind == SJA_POLICY_TIGHT_FIT)
-        launch_sorted_kb<3, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial);
+        launch_sorted_kb<3, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
     else
-        launch_sorted_kb<0, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial);
+        launch_sorted_kb<0, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
 }
 
 void launch_sorted(SelectKernel which, uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& jv,
-                   const Gap* sgaps, uint32_t G, uint32_t per_split, Partial* partial) {
+                   const Gap* sgaps, uint32_t G, uint32_t per_split, Partial* partial, const uint32_t* G_dev) {
     if (jv.tau_min != 0u || jv.tau_max != 0xFFFFFFFFu)
-        launch_sorted_b<true>(which, kind, grid, stream, jv, sgaps, G, per_split, partial);
+        launch_sorted_b<true>(which, kind, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
     else
-        launch_sorted_b<false>(which, kind, grid, stream, jv, sgaps, G, per_split, partial);
+        launch_sorted_b<false>(which, kind, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
 }
 
 template <uint32_t KIND, bool BOUNDED>
@@ -357,8 +361,10 @@ SelectPlan plan_select(const sja_ctx* c, uint32_t pflags, uint32_t G_act) {
 
 // `scratch`: candidate rows (n_chunks x G entries); nullptr = the context's own buffer, grown on demand.
 // `timed`: record profiling events (creates CUDA events on first use).
+// `G_dev`: optional device word with the number of gaps actually left (<= G_act, which then only sizes the launch).
 sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sgaps, uint32_t G_act,
-                      const uint32_t* blocked, Partial* scratch = nullptr, bool timed = true) {
+                      const uint32_t* blocked, Partial* scratch = nullptr, bool timed = true,
+                      const uint32_t* G_dev = nullptr) {
     const SelectPlan pl = plan_select(c, pflags, G_act);
     const uint32_t n_chunks = pl.n_chunks;
     // granularity of a gap split: a staging tile; the tile kernel also works in 32-gap steps, which a
@@ -386,18 +392,19 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
         JobView jv = job_view(c);
         jv.blocked = blocked;
         if (pl.kernel != SEL_SEARCH) {
-            launch_sorted(pl.kernel, kind, dim3(n_chunks, splits), c->stream, jv, sgaps, G_act, per_split, partial);
+            launch_sorted(pl.kernel, kind, dim3(n_chunks, splits), c->stream, jv, sgaps, G_act, per_split, partial,
+                          G_dev);
         } else {
             const bool opts = jv.late_start != 0u || jv.deadline != nullptr || jv.PW != nullptr;
             if (opts)
                 select_search_kernel<true><<<dim3(n_chunks, splits), SEARCH_THREADS, SEARCH_SMEM_BYTES, c->stream>>>(
-                    jv, sgaps, G_act, per_split, kind, partial);
+                    jv, sgaps, G_act, per_split, kind, partial, G_dev);
             else
                 select_search_kernel<false><<<dim3(n_chunks, splits), SEARCH_THREADS, SEARCH_SMEM_BYTES, c->stream>>>(
-                    jv, sgaps, G_act, per_split, kind, partial);
+                    jv, sgaps, G_act, per_split, kind, partial, G_dev);
         }
         finalize_awards_kernel<<<(G_act + 31) / 32, FINALIZE_WARPS * 32, 0, c->stream>>>(
-            jv, partial, n_chunks, sgaps, G_act, kind, c->awards.as<Award>(), c->widx.as<uint32_t>());
+            jv, partial, n_chunks, sgaps, G_act, kind, c->awards.as<Award>(), c->widx.as<uint32_t>(), G_dev);
     }
     c->prof = was_on;
     return SJA_OK;
@@ -474,7 +481,7 @@ sja_status sja_create(sja_ctx** out, int device, void* cuda_stream) {
         cudaDeviceProp prop;
         if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         c->n_sm = prop.multiProcessorCount;
-        if (cudaMallocHost(reinterpret_cast<void**>(&c->h_words), 64) != cudaSuccess) { st = SJA_ERR_OOM; break; }
+        if (cudaMallocHost(reinterpret_cast<void**>(&c->h_words), 512) != cudaSuccess) { st = SJA_ERR_OOM; break; }
         if ((st = reserve(c, c->flags, 8)) != SJA_OK) break;   // [0] status bits, [1] long-job count of a load
         if ((st = reserve(c, c->counter, 4)) != SJA_OK) break;
         if ((st = reserve(c, c->n_granted, 4)) != SJA_OK) break;
@@ -913,30 +920,45 @@ sja_status sja_round_reauction(sja_ctx* c, const sja_policy* policy, uint32_t ma
     const uint32_t kind = policy->kind, G = c->G, J = c->J;
     TRY(reserve(c, c->sgaps_alt, (size_t)G * sizeof(sja_gap)));
     TRY(reserve(c, c->blocked, (size_t)J * 4));
-    TRY(reserve(c, c->n_active, 16));   // per-pass report: orphans left, grants, flag word
     CU(cudaMemsetAsync(c->blocked.p, 0, (size_t)J * 4, c->stream));
 
+    // Passes are queued in batches without a host wait in between: the number of gaps a pass starts with lives
+    // in device memory (the report of the pass before it), launches are sized for the count at the last wait
+    // (it never grows), and a pass that finds nothing left does nothing.  The merge kernel does not take a
+    // device-side count: with SJA_FLAG_FORCE_MERGE every pass is waited for.
+    const uint32_t batch_max = (policy->flags & SJA_FLAG_FORCE_MERGE) ? 1u : (uint32_t)REAUCTION_BATCH;
+    TRY(reserve(c, c->n_active, (size_t)REAUCTION_BATCH * 16));
+    uint32_t* reports = c->n_active.as<uint32_t>();        // 4 words per pass of a batch
     const Gap* cur = c->sgaps.as<Gap>();
     Gap* spare = c->sgaps_alt.as<Gap>();
     Gap* const own = c->sgaps.as<Gap>();   // only ever written as the spare of a later pass, after it was read
     uint32_t g_act = G, total = 0, passes = 0;
-    bool overflow = false;
-    while (g_act > 0 && (max_passes == 0 || passes < max_passes)) {
-        TRY(run_select(c, kind, policy->flags, cur, g_act, c->blocked.as<uint32_t>()));
-        run_commit(c, c->blocked.as<uint32_t>());
-        collect_orphans_kernel<<<1, 1024, 0, c->stream>>>(cur, g_act, c->awards.as<Award>(), spare,
-                                                          c->n_granted.as<uint32_t>(), c->flags.as<uint32_t>(),
-                                                          c->n_active.as<uint32_t>());
-        CU(cudaGetLastError());
-        CU(cudaMemcpyAsync(c->h_words, c->n_active.p, 12, cudaMemcpyDeviceToHost, c->stream));
+    bool overflow = false, done = false;
+    while (!done && g_act > 0 && (max_passes == 0 || passes < max_passes)) {
+        uint32_t batch = batch_max;
+        if (max_passes != 0) batch = std::min(batch, max_passes - passes);
+        for (uint32_t k = 0; k < batch; ++k) {
+            const uint32_t* g_dev = k ? reports + 4 * (k - 1) : nullptr;   // gaps left after the pass before
+            TRY(run_select(c, kind, policy->flags, cur, g_act, c->blocked.as<uint32_t>(), nullptr, true, g_dev));
+            run_commit(c, c->blocked.as<uint32_t>());
+            collect_orphans_kernel<<<1, 1024, 0, c->stream>>>(cur, g_act, c->awards.as<Award>(), spare,
+                                                              c->n_granted.as<uint32_t>(), c->flags.as<uint32_t>(),
+                                                              reports + 4 * k, g_dev);
+            CU(cudaGetLastError());
+            cur = spare;
+            spare = (spare == c->sgaps_alt.as<Gap>()) ? own : c->sgaps_alt.as<Gap>();
+        }
+        CU(cudaMemcpyAsync(c->h_words, reports, (size_t)batch * 16, cudaMemcpyDeviceToHost, c->stream));
         CU(cudaStreamSynchronize(c->stream));
-        ++passes;
-        total += c->h_words[1];
-        if (c->h_words[2] & FLAG_OVF_READY) overflow = true;
-        if (c->h_words[1] == 0) break;          // nothing granted: the remaining gaps cannot be filled
-        g_act = c->h_words[0];
-        cur = spare;
-        spare = (spare == c->sgaps_alt.as<Gap>()) ? own : c->sgaps_alt.as<Gap>();
+        for (uint32_t k = 0; k < batch; ++k) {
+            const uint32_t* r = c->h_words + 4 * k;        // orphans left, grants, flags, gaps at the start
+            ++passes;
+            total += r[1];
+            if (r[2] & FLAG_OVF_READY) overflow = true;
+            g_act = r[0];
+            // nothing granted: no orphan has an interested job left (then none is kept either); nothing left
+            if (r[1] == 0 || r[0] == 0) { done = true; break; }
+        }
     }
     c->selected = false;
     c->committed = true;

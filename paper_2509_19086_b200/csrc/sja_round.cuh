@@ -62,8 +62,10 @@ static_assert((SEARCH_ROWS & (SEARCH_ROWS - 1)) == 0 && SEARCH_PAY_ROWS <= SEARC
 template <bool OPTS>
 __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
     JobView jv, const Gap* __restrict__ gaps, uint32_t G, uint32_t gaps_per_split, uint32_t kind,
-    Partial* __restrict__ partial_out) {
+    Partial* __restrict__ partial_out, const uint32_t* __restrict__ G_dev) {
     __shared__ Partial stage[SEARCH_GT][SEARCH_THREADS / 32];
+    const uint32_t G_now = G_dev ? min(G, *G_dev) : G;   // gaps actually left (see select_tile_kernel)
+    if (blockIdx.y * gaps_per_split >= G_now) return;
     extern __shared__ __align__(16) uint2 search_rows[];
     uint2* sDM = search_rows + threadIdx.x;                                     // row r of this thread: sDM[r * THREADS]
     uint2* sPay = search_rows + SEARCH_ROWS * SEARCH_THREADS + threadIdx.x;     // its policy payload (work or peak)
@@ -86,7 +88,7 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
     }
     const bool late = OPTS && jv.late_start != 0u;
     const uint32_t g_begin = blockIdx.y * gaps_per_split;
-    const uint32_t g_end = min(G, g_begin + gaps_per_split);
+    const uint32_t g_end = min(G_now, g_begin + gaps_per_split);
     // The first rows of the job in shared memory; the slots beyond its last row hold a sentinel that no
     // window admits (except T = C = 2^32-1, where the clamp below takes care), so every thread runs the
     // same five probes.  Each thread reads back only what it wrote: no barrier needed.
@@ -210,13 +212,14 @@ constexpr int FINALIZE_WARPS = 8;
 
 __global__ void __launch_bounds__(FINALIZE_WARPS * 32) finalize_awards_kernel(
     JobView jv, const Partial* __restrict__ partial, uint32_t n_rows, const Gap* __restrict__ sgaps, uint32_t G,
-    uint32_t kind, Award* __restrict__ awards, uint32_t* __restrict__ widx) {
+    uint32_t kind, Award* __restrict__ awards, uint32_t* __restrict__ widx, const uint32_t* __restrict__ G_dev) {
     __shared__ Partial fold[FINALIZE_WARPS][32];
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
     const uint32_t g = blockIdx.x * 32u + lane;     // position in the advertised (sorted) order
+    const uint32_t G_now = G_dev ? min(G, *G_dev) : G;   // G stays the row length of `partial`
     Partial best;
     best.key = 0; best.job = 0xFFFFFFFFu; best.cnt = 0;
-    if (g < G) {
+    if (g < G_now) {
         for (uint32_t r = wid; r < n_rows; r += FINALIZE_WARPS) {
             const Partial c = partial[(size_t)r * G + g];
             if (c.key > best.key || (c.key == best.key && c.job < best.job)) best = c;
@@ -224,7 +227,7 @@ __global__ void __launch_bounds__(FINALIZE_WARPS * 32) finalize_awards_kernel(
     }
     fold[wid][lane] = best;
     __syncthreads();
-    if (wid != 0 || g >= G) return;
+    if (wid != 0 || g >= G_now) return;
 #pragma unroll
     for (int w = 1; w < FINALIZE_WARPS; ++w) {
         const Partial c = fold[w][lane];
@@ -495,13 +498,16 @@ __global__ void __launch_bounds__(256) copy_gaps_kernel(const Gap* __restrict__ 
 // Re-auction: keep, in their advertised order, the gaps that had a winner but were not
 // granted (their winner accepted another gap).  One CTA walks the ordered list in tiles of
 // 1024 with a block-wide exclusive count.  report[0] receives the number of gaps kept, report[1] the grants
-// of the pass and report[2] the status flag word, so that the host reads one record per pass.
+// of the pass, report[2] the status flag word and report[3] the number of gaps the pass started with, so that
+// the host reads one 16-byte record per pass.  G_dev (optional): that number lives in device memory.
 __global__ void __launch_bounds__(1024) collect_orphans_kernel(const Gap* __restrict__ sgaps_in, uint32_t G_in,
                                                                const Award* __restrict__ awards,
                                                                Gap* __restrict__ sgaps_out,
                                                                const uint32_t* __restrict__ n_granted,
                                                                const uint32_t* __restrict__ flags,
-                                                               uint32_t* __restrict__ report) {
+                                                               uint32_t* __restrict__ report,
+                                                               const uint32_t* __restrict__ G_dev) {
+    if (G_dev) G_in = min(G_in, *G_dev);
     __shared__ uint32_t warp_cnt[32];
     __shared__ uint32_t tile_total;
     const uint32_t t = threadIdx.x, lane = t & 31u, wid = t >> 5;
@@ -535,7 +541,7 @@ __global__ void __launch_bounds__(1024) collect_orphans_kernel(const Gap* __rest
         carry += tile_total;
         __syncthreads();
     }
-    if (t == 0) { report[0] = carry; report[1] = *n_granted; report[2] = *flags; }
+    if (t == 0) { report[0] = carry; report[1] = G_in ? *n_granted : 0u; report[2] = *flags; report[3] = G_in; }
 }
 
 // ---------------------------------------------------------------------------------------
