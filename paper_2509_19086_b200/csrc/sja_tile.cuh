@@ -41,6 +41,9 @@ namespace sja {
 #ifndef SJA_TILE_GT
 #define SJA_TILE_GT 256
 #endif
+#ifndef SJA_TILE_MULTI
+#define SJA_TILE_MULTI 2
+#endif
 constexpr int TILE_WARPS = SJA_TILE_WARPS;
 constexpr int TILE_CTAS_PER_SM = SJA_TILE_CTAS_PER_SM;
 constexpr int TILE_RING = SJA_TILE_RING;     // rows per job ring (power of two)
@@ -152,6 +155,83 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
         if (threadIdx.x < gt) sg_w[threadIdx.x] = __ldg(reinterpret_cast<const uint4*>(sgaps) + g0 + threadIdx.x);
         __syncthreads();
         for (uint32_t sub = 0; sub < gt; sub += 32) {
+#if SJA_TILE_MULTI > 1
+            // Fast path: MULTI x 32 gaps of the class the cursors are in, MULTI per lane.  One set of cursor
+            // steps and one pass over the posted events serve all gaps of a lane; the PM is up to date (nothing
+            // was restarted), so no run detection, no catch-up and no rebuild are needed.
+            bool multi = !dirty && have_class && sub + 32u * SJA_TILE_MULTI <= gt;
+            if (multi) {
+                bool same = true;
+#pragma unroll
+                for (int q = 0; q < SJA_TILE_MULTI; ++q) same = same && sg[sub + 32 * q + lane].w == curC;
+                multi = __all_sync(0xFFFFFFFFu, same);
+            }
+            if (multi) {
+                uint32_t Tq[SJA_TILE_MULTI], eq[SJA_TILE_MULTI], iq[SJA_TILE_MULTI], cq[SJA_TILE_MULTI];
+                uint64_t kq[SJA_TILE_MULTI];
+#pragma unroll
+                for (int q = 0; q < SJA_TILE_MULTI; ++q) {
+                    const uint4 gq = sg[sub + 32 * q + lane];
+                    Tq[q] = BOUNDED ? min(gq.z, jv.tau_max) : gq.z;
+                    uint32_t e = 0;
+#pragma unroll
+                    for (uint32_t s = 16; s >= 1; s >>= 1) {
+                        const uint32_t v = __shfl_sync(0xFFFFFFFFu, sready, (e + s - 1u) & 31u);
+                        if (v <= gq.y) e += s;
+                    }
+                    if (e == 31u && sready_last <= gq.y) e = 32u;
+                    eq[q] = e;
+                    // base answer: PM[e - 1]; its row count is the owner's current cursor
+                    const uint32_t src = (e ? e - 1u : 0u) & 31u;
+                    const uint64_t k0 = __shfl_sync(0xFFFFFFFFu, pk, src);
+                    const uint32_t i0 = __shfl_sync(0xFFFFFFFFu, pi, src);
+                    const uint32_t c0 = __shfl_sync(0xFFFFFFFFu, w, 31u - i0);
+                    kq[q] = e ? k0 : 0ull; iq[q] = e ? i0 : 0u; cq[q] = e ? c0 : 0u;
+                }
+                const uint64_t pmr_k = __shfl_sync(0xFFFFFFFFu, pk, rank);
+                const uint32_t pmr_i = __shfl_sync(0xFFFFFFFFu, pi, rank);
+                const uint32_t T_hi = __shfl_sync(0xFFFFFFFFu, Tq[SJA_TILE_MULTI - 1], 31);
+                while (__any_sync(0xFFFFFFFFu, open && thr <= T_hi)) {
+                    bool post = false;
+                    if (open && thr <= T_hi) {
+                        uint32_t thr_e;
+                        do {
+                            thr_e = thr;
+                            step_cursor(curC);
+                            post = pair_ge(curKey, 31u - lane, pmr_k, pmr_i);
+                        } while (!post && open && thr <= T_hi);
+                        if (post) {
+                            ev[lane] = make_uint4(thr_e, rank, (uint32_t)curKey, (uint32_t)(curKey >> 32));
+                            evc[lane] = w;
+                        }
+                    }
+                    uint32_t m = __ballot_sync(0xFFFFFFFFu, post);
+                    if (m == 0u) continue;
+                    __syncwarp();
+                    while (m) {
+                        const uint32_t b = (uint32_t)__ffs((int)m) - 1u;
+                        m &= m - 1u;
+                        const uint4 q4 = ev[b];           // duration, rank of the job, key
+                        const uint32_t c = evc[b];
+                        const uint64_t k = pack64(q4.z, q4.w);
+                        const uint32_t ib = 31u - b;
+#pragma unroll
+                        for (int q = 0; q < SJA_TILE_MULTI; ++q)
+                            if (Tq[q] >= q4.x && q4.y < eq[q] && pair_ge(k, ib, kq[q], iq[q])) { kq[q] = k; iq[q] = ib; cq[q] = c; }
+                        if (lane >= q4.y && pair_ge(k, ib, pk, pi)) { pk = k; pi = ib; }
+                    }
+                    __syncwarp();
+                }
+#pragma unroll
+                for (int q = 0; q < SJA_TILE_MULTI; ++q) {
+                    Partial pr;
+                    pr.key = kq[q]; pr.job = kq[q] ? job0 + 31u - iq[q] : 0xFFFFFFFFu; pr.cnt = kq[q] ? cq[q] : 0u;
+                    stage[wid * TILE_GT + sub + 32 * q + lane] = pr;
+                }
+                sub += 32u * (SJA_TILE_MULTI - 1);
+                continue;
+            }
+#endif
             const bool in = sub + lane < gt;
             uint4 gq = make_uint4(0u, 0u, 0u, 0u);
             if (in) gq = sg[sub + lane];
