@@ -46,10 +46,11 @@ NCU_SCAN_SOURCE_SHA = "8b4aa85b4bb68d65"
 # Issue-slot roofline of the select kernel (it is bound by instruction issue, not HBM): warp instructions of one
 # launch on the large uniform workload from ncu (profiles/select_tile_kernel_cfg2-jobs32768.md, full-size line),
 # peak = SMs x 4 schedulers x SM clock.  The kernel's work is not proportional to the pair count, so the figure
-# holds for that workload only; it is reported while csrc/sja_tile.cuh is the file the counters were taken from.
+# holds for that workload only; it is reported while csrc/sja_tile.cuh is the file the counters were taken from
+# (its code: the hash was re-taken after a comment-only edit).
 NCU_TILE_WARP_INSTR_PER_LAUNCH = 90569842
 NCU_TILE_PAIRS = 65536 * 4096
-NCU_TILE_SOURCE_SHA = "cb7cd0e1f6f051df"
+NCU_TILE_SOURCE_SHA = "9470af5ea551c4a3"
 N_SM, SCHEDULERS_PER_SM = 148, 4
 
 

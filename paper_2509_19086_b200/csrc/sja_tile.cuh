@@ -21,6 +21,10 @@
 //    eligible ones, does it beat my best) and as PM entry (does it raise the prefix maximum
 //    at my rank), which leaves the PM ready for the next 32 gaps.
 //
+// Where the next 64 gaps all belong to the class the cursors are in, a lane takes two of them
+// at once (SJA_TILE_MULTI): one set of cursor steps and one pass over the posted events serve
+// both, and the bookkeeping of a step is paid once.
+//
 // The cost is therefore per (warp, 32 gaps) a small fixed part (the lookup) plus the cursor
 // steps, not the number of pairs.  The PM is rebuilt by a warp scan only after a restart of
 // the cursors (a new capacity class, or the start of a CTA's gap range).
