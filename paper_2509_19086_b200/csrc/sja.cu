@@ -397,7 +397,8 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
         } else {
             const bool opts = jv.late_start != 0u || jv.deadline != nullptr || jv.PW != nullptr;
             if (opts)
-                select_search_kernel<true><<<dim3(n_chunks, splits), SEARCH_THREADS, SEARCH_SMEM_BYTES, c->stream>>>(
+                select_search_kernel<true><<<dim3(n_chunks, splits), SEARCH_THREADS,
+                                             jv.PW ? SEARCH_SMEM_BYTES_POWER : SEARCH_SMEM_BYTES, c->stream>>>(
                     jv, sgaps, G_act, per_split, kind, partial, G_dev);
             else
                 select_search_kernel<false><<<dim3(n_chunks, splits), SEARCH_THREADS, SEARCH_SMEM_BYTES, c->stream>>>(
@@ -491,7 +492,7 @@ sja_status sja_create(sja_ctx** out, int device, void* cuda_stream) {
         if (cudaFuncSetAttribute(select_search_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  SEARCH_SMEM_BYTES) != cudaSuccess ||
             cudaFuncSetAttribute(select_search_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 SEARCH_SMEM_BYTES) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
+                                 SEARCH_SMEM_BYTES_POWER) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         if (sorted_smem_attr<0, false>() != cudaSuccess || sorted_smem_attr<1, false>() != cudaSuccess ||
             sorted_smem_attr<2, false>() != cudaSuccess || sorted_smem_attr<3, false>() != cudaSuccess ||
             sorted_smem_attr<0, true>() != cudaSuccess || sorted_smem_attr<1, true>() != cudaSuccess ||

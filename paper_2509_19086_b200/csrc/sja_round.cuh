@@ -56,6 +56,7 @@ constexpr int SEARCH_GT = 64;   // gaps per staging tile
 constexpr int SEARCH_ROWS = SJA_SEARCH_ROWS;          // boundary rows staged per job as {D - Dp, M} (a power of two)
 constexpr int SEARCH_PAY_ROWS = SJA_SEARCH_PAY_ROWS;  // of which the first ones also with their policy payload
 constexpr int SEARCH_SMEM_BYTES = (SEARCH_ROWS + SEARCH_PAY_ROWS) * SEARCH_THREADS * 8;   // [row][thread]
+constexpr int SEARCH_SMEM_BYTES_POWER = SEARCH_SMEM_BYTES + SEARCH_ROWS * SEARCH_THREADS * 4;   // + running power maxima
 static_assert((SEARCH_ROWS & (SEARCH_ROWS - 1)) == 0 && SEARCH_PAY_ROWS <= SEARCH_ROWS, "staging shape");
 
 // OPTS: a window option or a power cap is in force (compiled out otherwise).
@@ -69,6 +70,9 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
     extern __shared__ __align__(16) uint2 search_rows[];
     uint2* sDM = search_rows + threadIdx.x;                                     // row r of this thread: sDM[r * THREADS]
     uint2* sPay = search_rows + SEARCH_ROWS * SEARCH_THREADS + threadIdx.x;     // its policy payload (work or peak)
+    // with power caps in force the launch carries room for the rows' running power maxima as well
+    uint32_t* sPow = reinterpret_cast<uint32_t*>(search_rows + (SEARCH_ROWS + SEARCH_PAY_ROWS) * SEARCH_THREADS) + threadIdx.x;
+    const bool staged_power = OPTS && jv.PW != nullptr;
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
     const uint32_t j = blockIdx.x * SEARCH_THREADS + threadIdx.x;
 
@@ -103,6 +107,7 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
         }
         sDM[r * SEARCH_THREADS] = dm;
         if (r < (uint32_t)SEARCH_PAY_ROWS) sPay[r * SEARCH_THREADS] = pay;
+        if (staged_power) sPow[r * SEARCH_THREADS] = r < ns ? __ldg(&jv.PW[base + r].x) : 0xFFFFFFFFu;
     }
 
     for (uint32_t g0 = g_begin; g0 < g_end; g0 += SEARCH_GT) {
@@ -136,7 +141,7 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
             auto fits = [&](uint32_t idx) -> bool {
                 const uint2 r = sDM[idx * SEARCH_THREADS];
                 bool ok = r.x <= T && r.y <= C;
-                if (OPTS && capped && ok && idx < ns) ok = __ldg(&jv.PW[base + idx].x) <= cap;
+                if (OPTS && capped && ok && idx < ns) ok = sPow[idx * SEARCH_THREADS] <= cap;
                 return ok;
             };
             uint32_t lo = 0;
