@@ -65,6 +65,7 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
     JobView jv, const Gap* __restrict__ gaps, uint32_t G, uint32_t gaps_per_split, uint32_t kind,
     Partial* __restrict__ partial_out, const uint32_t* __restrict__ G_dev) {
     __shared__ Partial stage[SEARCH_GT][SEARCH_THREADS / 32];
+    __shared__ uint4 sgap[SEARCH_GT];
     const uint32_t G_now = G_dev ? min(G, *G_dev) : G;   // gaps actually left (see select_tile_kernel)
     if (blockIdx.y * gaps_per_split >= G_now) return;
     extern __shared__ __align__(16) uint2 search_rows[];
@@ -112,8 +113,13 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
 
     for (uint32_t g0 = g_begin; g0 < g_end; g0 += SEARCH_GT) {
         const uint32_t gt = min((uint32_t)SEARCH_GT, g_end - g0);
+        // the tile's gaps in shared memory; the next one is fetched while the current one is worked on
+        if (threadIdx.x < gt) sgap[threadIdx.x] = __ldg(reinterpret_cast<const uint4*>(gaps) + g0 + threadIdx.x);
+        __syncthreads();
+        uint4 gq_next = sgap[0];
         for (uint32_t gi = 0; gi < gt; ++gi) {
-            const uint4 gq = __ldg(reinterpret_cast<const uint4*>(gaps) + g0 + gi);
+            const uint4 gq = gq_next;
+            gq_next = sgap[min(gi + 1, gt - 1)];
             const uint32_t start = gq.y, C = gq.w;
             uint32_t T = gq.z, cap = 0xFFFFFFFFu;
             bool eligible = n != 0;
