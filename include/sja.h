@@ -3,8 +3,8 @@
  * Atomization (SJA) on one NVIDIA B200 (sm_100a).
  *
  * The paper defines the round in prose: the scheduler advertises execution gaps (a time
- * window on a MIG slice of some capacity), every waiting job answers "interest" if it
- * could safely generate a subjob for that time/capacity pair, the scheduler picks one
+ * window on a MIG slice of some capacity), every waiting job answers "interest" if a
+ * subjob of its own would fit that window and capacity safely, the scheduler picks one
  * interested job per gap by its policy, and only the granted job materialises the subjob
  * (Section 3.5; admissibility test in Sections 3.8 and 3.9; greedy slot filling in
  * Section 4.2).  This library fixes that prose as integer arithmetic:
@@ -64,7 +64,7 @@ typedef enum {
 
 typedef enum { SJA_MEM_HOST = 0, SJA_MEM_DEVICE = 1 } sja_memspace;
 
-/* One advertised execution gap: "time interval and slice capacity" (Section 3.5). 16 bytes. */
+/* One advertised execution gap: a window in time on a slice of a given memory capacity (Section 3.5). 16 bytes. */
 typedef struct {
     uint32_t slice;    /* MIG slice label, carried through, not used in scoring */
     uint32_t start_ms; /* absolute start of the window */
@@ -312,8 +312,8 @@ sja_status sja_load_power(sja_ctx* ctx, const uint64_t* off, const uint32_t* pow
 sja_status sja_advertise_power_caps(sja_ctx* ctx, const uint32_t* cap_W, sja_memspace where);
 
 /*
- * Re-profile one job.  Segmentation is on demand because the envelope U(t) "may evolve as runtime
- * predictions are refined" (Section 3.9): this call replaces the per-step durations and memory values of
+ * Re-profile one job.  Segmentation happens on demand, at offer time, because the envelope U(t) can change
+ * between offers as predictions improve (Section 3.9): this call replaces the per-step durations and memory values of
  * the steps job `job` has not been granted yet, steps p_job .. len_job - 1, n_steps = len_job - p_job of
  * them (SJA_ERR_BAD_PROFILE otherwise).  The job's safe boundaries stay where they are (a refined
  * prediction changes how long and how large a phase is, not where the checkpoints are), so only the
@@ -354,6 +354,17 @@ sja_status sja_profile_read(sja_ctx* ctx, sja_timing* out);
 
 /* Text of the most recent error on this context ("" if none).  Owned by the context. */
 const char* sja_last_error(const sja_ctx* ctx);
+
+/*
+ * Testing aid (the paper has no counterpart): host-side fault injection for the library's own device
+ * allocations.  After the call, the nth time (counting from 1) that a context buffer has to grow, the
+ * allocation is reported as failed (SJA_ERR_OOM) without being attempted; nth = 0 switches the injector off.
+ * Nothing on the GPU is touched: the failure is made on the host, so that the error paths of the entry
+ * points can be exercised without exhausting device memory.  A buffer whose growth fails keeps its old
+ * block; an sja_advertise that fails leaves the context without a batch (select / commit then return
+ * SJA_ERR_STATE) and with the loaded profiles intact.
+ */
+sja_status sja_debug_fail_alloc(sja_ctx* ctx, int nth);
 
 #ifdef __cplusplus
 }

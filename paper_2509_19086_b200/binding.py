@@ -34,7 +34,7 @@ AWARD_DTYPE = np.dtype([("job", "<u4"), ("end_step", "<u4"), ("dur_ms", "<u4"), 
 EXPORTS = [
     "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit", "sja_commit_masked", "sja_round_reauction", "sja_set_duration_bounds", "sja_set_window_options", "sja_update_profile", "sja_load_power", "sja_advertise_power_caps", "sja_get_bids", "sja_reduce_bids",
     "sja_get_awards", "sja_get_state", "sja_scan_size", "sja_get_scan", "sja_profile_enable",
-    "sja_profile_read", "sja_last_error",
+    "sja_profile_read", "sja_last_error", "sja_debug_fail_alloc",
 ]
 
 
@@ -94,6 +94,7 @@ def load_library() -> ctypes.CDLL:
     lib.sja_profile_enable.argtypes = [vp, i32]
     lib.sja_profile_read.argtypes = [vp, ctypes.POINTER(SjaTiming)]
     lib.sja_last_error.argtypes = [vp]
+    lib.sja_debug_fail_alloc.argtypes = [vp, i32]
     lib.sja_last_error.restype = ctypes.c_char_p
     for name in EXPORTS:
         if name != "sja_last_error":
@@ -345,6 +346,11 @@ class Sja:
         self._check(self._lib.sja_get_scan(self._h, boff.ctypes.data, k.ctypes.data, D.ctypes.data,
                                            M.ctypes.data, S.ctypes.data, W.ctypes.data, MEM_HOST))
         return dict(boff=boff, k=k, D=D, M=M, S=S, W=W)
+
+    # -- sja_debug_fail_alloc
+    def debug_fail_alloc(self, nth: int) -> None:
+        """Host-side fault injection: the nth growing allocation from now reports SJA_ERR_OOM (0 = off)."""
+        self._check(self._lib.sja_debug_fail_alloc(self._h, int(nth)))
 
     # -- profiling
     def profile_enable(self, on=True) -> None:

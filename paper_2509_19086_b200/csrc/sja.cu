@@ -52,6 +52,7 @@ struct sja_ctx {
     char err[320] = {0};
     bool poisoned = false;
     int n_sm = 148;
+    int fail_alloc_in = 0;             // sja_debug_fail_alloc: the n-th growing allocation from now fails (0 = off)
 
     // profiles / scan
     bool loaded = false;
@@ -136,17 +137,23 @@ struct DeviceGuard {
     }
 };
 
+// Grow a context buffer (contents are not kept).  The new block is allocated before the old one is let go, so
+// a failed allocation leaves the buffer as it was.  `fail_alloc_in` is the host-side fault injector of
+// sja_debug_fail_alloc: when it counts down to zero the allocation is reported as failed without being tried.
 sja_status reserve(sja_ctx* c, DevBuf& b, size_t bytes) {
     if (bytes <= b.cap) return SJA_OK;
+    const size_t want = (bytes + 255) & ~(size_t)255;
+    void* fresh = nullptr;
+    cudaError_t e = cudaSuccess;
+    if (c->fail_alloc_in > 0 && --c->fail_alloc_in == 0) e = cudaErrorMemoryAllocation;
+    else e = cudaMalloc(&fresh, want);
+    if (e != cudaSuccess) return cuda_fail(c, e, "cudaMalloc");
     if (b.p) {
-        CU(cudaStreamSynchronize(c->stream));   // a kernel in flight may still use the old buffer
-        CU(cudaFree(b.p));
-        b.p = nullptr;
-        b.cap = 0;
+        e = cudaStreamSynchronize(c->stream);   // a kernel in flight may still use the old buffer
+        if (e == cudaSuccess) e = cudaFree(b.p);
+        if (e != cudaSuccess) { cudaFree(fresh); return cuda_fail(c, e, "cudaFree"); }
     }
-    size_t want = (bytes + 255) & ~(size_t)255;
-    cudaError_t e = cudaMalloc(&b.p, want);
-    if (e != cudaSuccess) { b.p = nullptr; return cuda_fail(c, e, "cudaMalloc"); }
+    b.p = fresh;
     b.cap = want;
     return SJA_OK;
 }
@@ -530,9 +537,17 @@ sja_status sja_destroy(sja_ctx* c) {
 
 const char* sja_last_error(const sja_ctx* c) { return c ? c->err : ""; }
 
+sja_status sja_debug_fail_alloc(sja_ctx* c, int nth) {
+    TRY(check_ctx(c));
+    if (nth < 0) return fail(c, SJA_ERR_INVALID_ARG, "sja_debug_fail_alloc: nth must be >= 0");
+    c->fail_alloc_in = nth;
+    return SJA_OK;
+}
+
 sja_status sja_profile_enable(sja_ctx* c, int on) {
     TRY(check_ctx(c));
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     TRY(collect_spans(c));
     for (int i = 0; i < CAT_COUNT; ++i) { c->acc_ms[i] = 0.f; c->acc_n[i] = 0; }
     if (on < 0 || on > 2) return fail(c, SJA_ERR_INVALID_ARG, "sja_profile_enable: mode must be 0, 1 or 2");
@@ -544,6 +559,7 @@ sja_status sja_profile_read(sja_ctx* c, sja_timing* out) {
     TRY(check_ctx(c));
     if (!out) return fail(c, SJA_ERR_INVALID_ARG, "sja_profile_read: out is NULL");
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     TRY(collect_spans(c));
     out->scan_ms = c->acc_ms[CAT_SCAN];
     out->prep_ms = c->acc_ms[CAT_PREP];
@@ -766,6 +782,11 @@ sja_status sja_advertise(sja_ctx* c, uint32_t G, const sja_gap* gaps, sja_memspa
         return fail(c, SJA_ERR_INVALID_ARG, "sja_advertise: bad memspace");
     if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_advertise before sja_load_profiles");
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
+    // From here on the previous batch is gone, whatever happens below: if growing a buffer fails, a later
+    // select or commit must find no batch (SJA_ERR_STATE) rather than buffers that belong to two batches.
+    c->advertised = c->selected = c->committed = false;
+    c->have_caps = false;      // power caps belong to a batch
     TRY(reserve(c, c->gaps, (size_t)G * sizeof(sja_gap)));
     TRY(reserve(c, c->sgaps, (size_t)G * sizeof(sja_gap)));
     // u32 rank[G] (rounded up to 16 bytes), then u64 tile_key and u32 tile_idx, both padded to whole sort tiles
@@ -819,6 +840,7 @@ sja_status sja_select(sja_ctx* c, const sja_policy* policy, sja_award* out, sja_
         return fail(c, SJA_ERR_INVALID_ARG, "sja_select: bad memspace");
     TRY(check_policy(c, policy, "sja_select"));
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     const uint32_t kind = policy->kind;
     TRY(run_select(c, kind, policy->flags, c->sgaps.as<Gap>(), c->G, nullptr));
     CU(cudaGetLastError());
@@ -895,6 +917,7 @@ static sja_status commit_impl(sja_ctx* c, const uint8_t* accept, uint32_t* n_gra
 sja_status sja_commit(sja_ctx* c, uint32_t* n_granted) {
     TRY(check_ctx(c));
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     return commit_impl(c, nullptr, n_granted, "sja_commit");
 }
 
@@ -905,6 +928,7 @@ sja_status sja_commit_masked(sja_ctx* c, const uint8_t* accept, sja_memspace whe
         return fail(c, SJA_ERR_INVALID_ARG, "sja_commit_masked: bad memspace");
     if (!c->selected) return fail(c, SJA_ERR_STATE, "sja_commit_masked without a preceding sja_select");
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     TRY(reserve(c, c->accept, c->G));
     TRY(copy_in(c, c->accept.p, accept, c->G, where));
     const sja_status st = commit_impl(c, c->accept.as<uint8_t>(), n_granted, "sja_commit_masked");
@@ -918,6 +942,7 @@ sja_status sja_round_reauction(sja_ctx* c, const sja_policy* policy, uint32_t ma
     TRY(check_ctx(c));
     TRY(check_policy(c, policy, "sja_round_reauction"));
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     const uint32_t kind = policy->kind, G = c->G, J = c->J;
     TRY(reserve(c, c->sgaps_alt, (size_t)G * sizeof(sja_gap)));
     TRY(reserve(c, c->blocked, (size_t)J * 4));
@@ -993,6 +1018,7 @@ sja_status sja_update_profile(sja_ctx* c, uint32_t job, uint32_t n_steps, const 
     if (job >= c->J) return fail(c, SJA_ERR_INVALID_ARG, "sja_update_profile: job %u of %u", job, c->J);
     if (n_steps && (!dur_ms || !mem_MiB)) return fail(c, SJA_ERR_INVALID_ARG, "sja_update_profile: array is NULL");
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     const uint32_t *d_d = dur_ms, *d_m = mem_MiB;
     if (where == SJA_MEM_HOST && n_steps) {
         TRY(reserve(c, c->upd_d, (size_t)n_steps * 4));
@@ -1039,6 +1065,7 @@ sja_status sja_get_bids(sja_ctx* c, uint32_t job_base, uint32_t rank, sja_bid* o
     if ((uint64_t)job_base + c->J > 0xFFFFFFFFull)
         return fail(c, SJA_ERR_INVALID_ARG, "sja_get_bids: job_base + J does not fit a 32-bit job id");
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     Bid* d_out = reinterpret_cast<Bid*>(out);
     if (where == SJA_MEM_HOST) {
         TRY(reserve(c, c->st_bids, (size_t)c->G * sizeof(Bid)));
@@ -1064,6 +1091,7 @@ sja_status sja_reduce_bids(sja_ctx* c, uint32_t n_ranks, uint32_t my_rank, const
         return fail(c, SJA_ERR_INVALID_ARG, "sja_reduce_bids: bad memspace");
     if (!c->advertised) return fail(c, SJA_ERR_STATE, "sja_reduce_bids before sja_advertise");
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     const uint32_t G = c->G;
     const Bid* d_all = reinterpret_cast<const Bid*>(all);
     uint8_t* d_accept = accept;
@@ -1096,6 +1124,7 @@ sja_status sja_load_power(sja_ctx* c, const uint64_t* off, const uint32_t* power
     if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_load_power before sja_load_profiles");
     if (!off || (c->N > 0 && !power_W)) return fail(c, SJA_ERR_INVALID_ARG, "sja_load_power: off / power_W is NULL");
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     const uint64_t* d_off = off;
     const uint32_t* d_pw = power_W;
     if (where == SJA_MEM_HOST) {
@@ -1131,6 +1160,7 @@ sja_status sja_advertise_power_caps(sja_ctx* c, const uint32_t* cap_W, sja_memsp
         return fail(c, SJA_ERR_INVALID_ARG, "sja_advertise_power_caps: bad memspace");
     if (!c->advertised) return fail(c, SJA_ERR_STATE, "sja_advertise_power_caps before sja_advertise");
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     if (cap_W) {
         TRY(reserve(c, c->caps, (size_t)c->G * 4));
         TRY(copy_in(c, c->caps.p, cap_W, (size_t)c->G * 4, where));
@@ -1148,6 +1178,7 @@ sja_status sja_set_window_options(sja_ctx* c, uint32_t late_start, const uint32_
         return fail(c, SJA_ERR_INVALID_ARG, "sja_set_window_options: bad memspace");
     if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_set_window_options before sja_load_profiles");
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     if (deadline_ms) {
         TRY(reserve(c, c->deadline, (size_t)c->J * 4));
         TRY(copy_in(c, c->deadline.p, deadline_ms, (size_t)c->J * 4, where));
@@ -1165,6 +1196,7 @@ sja_status sja_get_awards(sja_ctx* c, sja_award* out, sja_memspace where) {
     if (!out) return fail(c, SJA_ERR_INVALID_ARG, "sja_get_awards: out is NULL");
     if (!c->selected && !c->committed) return fail(c, SJA_ERR_STATE, "sja_get_awards before sja_select");
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     TRY(copy_out(c, out, c->awards.p, (size_t)c->G * sizeof(sja_award), where));
     if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));
     return SJA_OK;
@@ -1174,6 +1206,7 @@ sja_status sja_get_state(sja_ctx* c, uint32_t* progress, uint32_t* ready_ms, sja
     TRY(check_ctx(c));
     if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_get_state before sja_load_profiles");
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     if (progress) TRY(copy_out(c, progress, c->p.p, (size_t)c->J * 4, where));
     if (ready_ms) TRY(copy_out(c, ready_ms, c->ready.p, (size_t)c->J * 4, where));
     if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));
@@ -1193,6 +1226,7 @@ sja_status sja_get_scan(sja_ctx* c, uint64_t* boff, uint32_t* k, uint32_t* D, ui
     TRY(check_ctx(c));
     if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_get_scan before sja_load_profiles");
     DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     const uint64_t n = c->n_rows;
     if (boff) TRY(copy_out(c, boff, c->boff.p, (size_t)(c->J + 1) * 8, where));
     if (n == 0) {

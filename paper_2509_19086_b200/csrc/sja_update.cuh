@@ -1,5 +1,5 @@
-// Re-profiling of one job (Section 3.9: the envelope U(t) may evolve as runtime predictions are
-// refined, which is why segmentation happens on demand).  The caller hands in new per-step
+// Re-profiling of one job (Section 3.9: segmentation is done at offer time because a job's envelope U(t)
+// can change between offers as its predictions improve).  The caller hands in new per-step
 // durations and memory values for the steps the job has not been granted yet; its safe
 // boundaries stay where they are, so the job keeps its rows of the boundary table and only
 // their contents are recomputed: cumulative duration, running maximum from the progress

@@ -340,6 +340,48 @@ def test_error_paths(sja_mod):
         assert e.value.status == 3
 
 
+def test_failed_allocation_leaves_a_usable_context(sja_mod, oracle_mod):
+    """A device allocation that fails inside sja_advertise (injected on the host: the n-th growing allocation
+    reports out-of-memory without being tried) must leave no half-built batch behind: select and commit answer
+    SJA_ERR_STATE and launch nothing, the loaded profiles stay usable, and the next advertise works."""
+    spec = wl.scaled(wl.SPECS[1], n_jobs=400, fixed_len=300, n_gaps=64)
+    prof = wl.make_profiles(spec, threads=1)
+    small, large = wl.make_gaps(spec), wl.make_gaps(spec, 1, n_gaps=9000)
+    zero = np.zeros(prof.n_jobs, np.uint32)
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof)
+        ctx.advertise(small)
+        want_small = oracle_mod.select(prof, zero, prof.ready_ms, small, spec.policy)
+        _assert_awards_equal(ctx.select(spec.policy, out="host"), want_small)
+        for nth in (1, 2, 3, 4, 5, 6):              # each of the six buffers a larger batch has to grow
+            ctx.debug_fail_alloc(nth)
+            with pytest.raises(sja_mod.SjaError) as e:
+                ctx.advertise(large[:1500 * nth])   # larger than any batch before: all six grow again
+            assert e.value.status == 5, nth         # SJA_ERR_OOM
+            for call in (lambda: ctx.select(spec.policy), ctx.commit, ctx.get_awards):
+                with pytest.raises(sja_mod.SjaError) as e:
+                    call()
+                assert e.value.status == 4, nth     # SJA_ERR_STATE: there is no batch
+            ctx.debug_fail_alloc(0)
+            ctx.advertise(small)                    # the context is still good
+            _assert_awards_equal(ctx.select(spec.policy, out="host"), want_small)
+        ctx.advertise(large)
+        want_large = oracle_mod.select(prof, zero, prof.ready_ms, large, spec.policy)
+        _assert_awards_equal(ctx.select(spec.policy, out="host"), want_large)
+        # a failure while select grows its candidate rows: the batch stays advertised, the next select works
+        ctx.advertise(wl.make_gaps(spec, 2, n_gaps=12000))
+        ctx.debug_fail_alloc(1)
+        with pytest.raises(sja_mod.SjaError) as e:
+            ctx.select(spec.policy)
+        assert e.value.status == 5
+        with pytest.raises(sja_mod.SjaError) as e:
+            ctx.commit()
+        assert e.value.status == 4
+        want = oracle_mod.select(prof, zero, prof.ready_ms, wl.make_gaps(spec, 2, n_gaps=12000), spec.policy)
+        _assert_awards_equal(ctx.select(spec.policy, out="host"), want)
+        assert ctx.commit() > 0
+
+
 def test_empty_and_degenerate_inputs(sja_mod, oracle_mod):
     # all jobs empty; a job that is already finished; gaps nobody fits
     prof = profiles_from_lists([([], [], []), ([], [], [])])

@@ -240,6 +240,40 @@ def test_p4_dense_prefix_matches_walk(oracle_mod):
         assert rows[-1][0] == length
 
 
+def test_p4_boundary_table_segment_maximum(oracle_mod):
+    """The segment-maximum column of the boundary rows.  Hand-computed example, then the property the column
+    exists for: started at any boundary row r0, the running maximum of the segment maxima over rows r0..r is
+    the window maximum max m[k_{r0-1} .. k_r), i.e. the M column of a scan that starts at progress k_{r0-1}
+    (library maximum.accumulate on the raw steps, not on the table)."""
+    oracle = oracle_mod
+    #            step  0  1  2  3  4  5  6  7
+    prof = profiles_from_lists([([1, 2, 3, 4, 5, 6, 7, 8], [5, 9, 2, 7, 7, 1, 8, 3], [0, 1, 0, 0, 1, 1, 0, 0])])
+    rows = oracle.boundary_table(prof, 0, 0)
+    assert [(r[0], r[3]) for r in rows] == [(2, 9), (5, 7), (6, 1), (8, 8)]          # (k, segment maximum)
+    assert [(r[1], r[2], r[4]) for r in rows] == [(3, 9, 23), (15, 9, 92), (21, 9, 98), (36, 9, 178)]   # D, M, W
+    rows = oracle.boundary_table(prof, 0, 3)          # from progress 3: the first segment is steps 3..4 only
+    assert [(r[0], r[3], r[2]) for r in rows] == [(5, 7, 7), (6, 1, 7), (8, 8, 8)]   # (k, segment max, M)
+    rng = np.random.default_rng(55)
+    jobs = random_small_profiles(rng, 12, 80, p_safe=0.25, dmax=30, mmax=500)
+    prof = profiles_from_lists(jobs)
+    for j in range(prof.n_jobs):
+        s = int(prof.off[j])
+        length = int(prof.off[j + 1]) - s
+        p0 = int(rng.integers(0, length))
+        rows = oracle.boundary_table(prof, j, p0)
+        ks = [p0] + [r[0] for r in rows]
+        m = prof.mem_MiB[s:s + length]
+        for r0 in range(len(rows)):
+            start = ks[r0]                               # progress point after committing up to row r0 - 1
+            run = 0
+            win = np.maximum.accumulate(m[start:])
+            for r in range(r0, len(rows)):
+                k, seg = rows[r][0], rows[r][3]
+                assert seg == int(m[ks[r]:k].max())      # the segment since the previous boundary, nothing else
+                run = max(run, seg)
+                assert run == int(win[k - start - 1]), (j, p0, r0, r)
+
+
 # ---------------------------------------------------------------- P5 closed form
 @pytest.mark.parametrize("a,b,q,n,T,wait", [
     (7, 11, 4, 100, 365, 0), (1, 1, 1, 50, 17, 999), (13, 5, 10, 95, 5000, 123456),
