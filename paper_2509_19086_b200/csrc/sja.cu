@@ -281,10 +281,10 @@ enum SelectKernel { SEL_TILE = 0, SEL_MERGE = 1, SEL_SEARCH = 2 };
 
 template <uint32_t KIND, bool BOUNDED>
 void launch_sorted_kb(SelectKernel which, dim3 grid, cudaStream_t stream, const JobView& jv, const Gap* sgaps,
-                      uint32_t G, uint32_t per_split, Partial* partial, const uint32_t* G_dev, uint32_t* flags) {
+                      uint32_t G, uint32_t per_split, Partial* partial, const uint32_t* G_dev) {
     if (which == SEL_TILE)
         select_tile_kernel<KIND, BOUNDED><<<grid, TILE_WARPS * 32, TILE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split,
-                                                                                             partial, G_dev, flags);
+                                                                                             partial, G_dev);
     else
         select_merge_kernel<KIND, BOUNDED><<<grid, MERGE_WARPS * 32, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G,
                                                                                                 per_split, partial);
@@ -292,25 +292,23 @@ void launch_sorted_kb(SelectKernel which, dim3 grid, cudaStream_t stream, const 
 
 template <bool BOUNDED>
 void launch_sorted_b(SelectKernel which, uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& jv,
-                     const Gap* sgaps, uint32_t G, uint32_t per_split, Partial* partial, const uint32_t* G_dev,
-                     uint32_t* flags) {
+                     const Gap* sgaps, uint32_t G, uint32_t per_split, Partial* partial, const uint32_t* G_dev) {
     if (kind == SJA_POLICY_FAIRNESS)
-        launch_sorted_kb<1, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev, flags);
+        launch_sorted_kb<1, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
     else if (kind == SJA_POLICY_SLA)
-        launch_sorted_kb<2, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev, flags);
+        launch_sorted_kb<2, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
     else if (kind == SJA_POLICY_TIGHT_FIT)
-        launch_sorted_kb<3, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev, flags);
+        launch_sorted_kb<3, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
     else
-        launch_sorted_kb<0, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev, flags);
+        launch_sorted_kb<0, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
 }
 
 void launch_sorted(SelectKernel which, uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& jv,
-                   const Gap* sgaps, uint32_t G, uint32_t per_split, Partial* partial, const uint32_t* G_dev,
-                   uint32_t* flags) {
+                   const Gap* sgaps, uint32_t G, uint32_t per_split, Partial* partial, const uint32_t* G_dev) {
     if (jv.tau_min != 0u || jv.tau_max != 0xFFFFFFFFu)
-        launch_sorted_b<true>(which, kind, grid, stream, jv, sgaps, G, per_split, partial, G_dev, flags);
+        launch_sorted_b<true>(which, kind, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
     else
-        launch_sorted_b<false>(which, kind, grid, stream, jv, sgaps, G, per_split, partial, G_dev, flags);
+        launch_sorted_b<false>(which, kind, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
 }
 
 template <uint32_t KIND, bool BOUNDED>
@@ -402,7 +400,7 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
         jv.blocked = blocked;
         if (pl.kernel != SEL_SEARCH) {
             launch_sorted(pl.kernel, kind, dim3(n_chunks, splits), c->stream, jv, sgaps, G_act, per_split, partial,
-                          G_dev, c->flags.as<uint32_t>());
+                          G_dev);
         } else {
             const bool opts = jv.late_start != 0u || jv.deadline != nullptr || jv.PW != nullptr;
             if (opts)

@@ -15,7 +15,6 @@ enum : uint32_t {
     FLAG_OVF_READY = 1u << 5,     // start + dur >= 2^32 at commit
     FLAG_INTERNAL = 1u << 6,      // self-check failed (boundary count mismatch)
     FLAG_NEED_ROWS = 1u << 7,     // the boundary table of this load needs more rows than the buffers given hold
-    FLAG_TIMEOUT = 1u << 8,       // a bounded wait inside a kernel gave up (results of that launch are not valid)
 };
 
 constexpr uint32_t SJA_NO_JOB_DEV = 0xFFFFFFFFu;

@@ -28,15 +28,6 @@
 // The cost is therefore per (warp, 32 gaps) a small fixed part (the lookup) plus the cursor
 // steps, not the number of pairs.  The PM is rebuilt by a warp scan only after a restart of
 // the cursors (a new capacity class, or the start of a CTA's gap range).
-//
-// The warps of a CTA never meet at a CTA-wide barrier while they sweep: how many cursor steps a
-// run of gaps costs differs from warp to warp, and a barrier per tile made every warp wait for
-// the slowest one of each tile.  Instead a warp drops its candidates of a tile of TILE_GT gaps
-// into its row of one of TILE_NB staging buffers and counts itself in on a shared-memory
-// counter; the warp that finds itself to be the last one folds the tile's rows into the CTA's
-// candidates and releases the buffer.  A warp only ever waits when it is TILE_NB tiles ahead of
-// the slowest warp of its CTA (the buffer it wants has not been folded yet); that wait is
-// bounded and raises FLAG_TIMEOUT if it gives up.
 #pragma once
 #include "sja_round.cuh"
 
@@ -52,10 +43,7 @@ namespace sja {
 #define SJA_TILE_RING 4
 #endif
 #ifndef SJA_TILE_GT
-#define SJA_TILE_GT 64
-#endif
-#ifndef SJA_TILE_NB
-#define SJA_TILE_NB 4
+#define SJA_TILE_GT 256
 #endif
 #ifndef SJA_TILE_MULTI
 #define SJA_TILE_MULTI 2
@@ -63,17 +51,16 @@ namespace sja {
 constexpr int TILE_WARPS = SJA_TILE_WARPS;
 constexpr int TILE_CTAS_PER_SM = SJA_TILE_CTAS_PER_SM;
 constexpr int TILE_RING = SJA_TILE_RING;     // rows per job ring (power of two)
-constexpr int TILE_GT = SJA_TILE_GT;         // gaps per staging tile (multiple of 32 x SJA_TILE_MULTI)
-constexpr int TILE_NB = SJA_TILE_NB;         // staging buffers: how many tiles the warps of a CTA may drift apart
+constexpr int TILE_GT = SJA_TILE_GT;         // gaps per staging tile (multiple of 32)
 constexpr int TILE_JOBS = TILE_WARPS * 32;
 constexpr int TILE_RING_BYTES = TILE_WARPS * TILE_RING * 32 * 16;
-constexpr int TILE_STAGE_BYTES = TILE_NB * TILE_WARPS * TILE_GT * 16;
+constexpr int TILE_STAGE_BYTES = TILE_WARPS * TILE_GT * 16;
+constexpr int TILE_GAP_BYTES = TILE_GT * 16;
 constexpr int TILE_EVENT_BYTES = TILE_WARPS * 32 * 16;   // posted events, one slot per lane
 constexpr int TILE_ECNT_BYTES = TILE_WARPS * 32 * 4;     // their row counts
-constexpr int TILE_SMEM_BYTES = TILE_RING_BYTES + TILE_STAGE_BYTES + TILE_EVENT_BYTES + TILE_ECNT_BYTES;
-constexpr uint32_t TILE_WAIT_LIMIT = 1u << 24;           // polls of a staging buffer before a warp gives up
+constexpr int TILE_SMEM_BYTES = TILE_RING_BYTES + TILE_STAGE_BYTES + TILE_GAP_BYTES + TILE_EVENT_BYTES + TILE_ECNT_BYTES;
 static_assert((TILE_RING & (TILE_RING - 1)) == 0, "ring size must be a power of two");
-static_assert(TILE_GT % (32 * SJA_TILE_MULTI) == 0, "a tile is a whole number of warp passes");
+static_assert(TILE_GT % 32 == 0 && TILE_GT <= TILE_JOBS, "one thread per gap of a staging tile");
 
 // Candidate order: larger key first, then the lower job id.
 __device__ __forceinline__ bool cand_better(uint64_t ka, uint32_t ja, uint64_t kb, uint32_t jb) {
@@ -90,7 +77,7 @@ __device__ __forceinline__ bool pair_ge(uint64_t ka, uint32_t ia, uint64_t kb, u
 template <uint32_t KIND, bool BOUNDED>
 __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile_kernel(
     JobView jv, const Gap* __restrict__ sgaps, uint32_t G, uint32_t gaps_per_split, Partial* __restrict__ partial_out,
-    const uint32_t* __restrict__ G_dev, uint32_t* __restrict__ flags) {
+    const uint32_t* __restrict__ G_dev) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // G is the gap count the launch was sized for (and the row length of partial_out); a re-auction hands
     // the count actually left in device memory, so that several passes can be queued without a host wait
@@ -98,15 +85,12 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
     if (blockIdx.y * gaps_per_split >= G_now) return;
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
     const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(smem_raw);
-    Partial* stage_all = reinterpret_cast<Partial*>(smem_raw + TILE_RING_BYTES);                   // [NB][WARPS][GT]
-    uint4* ev = reinterpret_cast<uint4*>(smem_raw + TILE_RING_BYTES + TILE_STAGE_BYTES) + wid * 32;
-    uint32_t* evc = reinterpret_cast<uint32_t*>(smem_raw + TILE_RING_BYTES + TILE_STAGE_BYTES + TILE_EVENT_BYTES) +
-                    wid * 32;
-    // hand-over of the staging buffers: warps counted in on the current tile of a buffer, tiles folded so far
-    __shared__ uint32_t arrived[TILE_NB];
-    __shared__ uint32_t folded[TILE_NB];
-    if (threadIdx.x < TILE_NB) { arrived[threadIdx.x] = 0u; folded[threadIdx.x] = 0u; }
-    __syncthreads();
+    Partial* stage = reinterpret_cast<Partial*>(smem_raw + TILE_RING_BYTES);                       // [WARPS][GT]
+    const uint4* sg = reinterpret_cast<const uint4*>(smem_raw + TILE_RING_BYTES + TILE_STAGE_BYTES);
+    uint4* sg_w = reinterpret_cast<uint4*>(smem_raw + TILE_RING_BYTES + TILE_STAGE_BYTES);
+    uint4* ev = reinterpret_cast<uint4*>(smem_raw + TILE_RING_BYTES + TILE_STAGE_BYTES + TILE_GAP_BYTES) + wid * 32;
+    uint32_t* evc = reinterpret_cast<uint32_t*>(smem_raw + TILE_RING_BYTES + TILE_STAGE_BYTES + TILE_GAP_BYTES +
+                                                TILE_EVENT_BYTES) + wid * 32;
     const uint32_t ring_s = smem_s + (wid * TILE_RING * 32 + lane) * 16;   // slot i of the ring: + i * 512
 
     // ---- the lane's job
@@ -172,21 +156,8 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
 
     for (uint32_t g0 = g_begin; g0 < g_end; g0 += TILE_GT) {
         const uint32_t gt = min((uint32_t)TILE_GT, g_end - g0);
-        const uint32_t tile_no = (g0 - g_begin) / TILE_GT;
-        const uint32_t buf = tile_no % TILE_NB, use = tile_no / TILE_NB;
-        if (use) {
-            // the tile that used this buffer last must have been folded (by the last warp that finished it)
-            uint32_t polls = 0;
-            while (*reinterpret_cast<volatile uint32_t*>(&folded[buf]) < use) {
-                __nanosleep(64);
-                if (++polls > TILE_WAIT_LIMIT) {
-                    if (lane == 0) atomicOr(flags, FLAG_TIMEOUT);
-                    break;
-                }
-            }
-            __threadfence_block();
-        }
-        Partial* stage = stage_all + (size_t)(buf * TILE_WARPS + wid) * TILE_GT;    // this warp's row of the buffer
+        if (threadIdx.x < gt) sg_w[threadIdx.x] = __ldg(reinterpret_cast<const uint4*>(sgaps) + g0 + threadIdx.x);
+        __syncthreads();
         for (uint32_t sub = 0; sub < gt; sub += 32) {
 #if SJA_TILE_MULTI > 1
             // Fast path: MULTI x 32 gaps of the class the cursors are in, MULTI per lane.  One set of cursor
@@ -196,7 +167,7 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
             if (multi) {
                 bool same = true;
 #pragma unroll
-                for (int q = 0; q < SJA_TILE_MULTI; ++q) same = same && __ldg(&sgaps[g0 + sub + 32 * q + lane].C) == curC;
+                for (int q = 0; q < SJA_TILE_MULTI; ++q) same = same && sg[sub + 32 * q + lane].w == curC;
                 multi = __all_sync(0xFFFFFFFFu, same);
             }
             if (multi) {
@@ -204,7 +175,7 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
                 uint64_t kq[SJA_TILE_MULTI];
 #pragma unroll
                 for (int q = 0; q < SJA_TILE_MULTI; ++q) {
-                    const uint4 gq = __ldg(reinterpret_cast<const uint4*>(sgaps) + g0 + sub + 32 * q + lane);
+                    const uint4 gq = sg[sub + 32 * q + lane];
                     Tq[q] = BOUNDED ? min(gq.z, jv.tau_max) : gq.z;
                     uint32_t e = 0;
 #pragma unroll
@@ -259,7 +230,7 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
                 for (int q = 0; q < SJA_TILE_MULTI; ++q) {
                     Partial pr;
                     pr.key = kq[q]; pr.job = kq[q] ? job0 + 31u - iq[q] : 0xFFFFFFFFu; pr.cnt = kq[q] ? cq[q] : 0u;
-                    stage[sub + 32 * q + lane] = pr;
+                    stage[wid * TILE_GT + sub + 32 * q + lane] = pr;
                 }
                 sub += 32u * (SJA_TILE_MULTI - 1);
                 continue;
@@ -267,7 +238,7 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
 #endif
             const bool in = sub + lane < gt;
             uint4 gq = make_uint4(0u, 0u, 0u, 0u);
-            if (in) gq = __ldg(reinterpret_cast<const uint4*>(sgaps) + g0 + sub + lane);
+            if (in) gq = sg[sub + lane];
             const uint32_t start = gq.y, C = gq.w;
             const uint32_t T = BOUNDED ? min(gq.z, jv.tau_max) : gq.z;
             // number of jobs of the warp that are ready by this gap's start (they are ranks 0 .. e-1)
@@ -375,36 +346,20 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
             if (in) {
                 Partial pr;
                 pr.key = bk; pr.job = bk ? job0 + 31u - bi : 0xFFFFFFFFu; pr.cnt = bk ? bc : 0u;
-                stage[sub + lane] = pr;
+                stage[wid * TILE_GT + sub + lane] = pr;
             }
         }
-        // count this warp in; the last one to arrive folds the tile and hands the buffer back
-        __syncwarp();
-        uint32_t before = 0;
-        if (lane == 0) {
-            __threadfence_block();
-            before = atomicAdd(&arrived[buf], 1u);
-        }
-        before = __shfl_sync(0xFFFFFFFFu, before, 0);
-        if (before == (uint32_t)TILE_WARPS - 1u) {
-            __threadfence_block();
-            const Partial* rows = stage_all + (size_t)buf * TILE_WARPS * TILE_GT;
-            for (uint32_t gi = lane; gi < gt; gi += 32) {
-                Partial bestp = rows[gi];
+        __syncthreads();
+        if (threadIdx.x < gt) {
+            Partial bestp = stage[threadIdx.x];
 #pragma unroll
-                for (int ww = 1; ww < TILE_WARPS; ++ww) {
-                    const Partial c = rows[ww * TILE_GT + gi];
-                    if (cand_better(c.key, c.job, bestp.key, bestp.job)) bestp = c;
-                }
-                partial_out[(size_t)blockIdx.x * G + g0 + gi] = bestp;
+            for (int ww = 1; ww < TILE_WARPS; ++ww) {
+                const Partial c = stage[ww * TILE_GT + threadIdx.x];
+                if (cand_better(c.key, c.job, bestp.key, bestp.job)) bestp = c;
             }
-            __syncwarp();
-            if (lane == 0) {
-                arrived[buf] = 0u;
-                __threadfence_block();
-                *reinterpret_cast<volatile uint32_t*>(&folded[buf]) = use + 1u;
-            }
+            partial_out[(size_t)blockIdx.x * G + g0 + threadIdx.x] = bestp;
         }
+        __syncthreads();
     }
     mg_wait<0>();
 }
