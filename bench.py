@@ -41,10 +41,17 @@ FALLBACK_HBM_GBS = 6650.0
 N_SM, SCHEDULERS_PER_SM = 148, 4
 
 # Kernels launched by one call of each entry point on the default path (counted from the launch list of this
-# command under ncu): load = count_boundaries, cta_offsets, row_offsets, init_state, scan_profiles; advertise =
-# sort_gap_tiles, rank_gap_tiles, place_gaps, count_classes (a batch of at most 1024 gaps: sort_gap_tiles alone);
-# select = select_tile (or select_search) + finalize_awards; commit = commit_vote, commit_apply, commit_refresh.
-LAUNCHES_LOAD, LAUNCHES_ADVERTISE, LAUNCHES_ADVERTISE_ONE_TILE, LAUNCHES_SELECT, LAUNCHES_COMMIT = 5, 4, 1, 2, 3
+# command under ncu): load = count_boundaries, cta_offsets, finish_load, scan_profiles; advertise = sort_gap_tiles,
+# rank_gap_tiles, place_gaps (a batch of at most 1024 gaps: sort_gap_tiles alone); select = select_tile, the
+# select_search launch that stands by for batches of very many capacity classes (it returns at once otherwise),
+# finalize_awards -- or select_search + finalize_awards where only the search runs; commit = commit_vote,
+# commit_apply, commit_refresh.
+LAUNCHES_LOAD, LAUNCHES_ADVERTISE, LAUNCHES_ADVERTISE_ONE_TILE, LAUNCHES_COMMIT = 4, 3, 1, 3
+
+
+def select_launches(pairs, flags, per_pair_window):
+    return 2 if (flags & 1) or per_pair_window or pairs < 65536 else 3
+
 
 # DRAM traffic of the scan kernel, from one ncu capture of dram__bytes_read.sum and dram__bytes_write.sum on the
 # large uniform configuration at full size: reads grow with the step count, writes with the number of boundary
@@ -403,6 +410,7 @@ def bench_workload(env, args, spec, *, streaming, steps, warmup, e2e_steps, samp
 
     launches = [0]
     adv_launches = LAUNCHES_ADVERTISE_ONE_TILE if G <= 1024 else LAUNCHES_ADVERTISE
+    LAUNCHES_SELECT = select_launches(pairs, flags, window_options or power_caps)
     round_gaps_dev, round_gaps_pinned = [], []
     if streaming:
         # one gap batch per round, resident on the device (and pinned on the host for the end-to-end leg)

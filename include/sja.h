@@ -180,9 +180,10 @@ sja_status sja_select(sja_ctx* ctx, const sja_policy* policy, sja_award* out, sj
  * cudaFree or other allocating routine and records no profiling events.
  *
  * Cost and limit: every GPU on which the library is used holds the array until the process
- * exits.  The call needs ceil(J / 512) * G candidate slots of 16 bytes (ceil(J / 1024) * G
- * with SJA_FLAG_FORCE_MERGE; ceil(J / 256) * G where the per-pair search runs, see the flags); if that exceeds the array it returns SJA_ERR_INVALID_ARG with the
- * numbers in sja_last_error() and does nothing.
+ * exits.  The call needs ceil(J / 256) * G candidate slots of 16 bytes (one per gap and per
+ * chunk of 256 jobs, the chunk of the per-pair search kernel, which runs or stands by in every
+ * select); if that exceeds the array it returns SJA_ERR_INVALID_ARG with the numbers in
+ * sja_last_error() and does nothing.
  *
  * The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
  * the context's device current); make that first call before starting any stream capture.

@@ -60,7 +60,7 @@ struct sja_ctx {
     uint64_t N = 0, n_rows = 0;
     bool have_wait = false, have_prio = false;
     uint32_t load_flags = 0;
-    DevBuf st_off, st_d, st_m, st_s, st_p;            // staging for host inputs / load-time progress
+    DevBuf st_off, st_d, st_m, st_s, st_p, st_ready, st_wait, st_prio;   // staging for host inputs
     DevBuf p, ready, pb, Dp, Wp, wait, prio;          // per-job state and attributes
     DevBuf nbj, cta_tot, cta_base, boff, boff_next, A, B, jobwin;   // row counting scratch, boundary table
     DevBuf flags, counter, n_granted;                 // small device words
@@ -78,7 +78,6 @@ struct sja_ctx {
     DevBuf st_bids, st_accept, st_global;              // sharded rounds: staging for host-side callers
     DevBuf upd_d, upd_m, upd_scratch, upd_status;   // sja_update_profile: staged inputs, segment values, verdict
     bool gaps_sorted = false;          // sgaps is ordered by (C, T); else it is the caller's order
-    uint32_t n_classes = 0;            // distinct capacities of the batch (valid when sorted)
     DevBuf gaps, sgaps, gap_info, gap_rank, awards, widx, partial, winners;
     DevBuf sgaps_alt, blocked, n_active, accept;   // re-auction: second ordered gap list, per-job block flags, gap counter
 
@@ -281,34 +280,34 @@ enum SelectKernel { SEL_TILE = 0, SEL_MERGE = 1, SEL_SEARCH = 2 };
 
 template <uint32_t KIND, bool BOUNDED>
 void launch_sorted_kb(SelectKernel which, dim3 grid, cudaStream_t stream, const JobView& jv, const Gap* sgaps,
-                      uint32_t G, uint32_t per_split, Partial* partial, const uint32_t* G_dev) {
+                      uint32_t G, uint32_t per_split, Partial* partial, const LaunchGate& gate) {
     if (which == SEL_TILE)
         select_tile_kernel<KIND, BOUNDED><<<grid, TILE_WARPS * 32, TILE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split,
-                                                                                             partial, G_dev);
+                                                                                             partial, gate);
     else
         select_merge_kernel<KIND, BOUNDED><<<grid, MERGE_WARPS * 32, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G,
-                                                                                                per_split, partial);
+                                                                                                per_split, partial, gate);
 }
 
 template <bool BOUNDED>
 void launch_sorted_b(SelectKernel which, uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& jv,
-                     const Gap* sgaps, uint32_t G, uint32_t per_split, Partial* partial, const uint32_t* G_dev) {
+                     const Gap* sgaps, uint32_t G, uint32_t per_split, Partial* partial, const LaunchGate& gate) {
     if (kind == SJA_POLICY_FAIRNESS)
-        launch_sorted_kb<1, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
+        launch_sorted_kb<1, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, gate);
     else if (kind == SJA_POLICY_SLA)
-        launch_sorted_kb<2, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
+        launch_sorted_kb<2, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, gate);
     else if (kind == SJA_POLICY_TIGHT_FIT)
-        launch_sorted_kb<3, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
+        launch_sorted_kb<3, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, gate);
     else
-        launch_sorted_kb<0, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
+        launch_sorted_kb<0, BOUNDED>(which, grid, stream, jv, sgaps, G, per_split, partial, gate);
 }
 
 void launch_sorted(SelectKernel which, uint32_t kind, dim3 grid, cudaStream_t stream, const JobView& jv,
-                   const Gap* sgaps, uint32_t G, uint32_t per_split, Partial* partial, const uint32_t* G_dev) {
+                   const Gap* sgaps, uint32_t G, uint32_t per_split, Partial* partial, const LaunchGate& gate) {
     if (jv.tau_min != 0u || jv.tau_max != 0xFFFFFFFFu)
-        launch_sorted_b<true>(which, kind, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
+        launch_sorted_b<true>(which, kind, grid, stream, jv, sgaps, G, per_split, partial, gate);
     else
-        launch_sorted_b<false>(which, kind, grid, stream, jv, sgaps, G, per_split, partial, G_dev);
+        launch_sorted_b<false>(which, kind, grid, stream, jv, sgaps, G, per_split, partial, gate);
 }
 
 template <uint32_t KIND, bool BOUNDED>
@@ -342,12 +341,40 @@ sja_status check_policy(sja_ctx* c, const sja_policy* policy, const char* who) {
 
 // Launch signal + score + select for the first G_act entries of `sgaps` (ordered or not);
 // awards and widx are written at the gaps' original indices.  `blocked` may be nullptr.
-struct SelectPlan { SelectKernel kernel; uint32_t jobs_per_cta, tile, n_chunks; };
+//
+// Which kernel: the per-pair search alone where only it can serve the round (it is asked for, a window option or
+// power caps are in force, the batch is not ordered) or where the round is small; else an ordered-gap kernel
+// (tile sweep, or the merge kernel on request) AND the search kernel behind it: the number of capacity classes
+// of the batch lives in device memory (the host does not wait for sja_advertise), so both are queued and each
+// looks at the count -- with very many classes the ordered-gap kernels would pay one cursor restart per class,
+// and the search serves the round instead.
+struct KernelPlan { SelectKernel kernel; uint32_t jobs_per_cta, n_chunks, splits, per_split; };
+struct SelectPlan { KernelPlan primary, alt; bool have_alt; uint32_t max_classes; uint32_t rows; };
+
+KernelPlan plan_kernel(const sja_ctx* c, SelectKernel k, uint32_t G_act) {
+    KernelPlan p;
+    p.kernel = k;
+    p.jobs_per_cta = k == SEL_TILE ? (uint32_t)TILE_JOBS : k == SEL_MERGE ? (uint32_t)MERGE_JOBS : (uint32_t)SEARCH_THREADS;
+    p.n_chunks = (c->J + p.jobs_per_cta - 1) / p.jobs_per_cta;
+    // granularity of a gap split: a staging tile; the tile kernel also works in 32-gap steps, which a
+    // small problem needs to put enough CTAs on the GPU
+    uint32_t tile = k == SEL_TILE ? (uint32_t)TILE_GT : k == SEL_MERGE ? (uint32_t)MERGE_GT : (uint32_t)SEARCH_GT;
+    if (k == SEL_TILE && (uint64_t)p.n_chunks * ((G_act + tile - 1) / tile) < (uint64_t)SJA_SELECT_CTAS_PER_SM * c->n_sm)
+        tile = 32u;
+    // split the gaps so that the grid covers the SMs several times over
+    uint32_t splits = (uint32_t)(((uint64_t)SJA_SELECT_CTAS_PER_SM * c->n_sm + p.n_chunks - 1) / p.n_chunks);
+    const uint32_t max_splits = (G_act + tile - 1) / tile;
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    uint32_t per_split = (G_act + splits - 1) / splits;
+    per_split = ((per_split + tile - 1) / tile) * tile;
+    p.per_split = per_split;
+    p.splits = (G_act + per_split - 1) / per_split;
+    return p;
+}
 
 SelectPlan plan_select(const sja_ctx* c, uint32_t pflags, uint32_t G_act) {
     SelectPlan p;
-    // The tile and merge kernels need the (capacity, T) order and pay one restart per capacity
-    // class; with very many classes (or an unsorted batch) the per-pair search is the better tool.
     const bool forced = (pflags & (SJA_FLAG_FORCE_MERGE | SJA_FLAG_FORCE_TILE)) != 0;
     // A round of a few thousand pairs cannot fill the GPU either way; there the cursors' sequential walk
     // through each capacity class is pure latency and the independent per-pair searches finish sooner.
@@ -356,63 +383,61 @@ SelectPlan plan_select(const sja_ctx* c, uint32_t pflags, uint32_t G_act) {
     const bool tiny = (uint64_t)c->J * c->G < (1ull << 16) || (G_act < c->G && (uint64_t)c->J * G_act < (1ull << 21));
     // with a window option the usable window differs from pair to pair: only the search kernel does that
     const bool per_pair_window = c->late_start || c->have_deadline || (c->have_power && c->have_caps);
-    const bool sorted_ok = !(pflags & SJA_FLAG_FORCE_SEARCH) && !per_pair_window && c->gaps_sorted && (forced || !tiny) &&
-                           c->n_classes <= std::max<uint32_t>(64u, c->G / 16u);
-    p.kernel = !sorted_ok ? SEL_SEARCH : (pflags & SJA_FLAG_FORCE_MERGE) ? SEL_MERGE : SEL_TILE;
-    p.jobs_per_cta = p.kernel == SEL_TILE ? (uint32_t)TILE_JOBS
-                                          : p.kernel == SEL_MERGE ? (uint32_t)MERGE_JOBS : (uint32_t)SEARCH_THREADS;
-    p.tile = p.kernel == SEL_TILE ? (uint32_t)TILE_GT : p.kernel == SEL_MERGE ? (uint32_t)MERGE_GT : (uint32_t)SEARCH_GT;
-    p.n_chunks = (c->J + p.jobs_per_cta - 1) / p.jobs_per_cta;
+    const bool search_only = (pflags & SJA_FLAG_FORCE_SEARCH) || per_pair_window || !c->gaps_sorted || (!forced && tiny);
+    p.max_classes = std::max<uint32_t>(64u, c->G / 16u);
+    p.have_alt = !search_only;
+    p.primary = plan_kernel(c, search_only ? SEL_SEARCH : (pflags & SJA_FLAG_FORCE_MERGE) ? SEL_MERGE : SEL_TILE, G_act);
+    p.alt = plan_kernel(c, SEL_SEARCH, G_act);
+    p.rows = p.have_alt ? std::max(p.primary.n_chunks, p.alt.n_chunks) : p.primary.n_chunks;
     return p;
 }
 
-// `scratch`: candidate rows (n_chunks x G entries); nullptr = the context's own buffer, grown on demand.
+// `scratch`: candidate rows (plan rows x G entries); nullptr = the context's own buffer, grown on demand.
 // `timed`: record profiling events (creates CUDA events on first use).
 // `G_dev`: optional device word with the number of gaps actually left (<= G_act, which then only sizes the launch).
 sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sgaps, uint32_t G_act,
                       const uint32_t* blocked, Partial* scratch = nullptr, bool timed = true,
                       const uint32_t* G_dev = nullptr) {
     const SelectPlan pl = plan_select(c, pflags, G_act);
-    const uint32_t n_chunks = pl.n_chunks;
-    // granularity of a gap split: a staging tile; the tile kernel also works in 32-gap steps, which a
-    // small problem needs to put enough CTAs on the GPU
-    uint32_t tile = pl.tile;
-    if (pl.kernel == SEL_TILE && (uint64_t)n_chunks * ((G_act + tile - 1) / tile) < (uint64_t)SJA_SELECT_CTAS_PER_SM * c->n_sm)
-        tile = 32u;
     Partial* partial = scratch;
     if (!partial) {
-        TRY(reserve(c, c->partial, (size_t)n_chunks * c->G * sizeof(Partial)));
+        TRY(reserve(c, c->partial, (size_t)pl.rows * c->G * sizeof(Partial)));
         partial = c->partial.as<Partial>();
     }
-    // split the gaps so that the grid covers the SMs several times over
-    uint32_t splits = (uint32_t)(((uint64_t)SJA_SELECT_CTAS_PER_SM * c->n_sm + n_chunks - 1) / n_chunks);
-    const uint32_t max_splits = (G_act + tile - 1) / tile;
-    if (splits > max_splits) splits = max_splits;
-    if (splits < 1) splits = 1;
-    uint32_t per_split = (G_act + splits - 1) / splits;
-    per_split = ((per_split + tile - 1) / tile) * tile;
-    splits = (G_act + per_split - 1) / per_split;
     const int was_on = c->prof;
     if (!timed) c->prof = 0;
     {
         ProfScope ps(c, CAT_SELECT);
         JobView jv = job_view(c);
         jv.blocked = blocked;
-        if (pl.kernel != SEL_SEARCH) {
-            launch_sorted(pl.kernel, kind, dim3(n_chunks, splits), c->stream, jv, sgaps, G_act, per_split, partial,
-                          G_dev);
-        } else {
+        LaunchGate gate;
+        gate.gaps_left = G_dev;
+        gate.n_classes = pl.have_alt ? &c->gap_info.as<GapInfo>()->n_classes : nullptr;
+        gate.max_classes = pl.max_classes;
+        gate.run_if_many = 0u;
+        auto launch_search = [&](const KernelPlan& kp, const LaunchGate& g) {
             const bool opts = jv.late_start != 0u || jv.deadline != nullptr || jv.PW != nullptr;
             if (opts)
-                select_search_kernel<true><<<dim3(n_chunks, splits), SEARCH_THREADS,
+                select_search_kernel<true><<<dim3(kp.n_chunks, kp.splits), SEARCH_THREADS,
                                              jv.PW ? SEARCH_SMEM_BYTES_POWER : SEARCH_SMEM_BYTES, c->stream>>>(
-                    jv, sgaps, G_act, per_split, kind, partial, G_dev);
+                    jv, sgaps, G_act, kp.per_split, kind, partial, g);
             else
-                select_search_kernel<false><<<dim3(n_chunks, splits), SEARCH_THREADS, SEARCH_SMEM_BYTES, c->stream>>>(
-                    jv, sgaps, G_act, per_split, kind, partial, G_dev);
+                select_search_kernel<false><<<dim3(kp.n_chunks, kp.splits), SEARCH_THREADS, SEARCH_SMEM_BYTES,
+                                              c->stream>>>(jv, sgaps, G_act, kp.per_split, kind, partial, g);
+        };
+        if (pl.primary.kernel != SEL_SEARCH)
+            launch_sorted(pl.primary.kernel, kind, dim3(pl.primary.n_chunks, pl.primary.splits), c->stream, jv, sgaps,
+                          G_act, pl.primary.per_split, partial, gate);
+        else
+            launch_search(pl.primary, gate);
+        if (pl.have_alt) {
+            LaunchGate many = gate;
+            many.run_if_many = 1u;
+            launch_search(pl.alt, many);
         }
         finalize_awards_kernel<<<(G_act + 31) / 32, FINALIZE_WARPS * 32, 0, c->stream>>>(
-            jv, partial, n_chunks, sgaps, G_act, kind, c->awards.as<Award>(), c->widx.as<uint32_t>(), G_dev);
+            jv, partial, pl.primary.n_chunks, pl.alt.n_chunks, sgaps, G_act, kind, c->awards.as<Award>(),
+            c->widx.as<uint32_t>(), gate);
     }
     c->prof = was_on;
     return SJA_OK;
@@ -522,7 +547,7 @@ sja_status sja_destroy(sja_ctx* c) {
     if (!c) return SJA_OK;
     DeviceGuard guard(c->device);
     cudaStreamSynchronize(c->stream);
-    DevBuf* bufs[] = {&c->st_off, &c->st_d, &c->st_m, &c->st_s, &c->st_p, &c->p, &c->ready, &c->pb, &c->Dp,
+    DevBuf* bufs[] = {&c->st_off, &c->st_d, &c->st_m, &c->st_s, &c->st_p, &c->st_ready, &c->st_wait, &c->st_prio, &c->p, &c->ready, &c->pb, &c->Dp,
                       &c->Wp, &c->wait, &c->prio, &c->nbj, &c->cta_tot, &c->cta_base, &c->boff, &c->boff_next, &c->A, &c->B, &c->jobwin,
                       &c->flags, &c->counter, &c->n_granted, &c->long_list, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->deadline, &c->PW, &c->caps, &c->st_power, &c->st_bids, &c->st_accept, &c->st_global, &c->upd_d, &c->upd_m, &c->upd_scratch, &c->upd_status, &c->awards, &c->widx, &c->partial,
                       &c->winners};
@@ -625,83 +650,62 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
     } else if ((!n_known || N > 0) && (!aligned16(dur_ms) || !aligned16(mem_MiB) || !aligned16(safe_bits))) {
         return fail(c, SJA_ERR_INVALID_ARG, "sja_load_profiles: device profile arrays must be 16-byte aligned");
     }
-    TRY(reserve(c, c->st_p, (size_t)J * 4));
     const uint32_t n_count_ctas = (J + COUNT_JOBS_PER_CTA - 1) / COUNT_JOBS_PER_CTA;
-    TRY(reserve(c, c->nbj, (size_t)J * 8));                       // per-job row offset inside its CTA
+    // scratch of the preparation pass and staging of host-side per-job inputs (none of it is loaded state)
+    TRY(reserve(c, c->nbj, (size_t)J * 8));                       // per-job row offset inside its counting CTA
     TRY(reserve(c, c->cta_tot, (size_t)n_count_ctas * 8));
     TRY(reserve(c, c->cta_base, (size_t)(n_count_ctas + 1) * 8));
     TRY(reserve(c, c->boff_next, (size_t)(J + 1) * 8));
-    if (progress) TRY(copy_in(c, c->st_p.p, progress, (size_t)J * 4, where));
-    else CU(cudaMemsetAsync(c->st_p.p, 0, (size_t)J * 4, c->stream));
+    TRY(reserve(c, c->long_list, (size_t)J * 4));
+    const uint32_t *d_p = progress, *d_ready = ready_ms, *d_wait = wait_ms;
+    const uint8_t* d_prio = prio;
+    if (where == SJA_MEM_HOST) {
+        TRY(reserve(c, c->st_ready, (size_t)J * 4));
+        TRY(copy_in(c, c->st_ready.p, ready_ms, (size_t)J * 4, where));
+        d_ready = c->st_ready.as<uint32_t>();
+        if (progress) {
+            TRY(reserve(c, c->st_p, (size_t)J * 4));
+            TRY(copy_in(c, c->st_p.p, progress, (size_t)J * 4, where));
+            d_p = c->st_p.as<uint32_t>();
+        }
+        if (wait_ms) {
+            TRY(reserve(c, c->st_wait, (size_t)J * 4));
+            TRY(copy_in(c, c->st_wait.p, wait_ms, (size_t)J * 4, where));
+            d_wait = c->st_wait.as<uint32_t>();
+        }
+        if (prio) {
+            TRY(reserve(c, c->st_prio, (size_t)J));
+            TRY(copy_in(c, c->st_prio.p, prio, (size_t)J, where));
+            d_prio = c->st_prio.as<uint8_t>();
+        }
+    }
 
-    // Device inputs and buffers of an earlier load at hand: the state kernel and the scan are launched right
-    // behind the validation pass and check its verdict on the device (they do nothing for a rejected load or
-    // one whose table outgrows the buffers), so the host waits once per load instead of twice.  Otherwise
-    // the host waits for the verdict and the row count first, as it must to size the table.
+    // The kernels of a load test the verdict of the validation pass on the device: the state kernel and the
+    // scan do nothing for a rejected load or for one whose table outgrows the buffers.  Where the context's
+    // buffers are large enough for this J they are therefore launched right behind the validation pass, and
+    // the host waits once per load; otherwise it waits for the verdict first, so that a rejected load never
+    // costs the previous one its buffers.
     const size_t need4 = (size_t)J * 4, need8 = (size_t)J * 8;
     const bool perjob_ready = c->p.cap >= need4 && c->ready.cap >= need4 && c->pb.cap >= need4 && c->Dp.cap >= need4 &&
-                              c->Wp.cap >= need8 && c->jobwin.cap >= need8 && (!wait_ms || c->wait.cap >= need4) &&
-                              (!prio || c->prio.cap >= (size_t)J);
-    const bool speculate = where == SJA_MEM_DEVICE && !n_known && perjob_ready && c->A.cap >= 32 && c->B.cap >= 24;
-    const uint64_t cap_rows = speculate ? std::min<uint64_t>(c->A.cap / 16 - 1, c->B.cap / 8 - 2) : ~0ull;
+                              c->Wp.cap >= need8 && c->jobwin.cap >= need8 &&
+                              (!wait_ms || c->wait.cap >= need4) && (!prio || c->prio.cap >= (size_t)J);
+    const bool speculate = perjob_ready && c->A.cap >= 32 && c->B.cap >= 24;
+    const uint64_t cap_now = speculate ? std::min<uint64_t>(c->A.cap / 16 - 1, c->B.cap / 8 - 2) : 0ull;
 
-    // pass 0: validate + count rows, then row offsets; nothing of the loaded state is touched yet
-    TRY(reserve(c, c->long_list, (size_t)J * 4));
-    CU(cudaMemsetAsync(c->flags.p, 0, 8, c->stream));
-    {
-        ProfScope ps(c, CAT_PREP);
-        count_boundaries_kernel<<<n_count_ctas, 256, 0, c->stream>>>(
-            d_off, d_s, c->st_p.as<uint32_t>(), J, c->nbj.as<uint64_t>(), c->cta_tot.as<uint64_t>(),
-            c->flags.as<uint32_t>(), c->long_list.as<uint32_t>());
-        cta_offsets_kernel<<<1, 1024, 0, c->stream>>>(c->cta_tot.as<uint64_t>(), n_count_ctas,
-                                                      c->cta_base.as<uint64_t>());
-        row_offsets_kernel<<<(J + 255) / 256, 256, 0, c->stream>>>(c->nbj.as<uint64_t>(), c->cta_base.as<uint64_t>(),
-                                                                   J, n_count_ctas, c->boff_next.as<uint64_t>(),
-                                                                   cap_rows, c->flags.as<uint32_t>());
-    }
-    CU(cudaGetLastError());
-
-    // verdict of pass 0 (waits for the stream): flags, row count and, if not known yet, N
-    uint64_t n_rows = 0;
-    uint32_t flags = 0;
-    bool n_resolved = n_known;
-    auto read_verdict = [&]() -> sja_status {
-        CU(cudaMemcpyAsync(c->h_words, c->flags.p, 4, cudaMemcpyDeviceToHost, c->stream));
-        CU(cudaMemcpyAsync(c->h_words + 2, c->boff_next.as<uint64_t>() + J, 8, cudaMemcpyDeviceToHost, c->stream));
-        if (!n_known) CU(cudaMemcpyAsync(c->h_words + 4, d_off + J, 8, cudaMemcpyDeviceToHost, c->stream));
-        CU(cudaStreamSynchronize(c->stream));
-        flags = c->h_words[0];
-        if (!n_known) {
-            memcpy(&N, c->h_words + 4, 8);
-            n_resolved = true;
-            if (N >= (1ull << 40) && !(flags & FLAG_BAD_PROFILE))
-                return fail(c, SJA_ERR_BAD_PROFILE, "off[J] = %llu is implausible", (unsigned long long)N);
-        }
-        if (flags & FLAG_BAD_PROFILE)
-            return fail(c, SJA_ERR_BAD_PROFILE,
-                        "profile CSR invalid (offsets not monotone, job too long, or progress > len)");
-        memcpy(&n_rows, c->h_words + 2, 8);
-        return SJA_OK;
-    };
-    // per-job state and the scan, reading the row offsets from boff_next (it becomes boff once the load stands)
-    auto launch_state_and_scan = [&]() -> sja_status {
+    // launched once or twice: row offsets and per-job state, then the scan
+    auto launch_state_and_scan = [&](uint64_t cap_rows) -> sja_status {
         {
             ProfScope ps(c, CAT_PREP);
-            const bool dev = where == SJA_MEM_DEVICE;
-            if (!dev) {
-                TRY(copy_in(c, c->ready.p, ready_ms, (size_t)J * 4, where));
-                if (wait_ms) TRY(copy_in(c, c->wait.p, wait_ms, (size_t)J * 4, where));
-                if (prio) TRY(copy_in(c, c->prio.p, prio, (size_t)J, where));
-            }
-            init_state_kernel<<<(J + 255) / 256, 256, 0, c->stream>>>(
-                J, c->st_p.as<uint32_t>(), dev ? ready_ms : nullptr, dev ? wait_ms : nullptr, dev ? prio : nullptr,
-                c->p.as<uint32_t>(), c->ready.as<uint32_t>(), c->wait.as<uint32_t>(), c->prio.as<uint8_t>(),
-                c->pb.as<uint32_t>(), c->Dp.as<uint32_t>(), c->Wp.as<uint64_t>(),
-                c->jobwin.as<unsigned long long>(), c->counter.as<uint32_t>(), c->flags.as<uint32_t>());
+            finish_load_kernel<<<(J + 255) / 256, 256, 0, c->stream>>>(
+                J, n_count_ctas, c->nbj.as<uint64_t>(), c->cta_base.as<uint64_t>(), c->boff_next.as<uint64_t>(), cap_rows,
+                d_p, d_ready, d_wait, d_prio, c->p.as<uint32_t>(), c->ready.as<uint32_t>(),
+                c->wait.as<uint32_t>(), c->prio.as<uint8_t>(), c->pb.as<uint32_t>(), c->Dp.as<uint32_t>(),
+                c->Wp.as<uint64_t>(), c->jobwin.as<unsigned long long>(),
+                c->counter.as<uint32_t>(), c->flags.as<uint32_t>());
         }
         ScanArgs a;
         a.off = d_off; a.d = d_d; a.m = d_m; a.sbits = d_s;
-        a.p0 = c->st_p.as<uint32_t>();
+        a.p0 = d_p;
         a.wait = wait_ms ? c->wait.as<uint32_t>() : nullptr;
         a.prio = prio ? c->prio.as<uint8_t>() : nullptr;
         a.boff = c->boff_next.as<uint64_t>();
@@ -711,7 +715,7 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
         a.counter = c->counter.as<uint32_t>();
         a.flags = c->flags.as<uint32_t>();
         a.long_list = c->long_list.as<uint32_t>();
-        if (!n_resolved || N > 0) {
+        if (!n_known || N > 0) {
             ProfScope ps(c, CAT_SCAN);
             const uint32_t ctas_per_sm = SCAN_CTAS_PER_SM;
             const uint32_t want = (J + SCAN_WARPS - 1) / SCAN_WARPS;
@@ -721,7 +725,46 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
         CU(cudaGetLastError());
         return SJA_OK;
     };
-    auto reserve_state = [&]() -> sja_status {
+
+    // pass 0: validate + count rows, offsets of the counting CTAs; nothing of the loaded
+    // state is touched yet
+    CU(cudaMemsetAsync(c->flags.p, 0, 8, c->stream));
+    {
+        ProfScope ps(c, CAT_PREP);
+        count_boundaries_kernel<<<n_count_ctas, 256, 0, c->stream>>>(
+            d_off, d_s, d_p, J, c->nbj.as<uint64_t>(), c->cta_tot.as<uint64_t>(), c->flags.as<uint32_t>(),
+            c->long_list.as<uint32_t>());
+        cta_offsets_kernel<<<1, 1024, 0, c->stream>>>(c->cta_tot.as<uint64_t>(), n_count_ctas,
+                                                      c->cta_base.as<uint64_t>());
+    }
+    CU(cudaGetLastError());
+    if (speculate) TRY(launch_state_and_scan(cap_now));
+
+    // verdict (waits for the stream): flags, row count and, if not known yet, N
+    uint64_t n_rows = 0;
+    uint32_t flags = 0;
+    CU(cudaMemcpyAsync(c->h_words, c->flags.p, 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaMemcpyAsync(c->h_words + 2, c->cta_base.as<uint64_t>() + n_count_ctas, 8, cudaMemcpyDeviceToHost, c->stream));
+    if (!n_known) CU(cudaMemcpyAsync(c->h_words + 4, d_off + J, 8, cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaStreamSynchronize(c->stream));
+    flags = c->h_words[0];
+    if (!n_known) {
+        memcpy(&N, c->h_words + 4, 8);
+        n_known = true;
+        if (N >= (1ull << 40) && !(flags & FLAG_BAD_PROFILE))
+            return fail(c, SJA_ERR_BAD_PROFILE, "off[J] = %llu is implausible", (unsigned long long)N);
+    }
+    if (flags & FLAG_BAD_PROFILE)     // a rejected load has touched nothing of the previous one
+        return fail(c, SJA_ERR_BAD_PROFILE, "profile CSR invalid (offsets not monotone, job too long, or progress > len)");
+    memcpy(&n_rows, c->h_words + 2, 8);
+
+    // from here on the previous load is replaced
+    c->loaded = false;
+    c->have_deadline = false;                // deadlines and power traces belong to the jobs of a load
+    c->have_power = false;
+    c->advertised = c->selected = c->committed = false;
+    if (!speculate || n_rows > cap_now) {
+        // buffers too small for this load (the kernels above, if launched, stood still): size them and run
         TRY(reserve(c, c->A, (size_t)n_rows * 16 + 16));
         TRY(reserve(c, c->B, (size_t)n_rows * 8 + 16));
         TRY(reserve(c, c->p, need4));
@@ -732,32 +775,13 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
         TRY(reserve(c, c->jobwin, need8));
         if (wait_ms) TRY(reserve(c, c->wait, need4));
         if (prio) TRY(reserve(c, c->prio, (size_t)J));
-        return SJA_OK;
-    };
-
-    if (speculate) {
-        TRY(launch_state_and_scan());
-        TRY(read_verdict());                     // a rejected load has touched nothing of the previous one
-        // from here on the previous load is replaced
-        c->loaded = false;
-        c->have_deadline = false;                // deadlines and power traces belong to the jobs of a load
-        c->have_power = false;
-        c->advertised = c->selected = c->committed = false;
         if (flags & FLAG_NEED_ROWS) {
-            // the table outgrew the buffers and the kernels stood still: size them and run again
-            TRY(reserve_state());
-            CU(cudaMemsetAsync(c->flags.p, 0, 4, c->stream));
-            TRY(launch_state_and_scan());
-            TRY(read_flags(c, &flags));
+            // clear that bit alone (the counters of the validation pass behind it stay)
+            flags &= ~FLAG_NEED_ROWS;
+            c->h_words[8] = flags;
+            CU(cudaMemcpyAsync(c->flags.p, c->h_words + 8, 4, cudaMemcpyHostToDevice, c->stream));
         }
-    } else {
-        TRY(read_verdict());
-        c->loaded = false;
-        c->have_deadline = false;
-        c->have_power = false;
-        c->advertised = c->selected = c->committed = false;
-        TRY(reserve_state());
-        TRY(launch_state_and_scan());
+        TRY(launch_state_and_scan(~0ull));
         TRY(read_flags(c, &flags));
     }
     std::swap(c->boff, c->boff_next);
@@ -798,7 +822,12 @@ sja_status sja_advertise(sja_ctx* c, uint32_t G, const sja_gap* gaps, sja_memspa
     const bool sortable = G <= SORT_MAX_GAPS;
     {
         ProfScope ps(c, CAT_ADVERTISE);
-        TRY(copy_in(c, c->gaps.p, gaps, (size_t)G * sizeof(sja_gap), where));
+        // host batches are copied into the context first; device batches are read in place by the first kernel,
+        // which also writes the context's copy (the commit needs the start times after the caller's array is gone)
+        const bool dev = where == SJA_MEM_DEVICE;
+        if (!dev) TRY(copy_in(c, c->gaps.p, gaps, (size_t)G * sizeof(sja_gap), where));
+        const Gap* src = dev ? reinterpret_cast<const Gap*>(gaps) : c->gaps.as<Gap>();
+        Gap* keep = dev ? c->gaps.as<Gap>() : nullptr;
         if (sortable) {
             // sorted tiles live behind the ranks in one buffer; the sort kernel clears the ranks and the class counter
             const uint32_t n_tiles = (G + SORT_TILE - 1) / SORT_TILE;
@@ -806,30 +835,24 @@ sja_status sja_advertise(sja_ctx* c, uint32_t G, const sja_gap* gaps, sja_memspa
             uint64_t* tile_key = reinterpret_cast<uint64_t*>(c->gap_rank.as<unsigned char>() + rank_bytes);
             uint32_t* tile_idx = reinterpret_cast<uint32_t*>(tile_key + (size_t)n_tiles * SORT_TILE);
             const bool one_tile = n_tiles == 1;
-            sort_gap_tiles_kernel<<<n_tiles, SORT_TILE, 0, c->stream>>>(c->gaps.as<Gap>(), G, tile_key, tile_idx, rank,
+            sort_gap_tiles_kernel<<<n_tiles, SORT_TILE, 0, c->stream>>>(src, G, tile_key, tile_idx, rank,
                                                                         c->gap_info.as<GapInfo>(),
-                                                                        one_tile ? c->sgaps.as<Gap>() : nullptr);
+                                                                        one_tile ? c->sgaps.as<Gap>() : nullptr, keep);
             if (!one_tile) {
                 rank_gap_tiles_kernel<<<dim3(n_tiles, n_tiles), SORT_TILE, 0, c->stream>>>(tile_key, tile_idx, rank);
-                place_gaps_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(c->gaps.as<Gap>(), G, rank,
-                                                                          c->sgaps.as<Gap>());
-                count_classes_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(c->sgaps.as<Gap>(), G,
-                                                                            c->gap_info.as<GapInfo>());
+                place_gaps_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(src, G, rank, c->sgaps.as<Gap>(),
+                                                                          c->gap_info.as<GapInfo>());
             }
-            CU(cudaMemcpyAsync(c->h_words + 4, c->gap_info.p, sizeof(GapInfo), cudaMemcpyDeviceToHost, c->stream));
         } else {
-            copy_gaps_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(c->gaps.as<Gap>(), G, c->sgaps.as<Gap>());
+            copy_gaps_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(src, G, c->sgaps.as<Gap>(), keep);
         }
     }
     CU(cudaGetLastError());
-    // the class count steers the kernel choice of sja_select, and a host buffer may be reused on return
-    CU(cudaStreamSynchronize(c->stream));
+    // a host array may be reused as soon as the call returns; a device batch is only queued
+    if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));
     c->gaps_sorted = sortable;
-    c->have_caps = false;      // power caps belong to a batch
-    c->n_classes = sortable ? c->h_words[4] : 0;
     c->G = G;
     c->advertised = true;
-    c->selected = c->committed = false;
     return SJA_OK;
 }
 
@@ -868,13 +891,15 @@ sja_status sja_select_static(sja_ctx* c, const sja_policy* policy, sja_award* ou
 
     const uint32_t kind = policy->kind, G = c->G, J = c->J;
     const SelectPlan pl = plan_select(c, policy->flags, G);
-    const uint64_t need = (uint64_t)pl.n_chunks * G;   // candidate slots: one per (CTA job chunk, gap)
+    const uint64_t need = (uint64_t)pl.rows * G;   // candidate slots: one per (CTA job chunk, gap)
     const uint64_t have = (uint64_t)SJA_STATIC_SCRATCH_BYTES / sizeof(Partial);
     if (need > have)
         return fail(c, SJA_ERR_INVALID_ARG,
                     "sja_select_static: %u jobs x %u gaps need %llu candidate slots (ceil(J/%u) x G), the fixed "
                     "scratch holds %llu; use sja_select for this size",
-                    J, G, (unsigned long long)need, pl.jobs_per_cta, (unsigned long long)have);
+                    J, G, (unsigned long long)need,
+                    pl.have_alt ? std::min(pl.primary.jobs_per_cta, pl.alt.jobs_per_cta) : pl.primary.jobs_per_cta,
+                    (unsigned long long)have);
     Partial* scratch = nullptr;
     TRY(static_scratch_for(c, c->device, &scratch));
     // Every slot that finalize_awards_kernel reads is written by the select kernel of this

@@ -19,7 +19,7 @@ constexpr uint32_t COUNT_LONG = 0x80000000u;   // marker: job left to the whole-
 
 __global__ void __launch_bounds__(256) count_boundaries_kernel(
     const uint64_t* __restrict__ off, const uint32_t* __restrict__ sbits,
-    const uint32_t* __restrict__ p0, uint32_t J, uint64_t* __restrict__ local_off,
+    const uint32_t* __restrict__ p0 /* may be nullptr: all 0 */, uint32_t J, uint64_t* __restrict__ local_off,
     uint64_t* __restrict__ cta_total, uint32_t* __restrict__ flags, uint32_t* __restrict__ long_list) {
     __shared__ uint32_t cnts[COUNT_JOBS_PER_CTA];
     __shared__ uint64_t warp_sums[COUNT_JOBS_PER_CTA / 32];
@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
         bool bad = false;
         if (j < J) {
             const uint64_t js = __ldg(off + j), je = __ldg(off + j + 1);
-            const uint32_t p = __ldg(p0 + j);
+            const uint32_t p = p0 ? __ldg(p0 + j) : 0u;
             bad = (je < js) || (je > N) || (je - js > 0xFFFFFFFFull) || ((uint64_t)p > je - js);
             if (j == 0 && js != 0) bad = true;
             if (!bad) {
@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
     for (uint32_t i = 0; i < COUNT_JOBS_PER_WARP; ++i) {
         if (cnts[slot0 + i] != COUNT_LONG) continue;   // same value in every lane
         const uint32_t j = jbase + i;
-        const uint64_t s = __ldg(off + j) + __ldg(p0 + j), e = __ldg(off + j + 1);
+        const uint64_t s = __ldg(off + j) + (p0 ? __ldg(p0 + j) : 0u), e = __ldg(off + j + 1);
         const uint64_t w0 = s >> 5, w1 = (e - 1) >> 5;
         uint32_t cnt = 0;
         for (uint64_t w = w0 + lane; w <= w1; w += 32) {
@@ -176,36 +176,32 @@ __global__ void __launch_bounds__(1024) cta_offsets_kernel(const uint64_t* __res
     if (t == 0) base_out[P] = carry;
 }
 
-// boff[j] = base of the job's CTA + offset inside the CTA; boff[J] = total row count.  A total above
-// `cap_rows` (what the table buffers handed to the following kernels can hold) raises FLAG_NEED_ROWS.
-__global__ void __launch_bounds__(256) row_offsets_kernel(const uint64_t* __restrict__ local_off,
-                                                          const uint64_t* __restrict__ cta_base, uint32_t J,
-                                                          uint32_t P, uint64_t* __restrict__ boff, uint64_t cap_rows,
-                                                          uint32_t* __restrict__ flags) {
+// Last preparation step of a load, one thread per job:
+//  * boff[j] = base of the job's counting CTA + offset inside it; boff[J] = total row count.  A total above
+//    `cap_rows` (what the table buffers handed to the scan can hold) raises FLAG_NEED_ROWS.
+//  * If the load stands (CSR valid, table fits): per-job state of a fresh load -- progress and attributes
+//    copied, cursors and commit votes cleared, the scan's job counter reset.  Otherwise nothing of the
+//    previously loaded state is touched.
+// Source pointers may be nullptr (attribute not given; progress = 0).
+__global__ void __launch_bounds__(256) finish_load_kernel(
+    uint32_t J, uint32_t P, const uint64_t* __restrict__ local_off, const uint64_t* __restrict__ cta_base,
+    uint64_t* __restrict__ boff, uint64_t cap_rows, const uint32_t* __restrict__ p_src,
+    const uint32_t* __restrict__ ready_src, const uint32_t* __restrict__ wait_src,
+    const uint8_t* __restrict__ prio_src, uint32_t* __restrict__ p, uint32_t* __restrict__ ready,
+    uint32_t* __restrict__ wait, uint8_t* __restrict__ prio, uint32_t* __restrict__ pb, uint32_t* __restrict__ Dp,
+    uint64_t* __restrict__ Wp, unsigned long long* __restrict__ jobwin, uint32_t* __restrict__ counter,
+    uint32_t* __restrict__ flags) {
     const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint64_t total = cta_base[P];
     if (j < J) boff[j] = cta_base[j / COUNT_JOBS_PER_CTA] + local_off[j];
     if (j == 0) {
-        const uint64_t total = cta_base[P];
         boff[J] = total;
         if (total > cap_rows) atomicOr(flags, FLAG_NEED_ROWS);
     }
-}
-
-// Per-job state of a fresh load in one launch: progress and attributes copied, cursors and
-// commit votes cleared, the scan's job counter reset.  Source pointers may be nullptr (then
-// the destination was filled by a host-to-device copy, or is not used).  Does nothing when the
-// validation pass rejected the load or the table buffers are too small (see sja_load_profiles).
-__global__ void __launch_bounds__(256) init_state_kernel(
-    uint32_t J, const uint32_t* __restrict__ p_src, const uint32_t* __restrict__ ready_src,
-    const uint32_t* __restrict__ wait_src, const uint8_t* __restrict__ prio_src, uint32_t* __restrict__ p,
-    uint32_t* __restrict__ ready, uint32_t* __restrict__ wait, uint8_t* __restrict__ prio, uint32_t* __restrict__ pb,
-    uint32_t* __restrict__ Dp, uint64_t* __restrict__ Wp, unsigned long long* __restrict__ jobwin,
-    uint32_t* __restrict__ counter, const uint32_t* __restrict__ flags) {
-    if (*flags & (FLAG_BAD_PROFILE | FLAG_NEED_ROWS)) return;
-    const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+    if ((*flags & FLAG_BAD_PROFILE) || total > cap_rows) return;     // same verdict in every thread
     if (j == 0) *counter = 0;
     if (j >= J) return;
-    p[j] = p_src[j];
+    p[j] = p_src ? p_src[j] : 0u;
     if (ready_src) ready[j] = ready_src[j];
     if (wait_src) wait[j] = wait_src[j];
     if (prio_src) prio[j] = prio_src[j];

@@ -27,6 +27,28 @@ struct JobView {
     uint32_t J;
 };
 
+// What a select launch has to find out on the device before it does anything.  The host queues the kernels of a
+// round without waiting for the GPU, so two facts may only exist in device memory when a kernel starts: how
+// many gaps are left (a later pass of a re-auction: `gaps_left`), and how many capacity classes the ordered
+// batch has (`n_classes`: with more than `max_classes` of them the ordered-gap kernels would restart their
+// cursors too often, and the per-pair search serves the round instead; both kernels are queued and the one
+// the count does not call for returns at once).
+struct LaunchGate {
+    const uint32_t* gaps_left;   // may be nullptr: all G gaps
+    const uint32_t* n_classes;   // may be nullptr: this launch runs whatever the class count
+    uint32_t max_classes;
+    uint32_t run_if_many;        // 0: run when n_classes <= max_classes, 1: run when it is larger
+};
+
+// Number of gaps this launch serves: 0 when the class count calls for the other kernel.
+__device__ __forceinline__ uint32_t gate_gaps(const LaunchGate& g, uint32_t G) {
+    if (g.n_classes) {
+        const bool many = *g.n_classes > g.max_classes;
+        if (many != (g.run_if_many != 0u)) return 0u;
+    }
+    return g.gaps_left ? min(G, *g.gaps_left) : G;
+}
+
 __device__ __forceinline__ uint32_t policy_factor(const JobView& jv, uint32_t kind, uint32_t j) {
     if (kind == 1) return 1u + __ldg(jv.wait + j) / 1000u;
     if (kind == 2) return (uint32_t)__ldg(jv.prio + j);
@@ -63,10 +85,10 @@ static_assert((SEARCH_ROWS & (SEARCH_ROWS - 1)) == 0 && SEARCH_PAY_ROWS <= SEARC
 template <bool OPTS>
 __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
     JobView jv, const Gap* __restrict__ gaps, uint32_t G, uint32_t gaps_per_split, uint32_t kind,
-    Partial* __restrict__ partial_out, const uint32_t* __restrict__ G_dev) {
+    Partial* __restrict__ partial_out, LaunchGate gate) {
     __shared__ Partial stage[SEARCH_GT][SEARCH_THREADS / 32];
     __shared__ uint4 sgap[SEARCH_GT];
-    const uint32_t G_now = G_dev ? min(G, *G_dev) : G;   // gaps actually left (see select_tile_kernel)
+    const uint32_t G_now = gate_gaps(gate, G);   // gaps actually left (G stays the row length of partial_out)
     if (blockIdx.y * gaps_per_split >= G_now) return;
     extern __shared__ __align__(16) uint2 search_rows[];
     uint2* sDM = search_rows + threadIdx.x;                                     // row r of this thread: sDM[r * THREADS]
@@ -222,12 +244,15 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
 constexpr int FINALIZE_WARPS = 8;
 
 __global__ void __launch_bounds__(FINALIZE_WARPS * 32) finalize_awards_kernel(
-    JobView jv, const Partial* __restrict__ partial, uint32_t n_rows, const Gap* __restrict__ sgaps, uint32_t G,
-    uint32_t kind, Award* __restrict__ awards, uint32_t* __restrict__ widx, const uint32_t* __restrict__ G_dev) {
+    JobView jv, const Partial* __restrict__ partial, uint32_t n_rows, uint32_t n_rows_many,
+    const Gap* __restrict__ sgaps, uint32_t G, uint32_t kind, Award* __restrict__ awards, uint32_t* __restrict__ widx,
+    LaunchGate gate) {
     __shared__ Partial fold[FINALIZE_WARPS][32];
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
     const uint32_t g = blockIdx.x * 32u + lane;     // position in the advertised (sorted) order
-    const uint32_t G_now = G_dev ? min(G, *G_dev) : G;   // G stays the row length of `partial`
+    const uint32_t G_now = gate.gaps_left ? min(G, *gate.gaps_left) : G;   // G stays the row length of `partial`
+    // the kernel that ran wrote one candidate row per job chunk of its own size
+    if (gate.n_classes && *gate.n_classes > gate.max_classes) n_rows = n_rows_many;
     Partial best;
     best.key = 0; best.job = 0xFFFFFFFFu; best.cnt = 0;
     if (g < G_now) {
@@ -383,12 +408,12 @@ namespace sja {
 //      each key of tile q, the number of smaller keys in tile t (a 10-probe binary search)
 //      to that gap's rank -- G * G/1024 searches instead of G * G comparisons, no pass
 //      waits on another;
-//   3. place_gaps_kernel writes gap i to position rank[i];
-//   4. count_classes_kernel counts the positions whose predecessor has another capacity.
+//   3. place_gaps_kernel writes gap i to position rank[i]; its last CTA counts the positions whose predecessor has
+//      another capacity (the class count, which decides between the ordered-gap kernels and the per-pair search).
 constexpr uint32_t SORT_MAX_GAPS = 65536;
 constexpr int SORT_TILE = 1024;
 
-struct GapInfo { uint32_t n_classes; uint32_t pad[3]; };
+struct GapInfo { uint32_t n_classes; uint32_t placed_ctas; uint32_t pad[2]; };
 
 __device__ __forceinline__ bool gap_key_less(uint64_t ka, uint32_t ia, uint64_t kb, uint32_t ib) {
     return ka < kb || (ka == kb && ia < ib);
@@ -396,19 +421,25 @@ __device__ __forceinline__ bool gap_key_less(uint64_t ka, uint32_t ia, uint64_t 
 
 // With `sorted_out` set (a batch of one tile) the kernel finishes the job alone: it writes the ordered gaps and
 // the class count.  Otherwise it stores the sorted tile for the ranking pass and clears the ranks and the counter.
+// `keep` (optional): the context's own copy of the batch, written here when the caller's array is read in place.
 __global__ void __launch_bounds__(SORT_TILE) sort_gap_tiles_kernel(const Gap* __restrict__ gaps, uint32_t G,
                                                                    uint64_t* __restrict__ tile_key,
                                                                    uint32_t* __restrict__ tile_idx,
                                                                    uint32_t* __restrict__ rank, GapInfo* __restrict__ info,
-                                                                   Gap* __restrict__ sorted_out) {
+                                                                   Gap* __restrict__ sorted_out, Gap* __restrict__ keep) {
     __shared__ uint64_t sk[SORT_TILE];
     __shared__ uint32_t si[SORT_TILE];
     const uint32_t t = threadIdx.x;
     const uint32_t i = blockIdx.x * SORT_TILE + t;
     uint64_t k = ~0ull;          // padding sorts last and is never smaller than a real key
     uint32_t x = 0xFFFFFFFFu;
-    if (i < G) { const Gap g = gaps[i]; k = ((uint64_t)g.C << 32) | g.T; x = i; }
-    if (i == 0) info->n_classes = 0;
+    if (i < G) {
+        const Gap g = gaps[i];
+        k = ((uint64_t)g.C << 32) | g.T;
+        x = i;
+        if (keep) keep[i] = g;
+    }
+    if (i == 0) { info->n_classes = 0; info->placed_ctas = 0; }
     // Bitonic network, one element per thread.  Partners less than 32 apart sit in the same warp and are
     // exchanged by shuffles; only the wider strides go through shared memory (15 barrier stages, not 55).
     for (uint32_t size = 2; size <= SORT_TILE; size <<= 1) {
@@ -439,7 +470,7 @@ __global__ void __launch_bounds__(SORT_TILE) sort_gap_tiles_kernel(const Gap* __
         const uint32_t src = si[t];
         const bool real = src != 0xFFFFFFFFu;
         if (real) {
-            const Gap g = gaps[src];
+            const Gap g = gaps[src];     // (the caller's array: `keep` may not be complete yet for other threads' rows)
             Gap o;
             o.slice = src;       // the original position travels in the slice field
             o.start = g.start; o.T = g.T; o.C = g.C;
@@ -476,31 +507,43 @@ __global__ void __launch_bounds__(SORT_TILE) rank_gap_tiles_kernel(const uint64_
     if (pos) atomicAdd(rank + x, pos);
 }
 
+// Placement by rank; the CTA that finishes last then counts the capacity classes of the ordered list (positions
+// whose predecessor has another capacity).  "Last" is decided by a counter that every CTA bumps after its own
+// stores are visible: nobody waits for anybody.
 __global__ void __launch_bounds__(256) place_gaps_kernel(const Gap* __restrict__ gaps, uint32_t G,
-                                                         const uint32_t* __restrict__ rank, Gap* __restrict__ sorted) {
+                                                         const uint32_t* __restrict__ rank, Gap* __restrict__ sorted,
+                                                         GapInfo* __restrict__ info) {
+    __shared__ uint32_t is_last;
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= G) return;
-    const Gap g = gaps[i];
-    Gap o;
-    o.slice = i;   // the original position travels in the slice field
-    o.start = g.start; o.T = g.T; o.C = g.C;
-    sorted[rank[i]] = o;
-}
-
-__global__ void __launch_bounds__(256) count_classes_kernel(const Gap* __restrict__ sorted, uint32_t G,
-                                                            GapInfo* __restrict__ info) {
-    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    const bool leader = i < G && (i == 0 || sorted[i - 1].C != sorted[i].C);
-    const uint32_t n = __popc(__ballot_sync(0xFFFFFFFFu, leader));
+    if (i < G) {
+        const Gap g = gaps[i];
+        Gap o;
+        o.slice = i;   // the original position travels in the slice field
+        o.start = g.start; o.T = g.T; o.C = g.C;
+        sorted[rank[i]] = o;
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = atomicAdd(&info->placed_ctas, 1u) == gridDim.x - 1u ? 1u : 0u;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    uint32_t leaders = 0;
+    for (uint32_t q = threadIdx.x; q < G; q += blockDim.x) {
+        const uint32_t c = __ldcg(&sorted[q].C);
+        if (q == 0 || __ldcg(&sorted[q - 1].C) != c) ++leaders;
+    }
+    const uint32_t n = __reduce_add_sync(0xFFFFFFFFu, leaders);
     if ((threadIdx.x & 31u) == 0 && n) atomicAdd(&info->n_classes, n);
 }
 
 // Identity order (used when the batch is too large for the one-CTA sort).
 __global__ void __launch_bounds__(256) copy_gaps_kernel(const Gap* __restrict__ gaps, uint32_t G,
-                                                        Gap* __restrict__ sorted) {
+                                                        Gap* __restrict__ sorted, Gap* __restrict__ keep) {
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= G) return;
     Gap g = gaps[i];
+    if (keep) keep[i] = g;
     g.slice = i;
     sorted[i] = g;
 }
@@ -623,8 +666,10 @@ __device__ __forceinline__ WarpBest warp_argmax_lowest_lane(uint64_t best, uint3
 // BOUNDED: the subjob duration thresholds are in force (off by default, and then compiled out).
 template <uint32_t KIND, bool BOUNDED>
 __global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_merge_kernel(
-    JobView jv, const Gap* __restrict__ sgaps, uint32_t G, uint32_t gaps_per_split, Partial* __restrict__ partial_out) {
+    JobView jv, const Gap* __restrict__ sgaps, uint32_t G, uint32_t gaps_per_split, Partial* __restrict__ partial_out,
+    LaunchGate gate) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    if (gate_gaps(gate, G) == 0u) return;      // the class count calls for the per-pair search
     Partial* stage = reinterpret_cast<Partial*>(smem_raw + MERGE_RING_BYTES);            // [GT][WARPS]
     uint4* sg = reinterpret_cast<uint4*>(smem_raw + MERGE_RING_BYTES + MERGE_GT * MERGE_WARPS * 16);
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;

@@ -37,7 +37,7 @@ struct ScanArgs {
     const uint32_t* d;       // [N]
     const uint32_t* m;       // [N]
     const uint32_t* sbits;   // [ceil(N/32)]
-    const uint32_t* p0;      // [J] progress at load
+    const uint32_t* p0;      // [J] progress at load, or nullptr (all 0)
     const uint32_t* wait;    // [J] or nullptr
     const uint8_t* prio;     // [J] or nullptr
     const uint64_t* boff;    // [J+1] row offsets
@@ -110,7 +110,7 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32, SCAN_CTAS_PER_SM) scan_profil
         }
 
         const uint64_t js = __ldg(a.off + j), je = __ldg(a.off + j + 1);
-        const uint32_t p = __ldg(a.p0 + j);
+        const uint32_t p = a.p0 ? __ldg(a.p0 + j) : 0u;
         const uint64_t s = js + p, e = je;
         if (s >= e) continue;
         if (c >= n_long && e - s > long_thresh) continue;   // scanned in the first phase

@@ -77,11 +77,11 @@ __device__ __forceinline__ bool pair_ge(uint64_t ka, uint32_t ia, uint64_t kb, u
 template <uint32_t KIND, bool BOUNDED>
 __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile_kernel(
     JobView jv, const Gap* __restrict__ sgaps, uint32_t G, uint32_t gaps_per_split, Partial* __restrict__ partial_out,
-    const uint32_t* __restrict__ G_dev) {
+    LaunchGate gate) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // G is the gap count the launch was sized for (and the row length of partial_out); a re-auction hands
     // the count actually left in device memory, so that several passes can be queued without a host wait
-    const uint32_t G_now = G_dev ? min(G, *G_dev) : G;
+    const uint32_t G_now = gate_gaps(gate, G);
     if (blockIdx.y * gaps_per_split >= G_now) return;
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
     const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(smem_raw);
