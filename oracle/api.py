@@ -52,13 +52,13 @@ def _load():
     lib.orc_pair.argtypes = [vp, vp, vp, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint32,
                              ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
                              ctypes.c_uint32, ctypes.c_uint32, ctypes.c_int, ctypes.c_uint32, vp, ctypes.c_uint32,
-                             u32p, u32p, u64p, u32p]
+                             ctypes.c_uint32, u32p, u32p, u64p, u32p]
     lib.orc_select.restype = ctypes.c_int
     lib.orc_select.argtypes = [ctypes.c_uint32, vp, vp, vp, vp, vp, vp, vp, vp,
                                ctypes.c_uint32, vp, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32,
-                               ctypes.c_int, vp, vp, vp, vp]
+                               ctypes.c_int, vp, vp, vp, ctypes.c_uint32, vp, vp, ctypes.c_uint32, vp]
     lib.orc_commit.restype = ctypes.c_int64
-    lib.orc_commit.argtypes = [ctypes.c_uint32, vp, vp, ctypes.c_uint32, vp, vp, ctypes.c_int]
+    lib.orc_commit.argtypes = [ctypes.c_uint32, vp, vp, ctypes.c_uint32, vp, vp, ctypes.c_int, vp]
     lib.orc_num_threads.restype = ctypes.c_int
     lib.orc_num_threads.argtypes = []
     del u8p
@@ -86,10 +86,12 @@ U32MAX = 0xFFFFFFFF
 
 def pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: int,
          tau_min_ms: int = 0, tau_max_ms: int = U32MAX, late_start: bool = False, deadline_ms: int = U32MAX,
-         want_peak: bool = False, power_W: Optional[np.ndarray] = None, power_cap_W: int = U32MAX):
+         want_peak: bool = False, power_W: Optional[np.ndarray] = None, power_cap_W: int = U32MAX,
+         min_slack_gain_MiB: int = 0):
     """R1-R3 (with the duration thresholds of R2' and the window options of R1'') for one (gap, job)
     pair: ``None`` for decline, else ``(k, dur, work)`` (``(k, dur, work, peak)`` with ``want_peak``).
-    ``power_W`` (u32 per step, aligned with the profile arrays) and ``power_cap_W`` switch on R2''."""
+    ``power_W`` (u32 per step, aligned with the profile arrays) and ``power_cap_W`` switch on R2'';
+    ``min_slack_gain_MiB`` > 0 switches on the hysteresis rule R3h."""
     lib = _load()
     k = ctypes.c_uint32()
     dur = ctypes.c_uint32()
@@ -99,7 +101,7 @@ def pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: i
                       prof.safe_bits.ctypes.data, int(prof.off[j]), int(prof.off[j + 1]),
                       int(p), int(ready_ms), int(start_ms), int(T_ms), int(C_MiB),
                       int(tau_min_ms), int(tau_max_ms), int(bool(late_start)), int(deadline_ms),
-                      _ptr(_as(power_W, np.uint32)), int(power_cap_W),
+                      _ptr(_as(power_W, np.uint32)), int(power_cap_W), int(min_slack_gain_MiB),
                       ctypes.byref(k), ctypes.byref(dur), ctypes.byref(work), ctypes.byref(peak))
     if not ok:
         return None
@@ -111,10 +113,13 @@ def pair(prof, j: int, p: int, ready_ms: int, start_ms: int, T_ms: int, C_MiB: i
 def select(prof, progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray,
            policy: int, tau_min_ms: int = 0, tau_max_ms: int = U32MAX, late_start: bool = False,
            deadline_ms: Optional[np.ndarray] = None, power_W: Optional[np.ndarray] = None,
-           power_cap_W: Optional[np.ndarray] = None) -> np.ndarray:
+           power_cap_W: Optional[np.ndarray] = None, min_slack_gain_MiB: int = 0,
+           ckpt_MiB: Optional[np.ndarray] = None, last_slice: Optional[np.ndarray] = None,
+           locality_weight: int = 0) -> np.ndarray:
     """R1-R5 for a batch of gaps; returns ``AWARD_DTYPE[G]`` (``granted`` all zero).
     ``late_start`` / ``deadline_ms`` (u32 per job) switch on the window options of R1''; ``power_W`` (u32 per
-    step) with ``power_cap_W`` (u32 per gap) the power envelope of R2''."""
+    step) with ``power_cap_W`` (u32 per gap) the power envelope of R2''; ``min_slack_gain_MiB`` the hysteresis
+    rule R3h; ``ckpt_MiB`` / ``last_slice`` (u32 per job) with ``locality_weight`` the locality penalty R4'."""
     lib = _load()
     off = _as(prof.off, np.uint64)
     d = _as(prof.dur_ms, np.uint32)
@@ -132,26 +137,33 @@ def select(prof, progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray,
     caps = _as(power_cap_W, np.uint32)
     assert power is None or power.shape[0] == d.shape[0]
     assert caps is None or caps.shape[0] == gaps.shape[0]
+    ckpt = _as(ckpt_MiB, np.uint32)
+    last = _as(last_slice, np.uint32)
+    assert ckpt is None or ckpt.shape[0] == off.shape[0] - 1
+    assert last is None or last.shape[0] == off.shape[0] - 1
     rc = lib.orc_select(off.shape[0] - 1, _ptr(off), _ptr(d), _ptr(m), _ptr(s),
                         _ptr(progress), _ptr(ready_ms), _ptr(wait), _ptr(prio),
                         gaps.shape[0], _ptr(gaps), int(policy), int(tau_min_ms), int(tau_max_ms),
-                        int(bool(late_start)), _ptr(deadline), _ptr(power), _ptr(caps), _ptr(awards))
+                        int(bool(late_start)), _ptr(deadline), _ptr(power), _ptr(caps), int(min_slack_gain_MiB),
+                        _ptr(ckpt), _ptr(last), int(locality_weight), _ptr(awards))
     if rc != 0:
         raise ValueError("oracle select: unknown policy or missing attribute array")
     return awards
 
 
 def commit(progress: np.ndarray, ready_ms: np.ndarray, gaps: np.ndarray,
-           awards: np.ndarray, late_start: bool = False) -> int:
+           awards: np.ndarray, late_start: bool = False, last_slice: Optional[np.ndarray] = None) -> int:
     """R6, in place on ``progress``, ``ready_ms`` and ``awards['granted']``.  With ``late_start`` a granted
-    subjob began at ``max(start, ready)`` (R1''), so that is what the new ready time counts from."""
+    subjob began at ``max(start, ready)`` (R1''), so that is what the new ready time counts from.  ``last_slice``
+    (u32 per job, in place): the slice of the granted gap is recorded for every granted job (R4')."""
     lib = _load()
     assert progress.dtype == np.uint32 and progress.flags.c_contiguous
     assert ready_ms.dtype == np.uint32 and ready_ms.flags.c_contiguous
     assert awards.dtype == AWARD_DTYPE and awards.flags.c_contiguous
     gaps = np.ascontiguousarray(gaps, dtype=GAP_DTYPE)
+    assert last_slice is None or (last_slice.dtype == np.uint32 and last_slice.flags.c_contiguous)
     n = lib.orc_commit(progress.shape[0], _ptr(progress), _ptr(ready_ms),
-                       gaps.shape[0], _ptr(gaps), _ptr(awards), int(bool(late_start)))
+                       gaps.shape[0], _ptr(gaps), _ptr(awards), int(bool(late_start)), _ptr(last_slice))
     if n < 0:
         raise OverflowError("oracle commit: begin + dur does not fit in 32 bits")
     return int(n)

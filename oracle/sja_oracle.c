@@ -56,10 +56,25 @@
  *                    power_W array and a per-gap cap, a candidate also needs
  *                    max power_W[p_j..k) <= cap_g; a cap of 2^32-1 means none.
  *
+ *   R3h hysteresis : optional guard against over-fragmentation (Section 3.9: a further subdivision is accepted
+ *                    only if it gains a minimum of slack).  Let k_T be the longest candidate when the memory
+ *                    capacity bound is lifted (every other rule stays) and k* the longest candidate proper.
+ *                    k* < k_T means the capacity forces the job to cut earlier than the window would allow -- a
+ *                    further subdivision.  What the cut gains is the demand it sheds,
+ *                    max m[p_j..k_T) - max m[p_j..k*); the job signals interest only if that gain is at least
+ *                    min_slack_gain MiB, else it declines and keeps the longer fragment for a window it fits.
+ *                    min_slack_gain = 0 switches the rule off.
+ *   R4' locality   : optional state- and locality-aware admission (Section 4.4, item 5; the Preference signal of
+ *                    Section 3.5): jobs declare a predicted checkpoint size ckpt_MiB_j and remember the slice
+ *                    their last fragment ran on.  A window on another slice means moving that state, so the
+ *                    policy score (the work for SLA, whose class stays) is lowered by weight * ckpt_MiB_j,
+ *                    not below zero; a window on the same slice, and a job that has not run yet, pay nothing.
+ *                    The commit records the granted gap's slice as the job's last slice.
+ *
  * The walk below visits one step at a time, exactly in that order: no prefix arrays,
  * no search, no blocking.  OpenMP only spreads independent gaps over host threads.
  *
- * Pins (tests/test_oracle_pins.py): exhaustive prefix enumeration on tiny inputs,
+ * Pins (tests/test_oracle_pins.py and the other tests/test_oracle_*_pins.py): exhaustive prefix enumeration on tiny inputs,
  * closed forms, reductions to numpy cumsum / searchsorted, monotonicity and symmetry
  * properties, the rigid-job special case, hand-computed policy examples, and the paper's
  * illustrative scenario.  The paper prints no numeric award values, so beyond those pins
@@ -92,35 +107,18 @@ static int step_is_safe(const uint32_t *safe_bits, uint64_t i)
 }
 
 /*
- * R1-R3 for one (gap, job) pair.  Returns 1 for interest (and fills k, dur, work),
- * 0 for decline.  [s, e) is the job's range of global step indices, p its progress.
+ * The walk of one pair: the longest candidate end index under the given bounds.  `begin` is when the subjob
+ * would start, `window_end` when the gap closes.  Returns 1 and fills k / dur / work / peak, or 0.
  */
-int orc_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *safe_bits,
-             uint64_t s, uint64_t e, uint32_t p, uint32_t ready_ms,
-             uint32_t start_ms, uint32_t T_ms, uint32_t C_MiB,
-             uint32_t tau_min_ms, uint32_t tau_max_ms,
-             int late_start, uint32_t deadline_ms,
-             const uint32_t *power_W /* per step like mem_MiB, or NULL */, uint32_t power_cap_W,
-             uint32_t *k_out, uint32_t *dur_out, uint64_t *work_out, uint32_t *peak_out /* may be NULL */)
+static int walk_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *safe_bits,
+                     uint64_t s, uint64_t e, uint32_t p, uint64_t begin, uint64_t window_end, uint32_t C_MiB,
+                     uint32_t tau_min_ms, uint32_t tau_max_ms, int has_deadline, uint32_t deadline_ms,
+                     const uint32_t *power_W, int has_cap, uint32_t power_cap_W,
+                     uint32_t *k_out, uint32_t *dur_out, uint64_t *work_out, uint32_t *peak_out)
 {
-    uint64_t len = e - s;
-    if ((uint64_t)p >= len) return 0;            /* R1: finished job */
-    uint64_t begin = start_ms;                   /* when the subjob would start running */
-    if (start_ms < ready_ms) {
-        if (!late_start) return 0;               /* R1: gap opens before the job is ready */
-        begin = ready_ms;                        /* R1'': start inside the window */
-    }
-    uint64_t window_end = (uint64_t)start_ms + (uint64_t)T_ms;
-    if (begin > window_end) return 0;            /* R1'': ready only after the window has closed */
-    const int has_deadline = deadline_ms != 0xFFFFFFFFu;          /* 2^32-1: no deadline */
-    if (has_deadline && begin > (uint64_t)deadline_ms) return 0; /* R1'': deadline already passed */
-
     uint64_t acc = 0, work = 0;
     uint32_t peak = 0, power_peak = 0;
-    const int has_cap = power_W != NULL && power_cap_W != 0xFFFFFFFFu;
     int found = 0;
-    uint32_t best_k = 0, best_dur = 0, best_peak = 0;
-    uint64_t best_work = 0;
     for (uint64_t i = s + p; i < e; ++i) {
         acc += dur_ms[i];
         if (mem_MiB[i] > peak) peak = mem_MiB[i];
@@ -135,23 +133,64 @@ int orc_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *sa
         if ((step_is_safe(safe_bits, i) || i + 1 == e)     /* R2: safe boundary after step i */
             && acc >= (uint64_t)tau_min_ms) {              /* R2': not shorter than the minimum subjob */
             found = 1;
-            best_k = (uint32_t)(i + 1 - s);
-            best_dur = (uint32_t)acc;
-            best_work = work;
-            best_peak = peak;
+            *k_out = (uint32_t)(i + 1 - s);
+            *dur_out = (uint32_t)acc;
+            *work_out = work;
+            *peak_out = peak;
         }
     }
-    if (!found) return 0;
-    *k_out = best_k;
-    *dur_out = best_dur;
-    *work_out = best_work;
-    if (peak_out) *peak_out = best_peak;
+    return found;
+}
+
+/*
+ * R1-R3 for one (gap, job) pair.  Returns 1 for interest (and fills k, dur, work),
+ * 0 for decline.  [s, e) is the job's range of global step indices, p its progress.
+ */
+int orc_pair(const uint32_t *dur_ms, const uint32_t *mem_MiB, const uint32_t *safe_bits,
+             uint64_t s, uint64_t e, uint32_t p, uint32_t ready_ms,
+             uint32_t start_ms, uint32_t T_ms, uint32_t C_MiB,
+             uint32_t tau_min_ms, uint32_t tau_max_ms,
+             int late_start, uint32_t deadline_ms,
+             const uint32_t *power_W /* per step like mem_MiB, or NULL */, uint32_t power_cap_W,
+             uint32_t min_slack_gain_MiB /* R3h, 0 = off */,
+             uint32_t *k_out, uint32_t *dur_out, uint64_t *work_out, uint32_t *peak_out /* may be NULL */)
+{
+    uint64_t len = e - s;
+    if ((uint64_t)p >= len) return 0;            /* R1: finished job */
+    uint64_t begin = start_ms;                   /* when the subjob would start running */
+    if (start_ms < ready_ms) {
+        if (!late_start) return 0;               /* R1: gap opens before the job is ready */
+        begin = ready_ms;                        /* R1'': start inside the window */
+    }
+    uint64_t window_end = (uint64_t)start_ms + (uint64_t)T_ms;
+    if (begin > window_end) return 0;            /* R1'': ready only after the window has closed */
+    const int has_deadline = deadline_ms != 0xFFFFFFFFu;          /* 2^32-1: no deadline */
+    if (has_deadline && begin > (uint64_t)deadline_ms) return 0; /* R1'': deadline already passed */
+    const int has_cap = power_W != NULL && power_cap_W != 0xFFFFFFFFu;
+
+    uint32_t k = 0, dur = 0, peak = 0;
+    uint64_t work = 0;
+    if (!walk_pair(dur_ms, mem_MiB, safe_bits, s, e, p, begin, window_end, C_MiB, tau_min_ms, tau_max_ms,
+                   has_deadline, deadline_ms, power_W, has_cap, power_cap_W, &k, &dur, &work, &peak))
+        return 0;
+    if (min_slack_gain_MiB > 0) {
+        /* R3h: the fragment the window alone would allow (capacity bound lifted) */
+        uint32_t k_T = 0, dur_T = 0, peak_T = 0;
+        uint64_t work_T = 0;
+        walk_pair(dur_ms, mem_MiB, safe_bits, s, e, p, begin, window_end, 0xFFFFFFFFu, tau_min_ms, tau_max_ms,
+                  has_deadline, deadline_ms, power_W, has_cap, power_cap_W, &k_T, &dur_T, &work_T, &peak_T);
+        if (k_T > k && peak_T - peak < min_slack_gain_MiB) return 0;   /* the cut gains too little: decline */
+    }
+    *k_out = k;
+    *dur_out = dur;
+    *work_out = work;
+    if (peak_out) *peak_out = peak;
     return 1;
 }
 
 /* R4: the policy key of an interested job, as (class, score). */
 static void policy_key(uint32_t policy, uint64_t work, uint32_t peak, uint32_t j,
-                       const uint32_t *wait_ms, const uint8_t *prio,
+                       const uint32_t *wait_ms, const uint8_t *prio, uint64_t penalty,
                        uint32_t *cls_out, uint64_t *score_out)
 {
     *cls_out = 0;
@@ -163,6 +202,8 @@ static void policy_key(uint32_t policy, uint64_t work, uint32_t peak, uint32_t j
     } else if (policy == ORC_TIGHT_FIT) {
         *score_out = peak;      /* largest peak <=> least slack C_g - peak */
     }
+    /* R4': the cost of moving the job's state to another slice, never below zero */
+    *score_out -= penalty < *score_out ? penalty : *score_out;
 }
 
 /*
@@ -178,6 +219,10 @@ int orc_select(uint32_t n_jobs, const uint64_t *off,
                uint32_t tau_min_ms, uint32_t tau_max_ms,
                int late_start, const uint32_t *deadline_ms /* per job, or NULL = none */,
                const uint32_t *power_W /* per step, or NULL */, const uint32_t *power_cap_W /* per gap, or NULL */,
+               uint32_t min_slack_gain_MiB /* R3h, 0 = off */,
+               const uint32_t *ckpt_MiB /* R4': per job, or NULL = off */,
+               const uint32_t *last_slice /* per job, 2^32-1 = has not run yet; NULL = none has */,
+               uint32_t locality_weight,
                orc_award *awards)
 {
     if (policy > ORC_TIGHT_FIT) return -1;
@@ -196,12 +241,14 @@ int orc_select(uint32_t n_jobs, const uint64_t *off,
             if (!orc_pair(dur_ms, mem_MiB, safe_bits, off[j], off[j + 1], progress[j],
                           ready_ms[j], gap.start_ms, gap.T_ms, gap.C_MiB, tau_min_ms, tau_max_ms,
                           late_start, deadline_ms ? deadline_ms[j] : 0xFFFFFFFFu,
-                          power_W, power_cap_W ? power_cap_W[g] : 0xFFFFFFFFu,
+                          power_W, power_cap_W ? power_cap_W[g] : 0xFFFFFFFFu, min_slack_gain_MiB,
                           &k, &dur, &work, &peak))
                 continue;                                      /* decline */
             uint32_t cls;
-            uint64_t score;
-            policy_key(policy, work, peak, j, wait_ms, prio, &cls, &score);
+            uint64_t score, penalty = 0;
+            if (ckpt_MiB && last_slice && last_slice[j] != 0xFFFFFFFFu && last_slice[j] != gap.slice)
+                penalty = (uint64_t)locality_weight * (uint64_t)ckpt_MiB[j];   /* R4': the state has to move */
+            policy_key(policy, work, peak, j, wait_ms, prio, penalty, &cls, &score);
             /* jobs are visited in ascending id, so a strict ">" keeps the lowest id on ties */
             if (!have || cls > best_cls || (cls == best_cls && score > best_score)) {
                 have = 1;
@@ -228,7 +275,8 @@ int orc_select(uint32_t n_jobs, const uint64_t *off,
  * jobs, returns the number of grants (or -1 if begin + dur does not fit in 32 bits).
  */
 int64_t orc_commit(uint32_t n_jobs, uint32_t *progress, uint32_t *ready_ms,
-                   uint32_t n_gaps, const orc_gap *gaps, orc_award *awards, int late_start)
+                   uint32_t n_gaps, const orc_gap *gaps, orc_award *awards, int late_start,
+                   uint32_t *last_slice /* R4': per job, updated for granted jobs; may be NULL */)
 {
     int64_t granted = 0;
     for (uint32_t g = 0; g < n_gaps; ++g) awards[g].granted = 0;
@@ -256,6 +304,7 @@ int64_t orc_commit(uint32_t n_jobs, uint32_t *progress, uint32_t *ready_ms,
         if (new_ready > 0xFFFFFFFFull) return -1;
         progress[j] = awards[g].end_step;
         ready_ms[j] = (uint32_t)new_ready;
+        if (last_slice) last_slice[j] = gaps[g].slice;     /* R4': where the job's state now lives */
         ++granted;
     }
     return granted;
