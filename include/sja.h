@@ -66,7 +66,7 @@ typedef enum { SJA_MEM_HOST = 0, SJA_MEM_DEVICE = 1 } sja_memspace;
 
 /* One advertised execution gap: a window in time on a slice of a given memory capacity (Section 3.5). 16 bytes. */
 typedef struct {
-    uint32_t slice;    /* MIG slice label, carried through, not used in scoring */
+    uint32_t slice;    /* MIG slice label; only sja_set_locality makes it count in scoring */
     uint32_t start_ms; /* absolute start of the window */
     uint32_t T_ms;     /* window length */
     uint32_t C_MiB;    /* slice memory capacity */
@@ -262,6 +262,40 @@ sja_status sja_set_duration_bounds(sja_ctx* ctx, uint32_t tau_min_ms, uint32_t t
  * select that has not been committed yet is discarded by the call: select again before commit.
  */
 sja_status sja_set_window_options(sja_ctx* ctx, uint32_t late_start, const uint32_t* deadline_ms, sja_memspace where);
+
+/*
+ * Hysteresis on slack gain (Section 3.9: against over-fragmentation by short-lived spikes, a further
+ * subdivision is accepted only if it gains a minimum of slack; longer, more stable fragments are preferred
+ * otherwise).  Reading taken here: let k_T be the longest subjob the window alone would allow (every rule but
+ * the memory capacity) and k* the longest one that also fits the capacity.  k* < k_T means the capacity
+ * forces the job to cut earlier -- a further subdivision -- and what the cut gains is the demand it sheds,
+ * max m[p..k_T) - max m[p..k*).  With min_slack_gain_MiB > 0 the job signals interest in such a pair only if
+ * that gain is at least the threshold; else it declines and keeps the longer fragment for a window it fits
+ * whole.  0 (the default) switches the rule off; a forced cut always sheds at least 1 MiB, so 1 changes
+ * nothing either.  Stays in force until changed.  With the rule on, every select runs the per-pair search
+ * kernel.  A select that has not been committed yet is discarded by the call.
+ */
+sja_status sja_set_hysteresis(sja_ctx* ctx, uint32_t min_slack_gain_MiB);
+
+/*
+ * State- and locality-aware admission (Section 4.4, item 5; the Preference signal of Section 3.5: jobs declare
+ * a predicted checkpoint size and a preference for the slice they ran on last, and admission penalises large
+ * checkpoints and favours locality).
+ *   ckpt_MiB    u32[J]  predicted checkpoint size of each job; NULL switches the feature off
+ *   last_slice  u32[J]  slice label (sja_gap.slice) of the job's last fragment, 0xFFFFFFFF = has not run yet;
+ *                       NULL = no job has run yet
+ *   weight              score units charged per MiB of checkpoint that has to move
+ * In a select, a job bidding for a gap on another slice than its last one has weight * ckpt_MiB_j taken off
+ * its policy score (off the work for SJA_POLICY_SLA, whose class stays), not below zero: a zero score still
+ * bids.  A gap on the same slice, and a job that has not run yet, pay nothing.  The reported score is the
+ * lowered one.  sja_commit records the slice of the granted gap as the job's last slice;
+ * sja_get_locality copies the current last slices out.  The arrays are copied; a new load drops them.  With
+ * the feature on every select runs the per-pair search kernel.  sja_set_locality discards a select that has
+ * not been committed yet.
+ */
+sja_status sja_set_locality(sja_ctx* ctx, const uint32_t* ckpt_MiB, const uint32_t* last_slice, uint32_t weight,
+                            sja_memspace where);
+sja_status sja_get_locality(sja_ctx* ctx, uint32_t* last_slice, sja_memspace where);
 
 /*
  * One scheduler over several GPUs (the paper has no counterpart; the round itself is Section 3.5).  The jobs

@@ -32,7 +32,7 @@ AWARD_DTYPE = np.dtype([("job", "<u4"), ("end_step", "<u4"), ("dur_ms", "<u4"), 
                         ("score", "<u8")])
 
 EXPORTS = [
-    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit", "sja_commit_masked", "sja_round_reauction", "sja_set_duration_bounds", "sja_set_window_options", "sja_update_profile", "sja_load_power", "sja_advertise_power_caps", "sja_get_bids", "sja_reduce_bids",
+    "sja_create", "sja_destroy", "sja_load_profiles", "sja_advertise", "sja_select", "sja_select_static", "sja_commit", "sja_commit_masked", "sja_round_reauction", "sja_set_duration_bounds", "sja_set_window_options", "sja_set_hysteresis", "sja_set_locality", "sja_get_locality", "sja_update_profile", "sja_load_power", "sja_advertise_power_caps", "sja_get_bids", "sja_reduce_bids",
     "sja_get_awards", "sja_get_state", "sja_scan_size", "sja_get_scan", "sja_profile_enable",
     "sja_profile_read", "sja_last_error", "sja_debug_fail_alloc",
 ]
@@ -81,6 +81,9 @@ def load_library() -> ctypes.CDLL:
     lib.sja_round_reauction.argtypes = [vp, ctypes.POINTER(SjaPolicy), u32, ctypes.POINTER(u32), ctypes.POINTER(u32)]
     lib.sja_set_duration_bounds.argtypes = [vp, u32, u32]
     lib.sja_set_window_options.argtypes = [vp, u32, vp, i32]
+    lib.sja_set_hysteresis.argtypes = [vp, u32]
+    lib.sja_set_locality.argtypes = [vp, vp, vp, u32, i32]
+    lib.sja_get_locality.argtypes = [vp, vp, i32]
     lib.sja_update_profile.argtypes = [vp, u32, u32, vp, vp, i32]
     lib.sja_load_power.argtypes = [vp, vp, vp, i32]
     lib.sja_get_bids.argtypes = [vp, u32, u32, vp, i32]
@@ -263,6 +266,25 @@ class Sja:
             raise ValueError("deadline_ms needs one entry per loaded job")
         self._check(self._lib.sja_set_window_options(self._h, 1 if late_start else 0, p,
                                                      MEM_HOST if space is None else space))
+
+    # -- sja_set_hysteresis
+    def set_hysteresis(self, min_slack_gain_MiB: int = 0) -> None:
+        self._check(self._lib.sja_set_hysteresis(self._h, int(min_slack_gain_MiB)))
+
+    # -- sja_set_locality / sja_get_locality
+    def set_locality(self, ckpt_MiB=None, last_slice=None, weight: int = 0) -> None:
+        """``ckpt_MiB`` / ``last_slice``: u32 per job (numpy or CUDA tensors); ``ckpt_MiB=None`` switches it off."""
+        pc, space, kc = _ptr_space(ckpt_MiB, None, np.uint32)
+        pl, space, kl = _ptr_space(last_slice, space, np.uint32)
+        for k in (kc, kl):
+            if k is not None and int(k.shape[0]) != self.n_jobs:
+                raise ValueError("locality arrays need one entry per loaded job")
+        self._check(self._lib.sja_set_locality(self._h, pc, pl, int(weight), MEM_HOST if space is None else space))
+
+    def get_locality(self) -> np.ndarray:
+        out = np.empty(self.n_jobs, dtype=np.uint32)
+        self._check(self._lib.sja_get_locality(self._h, out.ctypes.data, MEM_HOST))
+        return out
 
     # -- sja_get_bids / sja_reduce_bids (one scheduler over several GPUs)
     def get_bids(self, job_base: int, rank: int, out=None):

@@ -73,6 +73,10 @@ struct sja_ctx {
     uint32_t tau_min = 0, tau_max = 0xFFFFFFFFu;   // subjob duration thresholds for select
     bool late_start = false, have_deadline = false;   // window options (sja_set_window_options)
     DevBuf deadline;
+    uint32_t min_gain = 0;                             // hysteresis threshold (sja_set_hysteresis); 0 = off
+    bool have_locality = false;                        // checkpoint sizes and last slices loaded (sja_set_locality)
+    uint32_t loc_weight = 0;
+    DevBuf ckpt, last_slice;
     bool have_power = false, have_caps = false;        // power envelope (sja_load_power, sja_advertise_power_caps)
     DevBuf PW, caps, st_power;
     DevBuf st_bids, st_accept, st_global;              // sharded rounds: staging for host-side callers
@@ -256,6 +260,11 @@ JobView job_view(const sja_ctx* c) {
     v.late_start = c->late_start ? 1u : 0u;
     v.PW = (c->have_power && c->have_caps) ? c->PW.as<uint2>() : nullptr;
     v.caps = (c->have_power && c->have_caps) ? c->caps.as<uint32_t>() : nullptr;
+    v.min_gain = c->min_gain;
+    v.ckpt = c->have_locality ? c->ckpt.as<uint32_t>() : nullptr;
+    v.last_slice = c->have_locality ? c->last_slice.as<uint32_t>() : nullptr;
+    v.loc_weight = c->loc_weight;
+    v.gaps_orig = c->gaps.as<uint4>();
     v.J = c->J;
     return v;
 }
@@ -354,7 +363,9 @@ struct SelectPlan { KernelPlan primary, alt; bool have_alt; uint32_t max_classes
 KernelPlan plan_kernel(const sja_ctx* c, SelectKernel k, uint32_t G_act) {
     KernelPlan p;
     p.kernel = k;
-    p.jobs_per_cta = k == SEL_TILE ? (uint32_t)TILE_JOBS : k == SEL_MERGE ? (uint32_t)MERGE_JOBS : (uint32_t)SEARCH_THREADS;
+    // the search kernel gives every gap a thread: with few gaps it takes small job chunks, so that many CTAs share the jobs
+    p.jobs_per_cta = k == SEL_TILE ? (uint32_t)TILE_JOBS : k == SEL_MERGE ? (uint32_t)MERGE_JOBS
+                     : G_act <= 64u ? 32u : (uint32_t)SEARCH_JOBS;
     p.n_chunks = (c->J + p.jobs_per_cta - 1) / p.jobs_per_cta;
     // granularity of a gap split: a staging tile; the tile kernel also works in 32-gap steps, which a
     // small problem needs to put enough CTAs on the GPU
@@ -382,7 +393,8 @@ SelectPlan plan_select(const sja_ctx* c, uint32_t pflags, uint32_t G_act) {
     // 2^21 pairs the fixed start-up of the ordered-gap kernels outweighs what they save)
     const bool tiny = (uint64_t)c->J * c->G < (1ull << 16) || (G_act < c->G && (uint64_t)c->J * G_act < (1ull << 21));
     // with a window option the usable window differs from pair to pair: only the search kernel does that
-    const bool per_pair_window = c->late_start || c->have_deadline || (c->have_power && c->have_caps);
+    const bool per_pair_window = c->late_start || c->have_deadline || (c->have_power && c->have_caps) ||
+                                 c->min_gain != 0u || c->have_locality;
     const bool search_only = (pflags & SJA_FLAG_FORCE_SEARCH) || per_pair_window || !c->gaps_sorted || (!forced && tiny);
     p.max_classes = std::max<uint32_t>(64u, c->G / 16u);
     p.have_alt = !search_only;
@@ -401,7 +413,7 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
     const SelectPlan pl = plan_select(c, pflags, G_act);
     Partial* partial = scratch;
     if (!partial) {
-        TRY(reserve(c, c->partial, (size_t)pl.rows * c->G * sizeof(Partial)));
+        TRY(reserve(c, c->partial, (size_t)pl.rows * G_act * sizeof(Partial)));
         partial = c->partial.as<Partial>();
     }
     const int was_on = c->prof;
@@ -416,14 +428,16 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
         gate.max_classes = pl.max_classes;
         gate.run_if_many = 0u;
         auto launch_search = [&](const KernelPlan& kp, const LaunchGate& g) {
-            const bool opts = jv.late_start != 0u || jv.deadline != nullptr || jv.PW != nullptr;
+            const bool opts = jv.late_start != 0u || jv.deadline != nullptr || jv.PW != nullptr || jv.min_gain != 0u ||
+                              jv.ckpt != nullptr;
             if (opts)
                 select_search_kernel<true><<<dim3(kp.n_chunks, kp.splits), SEARCH_THREADS,
                                              jv.PW ? SEARCH_SMEM_BYTES_POWER : SEARCH_SMEM_BYTES, c->stream>>>(
-                    jv, sgaps, G_act, kp.per_split, kind, partial, g);
+                    jv, sgaps, G_act, kp.per_split, kind, partial, g, kp.jobs_per_cta);
             else
                 select_search_kernel<false><<<dim3(kp.n_chunks, kp.splits), SEARCH_THREADS, SEARCH_SMEM_BYTES,
-                                              c->stream>>>(jv, sgaps, G_act, kp.per_split, kind, partial, g);
+                                              c->stream>>>(jv, sgaps, G_act, kp.per_split, kind, partial, g,
+                                                           kp.jobs_per_cta);
         };
         if (pl.primary.kernel != SEL_SEARCH)
             launch_sorted(pl.primary.kernel, kind, dim3(pl.primary.n_chunks, pl.primary.splits), c->stream, jv, sgaps,
@@ -454,7 +468,8 @@ void run_commit(sja_ctx* c, uint32_t* blocked, const uint8_t* accept = nullptr) 
         c->awards.as<Award>(), c->gaps.as<Gap>(), c->widx.as<uint32_t>(), G, c->jobwin.as<unsigned long long>(),
         c->boff.as<uint64_t>(), c->A.as<uint4>(), c->p.as<uint32_t>(), c->ready.as<uint32_t>(), c->pb.as<uint32_t>(),
         c->Dp.as<uint32_t>(), c->Wp.as<uint64_t>(), c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(),
-        c->flags.as<uint32_t>(), blocked, accept, c->late_start ? 1u : 0u);
+        c->flags.as<uint32_t>(), blocked, accept, c->late_start ? 1u : 0u,
+        c->have_locality ? c->last_slice.as<uint32_t>() : nullptr);
     commit_refresh_kernel<<<(uint32_t)(((uint64_t)G * 32 + 255) / 256), 256, 0, c->stream>>>(
         c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(), G, c->boff.as<uint64_t>(), c->pb.as<uint32_t>(),
         c->A.as<uint4>(), c->B.as<uint2>(), c->jobwin.as<unsigned long long>(),
@@ -549,7 +564,7 @@ sja_status sja_destroy(sja_ctx* c) {
     cudaStreamSynchronize(c->stream);
     DevBuf* bufs[] = {&c->st_off, &c->st_d, &c->st_m, &c->st_s, &c->st_p, &c->st_ready, &c->st_wait, &c->st_prio, &c->p, &c->ready, &c->pb, &c->Dp,
                       &c->Wp, &c->wait, &c->prio, &c->nbj, &c->cta_tot, &c->cta_base, &c->boff, &c->boff_next, &c->A, &c->B, &c->jobwin,
-                      &c->flags, &c->counter, &c->n_granted, &c->long_list, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->deadline, &c->PW, &c->caps, &c->st_power, &c->st_bids, &c->st_accept, &c->st_global, &c->upd_d, &c->upd_m, &c->upd_scratch, &c->upd_status, &c->awards, &c->widx, &c->partial,
+                      &c->flags, &c->counter, &c->n_granted, &c->long_list, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->deadline, &c->ckpt, &c->last_slice, &c->PW, &c->caps, &c->st_power, &c->st_bids, &c->st_accept, &c->st_global, &c->upd_d, &c->upd_m, &c->upd_scratch, &c->upd_status, &c->awards, &c->widx, &c->partial,
                       &c->winners};
     for (DevBuf* b : bufs) release(*b);
     for (ProfSpan& s : c->spans) { cudaEventDestroy(s.a); cudaEventDestroy(s.b); }
@@ -760,8 +775,9 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
 
     // from here on the previous load is replaced
     c->loaded = false;
-    c->have_deadline = false;                // deadlines and power traces belong to the jobs of a load
+    c->have_deadline = false;                // deadlines, power traces, checkpoint sizes belong to the jobs of a load
     c->have_power = false;
+    c->have_locality = false;
     c->advertised = c->selected = c->committed = false;
     if (!speculate || n_rows > cap_now) {
         // buffers too small for this load (the kernels above, if launched, stood still): size them and run
@@ -1031,6 +1047,48 @@ sja_status sja_set_duration_bounds(sja_ctx* c, uint32_t tau_min_ms, uint32_t tau
         return fail(c, SJA_ERR_INVALID_ARG, "sja_set_duration_bounds: tau_min %u > tau_max %u", tau_min_ms, tau_max_ms);
     c->tau_min = tau_min_ms;
     c->tau_max = tau_max_ms;
+    return SJA_OK;
+}
+
+sja_status sja_set_hysteresis(sja_ctx* c, uint32_t min_slack_gain_MiB) {
+    TRY(check_ctx(c));
+    c->min_gain = min_slack_gain_MiB;
+    c->selected = false;   // awards chosen under the old threshold must not be committed under the new one
+    return SJA_OK;
+}
+
+sja_status sja_set_locality(sja_ctx* c, const uint32_t* ckpt_MiB, const uint32_t* last_slice, uint32_t weight,
+                            sja_memspace where) {
+    TRY(check_ctx(c));
+    if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_set_locality: bad memspace");
+    if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_set_locality before sja_load_profiles");
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
+    if (ckpt_MiB) {
+        TRY(reserve(c, c->ckpt, (size_t)c->J * 4));
+        TRY(reserve(c, c->last_slice, (size_t)c->J * 4));
+        TRY(copy_in(c, c->ckpt.p, ckpt_MiB, (size_t)c->J * 4, where));
+        if (last_slice) TRY(copy_in(c, c->last_slice.p, last_slice, (size_t)c->J * 4, where));
+        else CU(cudaMemsetAsync(c->last_slice.p, 0xFF, (size_t)c->J * 4, c->stream));   // nobody has run yet
+        if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));   // the caller may reuse its buffers
+    }
+    c->have_locality = ckpt_MiB != nullptr;
+    c->loc_weight = weight;
+    c->selected = false;   // awards chosen without the penalty must not be committed with it
+    return SJA_OK;
+}
+
+sja_status sja_get_locality(sja_ctx* c, uint32_t* last_slice, sja_memspace where) {
+    TRY(check_ctx(c));
+    if (!last_slice) return fail(c, SJA_ERR_INVALID_ARG, "sja_get_locality: out is NULL");
+    if (where != SJA_MEM_HOST && where != SJA_MEM_DEVICE)
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_get_locality: bad memspace");
+    if (!c->loaded || !c->have_locality) return fail(c, SJA_ERR_STATE, "sja_get_locality before sja_set_locality");
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
+    TRY(copy_out(c, last_slice, c->last_slice.p, (size_t)c->J * 4, where));
+    if (where == SJA_MEM_HOST) CU(cudaStreamSynchronize(c->stream));
     return SJA_OK;
 }
 

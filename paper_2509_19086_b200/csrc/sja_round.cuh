@@ -24,6 +24,11 @@ struct JobView {
     uint32_t late_start;        // non-zero: a job that turns ready inside a window may begin then
     const uint2* PW;            // may be nullptr; per row {running max, segment max} of the power trace (Section 4.4, item 1)
     const uint32_t* caps;       // may be nullptr; per gap (caller's index) power cap, 0xFFFFFFFF = none
+    uint32_t min_gain;          // hysteresis (Section 3.9): least slack gain that justifies a capacity-forced cut; 0 = off
+    const uint32_t* ckpt;       // may be nullptr; per job predicted checkpoint size in MiB (Section 4.4, item 5)
+    const uint32_t* last_slice; // with ckpt: per job the slice of its last fragment, 0xFFFFFFFF = has not run yet
+    uint32_t loc_weight;        // score units per MiB of checkpoint that has to move to another slice
+    const uint4* gaps_orig;     // the batch in the caller's order (the slice of a gap: ordered copies carry the index there)
     uint32_t J;
 };
 
@@ -56,184 +61,260 @@ __device__ __forceinline__ uint32_t policy_factor(const JobView& jv, uint32_t ki
 }
 
 // ---------------------------------------------------------------------------------------
-// Per-pair search kernel.  One thread owns one job and visits every gap of its gap range;
-// for each pair it finds the number of boundary rows that satisfy both monotone bounds
-// (D - Dp <= T and running max <= C) with a galloping + binary search over the rows above
-// the progress point, turns the last such row into a policy key, and the warp reduces the
-// 32 keys to one candidate per gap (largest key, then lowest job id).  Because every pair
-// is searched on its own, this is also the kernel for the window options, where the usable
-// window differs from pair to pair: with a late start the subjob begins at
-// max(start, ready) and only the rest of the window counts; with a deadline it must be over
-// by then.  The first SEARCH_ROWS rows of every job are staged in shared memory once per CTA
-// (most windows end inside them), so the usual pair is a five-probe search in shared memory;
-// only longer answers continue in global memory.
+// Per-pair search kernel.  Every (gap, job) pair is searched on its own: the number of the job's boundary rows
+// that satisfy both monotone bounds (D - Dp <= T and running max <= C) is found by a binary search over the rows
+// above the progress point, the last such row becomes a policy key, and the largest key per gap (ties: lowest job
+// id) is the candidate.  Because nothing is carried from one pair to the next, this is also the kernel for
+// everything that makes the test differ from pair to pair: a late start (the subjob begins at max(start, ready)
+// and only the rest of the window counts), a deadline (it must be over by then), a power cap (a second running
+// maximum), the hysteresis rule (a second search with the capacity lifted) and the locality penalty (the key
+// depends on the gap's slice).
+//
+// Work split: a CTA stages the first SEARCH_ROWS rows of a chunk of jobs in shared memory (most windows end
+// inside them; only longer answers continue in global memory) and owns a range of the gaps.  A THREAD owns a
+// gap and walks the staged jobs in ascending id: all lanes of a warp look at the same job at the same time, so
+// the job's constants are broadcast reads, the five probes of the lanes fall into the 32 banks of the job's
+// 128-byte row block without conflict, and the running best of a gap lives in its thread's registers -- no
+// reduction across lanes, no staging of candidates, one coalesced candidate row per CTA at the end.
 constexpr int SEARCH_THREADS = 256;
-constexpr int SEARCH_GT = 64;   // gaps per staging tile
+#ifndef SJA_SEARCH_JOBS
+#define SJA_SEARCH_JOBS 256
+#endif
 #ifndef SJA_SEARCH_ROWS
 #define SJA_SEARCH_ROWS 16
 #endif
-#ifndef SJA_SEARCH_PAY_ROWS
-#define SJA_SEARCH_PAY_ROWS 16
+#ifndef SJA_SEARCH_U
+#define SJA_SEARCH_U 4
 #endif
-constexpr int SEARCH_ROWS = SJA_SEARCH_ROWS;          // boundary rows staged per job as {D - Dp, M} (a power of two)
-constexpr int SEARCH_PAY_ROWS = SJA_SEARCH_PAY_ROWS;  // of which the first ones also with their policy payload
-constexpr int SEARCH_SMEM_BYTES = (SEARCH_ROWS + SEARCH_PAY_ROWS) * SEARCH_THREADS * 8;   // [row][thread]
-constexpr int SEARCH_SMEM_BYTES_POWER = SEARCH_SMEM_BYTES + SEARCH_ROWS * SEARCH_THREADS * 4;   // + running power maxima
-static_assert((SEARCH_ROWS & (SEARCH_ROWS - 1)) == 0 && SEARCH_PAY_ROWS <= SEARCH_ROWS, "staging shape");
+constexpr int SEARCH_U = SJA_SEARCH_U;                // jobs a thread has in flight
+constexpr int SEARCH_JOBS = SJA_SEARCH_JOBS;          // most jobs a CTA stages (a launch may ask for fewer)
+constexpr int SEARCH_GT = SEARCH_THREADS;             // granularity of a gap split: one gap per thread
+constexpr int SEARCH_ROWS = SJA_SEARCH_ROWS;          // boundary rows staged per job (a power of two)
+// per staged job: rows {D - Dp, M} and their policy payload, 14 words of constants; with power caps the rows'
+// running power maxima as well
+constexpr int SEARCH_JOB_WORDS = 14;
+constexpr int SEARCH_SMEM_BYTES = SEARCH_JOBS * (SEARCH_ROWS * 16 + SEARCH_JOB_WORDS * 4);
+constexpr int SEARCH_SMEM_BYTES_POWER = SEARCH_SMEM_BYTES + SEARCH_JOBS * SEARCH_ROWS * 4;
+static_assert((SEARCH_ROWS & (SEARCH_ROWS - 1)) == 0 && SEARCH_ROWS == 16, "a half-warp stages the rows of one job");
 
-// OPTS: a window option or a power cap is in force (compiled out otherwise).
+// Policy key with the locality penalty taken off the score first (never below zero).
+__device__ __forceinline__ uint64_t policy_key_less(uint32_t kind, uint64_t payload, uint32_t factor, uint64_t penalty) {
+    uint64_t score = kind == 1 ? payload * (uint64_t)factor : payload;
+    score -= min(score, penalty);
+    return kind == 2 ? ((uint64_t)factor << KEY_SLA_SHIFT) + score + 1ull : score + 1ull;
+}
+
+// OPTS: something that differs from pair to pair is in force (compiled out otherwise).
+// jobs_per_cta: jobs of one chunk (<= SEARCH_JOBS); the candidate row of chunk c is partial_out[c * G ...].
 template <bool OPTS>
 __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
     JobView jv, const Gap* __restrict__ gaps, uint32_t G, uint32_t gaps_per_split, uint32_t kind,
-    Partial* __restrict__ partial_out, LaunchGate gate) {
-    __shared__ Partial stage[SEARCH_GT][SEARCH_THREADS / 32];
-    __shared__ uint4 sgap[SEARCH_GT];
+    Partial* __restrict__ partial_out, LaunchGate gate, uint32_t jobs_per_cta) {
     const uint32_t G_now = gate_gaps(gate, G);   // gaps actually left (G stays the row length of partial_out)
     if (blockIdx.y * gaps_per_split >= G_now) return;
-    extern __shared__ __align__(16) uint2 search_rows[];
-    uint2* sDM = search_rows + threadIdx.x;                                     // row r of this thread: sDM[r * THREADS]
-    uint2* sPay = search_rows + SEARCH_ROWS * SEARCH_THREADS + threadIdx.x;     // its policy payload (work or peak)
-    // with power caps in force the launch carries room for the rows' running power maxima as well
-    uint32_t* sPow = reinterpret_cast<uint32_t*>(search_rows + (SEARCH_ROWS + SEARCH_PAY_ROWS) * SEARCH_THREADS) + threadIdx.x;
-    const bool staged_power = OPTS && jv.PW != nullptr;
+    extern __shared__ __align__(16) unsigned char search_smem[];
+    uint2* sDM = reinterpret_cast<uint2*>(search_smem);                                   // [job][row] {D - Dp, M}
+    uint2* sPay = sDM + SEARCH_JOBS * SEARCH_ROWS;                                        // [job][row] policy payload
+    uint32_t* sJob = reinterpret_cast<uint32_t*>(sPay + SEARCH_JOBS * SEARCH_ROWS);       // [word][job] constants
+    uint32_t* sPow = sJob + SEARCH_JOB_WORDS * SEARCH_JOBS;                               // [job][row], with power caps
+    // words of sJob: 0 n, 1 ready, 2 factor, 3 deadline, 4 home slice, 5 Dp, 6-7 first row index, 8-9 Wp, 10-11 penalty
+    const bool with_caps = OPTS && jv.PW != nullptr && jv.caps != nullptr;
+    const bool with_locality = OPTS && jv.ckpt != nullptr && jv.last_slice != nullptr;
+    const uint32_t min_gain = OPTS ? jv.min_gain : 0u;
+    const bool late = OPTS && jv.late_start != 0u;
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
-    const uint32_t j = blockIdx.x * SEARCH_THREADS + threadIdx.x;
+    const uint32_t job0 = blockIdx.x * jobs_per_cta;
+    const uint32_t n_jobs = min(jobs_per_cta, jv.J - job0);
 
-    uint64_t base = 0, Wp = 0;
-    uint32_t n = 0, Dp = 0, ready = 0xFFFFFFFFu, factor = 0, deadline = 0xFFFFFFFFu;
-    if (j < jv.J) {
+    // ---- stage the chunk: a half-warp per job, one row per lane (a coalesced 256-byte read of the table)
+    for (uint32_t jj = wid * 2u + (lane >> 4); jj < n_jobs; jj += (SEARCH_THREADS / 32) * 2u) {
+        const uint32_t j = job0 + jj, r = lane & 15u;
         const uint64_t b0 = jv.boff[j], b1 = jv.boff[j + 1];
         const uint32_t pb = jv.pb[j];
-        base = b0 + pb;
-        n = (uint32_t)(b1 - b0) - pb;
+        const uint64_t base = b0 + pb;
+        uint32_t n = (uint32_t)(b1 - b0) - pb;
         if (jv.blocked && jv.blocked[j]) n = 0;
-        Dp = jv.Dp[j];
-        Wp = jv.Wp[j];
-        ready = jv.ready[j];
-        factor = policy_factor(jv, kind, j);
-        if (OPTS && jv.deadline) deadline = jv.deadline[j];
-    }
-    const bool late = OPTS && jv.late_start != 0u;
-    const uint32_t g_begin = blockIdx.y * gaps_per_split;
-    const uint32_t g_end = min(G_now, g_begin + gaps_per_split);
-    // The first rows of the job in shared memory; the slots beyond its last row hold a sentinel that no
-    // window admits (except T = C = 2^32-1, where the clamp below takes care), so every thread runs the
-    // same five probes.  Each thread reads back only what it wrote: no barrier needed.
-    const uint32_t ns = min(n, (uint32_t)SEARCH_ROWS);
-    for (uint32_t r = 0; r < (uint32_t)SEARCH_ROWS; ++r) {
+        const uint32_t Dp = jv.Dp[j];
+        const uint64_t Wp = jv.Wp[j];
+        // rows beyond the job's last one hold a sentinel that no window admits (T = C = 2^32-1 is clamped below)
         uint2 dm = make_uint2(0xFFFFFFFFu, 0xFFFFFFFFu), pay = make_uint2(0u, 0u);
-        if (r < ns) {
+        uint32_t pw = 0xFFFFFFFFu;
+        if (r < n) {
             const uint4 row = __ldg(jv.A + base + r);
             const uint64_t pl = policy_payload(kind, row, Wp);
             dm = make_uint2(row.x - Dp, row.y);
             pay = make_uint2((uint32_t)pl, (uint32_t)(pl >> 32));
+            if (with_caps) pw = __ldg(&jv.PW[base + r].x);
         }
-        sDM[r * SEARCH_THREADS] = dm;
-        if (r < (uint32_t)SEARCH_PAY_ROWS) sPay[r * SEARCH_THREADS] = pay;
-        if (staged_power) sPow[r * SEARCH_THREADS] = r < ns ? __ldg(&jv.PW[base + r].x) : 0xFFFFFFFFu;
-    }
-
-    for (uint32_t g0 = g_begin; g0 < g_end; g0 += SEARCH_GT) {
-        const uint32_t gt = min((uint32_t)SEARCH_GT, g_end - g0);
-        // the tile's gaps in shared memory; the next one is fetched while the current one is worked on
-        if (threadIdx.x < gt) sgap[threadIdx.x] = __ldg(reinterpret_cast<const uint4*>(gaps) + g0 + threadIdx.x);
-        __syncthreads();
-        uint4 gq_next = sgap[0];
-        for (uint32_t gi = 0; gi < gt; ++gi) {
-            const uint4 gq = gq_next;
-            gq_next = sgap[min(gi + 1, gt - 1)];
-            const uint32_t start = gq.y, C = gq.w;
-            uint32_t T = gq.z, cap = 0xFFFFFFFFu;
-            bool eligible = n != 0;
-            if (OPTS) {
-                // power cap of the offer (the caller's gap index travels in the slice field)
-                if (jv.PW && jv.caps) cap = __ldg(jv.caps + gq.x);
-                // the window this pair sees: what is left of the gap once the job can begin, cut at its deadline
-                uint32_t begin = start;
-                if (start < ready) {
-                    const uint32_t late_by = ready - start;
-                    if (!late || late_by > T) eligible = false;
-                    begin = ready;
-                    T -= min(late_by, T);
-                }
-                if (deadline != 0xFFFFFFFFu) {
-                    if (begin > deadline) eligible = false;
-                    T = min(T, deadline - min(begin, deadline));
-                }
-            } else {
-                eligible = eligible && start >= ready;
+        sDM[jj * SEARCH_ROWS + r] = dm;
+        sPay[jj * SEARCH_ROWS + r] = pay;
+        if (with_caps) sPow[jj * SEARCH_ROWS + r] = pw;
+        if (r == 0) {
+            uint64_t penalty = 0;
+            uint32_t home = 0xFFFFFFFFu;
+            if (with_locality) {
+                home = jv.last_slice[j];
+                penalty = (uint64_t)jv.loc_weight * (uint64_t)jv.ckpt[j];
             }
-            T = min(T, jv.tau_max);
-            const bool capped = OPTS && cap != 0xFFFFFFFFu;
-            // number of staged rows that satisfy all bounds (they form a prefix): five probes, no branches
-            auto fits = [&](uint32_t idx) -> bool {
-                const uint2 r = sDM[idx * SEARCH_THREADS];
-                bool ok = r.x <= T && r.y <= C;
-                if (OPTS && capped && ok && idx < ns) ok = sPow[idx * SEARCH_THREADS] <= cap;
+            sJob[0 * SEARCH_JOBS + jj] = n;
+            sJob[1 * SEARCH_JOBS + jj] = jv.ready[j];
+            sJob[2 * SEARCH_JOBS + jj] = policy_factor(jv, kind, j);
+            sJob[3 * SEARCH_JOBS + jj] = (OPTS && jv.deadline) ? jv.deadline[j] : 0xFFFFFFFFu;
+            sJob[4 * SEARCH_JOBS + jj] = home;
+            sJob[5 * SEARCH_JOBS + jj] = Dp;
+            sJob[6 * SEARCH_JOBS + jj] = (uint32_t)base;
+            sJob[7 * SEARCH_JOBS + jj] = (uint32_t)(base >> 32);
+            sJob[8 * SEARCH_JOBS + jj] = (uint32_t)Wp;
+            sJob[9 * SEARCH_JOBS + jj] = (uint32_t)(Wp >> 32);
+            sJob[10 * SEARCH_JOBS + jj] = (uint32_t)penalty;
+            sJob[11 * SEARCH_JOBS + jj] = (uint32_t)(penalty >> 32);
+        }
+    }
+    __syncthreads();
+
+    const uint32_t g_begin = blockIdx.y * gaps_per_split;
+    const uint32_t g_end = min(G_now, g_begin + gaps_per_split);
+    for (uint32_t g = g_begin + threadIdx.x; g < g_end; g += SEARCH_THREADS) {
+        const uint4 gq = __ldg(reinterpret_cast<const uint4*>(gaps) + g);
+        const uint32_t start = gq.y, C = gq.w;
+        // (the caller's gap index travels in the slice field of the ordered copy)
+        const uint32_t cap = with_caps ? __ldg(jv.caps + gq.x) : 0xFFFFFFFFu;
+        const uint32_t slice = with_locality ? __ldg(&jv.gaps_orig[gq.x].x) : 0u;
+        uint64_t best_key = 0;
+        uint32_t best_job = 0xFFFFFFFFu, best_cnt = 0;
+
+        // SEARCH_U jobs are in flight per thread: their probe chains are independent, so the shared-memory latency
+        // of one search hides behind the others.
+        for (uint32_t j0 = 0; j0 < n_jobs; j0 += SEARCH_U) {
+            uint32_t Tq[SEARCH_U], nq[SEARCH_U], lo[SEARCH_U];
+            bool elig[SEARCH_U];
+#pragma unroll
+            for (int u = 0; u < SEARCH_U; ++u) {
+                const uint32_t jj = min(j0 + (uint32_t)u, n_jobs - 1u);      // (a pass beyond the chunk repeats its last job, not eligible)
+                const uint32_t n = sJob[0 * SEARCH_JOBS + jj];
+                const uint32_t ready = sJob[1 * SEARCH_JOBS + jj];
+                uint32_t T = gq.z;
+                bool eligible = n != 0u && j0 + (uint32_t)u < n_jobs;
+                if (OPTS) {
+                    // the window this pair sees: what is left of the gap once the job can begin, cut at its deadline
+                    const uint32_t deadline = sJob[3 * SEARCH_JOBS + jj];
+                    uint32_t begin = start;
+                    if (start < ready) {
+                        const uint32_t late_by = ready - start;
+                        if (!late || late_by > T) eligible = false;
+                        begin = ready;
+                        T -= min(late_by, T);
+                    }
+                    if (deadline != 0xFFFFFFFFu) {
+                        if (begin > deadline) eligible = false;
+                        T = min(T, deadline - min(begin, deadline));
+                    }
+                } else {
+                    eligible = eligible && start >= ready;
+                }
+                Tq[u] = min(T, jv.tau_max);
+                nq[u] = n;
+                elig[u] = eligible;
+                lo[u] = 0;
+            }
+            // does staged row idx of job jj fit a window of T ms under capacity Cx (and the gap's power cap)?
+            auto fits = [&](uint32_t jj, uint32_t idx, uint32_t T, uint32_t Cx, uint32_t ns) -> bool {
+                const uint2 r = sDM[jj * SEARCH_ROWS + idx];
+                bool ok = r.x <= T && r.y <= Cx;
+                if (OPTS && cap != 0xFFFFFFFFu && ok && idx < ns) ok = sPow[jj * SEARCH_ROWS + idx] <= cap;
                 return ok;
             };
-            uint32_t lo = 0;
+            // the probe chains, level by level: five probes per search, no branches
 #pragma unroll
-            for (uint32_t s = SEARCH_ROWS / 2; s > 0; s >>= 1) lo += fits(lo + s - 1) ? s : 0u;
-            lo += fits(lo) ? 1u : 0u;
-            lo = eligible ? min(lo, ns) : 0u;
-            if (eligible && lo == ns && ns < n) {
-                // every staged row fits: gallop on through global memory (rows ns, ns + 1, ns + 3, ...)
-                uint32_t hi = n, step = 1;
-                for (uint32_t idx = ns;;) {
-                    if (idx >= n) { hi = n; break; }
-                    const uint4 r = __ldg(jv.A + base + idx);
-                    bool ok = r.x - Dp <= T && r.y <= C;
-                    if (OPTS && ok && capped) ok = __ldg(&jv.PW[base + idx].x) <= cap;
-                    if (ok) { lo = idx + 1; idx += step; step <<= 1; }
-                    else { hi = idx; break; }
-                }
-                while (lo < hi) {
-                    const uint32_t mid = lo + ((hi - lo) >> 1);
-                    const uint4 r = __ldg(jv.A + base + mid);
-                    bool ok = r.x - Dp <= T && r.y <= C;
-                    if (OPTS && ok && capped) ok = __ldg(&jv.PW[base + mid].x) <= cap;
-                    if (ok) lo = mid + 1; else hi = mid;
+            for (uint32_t sp = SEARCH_ROWS / 2; sp > 0; sp >>= 1) {
+#pragma unroll
+                for (int u = 0; u < SEARCH_U; ++u) {
+                    const uint32_t jj = min(j0 + (uint32_t)u, n_jobs - 1u);
+                    lo[u] += fits(jj, lo[u] + sp - 1, Tq[u], C, min(nq[u], (uint32_t)SEARCH_ROWS)) ? sp : 0u;
                 }
             }
-            uint32_t cnt = lo;
-            uint64_t key = 0;
-            if (cnt) {
-                uint32_t dur;
+#pragma unroll
+            for (int u = 0; u < SEARCH_U; ++u) {
+                const uint32_t jj = min(j0 + (uint32_t)u, n_jobs - 1u);
+                const uint32_t n = nq[u], T = Tq[u];
+                const uint32_t ns = min(n, (uint32_t)SEARCH_ROWS);
+                // every staged row fits: rows ns, ns + 1, ns + 3, ... in global memory, then a binary search in the bracket
+                auto continue_global = [&](uint32_t lo_, uint32_t Cx) -> uint32_t {
+                    const uint64_t base = pack64(sJob[6 * SEARCH_JOBS + jj], sJob[7 * SEARCH_JOBS + jj]);
+                    const uint32_t Dp = sJob[5 * SEARCH_JOBS + jj];
+                    uint32_t hi = n, step = 1;
+                    for (uint32_t idx = ns;;) {
+                        if (idx >= n) { hi = n; break; }
+                        const uint4 r = __ldg(jv.A + base + idx);
+                        bool ok = r.x - Dp <= T && r.y <= Cx;
+                        if (OPTS && ok && cap != 0xFFFFFFFFu) ok = __ldg(&jv.PW[base + idx].x) <= cap;
+                        if (ok) { lo_ = idx + 1; idx += step; step <<= 1; }
+                        else { hi = idx; break; }
+                    }
+                    while (lo_ < hi) {
+                        const uint32_t mid = lo_ + ((hi - lo_) >> 1);
+                        const uint4 r = __ldg(jv.A + base + mid);
+                        bool ok = r.x - Dp <= T && r.y <= Cx;
+                        if (OPTS && ok && cap != 0xFFFFFFFFu) ok = __ldg(&jv.PW[base + mid].x) <= cap;
+                        if (ok) lo_ = mid + 1; else hi = mid;
+                    }
+                    return lo_;
+                };
+                uint32_t cnt = lo[u] + (fits(jj, lo[u], T, C, ns) ? 1u : 0u);
+                cnt = elig[u] ? min(cnt, ns) : 0u;
+                if (cnt == ns && ns < n && elig[u]) cnt = continue_global(cnt, C);
+                if (cnt == 0u) continue;
+                uint32_t dur, peak;
                 uint64_t pay;
-                if (cnt <= min(ns, (uint32_t)SEARCH_PAY_ROWS)) {
-                    dur = sDM[(cnt - 1) * SEARCH_THREADS].x;
-                    const uint2 pw = sPay[(cnt - 1) * SEARCH_THREADS];
+                if (cnt <= ns) {
+                    const uint2 r = sDM[jj * SEARCH_ROWS + cnt - 1];
+                    const uint2 pw = sPay[jj * SEARCH_ROWS + cnt - 1];
+                    dur = r.x; peak = r.y;
                     pay = pack64(pw.x, pw.y);
                 } else {
+                    const uint64_t base = pack64(sJob[6 * SEARCH_JOBS + jj], sJob[7 * SEARCH_JOBS + jj]);
                     const uint4 r = __ldg(jv.A + base + cnt - 1);
-                    dur = r.x - Dp;
-                    pay = policy_payload(kind, r, Wp);
+                    dur = r.x - sJob[5 * SEARCH_JOBS + jj]; peak = r.y;
+                    pay = policy_payload(kind, r, pack64(sJob[8 * SEARCH_JOBS + jj], sJob[9 * SEARCH_JOBS + jj]));
                 }
-                if (dur >= jv.tau_min) key = policy_key(kind, pay, factor);
-                else cnt = 0;   // the longest fitting subjob is shorter than the minimum: decline
-            }
-            const uint64_t mk = warp_max_u64(key);
-            const uint32_t jmin = __reduce_min_sync(0xFFFFFFFFu, (key == mk && key != 0) ? j : 0xFFFFFFFFu);
-            const uint32_t src = __ffs(__ballot_sync(0xFFFFFFFFu, key == mk && j == jmin)) - 1;
-            const uint32_t wcnt = __shfl_sync(0xFFFFFFFFu, cnt, src & 31u);
-            if (lane == 0) {
-                Partial pr;
-                pr.key = mk; pr.job = jmin; pr.cnt = mk ? wcnt : 0u;
-                stage[gi][wid] = pr;
-            }
-        }
-        __syncthreads();
-        if (threadIdx.x < gt) {
-            Partial best = stage[threadIdx.x][0];
+                if (dur < jv.tau_min) continue;    // the longest fitting subjob is shorter than the minimum: decline
+                if constexpr (OPTS) {
+                    if (min_gain != 0u && cnt < n) {
+                        // hysteresis: how far would the window alone let the job run (capacity lifted)?  If further,
+                        // the capacity forces this cut, and it is taken only if it sheds at least min_gain MiB
+                        uint32_t lt = 0;
 #pragma unroll
-            for (int w = 1; w < SEARCH_THREADS / 32; ++w) {
-                const Partial c = stage[threadIdx.x][w];
-                if (c.key > best.key || (c.key == best.key && c.job < best.job)) best = c;
+                        for (uint32_t sp = SEARCH_ROWS / 2; sp > 0; sp >>= 1) lt += fits(jj, lt + sp - 1, T, 0xFFFFFFFFu, ns) ? sp : 0u;
+                        lt += fits(jj, lt, T, 0xFFFFFFFFu, ns) ? 1u : 0u;
+                        lt = min(lt, ns);
+                        if (lt == ns && ns < n) lt = continue_global(lt, 0xFFFFFFFFu);
+                        if (lt > cnt) {
+                            uint32_t peak_t;
+                            if (lt <= ns) peak_t = sDM[jj * SEARCH_ROWS + lt - 1].y;
+                            else peak_t = __ldg(jv.A + pack64(sJob[6 * SEARCH_JOBS + jj], sJob[7 * SEARCH_JOBS + jj]) + lt - 1).y;
+                            if (peak_t - peak < min_gain) continue;
+                        }
+                    }
+                }
+                const uint32_t factor = sJob[2 * SEARCH_JOBS + jj];
+                uint64_t key;
+                if (OPTS) {
+                    uint64_t pen = 0;
+                    const uint32_t home = sJob[4 * SEARCH_JOBS + jj];
+                    if (with_locality && home != 0xFFFFFFFFu && home != slice)
+                        pen = pack64(sJob[10 * SEARCH_JOBS + jj], sJob[11 * SEARCH_JOBS + jj]);
+                    key = policy_key_less(kind, pay, factor, pen);
+                } else {
+                    key = policy_key(kind, pay, factor);
+                }
+                // jobs come in ascending id: only a larger key replaces the best, so ties stay with the lowest id
+                if (key > best_key) { best_key = key; best_job = job0 + jj; best_cnt = cnt; }
             }
-            partial_out[(size_t)blockIdx.x * G + g0 + threadIdx.x] = best;
         }
-        __syncthreads();
+
+        Partial pr;
+        pr.key = best_key; pr.job = best_job; pr.cnt = best_cnt;
+        partial_out[(size_t)blockIdx.x * G + g] = pr;
     }
 }
 
@@ -311,7 +392,7 @@ __global__ void __launch_bounds__(256) commit_apply_kernel(
     uint32_t* __restrict__ p, uint32_t* __restrict__ ready, uint32_t* __restrict__ pb, uint32_t* __restrict__ Dp,
     uint64_t* __restrict__ Wp, uint32_t* __restrict__ winners, uint32_t* __restrict__ n_granted,
     uint32_t* __restrict__ flags, uint32_t* __restrict__ blocked, const uint8_t* __restrict__ accept,
-    uint32_t late_start) {
+    uint32_t late_start, uint32_t* __restrict__ last_slice) {
     const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= G) return;
     if (accept && !accept[g]) return;
@@ -333,6 +414,7 @@ __global__ void __launch_bounds__(256) commit_apply_kernel(
     Dp[j] = r.x;
     Wp[j] = pack64(r.z, r.w);
     if (blocked) blocked[j] = 1u;   // re-auction: one subjob per job and round
+    if (last_slice) last_slice[j] = gaps[g].slice;   // where the job's state lives from now on (Section 4.4, item 5)
     winners[atomicAdd(n_granted, 1u)] = j;
 }
 
