@@ -180,8 +180,8 @@ sja_status sja_select(sja_ctx* ctx, const sja_policy* policy, sja_award* out, sj
  * cudaFree or other allocating routine and records no profiling events.
  *
  * Cost and limit: every GPU on which the library is used holds the array until the process
- * exits.  The call needs ceil(J / 256) * G candidate slots of 16 bytes (one per gap and per
- * chunk of 256 jobs, the chunk of the per-pair search kernel, which runs or stands by in every
+ * exits.  The call needs ceil(J / 128) * G candidate slots of 16 bytes (one per gap and per
+ * chunk of 128 jobs, the chunk of the per-pair search kernel, which runs or stands by in every
  * select); if that exceeds the array it returns SJA_ERR_INVALID_ARG with the numbers in
  * sja_last_error() and does nothing.
  *

@@ -1206,6 +1206,8 @@ sja_status sja_load_power(sja_ctx* c, const uint64_t* off, const uint32_t* power
         return fail(c, SJA_ERR_INVALID_ARG, "sja_load_power: bad memspace");
     if (!c->loaded) return fail(c, SJA_ERR_STATE, "sja_load_power before sja_load_profiles");
     if (!off || (c->N > 0 && !power_W)) return fail(c, SJA_ERR_INVALID_ARG, "sja_load_power: off / power_W is NULL");
+    if (where == SJA_MEM_DEVICE && c->N > 0 && !aligned16(power_W))
+        return fail(c, SJA_ERR_INVALID_ARG, "sja_load_power: the device trace must be 16-byte aligned");
     DeviceGuard guard(c->device);
     if (!guard.ok) return cuda_fail(c, cudaErrorInvalidDevice, "cudaSetDevice");
     const uint64_t* d_off = off;
@@ -1223,9 +1225,12 @@ sja_status sja_load_power(sja_ctx* c, const uint64_t* off, const uint32_t* power
     TRY(reserve(c, c->PW, (size_t)c->n_rows * 8 + 16));
     c->have_power = false;
     c->selected = false;       // awards chosen without the trace must not be committed with it
-    scan_power_kernel<<<(uint32_t)(((uint64_t)c->J * 32 + 255) / 256), 256, 0, c->stream>>>(
-        d_off, d_pw, c->J, c->boff.as<uint64_t>(), c->pb.as<uint32_t>(), c->p.as<uint32_t>(), c->B.as<uint2>(),
-        c->PW.as<uint2>(), c->flags.as<uint32_t>());
+    {
+        ProfScope ps(c, CAT_PREP);
+        scan_power_kernel<<<(c->J + POWER_WARPS - 1) / POWER_WARPS, POWER_WARPS * 32, 0, c->stream>>>(
+            d_off, d_pw, c->J, c->boff.as<uint64_t>(), c->pb.as<uint32_t>(), c->p.as<uint32_t>(), c->B.as<uint2>(),
+            c->PW.as<uint2>(), c->flags.as<uint32_t>());
+    }
     CU(cudaGetLastError());
     uint32_t flags = 0;
     TRY(read_flags(c, &flags));

@@ -8,17 +8,31 @@
 
 namespace sja {
 
-// One warp per job: 32 rows at a time, each lane walks the steps of its row's segment, then a
-// warp max-scan with a carry turns segment maxima into running maxima.  Rows below the
-// progress point are left alone (nothing reads them).  A job whose length in `off` differs
-// from the loaded one raises FLAG_BAD_PROFILE.
-__global__ void __launch_bounds__(256) scan_power_kernel(
+constexpr int POWER_WARPS = 8;          // warps per CTA, one job each
+constexpr int POWER_BLK = 512;          // steps per warp iteration (16 per lane)
+constexpr int POWER_BUF_BYTES = POWER_BLK * 4 + 64;    // a block's trace values + one boundary bit per step
+constexpr int POWER_WARP_BYTES = 2 * POWER_BUF_BYTES;  // two blocks in flight per warp
+
+// One warp per job streams the job's part of the trace from its progress point on, 512 steps at a time:
+// coalesced 16-byte cp.async copies into one of the warp's two shared-memory blocks (the next block is under way
+// while the current one is worked on; chunks XOR-swizzled so that the lanes' 128-bit reads of their 16
+// CONSECUTIVE steps are conflict-free), boundary bits of the block from the end indices of the table rows that
+// end in it (the next 64 row ends are fetched one block ahead), then the same two-level scheme as the profile
+// scan: every lane reduces its 16 steps, the warp combines the lane results with shuffles (running maximum =
+// plain prefix maximum, segment maximum = prefix maximum that restarts at every boundary), and every lane walks
+// its steps again to emit {Pm, Ps} for the rows that end there.  Rows below the progress point are left alone
+// (nothing reads them).  A job whose length in `off` differs from the loaded one raises FLAG_BAD_PROFILE.
+__global__ void __launch_bounds__(POWER_WARPS * 32) scan_power_kernel(
     const uint64_t* __restrict__ off, const uint32_t* __restrict__ power, uint32_t J,
     const uint64_t* __restrict__ boff, const uint32_t* __restrict__ pb, const uint32_t* __restrict__ p,
     const uint2* __restrict__ B, uint2* __restrict__ PW, uint32_t* __restrict__ flags) {
-    const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    __shared__ __align__(16) unsigned char smem[POWER_WARPS * POWER_WARP_BYTES];
+    const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
+    const uint32_t j = blockIdx.x * POWER_WARPS + wid;
     if (j >= J) return;
+    unsigned char* wbase = smem + wid * POWER_WARP_BYTES;
+    const uint32_t wbase_s = (uint32_t)__cvta_generic_to_shared(wbase);
+    const uint64_t N_total = off[J];
     const uint64_t b1 = boff[j + 1], base = boff[j] + pb[j];
     const uint32_t R = (uint32_t)(b1 - base), pj = p[j];
     const uint64_t s0 = off[j], len = off[j + 1] - s0;
@@ -27,24 +41,149 @@ __global__ void __launch_bounds__(256) scan_power_kernel(
         if (lane == 0) atomicOr(flags, FLAG_BAD_PROFILE);
         return;
     }
-    uint32_t carry = 0;
-    for (uint32_t r0 = 0; r0 < R; r0 += 32) {
-        const uint32_t r = r0 + lane;
-        uint32_t seg = 0;
-        if (r < R) {
-            const uint32_t a = r ? B[base + r - 1].x : pj, b = B[base + r].x;
-            for (uint32_t i = a; i < b; ++i) seg = max(seg, __ldg(power + s0 + i));
+    if (R == 0) return;
+    const uint64_t first = s0 + pj, end = s0 + len;       // global steps [first, end) are scanned
+    const uint64_t bs0 = first & ~3ull;
+    const uint64_t nblk = (end - bs0 + POWER_BLK - 1) / POWER_BLK;
+    // block t into buffer t & 1: chunk c = steps bs + 4c .. bs + 4c + 3 at swizzled slot c ^ ((c >> 3) & 3);
+    // bytes beyond the end of the trace are filled with zeros
+    auto stage = [&](uint64_t t) {
+        if (t < nblk) {
+            const uint64_t bs = bs0 + t * POWER_BLK;
+            const uint32_t dst = wbase_s + (uint32_t)(t & 1ull) * POWER_BUF_BYTES;
+#pragma unroll
+            for (uint32_t r = 0; r < 4; ++r) {
+                const uint32_t c = r * 32u + lane;
+                const uint64_t g = bs + 4ull * c;
+                uint32_t bytes = 0;
+                if (g < N_total) bytes = (N_total - g) >= 4ull ? 16u : (uint32_t)(N_total - g) * 4u;
+                cp_async16(dst + (c ^ ((c >> 3) & 3u)) * 16u, power + (bytes ? g : 0ull), bytes);
+            }
         }
-        uint32_t run = seg;
+        cp_async_commit();
+    };
+    // end index of table row r of the job (0 beyond its last row: a real end index is at least 1)
+    auto row_end = [&](uint32_t r) -> uint32_t { return r < R ? B[base + r].x : 0u; };
+
+    uint32_t row = 0;               // rows emitted so far
+    uint32_t carry_run = 0;         // maximum over all steps scanned so far
+    uint32_t carry_seg = 0;         // maximum since the last boundary
+    stage(0);
+    uint32_t k0 = row_end(lane), k1 = row_end(32u + lane);    // ends of rows row + lane and row + 32 + lane
+    for (uint64_t t = 0; t < nblk; ++t) {
+        const uint64_t bs = bs0 + t * POWER_BLK;
+        unsigned char* buf = wbase + (size_t)(t & 1ull) * POWER_BUF_BYTES;
+        const uint4* sv = reinterpret_cast<const uint4*>(buf);
+        uint32_t* sbits = reinterpret_cast<uint32_t*>(buf + POWER_BLK * 4);
+        stage(t + 1);
+        if (lane < 16) sbits[lane] = 0u;
+        cp_async_wait<1>();
+        __syncwarp();
+        // ---- boundary bits: the rows (from `row` on) whose last step lies in this block; row ends ascend, so
+        // they are a prefix of the rows still to come
+        uint32_t in_block = 0;
+        {
+            const uint64_t lim = bs + POWER_BLK - s0;         // a row ends in the block iff its end index <= lim
+            auto mark = [&](uint32_t k) -> uint32_t {
+                const bool here = k != 0u && (uint64_t)k <= lim;
+                if (here) {
+                    const uint32_t o = (uint32_t)(s0 + k - 1ull - bs);
+                    atomicOr(&sbits[o >> 5], 1u << (o & 31u));
+                }
+                return (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, here));
+            };
+            uint32_t f = mark(k0);
+            in_block = f;
+            if (f == 32u) {
+                f = mark(k1);
+                in_block += f;
+                for (uint32_t r0 = row + 64u; f == 32u; r0 += 32u) {     // denser than 64 rows per block: fetch on the spot
+                    f = mark(row_end(r0 + lane));
+                    in_block += f;
+                }
+            }
+        }
+        // the row ends the next block will want
+        const uint32_t k0n = row_end(row + in_block + lane), k1n = row_end(row + in_block + 32u + lane);
+        __syncwarp();
+        // ---- the lane's 16 consecutive steps
+        uint32_t v[16];
+#pragma unroll
+        for (uint32_t r = 0; r < 4; ++r) {
+            const uint32_t c = 4u * lane + r;
+            const uint4 q = sv[c ^ ((c >> 3) & 3u)];
+            v[4 * r + 0] = q.x; v[4 * r + 1] = q.y; v[4 * r + 2] = q.z; v[4 * r + 3] = q.w;
+        }
+        uint32_t bits = (sbits[lane >> 1] >> ((lane & 1u) * 16u)) & 0xFFFFu;
+        const uint64_t lane_base = bs + 16ull * lane;
+        if (lane_base < first || lane_base + 16 > end) {
+            // steps outside [first, end) count as 0 and carry no boundary
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+                if (lane_base + i < first || lane_base + i >= end) { v[i] = 0u; bits &= ~(1u << i); }
+        }
+        // first walk: maximum of all 16 steps, maximum since the lane's last boundary
+        uint32_t lmax = 0, tail = 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            lmax = max(lmax, v[i]);
+            tail = max(tail, v[i]);
+            if ((bits >> i) & 1u) tail = 0;
+        }
+        // running maximum before this lane: exclusive prefix maximum of the lane maxima
+        uint32_t inc = lmax;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, run, o);
-            if (lane >= (uint32_t)o) run = max(run, y);
+            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= (uint32_t)o) inc = max(inc, y);
         }
-        run = max(run, carry);
-        if (r < R) PW[base + r] = make_uint2(run, seg);
-        carry = __shfl_sync(0xFFFFFFFFu, run, 31);
+        uint32_t run = __shfl_up_sync(0xFFFFFFFFu, inc, 1);
+        run = lane == 0 ? carry_run : max(run, carry_run);
+        // maximum since the last boundary before this lane: prefix maximum of the tails that restarts at
+        // every lane holding a boundary
+        const uint32_t hm = __ballot_sync(0xFFFFFFFFu, bits != 0u);
+        const uint32_t below = hm & (0xFFFFFFFFu >> (31u - lane));   // lanes 0..lane
+        const int head = below ? (31 - __clz((int)below)) : -1;
+        uint32_t x = tail;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o);
+            if ((int)lane - o >= head && (int)lane >= o) x = max(x, y);
+        }
+        uint32_t seg = __shfl_up_sync(0xFFFFFFFFu, x, 1);
+        const bool none_before = (hm & ((1u << lane) - 1u)) == 0u;   // no boundary in lanes < lane
+        if (lane == 0) seg = carry_seg;
+        else if (none_before) seg = max(seg, carry_seg);
+        // rows this lane emits start at: rows of earlier blocks + boundaries of lower lanes
+        const uint32_t cnt = __popc(bits);
+        uint32_t pos = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, pos, o);
+            if (lane >= (uint32_t)o) pos += y;
+        }
+        pos = row + pos - cnt;
+        // second walk: emit {running maximum, segment maximum} at every boundary
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            seg = max(seg, v[i]);
+            run = max(run, v[i]);
+            if ((bits >> i) & 1u) {
+                if (pos < R) PW[base + pos] = make_uint2(run, seg);
+                ++pos;
+                seg = 0;
+            }
+        }
+        // carries for the next block
+        carry_run = max(carry_run, __shfl_sync(0xFFFFFFFFu, inc, 31));
+        const uint32_t x31 = __shfl_sync(0xFFFFFFFFu, x, 31);
+        carry_seg = hm ? x31 : max(x31, carry_seg);
+        row += in_block;
+        k0 = k0n;
+        k1 = k1n;
+        __syncwarp();   // everybody is done with the block before the one after the next overwrites it
     }
+    cp_async_wait<0>();
 }
 
 }  // namespace sja

@@ -78,7 +78,7 @@ __device__ __forceinline__ uint32_t policy_factor(const JobView& jv, uint32_t ki
 // reduction across lanes, no staging of candidates, one coalesced candidate row per CTA at the end.
 constexpr int SEARCH_THREADS = 256;
 #ifndef SJA_SEARCH_JOBS
-#define SJA_SEARCH_JOBS 256
+#define SJA_SEARCH_JOBS 128
 #endif
 #ifndef SJA_SEARCH_ROWS
 #define SJA_SEARCH_ROWS 16

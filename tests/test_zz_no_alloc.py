@@ -70,7 +70,7 @@ def test_static_select_allocates_nothing(oracle_mod):
     (host output and device output), and the ordinary select of the same problem must then lower it."""
     import torch
     from paper_2509_19086_b200 import binding
-    spec = wl.scaled(wl.SPECS[2], n_jobs=30000, fixed_len=64, n_gaps=16384)   # 118 job chunks x 16384 gaps x 16 B = 30 MiB
+    spec = wl.scaled(wl.SPECS[2], n_jobs=15000, fixed_len=64, n_gaps=16384)   # 118 job chunks x 16384 gaps x 16 B = 30 MiB
     prof = wl.make_profiles(spec, threads=2)
     gaps = wl.make_gaps(spec)
     sample = slice(0, 512)                 # the oracle on the first gaps; the rest through the ordinary select below
@@ -100,8 +100,8 @@ def test_static_select_allocates_nothing(oracle_mod):
 def test_static_select_refuses_sizes_beyond_the_fixed_array():
     from paper_2509_19086_b200 import binding
     slots = (32 * 1024 * 1024) // 16
-    n_jobs, n_gaps = 256 * 18, 1                     # 18 job chunks of the search kernel that stands by
-    while ((n_jobs + 255) // 256) * n_gaps <= slots:
+    n_jobs, n_gaps = 128 * 36, 1                     # 36 job chunks of the search kernel that stands by
+    while ((n_jobs + 127) // 128) * n_gaps <= slots:
         n_gaps *= 2
     spec = wl.scaled(wl.SPECS[0], n_jobs=n_jobs, fixed_len=16, n_gaps=n_gaps)
     prof = wl.make_profiles(spec, threads=1)
