@@ -30,9 +30,12 @@
  * DEVICE pointer on the context's device, as said by the `where` argument of the call.
  * The caller owns every buffer it passes; the library copies what it needs before the
  * call's work completes on the context's stream and never keeps a caller pointer.
- * Device-memspace calls are ordered on the context's stream and return without waiting;
- * host-memspace outputs are complete when the call returns.  Device input arrays dur_ms,
- * mem_MiB and safe_bits must be 16-byte aligned.
+ * Calls with device-memspace arguments are ordered on the context's stream and return
+ * without waiting for the GPU, so that a round (sja_advertise, sja_select, sja_commit) can be
+ * queued without a host round trip; the exceptions say so in their own comment (the loads
+ * return validation results and therefore wait).  Calls with host-memspace arguments wait:
+ * host inputs may be reused and host outputs are complete when the call returns.  Device
+ * input arrays dur_ms, mem_MiB, safe_bits and power_W must be 16-byte aligned.
  *
  * No call aborts the process or traps the device.  Every call returns an sja_status;
  * sja_last_error() gives a text for the most recent failure on that context.
@@ -153,7 +156,9 @@ sja_status sja_load_profiles(sja_ctx* ctx, uint32_t J, const uint64_t* off,
 
 /*
  * First protocol phase (Section 3.5): make G gaps visible to all jobs.  Replaces the
- * previous batch.  Gaps are taken as given (overlaps on a slice are not checked).
+ * previous batch (also when the call fails after its argument checks: the context then has
+ * no batch).  Gaps are taken as given (overlaps on a slice are not checked).  A device batch
+ * is read when the stream gets there: keep it unchanged until then.
  */
 sja_status sja_advertise(sja_ctx* ctx, uint32_t G, const sja_gap* gaps, sja_memspace where);
 
