@@ -470,8 +470,8 @@ def bench_workload(env, args, spec, *, streaming, steps, warmup, e2e_steps, samp
             ctx.advertise_power_caps(dev_caps)
         if reauction:
             _, passes = ctx.round_reauction(my_spec.policy, flags=flags)
-            # per pass: select, finalize, the commit kernels, orphan compaction
-            launches[0] += adv_launches + (LAUNCHES_SELECT + LAUNCHES_COMMIT + 1) * passes
+            # per pass: select, finalize, one kernel for the commit and the compaction of the gap list
+            launches[0] += adv_launches + 3 * passes
         else:
             ctx.select(my_spec.policy, flags=flags)
             ctx.commit(want_count=False)

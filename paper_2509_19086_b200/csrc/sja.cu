@@ -84,6 +84,7 @@ struct sja_ctx {
     bool gaps_sorted = false;          // sgaps is ordered by (C, T); else it is the caller's order
     DevBuf gaps, sgaps, gap_info, gap_rank, awards, widx, partial, winners;
     DevBuf sgaps_alt, blocked, n_active, accept;   // re-auction: second ordered gap list, per-job block flags, gap counter
+    DevBuf dirty;                                  // re-auction: job chunks whose candidate rows have to be found again
 
     // profiling
     int prof = 0;                      // 0 off, 1 every phase, 2 the scan kernel only
@@ -360,12 +361,14 @@ sja_status check_policy(sja_ctx* c, const sja_policy* policy, const char* who) {
 struct KernelPlan { SelectKernel kernel; uint32_t jobs_per_cta, n_chunks, splits, per_split; };
 struct SelectPlan { KernelPlan primary, alt; bool have_alt; uint32_t max_classes; uint32_t rows; };
 
-KernelPlan plan_kernel(const sja_ctx* c, SelectKernel k, uint32_t G_act) {
+// `fixed`: the passes of a re-auction keep the candidate rows of untouched job chunks from pass to pass, so the
+// kernel and its chunk size must not change with the number of gaps left.
+KernelPlan plan_kernel(const sja_ctx* c, SelectKernel k, uint32_t G_act, bool fixed) {
     KernelPlan p;
     p.kernel = k;
     // the search kernel gives every gap a thread: with few gaps it takes small job chunks, so that many CTAs share the jobs
     p.jobs_per_cta = k == SEL_TILE ? (uint32_t)TILE_JOBS : k == SEL_MERGE ? (uint32_t)MERGE_JOBS
-                     : G_act <= 64u ? 32u : (uint32_t)SEARCH_JOBS;
+                     : (G_act <= 64u && !fixed) ? 32u : (uint32_t)SEARCH_JOBS;
     p.n_chunks = (c->J + p.jobs_per_cta - 1) / p.jobs_per_cta;
     // granularity of a gap split: a staging tile; the tile kernel also works in 32-gap steps, which a
     // small problem needs to put enough CTAs on the GPU
@@ -384,22 +387,26 @@ KernelPlan plan_kernel(const sja_ctx* c, SelectKernel k, uint32_t G_act) {
     return p;
 }
 
-SelectPlan plan_select(const sja_ctx* c, uint32_t pflags, uint32_t G_act) {
+// `classes_known` (>= 0): the class count of the batch as read by the host; the choice is then made here and no
+// stand-by launch is needed.
+SelectPlan plan_select(const sja_ctx* c, uint32_t pflags, uint32_t G_act, bool fixed = false, int64_t classes_known = -1) {
     SelectPlan p;
     const bool forced = (pflags & (SJA_FLAG_FORCE_MERGE | SJA_FLAG_FORCE_TILE)) != 0;
     // A round of a few thousand pairs cannot fill the GPU either way; there the cursors' sequential walk
     // through each capacity class is pure latency and the independent per-pair searches finish sooner.
     // (a later pass of a re-auction with a handful of gaps left is such a round too, whatever J is: below
     // 2^21 pairs the fixed start-up of the ordered-gap kernels outweighs what they save)
-    const bool tiny = (uint64_t)c->J * c->G < (1ull << 16) || (G_act < c->G && (uint64_t)c->J * G_act < (1ull << 21));
+    const bool tiny = (uint64_t)c->J * c->G < (1ull << 16) ||
+                      (!fixed && G_act < c->G && (uint64_t)c->J * G_act < (1ull << 21));
     // with a window option the usable window differs from pair to pair: only the search kernel does that
     const bool per_pair_window = c->late_start || c->have_deadline || (c->have_power && c->have_caps) ||
                                  c->min_gain != 0u || c->have_locality;
-    const bool search_only = (pflags & SJA_FLAG_FORCE_SEARCH) || per_pair_window || !c->gaps_sorted || (!forced && tiny);
     p.max_classes = std::max<uint32_t>(64u, c->G / 16u);
-    p.have_alt = !search_only;
-    p.primary = plan_kernel(c, search_only ? SEL_SEARCH : (pflags & SJA_FLAG_FORCE_MERGE) ? SEL_MERGE : SEL_TILE, G_act);
-    p.alt = plan_kernel(c, SEL_SEARCH, G_act);
+    const bool search_only = (pflags & SJA_FLAG_FORCE_SEARCH) || per_pair_window || !c->gaps_sorted || (!forced && tiny) ||
+                             (classes_known >= 0 && classes_known > (int64_t)p.max_classes);
+    p.have_alt = !search_only && classes_known < 0;
+    p.primary = plan_kernel(c, search_only ? SEL_SEARCH : (pflags & SJA_FLAG_FORCE_MERGE) ? SEL_MERGE : SEL_TILE, G_act, fixed);
+    p.alt = plan_kernel(c, SEL_SEARCH, G_act, fixed);
     p.rows = p.have_alt ? std::max(p.primary.n_chunks, p.alt.n_chunks) : p.primary.n_chunks;
     return p;
 }
@@ -407,13 +414,18 @@ SelectPlan plan_select(const sja_ctx* c, uint32_t pflags, uint32_t G_act) {
 // `scratch`: candidate rows (plan rows x G entries); nullptr = the context's own buffer, grown on demand.
 // `timed`: record profiling events (creates CUDA events on first use).
 // `G_dev`: optional device word with the number of gaps actually left (<= G_act, which then only sizes the launch).
+// `dirty` (re-auction only): flags of the 128-job blocks whose chunks have to be evaluated again; the candidate
+// rows then have the whole batch as their length, are addressed by original gap index, and `classes_known` is the
+// batch's class count as read by the host.
 sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sgaps, uint32_t G_act,
                       const uint32_t* blocked, Partial* scratch = nullptr, bool timed = true,
-                      const uint32_t* G_dev = nullptr) {
-    const SelectPlan pl = plan_select(c, pflags, G_act);
+                      const uint32_t* G_dev = nullptr, const uint32_t* dirty = nullptr, int64_t classes_known = -1) {
+    const bool reauction = dirty != nullptr;
+    const SelectPlan pl = plan_select(c, pflags, G_act, reauction, classes_known);
     Partial* partial = scratch;
     if (!partial) {
-        TRY(reserve(c, c->partial, (size_t)pl.rows * G_act * sizeof(Partial)));
+        // (a re-auction sizes the rows for the whole batch before its first pass: nothing grows between passes)
+        TRY(reserve(c, c->partial, (size_t)pl.rows * (reauction ? c->G : G_act) * sizeof(Partial)));
         partial = c->partial.as<Partial>();
     }
     const int was_on = c->prof;
@@ -427,6 +439,9 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
         gate.n_classes = pl.have_alt ? &c->gap_info.as<GapInfo>()->n_classes : nullptr;
         gate.max_classes = pl.max_classes;
         gate.run_if_many = 0u;
+        gate.dirty = dirty;
+        gate.row_len = reauction ? c->G : 0u;
+        gate.stable = reauction ? 1u : 0u;
         auto launch_search = [&](const KernelPlan& kp, const LaunchGate& g) {
             const bool opts = jv.late_start != 0u || jv.deadline != nullptr || jv.PW != nullptr || jv.min_gain != 0u ||
                               jv.ckpt != nullptr;
@@ -457,23 +472,30 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
     return SJA_OK;
 }
 
+CommitArgs commit_args(sja_ctx* c, uint32_t* blocked, const uint8_t* accept, uint32_t* dirty_next) {
+    CommitArgs a;
+    a.awards = c->awards.as<Award>(); a.gaps = c->gaps.as<Gap>(); a.widx = c->widx.as<uint32_t>();
+    a.jobwin = c->jobwin.as<unsigned long long>(); a.boff = c->boff.as<uint64_t>();
+    a.A = c->A.as<uint4>(); a.B = c->B.as<uint2>();
+    a.p = c->p.as<uint32_t>(); a.ready = c->ready.as<uint32_t>(); a.pb = c->pb.as<uint32_t>(); a.Dp = c->Dp.as<uint32_t>();
+    a.Wp = c->Wp.as<uint64_t>(); a.winners = c->winners.as<uint32_t>(); a.n_granted = c->n_granted.as<uint32_t>();
+    a.flags = c->flags.as<uint32_t>(); a.blocked = blocked; a.accept = accept; a.late_start = c->late_start ? 1u : 0u;
+    a.last_slice = c->have_locality ? c->last_slice.as<uint32_t>() : nullptr;
+    a.dirty_next = dirty_next;
+    a.PW = c->have_power ? c->PW.as<uint2>() : nullptr;
+    return a;
+}
+
 // Launch the three commit kernels over all G awards.  `blocked` may be nullptr.
-void run_commit(sja_ctx* c, uint32_t* blocked, const uint8_t* accept = nullptr) {
+void run_commit(sja_ctx* c, uint32_t* blocked, const uint8_t* accept = nullptr, uint32_t* dirty_next = nullptr) {
     const uint32_t G = c->G;
     ProfScope ps(c, CAT_COMMIT);
     const uint32_t gb = (G + 255) / 256;
-    commit_vote_kernel<<<gb, 256, 0, c->stream>>>(c->awards.as<Award>(), G, c->jobwin.as<unsigned long long>(),
-                                                  c->n_granted.as<uint32_t>(), accept);
-    commit_apply_kernel<<<gb, 256, 0, c->stream>>>(
-        c->awards.as<Award>(), c->gaps.as<Gap>(), c->widx.as<uint32_t>(), G, c->jobwin.as<unsigned long long>(),
-        c->boff.as<uint64_t>(), c->A.as<uint4>(), c->p.as<uint32_t>(), c->ready.as<uint32_t>(), c->pb.as<uint32_t>(),
-        c->Dp.as<uint32_t>(), c->Wp.as<uint64_t>(), c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(),
-        c->flags.as<uint32_t>(), blocked, accept, c->late_start ? 1u : 0u,
-        c->have_locality ? c->last_slice.as<uint32_t>() : nullptr);
+    const CommitArgs a = commit_args(c, blocked, accept, dirty_next);
+    commit_vote_kernel<<<gb, 256, 0, c->stream>>>(a.awards, G, a.jobwin, a.n_granted, accept);
+    commit_apply_kernel<<<gb, 256, 0, c->stream>>>(a, G);
     commit_refresh_kernel<<<(uint32_t)(((uint64_t)G * 32 + 255) / 256), 256, 0, c->stream>>>(
-        c->winners.as<uint32_t>(), c->n_granted.as<uint32_t>(), G, c->boff.as<uint64_t>(), c->pb.as<uint32_t>(),
-        c->A.as<uint4>(), c->B.as<uint2>(), c->jobwin.as<unsigned long long>(),
-        c->have_power ? c->PW.as<uint2>() : nullptr);
+        a.winners, a.n_granted, G, a.boff, a.pb, a.A, a.B, a.jobwin, a.PW);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -564,7 +586,7 @@ sja_status sja_destroy(sja_ctx* c) {
     cudaStreamSynchronize(c->stream);
     DevBuf* bufs[] = {&c->st_off, &c->st_d, &c->st_m, &c->st_s, &c->st_p, &c->st_ready, &c->st_wait, &c->st_prio, &c->p, &c->ready, &c->pb, &c->Dp,
                       &c->Wp, &c->wait, &c->prio, &c->nbj, &c->cta_tot, &c->cta_base, &c->boff, &c->boff_next, &c->A, &c->B, &c->jobwin,
-                      &c->flags, &c->counter, &c->n_granted, &c->long_list, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->blocked, &c->n_active, &c->accept, &c->deadline, &c->ckpt, &c->last_slice, &c->PW, &c->caps, &c->st_power, &c->st_bids, &c->st_accept, &c->st_global, &c->upd_d, &c->upd_m, &c->upd_scratch, &c->upd_status, &c->awards, &c->widx, &c->partial,
+                      &c->flags, &c->counter, &c->n_granted, &c->long_list, &c->gaps, &c->sgaps, &c->gap_info, &c->gap_rank, &c->sgaps_alt, &c->dirty, &c->blocked, &c->n_active, &c->accept, &c->deadline, &c->ckpt, &c->last_slice, &c->PW, &c->caps, &c->st_power, &c->st_bids, &c->st_accept, &c->st_global, &c->upd_d, &c->upd_m, &c->upd_scratch, &c->upd_status, &c->awards, &c->widx, &c->partial,
                       &c->winners};
     for (DevBuf* b : bufs) release(*b);
     for (ProfSpan& s : c->spans) { cudaEventDestroy(s.a); cudaEventDestroy(s.b); }
@@ -988,6 +1010,23 @@ sja_status sja_round_reauction(sja_ctx* c, const sja_policy* policy, uint32_t ma
     TRY(reserve(c, c->sgaps_alt, (size_t)G * sizeof(sja_gap)));
     TRY(reserve(c, c->blocked, (size_t)J * 4));
     CU(cudaMemsetAsync(c->blocked.p, 0, (size_t)J * 4, c->stream));
+    // Candidate rows are kept from pass to pass: within a round nothing about a job changes except that granted
+    // jobs drop out, so the best candidate of a job chunk for a gap stays the best until one of the chunk's jobs is
+    // granted.  Two arrays of flags per block of 128 jobs: the select of a pass evaluates the chunks marked in one,
+    // the commit marks the chunks of the jobs it grants in the other, for the next pass.  All marked to begin with.
+    const uint32_t n_dirty = ((J + 127u) >> 7) + 8u;
+    TRY(reserve(c, c->dirty, (size_t)2 * n_dirty * 4));
+    uint32_t* dirty_cur = c->dirty.as<uint32_t>();
+    uint32_t* dirty_next = dirty_cur + n_dirty;
+    CU(cudaMemsetAsync(dirty_cur, 0xFF, (size_t)n_dirty * 4, c->stream));
+    CU(cudaMemsetAsync(dirty_next, 0, (size_t)n_dirty * 4, c->stream));
+    // the class count of the batch decides the kernel for every pass: read it once (the call waits for the GPU anyway)
+    int64_t classes_known = 0;
+    if (c->gaps_sorted) {
+        CU(cudaMemcpyAsync(c->h_words + 64, c->gap_info.p, 4, cudaMemcpyDeviceToHost, c->stream));
+        CU(cudaStreamSynchronize(c->stream));
+        classes_known = c->h_words[64];
+    }
 
     // Passes are queued in batches without a host wait in between: the number of gaps a pass starts with lives
     // in device memory (the report of the pass before it), launches are sized for the count at the last wait
@@ -1006,12 +1045,17 @@ sja_status sja_round_reauction(sja_ctx* c, const sja_policy* policy, uint32_t ma
         if (max_passes != 0) batch = std::min(batch, max_passes - passes);
         for (uint32_t k = 0; k < batch; ++k) {
             const uint32_t* g_dev = k ? reports + 4 * (k - 1) : nullptr;   // gaps left after the pass before
-            TRY(run_select(c, kind, policy->flags, cur, g_act, c->blocked.as<uint32_t>(), nullptr, true, g_dev));
-            run_commit(c, c->blocked.as<uint32_t>());
-            collect_orphans_kernel<<<1, 1024, 0, c->stream>>>(cur, g_act, c->awards.as<Award>(), spare,
-                                                              c->n_granted.as<uint32_t>(), c->flags.as<uint32_t>(),
-                                                              reports + 4 * k, g_dev);
+            TRY(run_select(c, kind, policy->flags, cur, g_act, c->blocked.as<uint32_t>(), nullptr, true, g_dev, dirty_cur,
+                           classes_known));
+            {
+                // commit of the pass and compaction of its gap list: one launch of one CTA
+                ProfScope ps(c, CAT_COMMIT);
+                reauction_resolve_kernel<<<1, 1024, 0, c->stream>>>(
+                    commit_args(c, c->blocked.as<uint32_t>(), nullptr, dirty_next), cur, g_act, spare, reports + 4 * k,
+                    g_dev, dirty_cur, n_dirty);
+            }
             CU(cudaGetLastError());
+            std::swap(dirty_cur, dirty_next);
             cur = spare;
             spare = (spare == c->sgaps_alt.as<Gap>()) ? own : c->sgaps_alt.as<Gap>();
         }

@@ -43,7 +43,15 @@ struct LaunchGate {
     const uint32_t* n_classes;   // may be nullptr: this launch runs whatever the class count
     uint32_t max_classes;
     uint32_t run_if_many;        // 0: run when n_classes <= max_classes, 1: run when it is larger
+    // Re-auction (several passes over a shrinking gap list inside one round): the candidate row of a job chunk
+    // stays valid from pass to pass unless one of its jobs was granted, so only the chunks marked dirty are
+    // evaluated again.  For that the rows are addressed by the gaps' original indices (stable while the list
+    // is compacted) and have the full batch as their length.
+    const uint32_t* dirty;       // may be nullptr (every chunk runs); else one word per block of 128 jobs
+    uint32_t row_len;            // length of a candidate row; 0 = the G the launch was sized for
+    uint32_t stable;             // non-zero: slot of a gap in a row = its original index, else its list position
 };
+constexpr uint32_t DIRTY_SHIFT = 7;   // jobs per dirty-flag block = 128 (every select kernel's chunk is a multiple)
 
 // Number of gaps this launch serves: 0 when the class count calls for the other kernel.
 __device__ __forceinline__ uint32_t gate_gaps(const LaunchGate& g, uint32_t G) {
@@ -52,6 +60,20 @@ __device__ __forceinline__ uint32_t gate_gaps(const LaunchGate& g, uint32_t G) {
         if (many != (g.run_if_many != 0u)) return 0u;
     }
     return g.gaps_left ? min(G, *g.gaps_left) : G;
+}
+
+// Does the chunk of `n` jobs from job `first` have to be evaluated in this launch?
+__device__ __forceinline__ bool chunk_dirty(const LaunchGate& g, uint32_t first, uint32_t n) {
+    if (!g.dirty) return true;
+    bool any = false;
+    for (uint32_t b = first >> DIRTY_SHIFT; b <= (first + n - 1u) >> DIRTY_SHIFT; ++b) any = any || g.dirty[b] != 0u;
+    return any;
+}
+
+// Slot of (job chunk, gap) in the candidate rows: `pos` is the gap's position in the list of this launch, `orig`
+// its original index.
+__device__ __forceinline__ size_t row_slot(const LaunchGate& g, uint32_t G, uint32_t chunk, uint32_t pos, uint32_t orig) {
+    return (size_t)chunk * (g.row_len ? g.row_len : G) + (g.stable ? orig : pos);
 }
 
 __device__ __forceinline__ uint32_t policy_factor(const JobView& jv, uint32_t kind, uint32_t j) {
@@ -110,8 +132,9 @@ template <bool OPTS>
 __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
     JobView jv, const Gap* __restrict__ gaps, uint32_t G, uint32_t gaps_per_split, uint32_t kind,
     Partial* __restrict__ partial_out, LaunchGate gate, uint32_t jobs_per_cta) {
-    const uint32_t G_now = gate_gaps(gate, G);   // gaps actually left (G stays the row length of partial_out)
+    const uint32_t G_now = gate_gaps(gate, G);   // gaps actually left
     if (blockIdx.y * gaps_per_split >= G_now) return;
+    if (!chunk_dirty(gate, blockIdx.x * jobs_per_cta, jobs_per_cta)) return;   // its candidate row still stands
     extern __shared__ __align__(16) unsigned char search_smem[];
     uint2* sDM = reinterpret_cast<uint2*>(search_smem);                                   // [job][row] {D - Dp, M}
     uint2* sPay = sDM + SEARCH_JOBS * SEARCH_ROWS;                                        // [job][row] policy payload
@@ -314,7 +337,7 @@ __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
 
         Partial pr;
         pr.key = best_key; pr.job = best_job; pr.cnt = best_cnt;
-        partial_out[(size_t)blockIdx.x * G + g] = pr;
+        partial_out[row_slot(gate, G, blockIdx.x, g, gq.x)] = pr;
     }
 }
 
@@ -337,8 +360,10 @@ __global__ void __launch_bounds__(FINALIZE_WARPS * 32) finalize_awards_kernel(
     Partial best;
     best.key = 0; best.job = 0xFFFFFFFFu; best.cnt = 0;
     if (g < G_now) {
+        const uint32_t slot = gate.stable ? sgaps[g].slice : g;
+        const size_t row_len = gate.row_len ? gate.row_len : G;
         for (uint32_t r = wid; r < n_rows; r += FINALIZE_WARPS) {
-            const Partial c = partial[(size_t)r * G + g];
+            const Partial c = partial[(size_t)r * row_len + slot];
             if (c.key > best.key || (c.key == best.key && c.job < best.job)) best = c;
         }
     }
@@ -371,13 +396,9 @@ __global__ void __launch_bounds__(FINALIZE_WARPS * 32) finalize_awards_kernel(
 // ---------------------------------------------------------------------------------------
 // Commit, step 1: every winning job records the gap it accepts: largest end_step, then
 // lowest gap id (one atomicMax on a packed key; the order of the atomics does not matter).
-__global__ void __launch_bounds__(256) commit_vote_kernel(const Award* __restrict__ awards, uint32_t G,
-                                                          unsigned long long* __restrict__ jobwin,
-                                                          uint32_t* __restrict__ n_granted,
-                                                          const uint8_t* __restrict__ accept) {
-    const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
-    if (g == 0) *n_granted = 0;
-    if (g >= G) return;
+__device__ __forceinline__ void commit_vote_one(const Award* __restrict__ awards, uint32_t g,
+                                                unsigned long long* __restrict__ jobwin,
+                                                const uint8_t* __restrict__ accept) {
     if (accept && !accept[g]) return;   // grant not taken up (failed subjob): no part in the commit
     const uint32_t j = awards[g].job;
     if (j == 0xFFFFFFFFu || awards[g].granted) return;   // granted: settled in an earlier pass of this round
@@ -385,50 +406,64 @@ __global__ void __launch_bounds__(256) commit_vote_kernel(const Award* __restric
     atomicMax(jobwin + j, key);
 }
 
-// Commit, step 2: the accepted gap of each job is granted and the job's state advances.
-__global__ void __launch_bounds__(256) commit_apply_kernel(
-    Award* __restrict__ awards, const Gap* __restrict__ gaps, const uint32_t* __restrict__ widx, uint32_t G,
-    const unsigned long long* __restrict__ jobwin, const uint64_t* __restrict__ boff, const uint4* __restrict__ A,
-    uint32_t* __restrict__ p, uint32_t* __restrict__ ready, uint32_t* __restrict__ pb, uint32_t* __restrict__ Dp,
-    uint64_t* __restrict__ Wp, uint32_t* __restrict__ winners, uint32_t* __restrict__ n_granted,
-    uint32_t* __restrict__ flags, uint32_t* __restrict__ blocked, const uint8_t* __restrict__ accept,
-    uint32_t late_start, uint32_t* __restrict__ last_slice) {
+__global__ void __launch_bounds__(256) commit_vote_kernel(const Award* __restrict__ awards, uint32_t G,
+                                                          unsigned long long* __restrict__ jobwin,
+                                                          uint32_t* __restrict__ n_granted,
+                                                          const uint8_t* __restrict__ accept) {
     const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
+    if (g == 0) *n_granted = 0;
     if (g >= G) return;
-    if (accept && !accept[g]) return;
-    Award a = awards[g];
+    commit_vote_one(awards, g, jobwin, accept);
+}
+
+// What the apply step works on (one struct, so that the stand-alone kernel and the re-auction's one-CTA kernel
+// share the code).
+struct CommitArgs {
+    Award* awards; const Gap* gaps; const uint32_t* widx; unsigned long long* jobwin; const uint64_t* boff;
+    uint4* A; const uint2* B; uint32_t *p, *ready, *pb, *Dp; uint64_t* Wp; uint32_t *winners, *n_granted, *flags;
+    uint32_t* blocked; const uint8_t* accept; uint32_t late_start; uint32_t* last_slice; uint32_t* dirty_next;
+    uint2* PW;
+};
+
+// Commit, step 2: the accepted gap of each job is granted and the job's state advances.
+__device__ __forceinline__ void commit_apply_one(const CommitArgs& c, uint32_t g) {
+    if (c.accept && !c.accept[g]) return;
+    Award a = c.awards[g];
     if (a.job == 0xFFFFFFFFu || a.granted) return;   // granted: settled in an earlier pass of this round
     const unsigned long long key = ((unsigned long long)a.end_step << 32) | (0xFFFFFFFFu - g);
-    if (jobwin[a.job] != key) { awards[g].granted = 0; return; }
+    if (c.jobwin[a.job] != key) { c.awards[g].granted = 0; return; }
     const uint32_t j = a.job;
-    const uint32_t row_rel = pb[j] + widx[g] - 1;
-    const uint4 r = A[boff[j] + row_rel];
+    const uint32_t row_rel = c.pb[j] + c.widx[g] - 1;
+    const uint4 r = c.A[c.boff[j] + row_rel];
     // the subjob began when the gap opened, or when the job turned ready inside it (late start)
-    const uint32_t begin = late_start ? max(gaps[g].start, ready[j]) : gaps[g].start;
+    const uint32_t begin = c.late_start ? max(c.gaps[g].start, c.ready[j]) : c.gaps[g].start;
     const uint64_t new_ready = (uint64_t)begin + (uint64_t)a.dur;
-    if (new_ready > 0xFFFFFFFFull) atomicOr(flags, FLAG_OVF_READY);
-    awards[g].granted = 1;
-    p[j] = a.end_step;
-    ready[j] = new_ready > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)new_ready;
-    pb[j] = row_rel + 1;
-    Dp[j] = r.x;
-    Wp[j] = pack64(r.z, r.w);
-    if (blocked) blocked[j] = 1u;   // re-auction: one subjob per job and round
-    if (last_slice) last_slice[j] = gaps[g].slice;   // where the job's state lives from now on (Section 4.4, item 5)
-    winners[atomicAdd(n_granted, 1u)] = j;
+    if (new_ready > 0xFFFFFFFFull) atomicOr(c.flags, FLAG_OVF_READY);
+    c.awards[g].granted = 1;
+    c.p[j] = a.end_step;
+    c.ready[j] = new_ready > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)new_ready;
+    c.pb[j] = row_rel + 1;
+    c.Dp[j] = r.x;
+    c.Wp[j] = pack64(r.z, r.w);
+    if (c.blocked) c.blocked[j] = 1u;   // re-auction: one subjob per job and round
+    if (c.dirty_next) c.dirty_next[j >> DIRTY_SHIFT] = 1u;   // ... and its chunk's candidates have to be found again
+    if (c.last_slice) c.last_slice[j] = c.gaps[g].slice;   // where the job's state lives from now on (Section 4.4, item 5)
+    c.winners[atomicAdd(c.n_granted, 1u)] = j;
+}
+
+__global__ void __launch_bounds__(256) commit_apply_kernel(CommitArgs c, uint32_t G) {
+    const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= G) return;
+    commit_apply_one(c, g);
 }
 
 // Commit, step 3: one warp per granted job rebuilds the running-maximum column from the
 // new progress point (the maximum of a window is not derivable from the previous column),
 // stopping as soon as the new and the old column agree, and clears the job's vote.
-__global__ void __launch_bounds__(256) commit_refresh_kernel(
-    const uint32_t* __restrict__ winners, const uint32_t* __restrict__ n_granted, uint32_t G,
-    const uint64_t* __restrict__ boff, const uint32_t* __restrict__ pb, uint4* __restrict__ A,
-    const uint2* __restrict__ B, unsigned long long* __restrict__ jobwin, uint2* __restrict__ PW) {
-    const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (w >= G || w >= *n_granted) return;
-    const uint32_t j = winners[w];
+__device__ __forceinline__ void commit_refresh_one(uint32_t j, uint32_t lane, const uint64_t* __restrict__ boff,
+                                                   const uint32_t* __restrict__ pb, uint4* __restrict__ A,
+                                                   const uint2* __restrict__ B, unsigned long long* __restrict__ jobwin,
+                                                   uint2* __restrict__ PW) {
     if (lane == 0) jobwin[j] = 0ull;
     const uint64_t base = boff[j] + pb[j];
     const uint32_t n = (uint32_t)(boff[j + 1] - base);
@@ -473,6 +508,16 @@ __global__ void __launch_bounds__(256) commit_refresh_kernel(
         if (v_last == old_last) break;
         carry = v_last;
     }
+}
+
+__global__ void __launch_bounds__(256) commit_refresh_kernel(
+    const uint32_t* __restrict__ winners, const uint32_t* __restrict__ n_granted, uint32_t G,
+    const uint64_t* __restrict__ boff, const uint32_t* __restrict__ pb, uint4* __restrict__ A,
+    const uint2* __restrict__ B, unsigned long long* __restrict__ jobwin, uint2* __restrict__ PW) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (w >= G || w >= *n_granted) return;
+    commit_refresh_one(winners[w], lane, boff, pb, A, B, jobwin, PW);
 }
 
 }  // namespace sja
@@ -631,22 +676,34 @@ __global__ void __launch_bounds__(256) copy_gaps_kernel(const Gap* __restrict__ 
 }
 
 // ---------------------------------------------------------------------------------------
-// Re-auction: keep, in their advertised order, the gaps that had a winner but were not
-// granted (their winner accepted another gap).  One CTA walks the ordered list in tiles of
-// 1024 with a block-wide exclusive count.  report[0] receives the number of gaps kept, report[1] the grants
-// of the pass, report[2] the status flag word and report[3] the number of gaps the pass started with, so that
-// the host reads one 16-byte record per pass.  G_dev (optional): that number lives in device memory.
-__global__ void __launch_bounds__(1024) collect_orphans_kernel(const Gap* __restrict__ sgaps_in, uint32_t G_in,
-                                                               const Award* __restrict__ awards,
-                                                               Gap* __restrict__ sgaps_out,
-                                                               const uint32_t* __restrict__ n_granted,
-                                                               const uint32_t* __restrict__ flags,
-                                                               uint32_t* __restrict__ report,
-                                                               const uint32_t* __restrict__ G_dev) {
+// The commit of a re-auction pass and the compaction of its gap list in ONE launch of one CTA: votes of the
+// gaps still in the list, barrier, grants, barrier, running-maximum refresh of the granted jobs (a warp each),
+// then the compaction: the gaps that had a winner but were not granted (their winner accepted another gap) are kept,
+// in their advertised order, for the next pass (a block-wide exclusive count per tile of 1024; report[0] receives the
+// number of gaps kept, report[1] the grants of the pass, report[2] the status flag word and report[3] the number of
+// gaps the pass started with, so that the host reads one 16-byte record per pass; G_dev (optional): that number
+// lives in device memory).  A pass of a re-auction has at most a few thousand gaps and grants a
+// handful of jobs, so four launches that are each bound by their start-up cost become one; every phase only reads
+// what earlier phases of this same CTA wrote, so nothing waits on another CTA.
+__global__ void __launch_bounds__(1024) reauction_resolve_kernel(CommitArgs c, const Gap* __restrict__ sgaps_in,
+                                                                 uint32_t G_in, Gap* __restrict__ sgaps_out,
+                                                                 uint32_t* __restrict__ report,
+                                                                 const uint32_t* __restrict__ G_dev,
+                                                                 uint32_t* __restrict__ dirty_done, uint32_t n_dirty) {
     if (G_dev) G_in = min(G_in, *G_dev);
     __shared__ uint32_t warp_cnt[32];
     __shared__ uint32_t tile_total;
     const uint32_t t = threadIdx.x, lane = t & 31u, wid = t >> 5;
+    for (uint32_t i = t; i < n_dirty; i += blockDim.x) dirty_done[i] = 0u;   // flags this pass's select has consumed
+    if (t == 0) *c.n_granted = 0;
+    // (awards are stored at the gaps' original indices, which ride in the slice field of the ordered list)
+    for (uint32_t i = t; i < G_in; i += blockDim.x) commit_vote_one(c.awards, sgaps_in[i].slice, c.jobwin, nullptr);
+    __syncthreads();
+    for (uint32_t i = t; i < G_in; i += blockDim.x) commit_apply_one(c, sgaps_in[i].slice);
+    __syncthreads();
+    const uint32_t n_won = *c.n_granted;
+    for (uint32_t w = wid; w < n_won; w += blockDim.x / 32) commit_refresh_one(c.winners[w], lane, c.boff, c.pb, c.A, c.B, c.jobwin, c.PW);
+    // keep, in order, the gaps that had a winner but were not granted
     uint32_t carry = 0;
     for (uint32_t base = 0; base < G_in; base += 1024) {
         const uint32_t i = base + t;
@@ -654,7 +711,7 @@ __global__ void __launch_bounds__(1024) collect_orphans_kernel(const Gap* __rest
         bool keep = false;
         if (i < G_in) {
             g = sgaps_in[i];
-            const Award a = awards[g.slice];
+            const Award a = c.awards[g.slice];
             keep = a.job != 0xFFFFFFFFu && a.granted == 0u;
         }
         const uint32_t ball = __ballot_sync(0xFFFFFFFFu, keep);
@@ -677,7 +734,7 @@ __global__ void __launch_bounds__(1024) collect_orphans_kernel(const Gap* __rest
         carry += tile_total;
         __syncthreads();
     }
-    if (t == 0) { report[0] = carry; report[1] = G_in ? *n_granted : 0u; report[2] = *flags; report[3] = G_in; }
+    if (t == 0) { report[0] = carry; report[1] = G_in ? n_won : 0u; report[2] = *c.flags; report[3] = G_in; }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -752,6 +809,7 @@ __global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_me
     LaunchGate gate) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     if (gate_gaps(gate, G) == 0u) return;      // the class count calls for the per-pair search
+    if (!chunk_dirty(gate, blockIdx.x * MERGE_JOBS, MERGE_JOBS)) return;
     Partial* stage = reinterpret_cast<Partial*>(smem_raw + MERGE_RING_BYTES);            // [GT][WARPS]
     uint4* sg = reinterpret_cast<uint4*>(smem_raw + MERGE_RING_BYTES + MERGE_GT * MERGE_WARPS * 16);
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
@@ -901,7 +959,7 @@ __global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_me
                 const Partial c = stage[threadIdx.x * MERGE_WARPS + ww];
                 if (c.key > bestp.key || (c.key == bestp.key && c.job < bestp.job)) bestp = c;
             }
-            partial_out[(size_t)blockIdx.x * G + g0 + threadIdx.x] = bestp;
+            partial_out[row_slot(gate, G, blockIdx.x, g0 + threadIdx.x, sg[threadIdx.x].x)] = bestp;
         }
         __syncthreads();
     }

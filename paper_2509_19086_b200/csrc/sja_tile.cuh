@@ -83,6 +83,7 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
     // the count actually left in device memory, so that several passes can be queued without a host wait
     const uint32_t G_now = gate_gaps(gate, G);
     if (blockIdx.y * gaps_per_split >= G_now) return;
+    if (!chunk_dirty(gate, blockIdx.x * TILE_JOBS, TILE_JOBS)) return;   // re-auction: its candidate row still stands
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
     const uint32_t smem_s = (uint32_t)__cvta_generic_to_shared(smem_raw);
     Partial* stage = reinterpret_cast<Partial*>(smem_raw + TILE_RING_BYTES);                       // [WARPS][GT]
@@ -357,7 +358,7 @@ __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile
                 const Partial c = stage[ww * TILE_GT + threadIdx.x];
                 if (cand_better(c.key, c.job, bestp.key, bestp.job)) bestp = c;
             }
-            partial_out[(size_t)blockIdx.x * G + g0 + threadIdx.x] = bestp;
+            partial_out[row_slot(gate, G, blockIdx.x, g0 + threadIdx.x, sg[threadIdx.x].x)] = bestp;
         }
         __syncthreads();
     }
