@@ -85,7 +85,17 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
         const uint64_t s = __ldg(off + j) + (p0 ? __ldg(p0 + j) : 0u), e = __ldg(off + j + 1);
         const uint64_t w0 = s >> 5, w1 = (e - 1) >> 5;
         uint32_t cnt = 0;
-        for (uint64_t w = w0 + lane; w <= w1; w += 32) {
+        // interior words eight at a time (eight independent loads in flight per lane), then the edges one by one
+        uint64_t w = w0 + lane;
+        for (; w + 7 * 32 < w1; w += 8 * 32) {
+            uint32_t x[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) x[u] = __ldg(sbits + w + 32 * u);
+            if (w == w0) x[0] &= 0xFFFFFFFFu << (uint32_t)(s & 31);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) cnt += __popc(x[u]);
+        }
+        for (; w <= w1; w += 32) {
             uint32_t x = __ldg(sbits + w);
             if (w == w0) x &= 0xFFFFFFFFu << (uint32_t)(s & 31);
             if (w == w1) x &= 0xFFFFFFFFu >> (31u - (uint32_t)((e - 1) & 31));

@@ -655,10 +655,22 @@ __global__ void __launch_bounds__(256) place_gaps_kernel(const Gap* __restrict__
     __syncthreads();
     if (!is_last) return;
     __threadfence();
+    // every thread takes a contiguous stretch of the list, eight independent loads in flight
+    const uint32_t per = (G + blockDim.x - 1) / blockDim.x;
+    const uint32_t q0 = threadIdx.x * per, q1 = min(G, q0 + per);
     uint32_t leaders = 0;
-    for (uint32_t q = threadIdx.x; q < G; q += blockDim.x) {
-        const uint32_t c = __ldcg(&sorted[q].C);
-        if (q == 0 || __ldcg(&sorted[q - 1].C) != c) ++leaders;
+    uint32_t prev = (q0 > 0 && q0 < G) ? __ldcg(&sorted[q0 - 1].C) : 0u;
+    for (uint32_t q = q0; q < q1; q += 8) {
+        uint32_t cv[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) cv[u] = (q + u < q1) ? __ldcg(&sorted[q + u].C) : 0u;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (q + u < q1) {
+                if (q + u == 0 || cv[u] != prev) ++leaders;
+                prev = cv[u];
+            }
+        }
     }
     const uint32_t n = __reduce_add_sync(0xFFFFFFFFu, leaders);
     if ((threadIdx.x & 31u) == 0 && n) atomicAdd(&info->n_classes, n);
