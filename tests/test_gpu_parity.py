@@ -425,6 +425,35 @@ def test_select_very_large_gap_batch_unsorted_path(sja_mod, oracle_mod):
         _assert_awards_equal(got, want[:65536])
 
 
+def test_very_many_capacity_classes_take_the_standby_search(sja_mod, oracle_mod):
+    """More distinct capacities than max(64, G/16): the ordered-gap kernel that was queued returns at once and the
+    per-pair search kernel queued behind it serves the round (the class count never leaves the device); device
+    batches are read in place.  Plain rounds, a forced tile / merge request, and a re-auction (which reads the count
+    once and then queues the search alone) all match the oracle."""
+    import torch
+    spec = wl.scaled(wl.SPECS[3], n_jobs=3000, zipf_max=2500, n_gaps=1000)
+    prof = wl.make_profiles(spec, threads=2)
+    gaps = wl.make_gaps(spec)
+    rng = np.random.default_rng(808)
+    gaps["C_MiB"] = rng.choice(np.arange(1500, 82000, 97), gaps.shape[0])      # several hundred distinct capacities
+    assert np.unique(gaps["C_MiB"]).size > 200
+    progress = np.zeros(prof.n_jobs, np.uint32)
+    ready = prof.ready_ms.copy()
+    dev_gaps = torch.from_numpy(gaps.view(np.uint8).reshape(-1).copy()).cuda()
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof)
+        for policy, flags in ((0, 0), (2, 0), (3, sja_mod.FLAG_FORCE_TILE), (0, sja_mod.FLAG_FORCE_MERGE)):
+            ctx.advertise(dev_gaps)
+            want = oracle_mod.select(prof, progress, ready, gaps, policy)
+            _assert_awards_equal(ctx.select(policy, flags=flags, out="host"), want)
+        n_gpu, passes = ctx.round_reauction(2)
+        aw_o, n_cpu, passes_o = oracle_mod.round_with_reauction(prof, progress, ready, gaps, 2)
+        assert (n_gpu, passes) == (n_cpu, passes_o) and n_gpu > 0
+        _assert_awards_equal(ctx.get_awards(), aw_o, fields=("job", "end_step", "dur_ms", "score", "granted"))
+        p, r = ctx.get_state()
+        assert np.array_equal(p, progress) and np.array_equal(r, ready)
+
+
 def test_reloads_from_device_arrays(sja_mod, oracle_mod):
     """Loads from device-resident arrays into a context that already holds a load take the path with a
     single host wait (the validation verdict is checked on the device).  Covered here: a same-size reload,
