@@ -43,21 +43,35 @@ __global__ void __launch_bounds__(POWER_WARPS * 32) scan_power_kernel(
     }
     if (R == 0) return;
     const uint64_t first = s0 + pj, end = s0 + len;       // global steps [first, end) are scanned
-    const uint64_t bs0 = first & ~3ull;
-    const uint64_t nblk = (end - bs0 + POWER_BLK - 1) / POWER_BLK;
-    // block t into buffer t & 1: chunk c = steps bs + 4c .. bs + 4c + 3 at swizzled slot c ^ ((c >> 3) & 3);
+    const uint64_t bs0 = first & ~3ull;                   // blocks start 16-byte aligned
+    // everything below counts steps from bs0 in 32 bits (a job has fewer than 2^32 steps)
+    const uint32_t lead = (uint32_t)(first - bs0);        // 0..3 steps of the first block precede the scan
+    const uint32_t span = (uint32_t)(end - bs0);          // steps from bs0 to the end of the job
+    const uint32_t nblk = (span + POWER_BLK - 1) / POWER_BLK;
+    const uint32_t* src0 = power + bs0;
+    const uint64_t room = N_total - bs0;                  // steps of the trace from bs0 on
+    // block t into buffer t & 1: chunk c = steps 4c .. 4c + 3 of the block at swizzled slot c ^ ((c >> 3) & 3);
     // bytes beyond the end of the trace are filled with zeros
-    auto stage = [&](uint64_t t) {
+    auto stage = [&](uint32_t t) {
         if (t < nblk) {
-            const uint64_t bs = bs0 + t * POWER_BLK;
-            const uint32_t dst = wbase_s + (uint32_t)(t & 1ull) * POWER_BUF_BYTES;
+            const uint32_t dst = wbase_s + (t & 1u) * POWER_BUF_BYTES;
+            const uint32_t* src = src0 + (size_t)t * POWER_BLK + 4u * lane;
+            if ((uint64_t)(t + 1u) * POWER_BLK <= room) {
+                // the whole block lies inside the trace: plain copies
 #pragma unroll
-            for (uint32_t r = 0; r < 4; ++r) {
-                const uint32_t c = r * 32u + lane;
-                const uint64_t g = bs + 4ull * c;
-                uint32_t bytes = 0;
-                if (g < N_total) bytes = (N_total - g) >= 4ull ? 16u : (uint32_t)(N_total - g) * 4u;
-                cp_async16(dst + (c ^ ((c >> 3) & 3u)) * 16u, power + (bytes ? g : 0ull), bytes);
+                for (uint32_t r = 0; r < 4; ++r) {
+                    const uint32_t c = r * 32u + lane;
+                    cp_async16(dst + (c ^ ((c >> 3) & 3u)) * 16u, src + r * 128u, 16u);
+                }
+            } else {
+#pragma unroll
+                for (uint32_t r = 0; r < 4; ++r) {
+                    const uint32_t c = r * 32u + lane;
+                    const uint64_t g = (uint64_t)t * POWER_BLK + 4ull * c;      // steps from bs0
+                    uint32_t bytes = 0;
+                    if (g < room) bytes = (room - g) >= 4ull ? 16u : (uint32_t)(room - g) * 4u;
+                    cp_async16(dst + (c ^ ((c >> 3) & 3u)) * 16u, bytes ? src + r * 128u : power, bytes);
+                }
             }
         }
         cp_async_commit();
@@ -70,9 +84,12 @@ __global__ void __launch_bounds__(POWER_WARPS * 32) scan_power_kernel(
     uint32_t carry_seg = 0;         // maximum since the last boundary
     stage(0);
     uint32_t k0 = row_end(lane), k1 = row_end(32u + lane);    // ends of rows row + lane and row + 32 + lane
-    for (uint64_t t = 0; t < nblk; ++t) {
-        const uint64_t bs = bs0 + t * POWER_BLK;
-        unsigned char* buf = wbase + (size_t)(t & 1ull) * POWER_BUF_BYTES;
+    // a table row with end index k ends at step k - 1 of the job = step k - 1 - pj + lead from bs0
+    const uint32_t k_shift = pj + 1u - lead;      // (lead <= 3 and end indices above pj: no wrap for rows that count)
+    uint2* out = PW + base;
+    for (uint32_t t = 0; t < nblk; ++t) {
+        const uint32_t bs = t * POWER_BLK;        // the block's first step, counted from bs0
+        unsigned char* buf = wbase + (size_t)(t & 1u) * POWER_BUF_BYTES;
         const uint4* sv = reinterpret_cast<const uint4*>(buf);
         uint32_t* sbits = reinterpret_cast<uint32_t*>(buf + POWER_BLK * 4);
         stage(t + 1);
@@ -83,13 +100,10 @@ __global__ void __launch_bounds__(POWER_WARPS * 32) scan_power_kernel(
         // they are a prefix of the rows still to come
         uint32_t in_block = 0;
         {
-            const uint64_t lim = bs + POWER_BLK - s0;         // a row ends in the block iff its end index <= lim
             auto mark = [&](uint32_t k) -> uint32_t {
-                const bool here = k != 0u && (uint64_t)k <= lim;
-                if (here) {
-                    const uint32_t o = (uint32_t)(s0 + k - 1ull - bs);
-                    atomicOr(&sbits[o >> 5], 1u << (o & 31u));
-                }
+                const uint32_t o = k - k_shift - bs;          // offset of the row's last step in this block
+                const bool here = k != 0u && o < (uint32_t)POWER_BLK;   // (earlier rows are emitted, later ones wrap or exceed)
+                if (here) atomicOr(&sbits[o >> 5], 1u << (o & 31u));
                 return (uint32_t)__popc(__ballot_sync(0xFFFFFFFFu, here));
             };
             uint32_t f = mark(k0);
@@ -115,12 +129,12 @@ __global__ void __launch_bounds__(POWER_WARPS * 32) scan_power_kernel(
             v[4 * r + 0] = q.x; v[4 * r + 1] = q.y; v[4 * r + 2] = q.z; v[4 * r + 3] = q.w;
         }
         uint32_t bits = (sbits[lane >> 1] >> ((lane & 1u) * 16u)) & 0xFFFFu;
-        const uint64_t lane_base = bs + 16ull * lane;
-        if (lane_base < first || lane_base + 16 > end) {
-            // steps outside [first, end) count as 0 and carry no boundary
+        const uint32_t lane_base = bs + 16u * lane;
+        if (lane_base < lead || lane_base + 16u > span) {
+            // steps outside the job's part [lead, span) count as 0 and carry no boundary
 #pragma unroll
             for (int i = 0; i < 16; ++i)
-                if (lane_base + i < first || lane_base + i >= end) { v[i] = 0u; bits &= ~(1u << i); }
+                if (lane_base + i < lead || lane_base + i >= span) { v[i] = 0u; bits &= ~(1u << i); }
         }
         // first walk: maximum of all 16 steps, maximum since the lane's last boundary
         uint32_t lmax = 0, tail = 0;
@@ -163,15 +177,19 @@ __global__ void __launch_bounds__(POWER_WARPS * 32) scan_power_kernel(
             if (lane >= (uint32_t)o) pos += y;
         }
         pos = row + pos - cnt;
-        // second walk: emit {running maximum, segment maximum} at every boundary
+        // second walk: emit {running maximum, segment maximum} at every boundary (lanes without one skip it)
+        if (bits) {
+            uint2* o = out + pos;
+            const uint2* o_end = out + R;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            seg = max(seg, v[i]);
-            run = max(run, v[i]);
-            if ((bits >> i) & 1u) {
-                if (pos < R) PW[base + pos] = make_uint2(run, seg);
-                ++pos;
-                seg = 0;
+            for (int i = 0; i < 16; ++i) {
+                seg = max(seg, v[i]);
+                run = max(run, v[i]);
+                if ((bits >> i) & 1u) {
+                    if (o < o_end) *o = make_uint2(run, seg);
+                    ++o;
+                    seg = 0;
+                }
             }
         }
         // carries for the next block
