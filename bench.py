@@ -63,9 +63,9 @@ NCU_SCAN = {"source_sha": "351669ab0df1e1e6", "read_bytes_per_step": 2184044544 
 # Warp instructions of one select_tile_kernel launch (ncu smsp__inst_executed.sum, one pass, full size), per
 # workload; valid while csrc/sja_tile.cuh is the file they were taken from.  The kernel's work is not proportional
 # to the pair count, so each figure holds for its workload only.
-NCU_TILE = {"source_sha": "c1eae935f84bb65e",
-            "warp_instr_per_launch": {"cfg3-heavy-tailed": 769451495, "cfg2-large-uniform": 90760306,
-                                      "cfg4-streaming": 187134035}}
+NCU_TILE = {"source_sha": "eb40ed91a9a31e13",
+            "warp_instr_per_launch": {"cfg3-heavy-tailed": 769500647, "cfg2-large-uniform": 90793074,
+                                      "cfg4-streaming": 187177939}}
 
 
 def _source_sha(name: str):

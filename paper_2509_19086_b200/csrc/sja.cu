@@ -284,6 +284,28 @@ __global__ void export_rows_kernel(const uint4* __restrict__ A, const uint2* __r
     if (W) W[i] = pack64(a.z, a.w);
 }
 
+// Launch a kernel of the round so that it may be brought onto the GPU while the kernel before it in the stream is
+// still running (programmatic dependent launch): all kernels launched here begin with dep_wait(), which holds them
+// until that kernel has completed and its writes are visible.  The launch gap between two small dependent
+// kernels shrinks to what the hardware needs to hand over.
+#ifndef SJA_DEP_LAUNCH
+#define SJA_DEP_LAUNCH 1
+#endif
+template <typename... P, typename... A>
+void launch_dep(void (*kernel)(P...), dim3 grid, uint32_t threads, size_t smem, cudaStream_t stream, A&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = SJA_DEP_LAUNCH ? 1u : 0u;
+    (void)cudaLaunchKernelEx(&cfg, kernel, P(args)...);   // a failure stays in the runtime's last-error slot
+}
+
 // The merge and tile kernels are templated on the policy and on whether the subjob duration
 // thresholds are in force; these helpers pick the instance.
 enum SelectKernel { SEL_TILE = 0, SEL_MERGE = 1, SEL_SEARCH = 2 };
@@ -292,11 +314,11 @@ template <uint32_t KIND, bool BOUNDED>
 void launch_sorted_kb(SelectKernel which, dim3 grid, cudaStream_t stream, const JobView& jv, const Gap* sgaps,
                       uint32_t G, uint32_t per_split, Partial* partial, const LaunchGate& gate) {
     if (which == SEL_TILE)
-        select_tile_kernel<KIND, BOUNDED><<<grid, TILE_WARPS * 32, TILE_SMEM_BYTES, stream>>>(jv, sgaps, G, per_split,
-                                                                                             partial, gate);
+        launch_dep(select_tile_kernel<KIND, BOUNDED>, grid, TILE_WARPS * 32, TILE_SMEM_BYTES, stream, jv, sgaps, G,
+                   per_split, partial, gate);
     else
-        select_merge_kernel<KIND, BOUNDED><<<grid, MERGE_WARPS * 32, MERGE_SMEM_BYTES, stream>>>(jv, sgaps, G,
-                                                                                                per_split, partial, gate);
+        launch_dep(select_merge_kernel<KIND, BOUNDED>, grid, MERGE_WARPS * 32, MERGE_SMEM_BYTES, stream, jv, sgaps, G,
+                   per_split, partial, gate);
 }
 
 template <bool BOUNDED>
@@ -446,13 +468,12 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
             const bool opts = jv.late_start != 0u || jv.deadline != nullptr || jv.PW != nullptr || jv.min_gain != 0u ||
                               jv.ckpt != nullptr;
             if (opts)
-                select_search_kernel<true><<<dim3(kp.n_chunks, kp.splits), SEARCH_THREADS,
-                                             jv.PW ? SEARCH_SMEM_BYTES_POWER : SEARCH_SMEM_BYTES, c->stream>>>(
-                    jv, sgaps, G_act, kp.per_split, kind, partial, g, kp.jobs_per_cta);
+                launch_dep(select_search_kernel<true>, dim3(kp.n_chunks, kp.splits), SEARCH_THREADS,
+                           jv.PW ? SEARCH_SMEM_BYTES_POWER : SEARCH_SMEM_BYTES, c->stream, jv, sgaps, G_act,
+                           kp.per_split, kind, partial, g, kp.jobs_per_cta);
             else
-                select_search_kernel<false><<<dim3(kp.n_chunks, kp.splits), SEARCH_THREADS, SEARCH_SMEM_BYTES,
-                                              c->stream>>>(jv, sgaps, G_act, kp.per_split, kind, partial, g,
-                                                           kp.jobs_per_cta);
+                launch_dep(select_search_kernel<false>, dim3(kp.n_chunks, kp.splits), SEARCH_THREADS, SEARCH_SMEM_BYTES,
+                           c->stream, jv, sgaps, G_act, kp.per_split, kind, partial, g, kp.jobs_per_cta);
         };
         if (pl.primary.kernel != SEL_SEARCH)
             launch_sorted(pl.primary.kernel, kind, dim3(pl.primary.n_chunks, pl.primary.splits), c->stream, jv, sgaps,
@@ -464,9 +485,9 @@ sja_status run_select(sja_ctx* c, uint32_t kind, uint32_t pflags, const Gap* sga
             many.run_if_many = 1u;
             launch_search(pl.alt, many);
         }
-        finalize_awards_kernel<<<(G_act + 31) / 32, FINALIZE_WARPS * 32, 0, c->stream>>>(
-            jv, partial, pl.primary.n_chunks, pl.alt.n_chunks, sgaps, G_act, kind, c->awards.as<Award>(),
-            c->widx.as<uint32_t>(), gate);
+        launch_dep(finalize_awards_kernel, dim3((G_act + 31) / 32), FINALIZE_WARPS * 32, 0, c->stream, jv, partial,
+                   pl.primary.n_chunks, pl.alt.n_chunks, sgaps, G_act, kind, c->awards.as<Award>(),
+                   c->widx.as<uint32_t>(), gate);
     }
     c->prof = was_on;
     return SJA_OK;
@@ -492,10 +513,10 @@ void run_commit(sja_ctx* c, uint32_t* blocked, const uint8_t* accept = nullptr, 
     ProfScope ps(c, CAT_COMMIT);
     const uint32_t gb = (G + 255) / 256;
     const CommitArgs a = commit_args(c, blocked, accept, dirty_next);
-    commit_vote_kernel<<<gb, 256, 0, c->stream>>>(a.awards, G, a.jobwin, a.n_granted, accept);
-    commit_apply_kernel<<<gb, 256, 0, c->stream>>>(a, G);
-    commit_refresh_kernel<<<(uint32_t)(((uint64_t)G * 32 + 255) / 256), 256, 0, c->stream>>>(
-        a.winners, a.n_granted, G, a.boff, a.pb, a.A, a.B, a.jobwin, a.PW);
+    launch_dep(commit_vote_kernel, dim3(gb), 256, 0, c->stream, a.awards, G, a.jobwin, a.n_granted, accept);
+    launch_dep(commit_apply_kernel, dim3(gb), 256, 0, c->stream, a, G);
+    launch_dep(commit_refresh_kernel, dim3((uint32_t)(((uint64_t)G * 32 + 255) / 256)), 256, 0, c->stream, a.winners,
+               a.n_granted, G, a.boff, a.pb, a.A, a.B, a.jobwin, a.PW);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -733,7 +754,7 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
     auto launch_state_and_scan = [&](uint64_t cap_rows) -> sja_status {
         {
             ProfScope ps(c, CAT_PREP);
-            finish_load_kernel<<<(J + 255) / 256, 256, 0, c->stream>>>(
+            launch_dep(finish_load_kernel, dim3((J + 255) / 256), 256, 0, c->stream,
                 J, n_count_ctas, c->nbj.as<uint64_t>(), c->cta_base.as<uint64_t>(), c->boff_next.as<uint64_t>(), cap_rows,
                 d_p, d_ready, d_wait, d_prio, c->p.as<uint32_t>(), c->ready.as<uint32_t>(),
                 c->wait.as<uint32_t>(), c->prio.as<uint8_t>(), c->pb.as<uint32_t>(), c->Dp.as<uint32_t>(),
@@ -771,8 +792,8 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
         count_boundaries_kernel<<<n_count_ctas, 256, 0, c->stream>>>(
             d_off, d_s, d_p, J, c->nbj.as<uint64_t>(), c->cta_tot.as<uint64_t>(), c->flags.as<uint32_t>(),
             c->long_list.as<uint32_t>());
-        cta_offsets_kernel<<<1, 1024, 0, c->stream>>>(c->cta_tot.as<uint64_t>(), n_count_ctas,
-                                                      c->cta_base.as<uint64_t>());
+        launch_dep(cta_offsets_kernel, dim3(1), 1024, 0, c->stream, c->cta_tot.as<uint64_t>(), n_count_ctas,
+                   c->cta_base.as<uint64_t>());
     }
     CU(cudaGetLastError());
     if (speculate) TRY(launch_state_and_scan(cap_now));
@@ -873,16 +894,16 @@ sja_status sja_advertise(sja_ctx* c, uint32_t G, const sja_gap* gaps, sja_memspa
             uint64_t* tile_key = reinterpret_cast<uint64_t*>(c->gap_rank.as<unsigned char>() + rank_bytes);
             uint32_t* tile_idx = reinterpret_cast<uint32_t*>(tile_key + (size_t)n_tiles * SORT_TILE);
             const bool one_tile = n_tiles == 1;
-            sort_gap_tiles_kernel<<<n_tiles, SORT_TILE, 0, c->stream>>>(src, G, tile_key, tile_idx, rank,
-                                                                        c->gap_info.as<GapInfo>(),
-                                                                        one_tile ? c->sgaps.as<Gap>() : nullptr, keep);
+            launch_dep(sort_gap_tiles_kernel, dim3(n_tiles), SORT_TILE, 0, c->stream, src, G, tile_key, tile_idx, rank,
+                       c->gap_info.as<GapInfo>(), one_tile ? c->sgaps.as<Gap>() : nullptr, keep);
             if (!one_tile) {
-                rank_gap_tiles_kernel<<<dim3(n_tiles, n_tiles), SORT_TILE, 0, c->stream>>>(tile_key, tile_idx, rank);
-                place_gaps_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(src, G, rank, c->sgaps.as<Gap>(),
-                                                                          c->gap_info.as<GapInfo>());
+                launch_dep(rank_gap_tiles_kernel, dim3(n_tiles, n_tiles), SORT_TILE, 0, c->stream, tile_key, tile_idx,
+                           rank);
+                launch_dep(place_gaps_kernel, dim3((G + 255) / 256), 256, 0, c->stream, src, G, rank,
+                           c->sgaps.as<Gap>(), c->gap_info.as<GapInfo>());
             }
         } else {
-            copy_gaps_kernel<<<(G + 255) / 256, 256, 0, c->stream>>>(src, G, c->sgaps.as<Gap>(), keep);
+            launch_dep(copy_gaps_kernel, dim3((G + 255) / 256), 256, 0, c->stream, src, G, c->sgaps.as<Gap>(), keep);
         }
     }
     CU(cudaGetLastError());
@@ -1050,9 +1071,9 @@ sja_status sja_round_reauction(sja_ctx* c, const sja_policy* policy, uint32_t ma
             {
                 // commit of the pass and compaction of its gap list: one launch of one CTA
                 ProfScope ps(c, CAT_COMMIT);
-                reauction_resolve_kernel<<<1, 1024, 0, c->stream>>>(
-                    commit_args(c, c->blocked.as<uint32_t>(), nullptr, dirty_next), cur, g_act, spare, reports + 4 * k,
-                    g_dev, dirty_cur, n_dirty);
+                launch_dep(reauction_resolve_kernel, dim3(1), 1024, 0, c->stream,
+                           commit_args(c, c->blocked.as<uint32_t>(), nullptr, dirty_next), cur, g_act, spare,
+                           reports + 4 * k, g_dev, dirty_cur, n_dirty);
             }
             CU(cudaGetLastError());
             std::swap(dirty_cur, dirty_next);

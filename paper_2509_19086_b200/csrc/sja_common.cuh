@@ -19,6 +19,17 @@ enum : uint32_t {
 
 constexpr uint32_t SJA_NO_JOB_DEV = 0xFFFFFFFFu;
 
+// Programmatic dependent launch (griddepcontrol, sm_90 and later).  The small kernels of a round follow one another
+// in one stream, each reading what the one before wrote, and the gap between two such launches is longer than most
+// of them run.  A kernel launched with the programmatic-stream-serialization attribute may be made resident while
+// the kernel before it is still running: dep_wait() then holds it until that grid has completed and its writes are
+// visible, and dep_launch() tells the hardware that the NEXT kernel in the stream may be brought in.  Every kernel
+// that is launched with the attribute calls dep_wait() as its first statement, before any early return (a kernel
+// that left without waiting could complete before its predecessor, and release its own successor too early); in a
+// kernel launched without the attribute both calls do nothing.
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // A job counts as "long" for the scan's hand-out order when it has more steps left than twice the
 // mean job length (and at least 8192): such jobs are scanned first, so that none of them starts late and
 // stretches the kernel's tail.  The row-counting kernel lists them, the scan kernel skips them later.

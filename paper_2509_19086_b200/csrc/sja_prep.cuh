@@ -21,6 +21,7 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
     const uint64_t* __restrict__ off, const uint32_t* __restrict__ sbits,
     const uint32_t* __restrict__ p0 /* may be nullptr: all 0 */, uint32_t J, uint64_t* __restrict__ local_off,
     uint64_t* __restrict__ cta_total, uint32_t* __restrict__ flags, uint32_t* __restrict__ long_list) {
+    dep_launch();   // the one-CTA offsets kernel may be brought in meanwhile
     __shared__ uint32_t cnts[COUNT_JOBS_PER_CTA];
     __shared__ uint64_t warp_sums[COUNT_JOBS_PER_CTA / 32];
     const uint64_t N = __ldg(off + J);   // total step count
@@ -140,6 +141,8 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
 // array in tiles of 8192 with a running carry.
 __global__ void __launch_bounds__(1024) cta_offsets_kernel(const uint64_t* __restrict__ totals, uint32_t P,
                                                            uint64_t* __restrict__ base_out) {
+    dep_wait();
+    dep_launch();
     __shared__ uint64_t warp_sums[32];
     __shared__ uint64_t warp_excl[32];
     __shared__ uint64_t tile_total;
@@ -201,6 +204,8 @@ __global__ void __launch_bounds__(256) finish_load_kernel(
     uint32_t* __restrict__ wait, uint8_t* __restrict__ prio, uint32_t* __restrict__ pb, uint32_t* __restrict__ Dp,
     uint64_t* __restrict__ Wp, unsigned long long* __restrict__ jobwin, uint32_t* __restrict__ counter,
     uint32_t* __restrict__ flags) {
+    dep_wait();
+    dep_launch();
     const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
     const uint64_t total = cta_base[P];
     if (j < J) boff[j] = cta_base[j / COUNT_JOBS_PER_CTA] + local_off[j];

@@ -132,6 +132,8 @@ template <bool OPTS>
 __global__ void __launch_bounds__(SEARCH_THREADS) select_search_kernel(
     JobView jv, const Gap* __restrict__ gaps, uint32_t G, uint32_t gaps_per_split, uint32_t kind,
     Partial* __restrict__ partial_out, LaunchGate gate, uint32_t jobs_per_cta) {
+    dep_wait();
+    dep_launch();
     const uint32_t G_now = gate_gaps(gate, G);   // gaps actually left
     if (blockIdx.y * gaps_per_split >= G_now) return;
     if (!chunk_dirty(gate, blockIdx.x * jobs_per_cta, jobs_per_cta)) return;   // its candidate row still stands
@@ -351,6 +353,8 @@ __global__ void __launch_bounds__(FINALIZE_WARPS * 32) finalize_awards_kernel(
     JobView jv, const Partial* __restrict__ partial, uint32_t n_rows, uint32_t n_rows_many,
     const Gap* __restrict__ sgaps, uint32_t G, uint32_t kind, Award* __restrict__ awards, uint32_t* __restrict__ widx,
     LaunchGate gate) {
+    dep_wait();
+    dep_launch();
     __shared__ Partial fold[FINALIZE_WARPS][32];
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
     const uint32_t g = blockIdx.x * 32u + lane;     // position in the advertised (sorted) order
@@ -410,6 +414,8 @@ __global__ void __launch_bounds__(256) commit_vote_kernel(const Award* __restric
                                                           unsigned long long* __restrict__ jobwin,
                                                           uint32_t* __restrict__ n_granted,
                                                           const uint8_t* __restrict__ accept) {
+    dep_wait();
+    dep_launch();
     const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g == 0) *n_granted = 0;
     if (g >= G) return;
@@ -452,6 +458,8 @@ __device__ __forceinline__ void commit_apply_one(const CommitArgs& c, uint32_t g
 }
 
 __global__ void __launch_bounds__(256) commit_apply_kernel(CommitArgs c, uint32_t G) {
+    dep_wait();
+    dep_launch();
     const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= G) return;
     commit_apply_one(c, g);
@@ -514,6 +522,8 @@ __global__ void __launch_bounds__(256) commit_refresh_kernel(
     const uint32_t* __restrict__ winners, const uint32_t* __restrict__ n_granted, uint32_t G,
     const uint64_t* __restrict__ boff, const uint32_t* __restrict__ pb, uint4* __restrict__ A,
     const uint2* __restrict__ B, unsigned long long* __restrict__ jobwin, uint2* __restrict__ PW) {
+    dep_wait();
+    dep_launch();
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (w >= G || w >= *n_granted) return;
@@ -554,6 +564,8 @@ __global__ void __launch_bounds__(SORT_TILE) sort_gap_tiles_kernel(const Gap* __
                                                                    uint32_t* __restrict__ tile_idx,
                                                                    uint32_t* __restrict__ rank, GapInfo* __restrict__ info,
                                                                    Gap* __restrict__ sorted_out, Gap* __restrict__ keep) {
+    dep_wait();
+    dep_launch();
     __shared__ uint64_t sk[SORT_TILE];
     __shared__ uint32_t si[SORT_TILE];
     const uint32_t t = threadIdx.x;
@@ -616,6 +628,8 @@ __global__ void __launch_bounds__(SORT_TILE) sort_gap_tiles_kernel(const Gap* __
 __global__ void __launch_bounds__(SORT_TILE) rank_gap_tiles_kernel(const uint64_t* __restrict__ tile_key,
                                                                    const uint32_t* __restrict__ tile_idx,
                                                                    uint32_t* __restrict__ rank) {
+    dep_wait();
+    dep_launch();
     __shared__ uint64_t sk[SORT_TILE];
     __shared__ uint32_t si[SORT_TILE];
     const uint32_t t = threadIdx.x;
@@ -640,6 +654,8 @@ __global__ void __launch_bounds__(SORT_TILE) rank_gap_tiles_kernel(const uint64_
 __global__ void __launch_bounds__(256) place_gaps_kernel(const Gap* __restrict__ gaps, uint32_t G,
                                                          const uint32_t* __restrict__ rank, Gap* __restrict__ sorted,
                                                          GapInfo* __restrict__ info) {
+    dep_wait();
+    dep_launch();
     __shared__ uint32_t is_last;
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < G) {
@@ -679,6 +695,8 @@ __global__ void __launch_bounds__(256) place_gaps_kernel(const Gap* __restrict__
 // Identity order (used when the batch is too large for the one-CTA sort).
 __global__ void __launch_bounds__(256) copy_gaps_kernel(const Gap* __restrict__ gaps, uint32_t G,
                                                         Gap* __restrict__ sorted, Gap* __restrict__ keep) {
+    dep_wait();
+    dep_launch();
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= G) return;
     Gap g = gaps[i];
@@ -702,6 +720,8 @@ __global__ void __launch_bounds__(1024) reauction_resolve_kernel(CommitArgs c, c
                                                                  uint32_t* __restrict__ report,
                                                                  const uint32_t* __restrict__ G_dev,
                                                                  uint32_t* __restrict__ dirty_done, uint32_t n_dirty) {
+    dep_wait();
+    dep_launch();
     if (G_dev) G_in = min(G_in, *G_dev);
     __shared__ uint32_t warp_cnt[32];
     __shared__ uint32_t tile_total;
@@ -819,6 +839,8 @@ template <uint32_t KIND, bool BOUNDED>
 __global__ void __launch_bounds__(MERGE_WARPS * 32, MERGE_CTAS_PER_SM) select_merge_kernel(
     JobView jv, const Gap* __restrict__ sgaps, uint32_t G, uint32_t gaps_per_split, Partial* __restrict__ partial_out,
     LaunchGate gate) {
+    dep_wait();
+    dep_launch();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     if (gate_gaps(gate, G) == 0u) return;      // the class count calls for the per-pair search
     if (!chunk_dirty(gate, blockIdx.x * MERGE_JOBS, MERGE_JOBS)) return;

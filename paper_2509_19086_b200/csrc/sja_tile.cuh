@@ -78,6 +78,8 @@ template <uint32_t KIND, bool BOUNDED>
 __global__ void __launch_bounds__(TILE_WARPS * 32, TILE_CTAS_PER_SM) select_tile_kernel(
     JobView jv, const Gap* __restrict__ sgaps, uint32_t G, uint32_t gaps_per_split, Partial* __restrict__ partial_out,
     LaunchGate gate) {
+    dep_wait();
+    dep_launch();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // G is the gap count the launch was sized for (and the row length of partial_out); a re-auction hands
     // the count actually left in device memory, so that several passes can be queued without a host wait
