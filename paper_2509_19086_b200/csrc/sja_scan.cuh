@@ -30,7 +30,16 @@ constexpr int SCAN_STAGES = SJA_SCAN_STAGES;        // cp.async ring depth per w
 constexpr int SCAN_WARPS = SJA_SCAN_WARPS;          // warps per CTA
 constexpr int SCAN_CTAS_PER_SM = SJA_SCAN_CTAS_PER_SM;
 constexpr int SCAN_STAGE_BYTES = 2048 + 2048 + 64;  // d, m, 16 safe words
-constexpr int SCAN_SMEM_BYTES = SCAN_WARPS * SCAN_STAGES * SCAN_STAGE_BYTES;
+// Per warp, between its two ring slots: 3 KB that belong to the row buffer only.  A consumed slot alone holds the
+// rows of a block with boundaries up to one in three steps; with the region next to it (behind slot 0, before
+// slot 1: contiguous with either) up to 301 rows, i.e. boundaries denser than one in two, leave through the buffer
+// with coalesced stores.  2 CTAs x 10 warps x 11 392 B = 222.5 KB of the SM's 227 KB.
+#ifndef SJA_SCAN_EXTRA_BYTES
+#define SJA_SCAN_EXTRA_BYTES 3072
+#endif
+constexpr int SCAN_EXTRA_BYTES = SJA_SCAN_EXTRA_BYTES;
+constexpr int SCAN_WARP_BYTES = SCAN_STAGES * SCAN_STAGE_BYTES + SCAN_EXTRA_BYTES;
+constexpr int SCAN_SMEM_BYTES = SCAN_WARPS * SCAN_WARP_BYTES;
 
 struct ScanArgs {
     const uint64_t* off;     // [J+1]
@@ -73,19 +82,27 @@ __device__ __forceinline__ uint32_t swz(uint32_t c) { return c ^ ((c >> 3) & 3u)
 // Per 512-step block a warp knows, after one popcount scan, how many rows the block emits.
 // Usual case (at most SCAN_STAGE_ROWS rows): each lane walks its 16 steps ONCE, keeping
 // lane-local sums, and drops a lane-relative row into shared memory at every safe bit (the
-// just-consumed input slot of the ring is reused as the row buffer).  The warp then scans the
+// just-consumed input slot of the ring, lengthened by the region next to it, is the row buffer).  The warp then scans the
 // 32 lane totals and a second, row-indexed phase (32 rows per iteration, i.e. about a tenth of
 // the steps) adds each row's lane offset, derives the running maximum as a prefix maximum over
 // the rows' segment maxima, and writes the finished rows with fully coalesced 512-byte and
-// 256-byte stores.  Blocks with more rows (boundaries denser than one in three steps) take
-// the two-pass route: lane totals first, then a second walk that stores rows directly.
-constexpr int SCAN_STAGE_ROWS = 168;   // 168 * 24 B = 4032 B <= the 4096 B of a consumed d+m slot
+// 256-byte stores.  Blocks with more rows (boundaries denser than about three in five steps)
+// take the two-pass route: lane totals first, then a second walk that produces finished rows,
+// the first SCAN_STAGE_ROWS through the buffer, the rest stored directly.
+constexpr int SCAN_STAGE_ROWS = (SCAN_EXTRA_BYTES ? SCAN_STAGE_BYTES + SCAN_EXTRA_BYTES : 4096) / 24;   // 301 rows of 24 B
+#ifndef SJA_SCAN_STAGED_MAX
+#define SJA_SCAN_STAGED_MAX SCAN_STAGE_ROWS
+#endif
+constexpr int SCAN_STAGED_MAX = SJA_SCAN_STAGED_MAX;   // blocks with more rows take the two-pass route
+static_assert(SCAN_STAGED_MAX <= SCAN_STAGE_ROWS, "staged rows must fit the row buffer");
+static_assert(SCAN_EXTRA_BYTES == 0 || SCAN_STAGES == 2, "the extra region sits between two slots");
+static_assert(SCAN_EXTRA_BYTES % 16 == 0, "row buffer alignment");
 
 __global__ void __launch_bounds__(SCAN_WARPS * 32, SCAN_CTAS_PER_SM) scan_profiles_kernel(ScanArgs a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t wid = threadIdx.x >> 5;
-    unsigned char* wbase = smem_raw + (size_t)wid * SCAN_STAGES * SCAN_STAGE_BYTES;
+    unsigned char* wbase = smem_raw + (size_t)wid * SCAN_WARP_BYTES;
     const uint32_t wbase_s = (uint32_t)__cvta_generic_to_shared(wbase);
     // a load that was rejected by the validation pass, or whose table does not fit the buffers, is not scanned
     if (*reinterpret_cast<volatile const uint32_t*>(a.flags) & (FLAG_BAD_PROFILE | FLAG_NEED_ROWS)) return;
@@ -123,7 +140,7 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32, SCAN_CTAS_PER_SM) scan_profil
         auto issue = [&](uint64_t t) {
             if (t < nblk) {
                 const uint64_t bs = blk0 + t * SCAN_BLK;
-                const uint32_t st = wbase_s + (uint32_t)(t % SCAN_STAGES) * SCAN_STAGE_BYTES;
+                const uint32_t st = wbase_s + (uint32_t)(t % SCAN_STAGES) * (SCAN_STAGE_BYTES + SCAN_EXTRA_BYTES);
                 if (bs >= s && bs + SCAN_BLK <= e) {
                     // block entirely inside the job: plain 16-byte copies, no clipping
                     const uint32_t* dp = a.d + bs + 4u * lane;
@@ -175,7 +192,7 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32, SCAN_CTAS_PER_SM) scan_profil
             cp_async_wait<SCAN_STAGES - 1>();
             __syncwarp();
 
-            unsigned char* st = wbase + (size_t)(t % SCAN_STAGES) * SCAN_STAGE_BYTES;
+            unsigned char* st = wbase + (size_t)(t % SCAN_STAGES) * (SCAN_STAGE_BYTES + SCAN_EXTRA_BYTES);
             const uint4* sd = reinterpret_cast<const uint4*>(st);
             const uint4* sm = reinterpret_cast<const uint4*>(st + 2048);
             const uint32_t* ss = reinterpret_cast<const uint32_t*>(st + 4096);
@@ -218,10 +235,12 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32, SCAN_CTAS_PER_SM) scan_profil
                 if (lane >= (uint32_t)o) incC += yc;
             }
             const uint32_t c_total = __shfl_sync(0xFFFFFFFFu, incC, 31);
-            const bool staged = c_total <= (uint32_t)SCAN_STAGE_ROWS;   // warp-uniform
+            const bool staged = c_total <= (uint32_t)SCAN_STAGED_MAX;   // warp-uniform
 
-            uint4* rowA = reinterpret_cast<uint4*>(st);
-            uint2* rowB = reinterpret_cast<uint2*>(st + 16 * SCAN_STAGE_ROWS);
+            // the row buffer: the consumed slot, plus the extra region next to it (behind slot 0, before slot 1)
+            unsigned char* rbuf = (SCAN_EXTRA_BYTES && (t % SCAN_STAGES)) ? st - SCAN_EXTRA_BYTES : st;
+            uint4* rowA = reinterpret_cast<uint4*>(rbuf);
+            uint2* rowB = reinterpret_cast<uint2*>(rbuf + 16 * SCAN_STAGE_ROWS);
 
             // ---- walk the 16 steps: lane totals, and (staged route) lane-relative rows
             uint32_t td = 0, tail = 0, orv = 0;

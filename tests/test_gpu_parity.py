@@ -87,6 +87,30 @@ def test_scan_matches_oracle_dense_boundaries_and_large_values(sja_mod, oracle_m
         _check_scan(oracle_mod, ctx, prof, progress)
 
 
+def test_scan_matches_oracle_boundary_densities_around_the_row_buffer(sja_mod, oracle_mod):
+    """Boundary densities on both sides of what the warp's row buffer holds per 512-step block (about 300 rows):
+    blocks that leave through the buffer (in either of its two positions: even and odd blocks), blocks that
+    overflow it, and jobs that switch between the two from block to block."""
+    rng = np.random.default_rng(103)
+    jobs = []
+    for dens in (0.3, 0.36, 0.45, 0.52, 0.56, 0.58, 0.59, 0.6, 0.62, 0.7, 0.9):
+        for n in (3000, 1111):
+            d = rng.integers(0, 60, n).tolist()
+            m = rng.integers(0, 90000, n).tolist()
+            s = (rng.random(n) < dens).astype(int).tolist()
+            jobs.append((d, m, s))
+    # density that changes along the job: sparse, dense, sparse ... in 512-step stretches that do not align with the blocks
+    n = 6000
+    dens = np.where((np.arange(n) // 700) % 2 == 0, 0.05, 0.75)
+    jobs.append((rng.integers(1, 50, n).tolist(), rng.integers(1, 81920, n).tolist(), (rng.random(n) < dens).astype(int).tolist()))
+    prof = profiles_from_lists(jobs, ready=rng.integers(0, 100, len(jobs)))
+    lens = np.diff(prof.off).astype(np.int64)
+    progress = (lens * rng.random(len(jobs)) * (rng.random(len(jobs)) < 0.5)).astype(np.uint32)
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof, progress)
+        _check_scan(oracle_mod, ctx, prof, progress)
+
+
 def test_scan_cfg1_sampled_jobs(sja_mod, oracle_mod):
     spec = wl.SPECS[1]
     prof = wl.make_profiles(spec)
