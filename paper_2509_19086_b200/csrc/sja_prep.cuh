@@ -10,12 +10,15 @@ namespace sja {
 // bits above the progress point; the end of a job always counts).  The kernel is bound by
 // memory latency, so it wants many warps with several loads in flight each: a CTA of 8
 // warps owns 64 consecutive jobs, a warp counts 8 of them, four at a time with eight lanes
-// per job (lanes stride over the job's safe words, four independent loads per lane).  The
-// CTA scans its 64 counts and writes each job's offset relative to the CTA plus the CTA
-// total.  Two tiny kernels then turn CTA totals into global offsets.
+// per job (lanes stride over the job's safe words, four independent loads per lane); jobs of
+// more than 256 safe words are left to a second phase in which the whole CTA counts them one
+// after the other (on a heavy-tailed mix they hold most of the bits, and a warp that met
+// several of them would keep the other seven waiting).  The CTA scans its 64 counts and
+// writes each job's offset relative to the CTA plus the CTA total.  Two tiny kernels then
+// turn CTA totals into global offsets.
 constexpr int COUNT_JOBS_PER_CTA = 64;
 constexpr int COUNT_JOBS_PER_WARP = 8;
-constexpr uint32_t COUNT_LONG = 0x80000000u;   // marker: job left to the whole-warp pass
+constexpr uint32_t COUNT_LONG = 0x80000000u;   // marker: job left to the whole-CTA pass
 
 __global__ void __launch_bounds__(256) count_boundaries_kernel(
     const uint64_t* __restrict__ off, const uint32_t* __restrict__ sbits,
@@ -23,7 +26,14 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
     uint64_t* __restrict__ cta_total, uint32_t* __restrict__ flags, uint32_t* __restrict__ long_list) {
     dep_launch();   // the one-CTA offsets kernel may be brought in meanwhile
     __shared__ uint32_t cnts[COUNT_JOBS_PER_CTA];
+    __shared__ uint32_t is_long[COUNT_JOBS_PER_CTA];
+    __shared__ uint32_t long_cnt[COUNT_JOBS_PER_CTA];   // boundary rows of the jobs the whole CTA counts
+    __shared__ uint4 ldesc[COUNT_JOBS_PER_CTA];         // those jobs: {first word lo, hi, last word - first word, first bit | last bit << 8 | slot << 16}
+    __shared__ uint32_t n_long_cta;
     __shared__ uint64_t warp_sums[COUNT_JOBS_PER_CTA / 32];
+    if (threadIdx.x < COUNT_JOBS_PER_CTA) long_cnt[threadIdx.x] = 0u;
+    if (threadIdx.x == 0) n_long_cta = 0u;
+    __syncthreads();
     const uint64_t N = __ldg(off + J);   // total step count
     const uint64_t long_thresh = long_job_threshold(N, J);
     const uint32_t lane = threadIdx.x & 31u, wid = threadIdx.x >> 5;
@@ -35,7 +45,7 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
         const uint32_t i = it * 4u + grp;
         const uint32_t j = jbase + i;
         uint32_t cnt = 0;
-        bool bad = false;
+        bool bad = false, lng = false;
         if (j < J) {
             const uint64_t js = __ldg(off + j), je = __ldg(off + j + 1);
             const uint32_t p = p0 ? __ldg(p0 + j) : 0u;
@@ -43,10 +53,15 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
             if (j == 0 && js != 0) bad = true;
             if (!bad) {
                 const uint64_t s = js + p, e = je;
-                // long jobs go on the list the scan works off first (flags[1] counts them)
-                if (sub == 0 && e - s > long_thresh) long_list[atomicAdd(flags + 1, 1u)] = j;
+                lng = e - s > long_thresh;   // goes on the list the scan works off first
                 if (s < e && ((e - 1) >> 5) - (s >> 5) >= 256) {
-                    cnt = COUNT_LONG;   // long job: counted by the whole warp below
+                    cnt = COUNT_LONG;   // long job: counted by the whole CTA below
+                    if (sub == 0) {
+                        const uint64_t w0 = s >> 5;
+                        ldesc[atomicAdd(&n_long_cta, 1u)] =
+                            make_uint4((uint32_t)w0, (uint32_t)(w0 >> 32), (uint32_t)(((e - 1) >> 5) - w0),
+                                       (uint32_t)(s & 31) | ((uint32_t)((e - 1) & 31) << 8) | ((slot0 + i) << 16));
+                    }
                 } else if (s < e) {
                     const uint64_t w0 = s >> 5, w1 = (e - 1) >> 5;
                     const uint32_t m0 = 0xFFFFFFFFu << (uint32_t)(s & 31);
@@ -76,44 +91,84 @@ __global__ void __launch_bounds__(256) count_boundaries_kernel(
             cnt += __shfl_xor_sync(0xFFu << (lane & 24u), cnt, 2);
             cnt += __shfl_xor_sync(0xFFu << (lane & 24u), cnt, 4);
         }
-        if (sub == 0) cnts[slot0 + i] = cnt;
+        if (sub == 0) { cnts[slot0 + i] = cnt; is_long[slot0 + i] = lng ? 1u : 0u; }
     }
-    __syncwarp();
-    // long jobs (more than 256 safe words): all 32 lanes stride over the words of one job
-    for (uint32_t i = 0; i < COUNT_JOBS_PER_WARP; ++i) {
-        if (cnts[slot0 + i] != COUNT_LONG) continue;   // same value in every lane
-        const uint32_t j = jbase + i;
-        const uint64_t s = __ldg(off + j) + (p0 ? __ldg(p0 + j) : 0u), e = __ldg(off + j + 1);
-        const uint64_t w0 = s >> 5, w1 = (e - 1) >> 5;
-        uint32_t cnt = 0;
-        // interior words eight at a time (eight independent loads in flight per lane), then the edges one by one
-        uint64_t w = w0 + lane;
-        for (; w + 7 * 32 < w1; w += 8 * 32) {
-            uint32_t x[8];
+    __syncthreads();
+    // long jobs (more than 256 safe words), by the whole CTA: every thread takes up to eight words of a job, 256
+    // apart, and two jobs are under way at a time (sixteen independent loads in flight per thread), so that all
+    // warps of the CTA carry the long jobs of any one of them and a job costs about half a memory round trip.
+    // A warp adds its part to the job's counter in shared memory.  The thread that holds a job's last word also
+    // counts the end of the job where its bit is not set.
+    {
+        const uint32_t n_long = n_long_cta;
+        // words [base, base + 8 * 256) of the job, relative to its first word
+        auto load8 = [&](const uint4& dsc, uint32_t base, uint32_t (&x)[8]) {
+            const uint64_t w0 = pack64(dsc.x, dsc.y);
 #pragma unroll
-            for (int u = 0; u < 8; ++u) x[u] = __ldg(sbits + w + 32 * u);
-            if (w == w0) x[0] &= 0xFFFFFFFFu << (uint32_t)(s & 31);
+            for (int u = 0; u < 8; ++u) {
+                const uint32_t r = base + threadIdx.x + 256u * u;
+                x[u] = r <= dsc.z ? __ldg(sbits + w0 + r) : 0u;
+            }
+        };
+        auto tally8 = [&](const uint4& dsc, uint32_t base, uint32_t (&x)[8]) -> uint32_t {
+            const uint32_t first_bit = dsc.w & 31u, last_bit = (dsc.w >> 8) & 31u;
+            uint32_t cnt = 0;
 #pragma unroll
-            for (int u = 0; u < 8; ++u) cnt += __popc(x[u]);
+            for (int u = 0; u < 8; ++u) {
+                const uint32_t r = base + threadIdx.x + 256u * u;
+                if (r == 0u) x[u] &= 0xFFFFFFFFu << first_bit;
+                if (r == dsc.z) {
+                    cnt += 1u - ((x[u] >> last_bit) & 1u);
+                    x[u] &= 0xFFFFFFFFu >> (31u - last_bit);
+                }
+                cnt += __popc(x[u]);
+            }
+            return cnt;
+        };
+        auto add = [&](const uint4& dsc, uint32_t cnt) {
+            cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+            if (lane == 0 && cnt) atomicAdd(&long_cnt[dsc.w >> 16], cnt);
+        };
+        for (uint32_t q = 0; q < n_long; q += 2) {
+            const bool two = q + 1 < n_long;
+            const uint4 da = ldesc[q];
+            const uint4 db = two ? ldesc[q + 1] : make_uint4(0u, 0u, 0u, 0u);
+            uint32_t xa[8], xb[8];
+            load8(da, 0u, xa);
+            if (two) load8(db, 0u, xb);
+            uint32_t ca = tally8(da, 0u, xa);
+            uint32_t cb = two ? tally8(db, 0u, xb) : 0u;
+            // jobs of more than 2048 words: the rest, one job at a time
+            for (uint32_t base = 8u * 256u; base <= da.z; base += 8u * 256u) {
+                load8(da, base, xa);
+                ca += tally8(da, base, xa);
+            }
+            if (two)
+                for (uint32_t base = 8u * 256u; base <= db.z; base += 8u * 256u) {
+                    load8(db, base, xb);
+                    cb += tally8(db, base, xb);
+                }
+            add(da, ca);
+            if (two) add(db, cb);
         }
-        for (; w <= w1; w += 32) {
-            uint32_t x = __ldg(sbits + w);
-            if (w == w0) x &= 0xFFFFFFFFu << (uint32_t)(s & 31);
-            if (w == w1) x &= 0xFFFFFFFFu >> (31u - (uint32_t)((e - 1) & 31));
-            cnt += __popc(x);
-        }
-        cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
-        cnt += 1u - ((__ldg(sbits + w1) >> (uint32_t)((e - 1) & 31)) & 1u);
-        __syncwarp();
-        if (lane == 0) cnts[slot0 + i] = cnt;
-        __syncwarp();
     }
     __syncthreads();
     // exclusive scan of the CTA's counts by its first warps, one job per thread
     uint32_t mine = 0;
     uint64_t inc = 0;
     if (threadIdx.x < COUNT_JOBS_PER_CTA) {
+        // the list of long jobs (flags[1] counts them): one atomic per warp of 32 jobs, not one per job --
+        // on a heavy-tailed mix every eighth job is long, and that many atomics on one word take longer than the count
+        const bool lng = is_long[threadIdx.x] != 0u;
+        const uint32_t lb = __ballot_sync(0xFFFFFFFFu, lng);
+        if (lb) {
+            uint32_t base = 0;
+            if (lane == 0) base = atomicAdd(flags + 1, (uint32_t)__popc(lb));
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            if (lng) long_list[base + __popc(lb & ((1u << lane) - 1u))] = blockIdx.x * COUNT_JOBS_PER_CTA + threadIdx.x;
+        }
         mine = cnts[threadIdx.x];
+        if (mine == COUNT_LONG) mine = long_cnt[threadIdx.x];
         inc = mine;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
