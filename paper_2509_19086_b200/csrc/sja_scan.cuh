@@ -112,12 +112,14 @@ __global__ void __launch_bounds__(SCAN_WARPS * 32, SCAN_CTAS_PER_SM) scan_profil
     const uint32_t lane_sw = (lane ^ ((lane >> 3) & 3u)) * 16u;   // swz(32 r + lane) * 16 - 512 r
     const uint32_t rd_x = (lane >> 1) & 3u;                        // swz(4 lane + r) = 4 lane + (r ^ rd_x)
 
+    // hand-out order: the listed long jobs first, then all jobs in id order (neighbouring warps stream
+    // neighbouring memory), the long ones skipped.  A warp draws its next number when it starts on a job, so
+    // that the counter's round trip is over by the time the job is done.
+    uint32_t drawn = 0;
+    if (lane == 0) drawn = atomicAdd(a.counter, 1u);
     for (;;) {
-        // hand-out order: the listed long jobs first, then all jobs in id order (neighbouring warps stream
-        // neighbouring memory), the long ones skipped
-        uint32_t c = 0;
-        if (lane == 0) c = atomicAdd(a.counter, 1u);
-        c = __shfl_sync(0xFFFFFFFFu, c, 0);
+        const uint32_t c = __shfl_sync(0xFFFFFFFFu, drawn, 0);
+        if (lane == 0) drawn = atomicAdd(a.counter, 1u);
         uint32_t j;
         if (c < n_long) {
             j = __ldg(a.long_list + c);
