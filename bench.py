@@ -57,8 +57,8 @@ def select_launches(pairs, flags, per_pair_window):
 # large uniform configuration at full size: reads grow with the step count, writes with the number of boundary
 # rows.  The figures are reported only while csrc/sja_scan.cuh is the file they were taken from (first 16 hex
 # digits of its sha256); otherwise "traffic" is null.
-NCU_SCAN = {"source_sha": "351669ab0df1e1e6", "read_bytes_per_step": 2184044544 / 268435456,
-            "write_bytes_per_row": 625089536 / 26906044}
+NCU_SCAN = {"source_sha": "06cf166b6a8a770f", "read_bytes_per_step": 2184370432 / 268435456,
+            "write_bytes_per_row": 625901568 / 26906044}
 
 # Warp instructions of one select_tile_kernel launch (ncu smsp__inst_executed.sum, one pass, full size), per
 # workload; valid while csrc/sja_tile.cuh is the file they were taken from.  The kernel's work is not proportional
