@@ -20,7 +20,7 @@ constexpr int COUNT_JOBS_PER_CTA = 64;
 constexpr int COUNT_JOBS_PER_WARP = 8;
 constexpr uint32_t COUNT_LONG = 0x80000000u;   // marker: job left to the whole-CTA pass
 
-__global__ void __launch_bounds__(256) count_boundaries_kernel(
+__global__ void __launch_bounds__(256, 8) count_boundaries_kernel(
     const uint64_t* __restrict__ off, const uint32_t* __restrict__ sbits,
     const uint32_t* __restrict__ p0 /* may be nullptr: all 0 */, uint32_t J, uint64_t* __restrict__ local_off,
     uint64_t* __restrict__ cta_total, uint32_t* __restrict__ flags, uint32_t* __restrict__ long_list) {
