@@ -18,6 +18,10 @@ namespace sja {
 // turn CTA totals into global offsets.
 constexpr int COUNT_JOBS_PER_CTA = 64;
 constexpr int COUNT_JOBS_PER_WARP = 8;
+#ifndef SJA_COUNT_COOP_WORDS
+#define SJA_COUNT_COOP_WORDS 256
+#endif
+constexpr uint32_t COUNT_COOP_WORDS = SJA_COUNT_COOP_WORDS;   // jobs of this many safe words or more: whole-CTA pass (swept 16 .. 1024)
 constexpr uint32_t COUNT_LONG = 0x80000000u;   // marker: job left to the whole-CTA pass
 
 __global__ void __launch_bounds__(256, 8) count_boundaries_kernel(
@@ -54,7 +58,7 @@ __global__ void __launch_bounds__(256, 8) count_boundaries_kernel(
             if (!bad) {
                 const uint64_t s = js + p, e = je;
                 lng = e - s > long_thresh;   // goes on the list the scan works off first
-                if (s < e && ((e - 1) >> 5) - (s >> 5) >= 256) {
+                if (s < e && ((e - 1) >> 5) - (s >> 5) >= COUNT_COOP_WORDS) {
                     cnt = COUNT_LONG;   // long job: counted by the whole CTA below
                     if (sub == 0) {
                         const uint64_t w0 = s >> 5;
