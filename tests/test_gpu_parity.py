@@ -111,6 +111,35 @@ def test_scan_matches_oracle_boundary_densities_around_the_row_buffer(sja_mod, o
         _check_scan(oracle_mod, ctx, prof, progress)
 
 
+def test_scan_long_jobs_counted_by_the_whole_cta(sja_mod, oracle_mod):
+    """Jobs of more than 8192 steps (256 safe words) are counted by the whole counting CTA, two at a time, and jobs of
+    more than 65 536 steps take several trips; an even and an odd number of them per block of 64 jobs, some entered
+    at a progress point that is not word-aligned, between short jobs."""
+    rng = np.random.default_rng(104)
+    lens = [int(x) for x in rng.integers(1, 600, 140)]
+    for pos, n in ((3, 150_000), (4, 70_000), (17, 9_000), (40, 8_225), (41, 66_000), (63, 12_345),   # six in block 0
+                   (64, 65_536 + 31), (90, 8_193), (127, 30_000),                                     # three in block 1
+                   (139, 100_001)):                                                                   # one in block 2
+        lens[pos] = n
+    jobs = []
+    for n in lens:
+        d = rng.integers(1, 50, n).astype(np.uint32)
+        m = rng.integers(1, 81920, n).astype(np.uint32)
+        s = (rng.random(n) < 0.1).astype(np.uint8)
+        jobs.append((d, m, s))
+    off = np.zeros(len(jobs) + 1, np.uint64)
+    off[1:] = np.cumsum(lens)
+    prof = wl.Profiles(off, np.concatenate([j[0] for j in jobs]), np.concatenate([j[1] for j in jobs]),
+                       wl.pack_safe_bits(np.concatenate([j[2] for j in jobs])),
+                       rng.integers(0, 100, len(jobs)).astype(np.uint32), None, None)
+    progress = np.zeros(len(jobs), np.uint32)
+    for pos, p in ((3, 70_001), (4, 33), (41, 500), (64, 31), (127, 21_000), (139, 99_990)):
+        progress[pos] = p
+    with sja_mod.Sja() as ctx:
+        _load(ctx, prof, progress)
+        _check_scan(oracle_mod, ctx, prof, progress)
+
+
 def test_scan_cfg1_sampled_jobs(sja_mod, oracle_mod):
     spec = wl.SPECS[1]
     prof = wl.make_profiles(spec)
