@@ -58,6 +58,7 @@ struct sja_ctx {
     bool loaded = false;
     uint32_t J = 0;
     uint64_t N = 0, n_rows = 0;
+    uint32_t n_long = 0;               // jobs the load listed as long (many more steps than the mean)
     bool have_wait = false, have_prio = false;
     uint32_t load_flags = 0;
     DevBuf st_off, st_d, st_m, st_s, st_p, st_ready, st_wait, st_prio;   // staging for host inputs
@@ -574,7 +575,7 @@ sja_status sja_create(sja_ctx** out, int device, void* cuda_stream) {
         c->n_sm = prop.multiProcessorCount;
         if (cudaMallocHost(reinterpret_cast<void**>(&c->h_words), 512) != cudaSuccess) { st = SJA_ERR_OOM; break; }
         if ((st = reserve(c, c->flags, 8)) != SJA_OK) break;   // [0] status bits, [1] long-job count of a load
-        if ((st = reserve(c, c->counter, 4)) != SJA_OK) break;
+        if ((st = reserve(c, c->counter, 8)) != SJA_OK) break;
         if ((st = reserve(c, c->n_granted, 4)) != SJA_OK) break;
         if (cudaMemsetAsync(c->flags.p, 0, 8, c->stream) != cudaSuccess) { st = SJA_ERR_CUDA; break; }
         if (cudaFuncSetAttribute(scan_profiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -801,11 +802,12 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
     // verdict (waits for the stream): flags, row count and, if not known yet, N
     uint64_t n_rows = 0;
     uint32_t flags = 0;
-    CU(cudaMemcpyAsync(c->h_words, c->flags.p, 4, cudaMemcpyDeviceToHost, c->stream));
+    CU(cudaMemcpyAsync(c->h_words, c->flags.p, 8, cudaMemcpyDeviceToHost, c->stream));   // status, long jobs listed
     CU(cudaMemcpyAsync(c->h_words + 2, c->cta_base.as<uint64_t>() + n_count_ctas, 8, cudaMemcpyDeviceToHost, c->stream));
     if (!n_known) CU(cudaMemcpyAsync(c->h_words + 4, d_off + J, 8, cudaMemcpyDeviceToHost, c->stream));
     CU(cudaStreamSynchronize(c->stream));
     flags = c->h_words[0];
+    const uint32_t n_long_jobs = c->h_words[1];
     if (!n_known) {
         memcpy(&N, c->h_words + 4, 8);
         n_known = true;
@@ -853,6 +855,7 @@ sja_status sja_load_profiles(sja_ctx* c, uint32_t J, const uint64_t* off, const 
     if (flags & FLAG_OVF_DURATION) return fail(c, SJA_ERR_OVERFLOW, "a job's total duration does not fit in 32 bits");
     if (flags & FLAG_OVF_WORK) return fail(c, SJA_ERR_OVERFLOW, "a job's total work is >= 2^63");
     c->load_flags = flags;
+    c->n_long = n_long_jobs;
     c->loaded = true;
     return SJA_OK;
 }
@@ -1292,9 +1295,24 @@ sja_status sja_load_power(sja_ctx* c, const uint64_t* off, const uint32_t* power
     c->selected = false;       // awards chosen without the trace must not be committed with it
     {
         ProfScope ps(c, CAT_PREP);
-        scan_power_kernel<<<(c->J + POWER_WARPS - 1) / POWER_WARPS, POWER_WARPS * 32, 0, c->stream>>>(
-            d_off, d_pw, c->J, c->boff.as<uint64_t>(), c->pb.as<uint32_t>(), c->p.as<uint32_t>(), c->B.as<uint2>(),
-            c->PW.as<uint2>(), c->flags.as<uint32_t>());
+        // Jobs of about equal length: a warp per job, as many CTAs as that takes.  A load that listed long jobs:
+        // a persistent grid (as many CTAs as the GPU holds at once) whose warps draw jobs from two counters, the
+        // long ones first -- with a warp per job the CTA of a long job would hold seven idle warps' places.
+        const uint32_t want = (c->J + POWER_WARPS - 1) / POWER_WARPS;
+        uint32_t grid = want;
+        if (c->n_long) {
+            int per_sm = 0;
+            CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, scan_power_kernel<true>, POWER_WARPS * 32, 0));
+            grid = std::min<uint32_t>(want, (uint32_t)c->n_sm * (uint32_t)std::max(per_sm, 1));
+            CU(cudaMemsetAsync(c->counter.p, 0, 8, c->stream));
+            scan_power_kernel<true><<<grid, POWER_WARPS * 32, 0, c->stream>>>(
+                d_off, d_pw, c->J, c->boff.as<uint64_t>(), c->pb.as<uint32_t>(), c->p.as<uint32_t>(), c->B.as<uint2>(),
+                c->PW.as<uint2>(), c->flags.as<uint32_t>(), c->counter.as<uint32_t>());
+        } else {
+            scan_power_kernel<false><<<grid, POWER_WARPS * 32, 0, c->stream>>>(
+                d_off, d_pw, c->J, c->boff.as<uint64_t>(), c->pb.as<uint32_t>(), c->p.as<uint32_t>(), c->B.as<uint2>(),
+                c->PW.as<uint2>(), c->flags.as<uint32_t>(), c->counter.as<uint32_t>());
+        }
     }
     CU(cudaGetLastError());
     uint32_t flags = 0;

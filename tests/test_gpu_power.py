@@ -132,3 +132,40 @@ def test_power_errors_and_lifetime(oracle_mod):
         ctx.advertise(gaps)
         ctx.advertise_power_caps(np.full(gaps.shape[0], 0, np.uint32))
         _same(ctx.select(spec.policy, out="host"), oracle_mod.select(prof, z, prof.ready_ms, gaps, spec.policy))
+
+
+def test_power_trace_on_a_load_with_long_jobs(oracle_mod):
+    """A load that lists long jobs (far more steps left than the mean, at least 8192) takes the power scan's other
+    hand-out: warps draw jobs from counters, the long ones first.  Long windows and loose capacities, so that awards
+    reach deep into the long jobs' rows; some jobs entered at a progress point."""
+    from paper_2509_19086_b200 import binding
+    rng = np.random.default_rng(1400)
+    lens = [int(x) for x in rng.integers(1, 700, 300)]
+    for pos, n in ((0, 20_000), (7, 9_500), (8, 33_000), (150, 8_700), (299, 12_000)):
+        lens[pos] = n
+    N = int(np.sum(lens))
+    off = np.zeros(len(lens) + 1, np.uint64)
+    off[1:] = np.cumsum(lens)
+    safe = (rng.random(N) < 0.1).astype(np.uint8)
+    prof = wl.Profiles(off, rng.integers(1, 50, N).astype(np.uint32), rng.integers(1, 81920, N).astype(np.uint32),
+                       wl.pack_safe_bits(safe), rng.integers(0, 100, len(lens)).astype(np.uint32), None, None)
+    progress = np.zeros(len(lens), np.uint32)
+    for pos, p in ((0, 10_001), (8, 7), (150, 8_000), (20, 100)):
+        progress[pos] = min(p, lens[pos])
+    power = rng.integers(50, 400, N).astype(np.uint32)
+    G = 160
+    gaps = gaps_from_lists([(int(rng.integers(0, 7)), int(rng.integers(100, 2000)),
+                             int(rng.choice([500, 5_000, 100_000, 1_000_000])), int(rng.choice([40960, 81920])))
+                            for _ in range(G)])
+    caps = rng.integers(300, 420, G).astype(np.uint32)
+    caps[rng.random(G) < 0.3] = U32MAX
+    with binding.Sja() as ctx:
+        _load(ctx, prof, progress)
+        ctx.load_power(prof.off, power)
+        ctx.advertise(gaps)
+        ctx.advertise_power_caps(caps)
+        want = oracle_mod.select(prof, progress, prof.ready_ms, gaps, 0, power_W=power, power_cap_W=caps)
+        got = ctx.select(0, out="host")
+        _same(got, want)
+        assert (want["job"] != U32MAX).sum() > G // 4
+        assert want["end_step"].max() > 1000      # some award runs far into a long job
