@@ -59,6 +59,7 @@ struct sja_ctx {
     uint32_t J = 0;
     uint64_t N = 0, n_rows = 0;
     uint32_t n_long = 0;               // jobs the load listed as long (many more steps than the mean)
+    bool reauction_later_pass = false; // set by sja_round_reauction around the select of its passes after the first
     bool have_wait = false, have_prio = false;
     uint32_t load_flags = 0;
     DevBuf st_off, st_d, st_m, st_s, st_p, st_ready, st_wait, st_prio;   // staging for host inputs
@@ -386,6 +387,9 @@ struct SelectPlan { KernelPlan primary, alt; bool have_alt; uint32_t max_classes
 
 // `fixed`: the passes of a re-auction keep the candidate rows of untouched job chunks from pass to pass, so the
 // kernel and its chunk size must not change with the number of gaps left.
+#ifndef SJA_REAUC_SPLIT_GAPS
+#define SJA_REAUC_SPLIT_GAPS 256
+#endif
 KernelPlan plan_kernel(const sja_ctx* c, SelectKernel k, uint32_t G_act, bool fixed) {
     KernelPlan p;
     p.kernel = k;
@@ -403,6 +407,12 @@ KernelPlan plan_kernel(const sja_ctx* c, SelectKernel k, uint32_t G_act, bool fi
     const uint32_t max_splits = (G_act + tile - 1) / tile;
     if (splits > max_splits) splits = max_splits;
     if (splits < 1) splits = 1;
+#if SJA_REAUC_SPLIT_GAPS > 0
+    // Later passes of a re-auction evaluate a handful of job chunks only (the others keep their candidate rows):
+    // the grid is nearly empty and a pass lasts as long as one CTA needs for its gaps, so the gaps are cut finer.
+    if (fixed && c->reauction_later_pass && k != SEL_SEARCH)
+        splits = std::min(max_splits, std::max(splits, (G_act + SJA_REAUC_SPLIT_GAPS - 1) / SJA_REAUC_SPLIT_GAPS));
+#endif
     uint32_t per_split = (G_act + splits - 1) / splits;
     per_split = ((per_split + tile - 1) / tile) * tile;
     p.per_split = per_split;
@@ -1069,6 +1079,7 @@ sja_status sja_round_reauction(sja_ctx* c, const sja_policy* policy, uint32_t ma
         if (max_passes != 0) batch = std::min(batch, max_passes - passes);
         for (uint32_t k = 0; k < batch; ++k) {
             const uint32_t* g_dev = k ? reports + 4 * (k - 1) : nullptr;   // gaps left after the pass before
+            c->reauction_later_pass = passes + k > 0;
             TRY(run_select(c, kind, policy->flags, cur, g_act, c->blocked.as<uint32_t>(), nullptr, true, g_dev, dirty_cur,
                            classes_known));
             {
